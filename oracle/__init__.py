@@ -1,0 +1,15 @@
+"""CPU oracle for the full-FP4 Direct-P attention forward.
+
+TEST INFRASTRUCTURE ONLY.  Plain, slow, fp64 NumPy restatement of what the hot path
+computes, written from the paper.  It shares no code with the CUDA path and must never
+be imported by the product package; only tests, the smoke check and the benchmark's
+cpu-baseline leg may call it.
+
+Pinned by tests/test_oracle_*.py (run with -m "not gpu"):
+  formats.py    E2M1 / E8M0 / E4M3 coders      -> printed codebook and boundaries, exhaustive
+                                                  enumeration, closed forms, Table "p-range"
+  quantize.py   MXFP4 / NVFP4 operand quantizers -> closed forms, brute force, error bounds
+  attention.py  tiled Direct-P forward          -> tile-size / tile-order invariance, V == 1,
+                                                  equal keys, dominant key, brute-force exact
+                                                  attention on losslessly representable inputs
+"""

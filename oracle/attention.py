@@ -1,0 +1,146 @@
+"""Tiled Direct-P attention forward (oracle side, test infrastructure only).
+
+Follows, in the paper's order and notation:
+  * the online recurrence over key tiles (Eq. "online-recurrence"),
+  * Algorithm "direct-p-pack" for every N32 score fragment: block maximum -> power-of-two
+    amplitude alpha_B = 2**e_B with byte u_B = e_B + 127 (a block whose byte would fall
+    below 1 is a zero block) -> x = (z - m)*log2(e) - e_B + log2(6) -> q = Q_E2M1(2**x)
+    (Eq. "ideal-code-path") -> code sum c_B,
+  * the represented numerator / denominator (Eqs. "represented-contributions",
+    "represented-output"), with the denominator term evaluated as alpha_B * (c_B / 6) in that
+    association (Algorithm "sampled-guard", steps 4-5).
+
+Readings where the paper leaves a choice (listed in the design notes of the repository):
+  * row reference m_i: the running maximum rounded UP to an integer in the log2 domain,
+    mu_i = max over tiles seen so far of ceil(max_j y_ij), y = z*log2(e).  With an integer
+    reference every online rescale factor is an exact power of two and
+    x = y - E_B + log2(6) no longer depends on the reference, so the represented
+    probabilities do not depend on tile size, tile order or rescale policy;
+  * block exponent: E_B = ceil(max_{j in B} y_ij) (absolute), e_B = E_B - mu_i;
+  * "fp32 accumulate": the score handed to softmax is the exact block-scaled product rounded
+    once to float32; y used for the integer decisions is the float32 product fl32(s32*c32).
+  * LSE is the natural log of the represented denominator.
+
+Everything else is float64.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+from .formats import E2M1_VALUES, e2m1_encode_mag
+from .quantize import dequantize
+
+LOG2E_32 = np.float32(1.4426950408889634)
+LOG2_6_32 = np.float32(math.log2(6.0))
+P_BLOCK = 32
+
+
+def score_constant(qd: dict, kd: dict, d: int, softmax_scale=None) -> np.float32:
+    """c32: multiplies the tensor-core-facing score S_hw to give y = z*log2(e).
+
+    MXFP4 x MXFP4: S_hw carries 6*6 (amplitude convention) -> c = fl32(fl32(log2e*scale)/36).
+    NVFP4 x NVFP4: S_hw carries G_q*G_k              -> c = fl32(fl32(log2e*scale)/fl32(G_q*G_k)).
+    """
+    scale = np.float32(1.0 / math.sqrt(d)) if softmax_scale is None else np.float32(softmax_scale)
+    base = np.float32(LOG2E_32 * scale)
+    if qd["fmt"] == "mx" and kd["fmt"] == "mx":
+        return np.float32(base / np.float32(36.0))
+    assert qd["fmt"] == "nv" and kd["fmt"] == "nv"
+    return np.float32(base / np.float32(np.float32(qd["G"]) * np.float32(kd["G"])))
+
+
+def scores_fp32(qd: dict, kd: dict, b: int, h: int, rows=None) -> np.ndarray:
+    """S_hw[i, j] = sum_k (scale*code)_Q[i,k] * (scale*code)_K[j,k], exact, rounded once to fp32."""
+    A = dequantize({**qd, "nib": qd["nib"][b, h][None, None], "sf": qd["sf"][b, h][None, None]}, hw=True)[0, 0]
+    Bm = dequantize({**kd, "nib": kd["nib"][b, h][None, None], "sf": kd["sf"][b, h][None, None]}, hw=True)[0, 0]
+    if rows is not None:
+        A = A[rows]
+    return (A @ Bm.T).astype(np.float32)
+
+
+def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int = 128, tile_order=None):
+    """Direct-P online softmax + PV for a set of query rows of one (batch, head).
+
+    s32  [R, N] float32 tensor-core-facing scores;  Vhat [N, d] float64 reconstructed V.
+    Returns O [R, d] float64, LSE [R] float64, and the represented probabilities' pieces
+    (codes [R, N] uint8, block exponents E_B [R, N/32] int64, final reference mu [R]).
+    """
+    R, N = s32.shape
+    assert N % P_BLOCK == 0 and tile % P_BLOCK == 0 and N % tile == 0
+    y32 = (s32 * np.float32(c32)).astype(np.float32)             # decision variable, fp32
+    yx = s32.astype(np.float64) * np.float64(c32)                # converter input, fp64
+    mu = np.full(R, -np.inf)
+    L = np.zeros(R)
+    O = np.zeros((R, Vhat.shape[1]))
+    codes_all = np.zeros((R, N), dtype=np.uint8)
+    EB_all = np.zeros((R, N // P_BLOCK), dtype=np.int64)
+    order = range(N // tile) if tile_order is None else tile_order
+    for t in order:
+        j0 = t * tile
+        m_tile = np.ceil(y32[:, j0:j0 + tile].max(axis=1).astype(np.float64))
+        mu_new = np.maximum(mu, m_tile)
+        f = np.where(np.isinf(mu), 0.0, np.exp2(mu - mu_new))     # exact power of two
+        L *= f
+        O *= f[:, None]
+        mu = mu_new
+        for bj in range(j0, j0 + tile, P_BLOCK):
+            E_B = np.ceil(y32[:, bj:bj + P_BLOCK].max(axis=1).astype(np.float64))
+            e_B = E_B - mu
+            live = (e_B + 127) >= 1
+            b_B = np.float32(LOG2_6_32 - E_B.astype(np.float32)).astype(np.float64)
+            x = yx[:, bj:bj + P_BLOCK] + b_B[:, None]
+            code = e2m1_encode_mag(np.exp2(x))
+            code = np.where(live[:, None], code, 0).astype(np.uint8)
+            q = E2M1_VALUES[code]
+            alpha = np.where(live, np.exp2(e_B), 0.0)
+            c_B = q.sum(axis=1)
+            L += alpha * (c_B / 6.0)
+            O += (alpha / 6.0)[:, None] * (q @ Vhat[bj:bj + P_BLOCK])
+            codes_all[:, bj:bj + P_BLOCK] = code
+            EB_all[:, bj // P_BLOCK] = E_B.astype(np.int64)
+    Oout = O / L[:, None]
+    lse = math.log(2.0) * (mu + np.log2(L))
+    return Oout, lse, codes_all, EB_all, mu
+
+
+def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int = 128,
+                     rows=None, heads=None, tile_order=None):
+    """Whole-operator oracle.  qd/kd/vd come from oracle.quantize.quantize_qk / quantize_v.
+
+    rows : optional 1-D index array of query rows evaluated for every (b, h) (rows are
+           independent); heads : optional list of (b, h) pairs.  Returns O [n_heads, R, d]
+           float64 and LSE [n_heads, R] float64 in the order of `heads`.
+    """
+    B, H, N, d = qd["nib"].shape
+    heads = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
+    c32 = score_constant(qd, kd, d, softmax_scale)
+    Os, Ls = [], []
+    for (b, h) in heads:
+        s32 = scores_fp32(qd, kd, b, h, rows)
+        Vhat = dequantize({**vd, "nib": vd["nib"][b, h][None, None], "sf": vd["sf"][b, h][None, None]})[0, 0].T
+        O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order)
+        Os.append(O)
+        Ls.append(lse)
+    return np.stack(Os), np.stack(Ls)
+
+
+def exact_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray, softmax_scale=None, rows=None):
+    """Eq. "exact-attention" in float64 for one head: Q [N,d], K [N,d], V [N,d] -> O, LSE."""
+    d = Q.shape[1]
+    scale = 1.0 / math.sqrt(d) if softmax_scale is None else float(softmax_scale)
+    Qr = Q if rows is None else Q[rows]
+    z = (Qr @ K.T) * scale
+    m = z.max(axis=1, keepdims=True)
+    p = np.exp(z - m)
+    l = p.sum(axis=1, keepdims=True)
+    return (p @ V) / l, (m + np.log(l))[:, 0]
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """float64 -> nearest bfloat16 value (ties to even), returned as float64."""
+    x = np.asarray(x, dtype=np.float64)
+    _, e = np.frexp(x)                    # |x| in [2**(e-1), 2**e)
+    step = np.ldexp(1.0, e - 8)           # 8 significant bits
+    return np.rint(x / step) * step       # rint is round-half-even

@@ -1,0 +1,163 @@
+"""Operand quantizers of the path (oracle side, test infrastructure only).
+
+MXFP4 (Eq. "mx-scale", amplitude convention): a block of 32 values with maximum
+magnitude a stores the power-of-two amplitude alpha = 2**ceil(log2 a) as the E8M0 byte
+u = 127 + ceil(log2 a) and the codes q = Q_E2M1(6 v / alpha); a value is reconstructed
+as alpha * q / 6.  Reading taken here: the ceiling of the two powers the paper allows,
+so the block maximum lands in (3, 6] and never saturates.
+
+NVFP4 (Table "fp4-formats", Eq. "nv-scale"): a block of 16 values stores
+S_B = Q_E4M3(G a_B / 6) and q = Q_E2M1(G v / S_B); reconstruction S_B q / G.  Reading
+taken here: one encode factor G = 448*6 / max|x| per tensor; the scale arithmetic is
+carried in float32 in a fixed order so that a GPU can reproduce the bytes exactly.
+
+Q and K are blocked along the head dimension (the contraction of QK^T); V is blocked
+along the key index (the contraction of PV) and is emitted transposed, [.., d, N].
+
+Layouts of the bytes handed to the attention kernel are restated at the end of the file
+(packing two nibbles per byte, and the 128x4 scale atom the block-scaled tensor-core
+instruction reads).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from .formats import (ceil_log2, e2m1_decode, e2m1_encode, e4m3_decode,
+                      e4m3_encode_unsigned, e8m0_decode)
+
+MX_BLOCK = 32
+NV_BLOCK = 16
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    u = np.asarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return u.view(np.float32).astype(np.float64)
+
+
+# --------------------------------------------------------------------------- MXFP4
+def mx_quantize_lastdim(x: np.ndarray):
+    """x float64 [..., L], L % 32 == 0, blocks of 32 along the last axis.
+
+    Returns (nibbles uint8 [..., L], scale bytes uint8 [..., L/32]).
+    """
+    L = x.shape[-1]
+    assert L % MX_BLOCK == 0
+    xb = x.reshape(x.shape[:-1] + (L // MX_BLOCK, MX_BLOCK))
+    a = np.abs(xb).max(axis=-1)
+    nz = a > 0
+    e = ceil_log2(np.where(nz, a, 1.0))
+    u = np.clip(e + 127, 1, 254)
+    u = np.where(nz, u, 0).astype(np.uint8)
+    alpha = e8m0_decode(u)
+    codes = e2m1_encode(6.0 * xb / alpha[..., None])
+    codes = np.where(nz[..., None], codes, 0).astype(np.uint8)
+    return codes.reshape(x.shape), u
+
+
+def mx_dequantize_lastdim(nib: np.ndarray, u: np.ndarray, hw: bool = False) -> np.ndarray:
+    """alpha*q/6 (hw=False) or the tensor-core-facing alpha*q (hw=True)."""
+    L = nib.shape[-1]
+    q = e2m1_decode(nib).reshape(nib.shape[:-1] + (L // MX_BLOCK, MX_BLOCK))
+    alpha = np.where(u == 0, 0.0, e8m0_decode(u))
+    v = q * alpha[..., None]
+    if not hw:
+        v = v / 6.0
+    return v.reshape(nib.shape)
+
+
+# --------------------------------------------------------------------------- NVFP4
+def nv_tensor_scale(x: np.ndarray) -> np.float32:
+    """Encode factor G = fl32(2688 / max|x|) (G = 1 for an all-zero tensor)."""
+    aT = np.float32(np.abs(x).max())
+    if aT == 0:
+        return np.float32(1.0)
+    return np.float32(np.float32(2688.0) / aT)
+
+
+def nv_quantize_lastdim(x: np.ndarray, G: np.float32):
+    """x float64 holding bf16 values, [..., L], L % 16 == 0.
+
+    float32 steps, in this order:  t = fl32(fl32(a_B * G) / 6);  S_B = Q_E4M3(t);
+    r = fl32(G / S_B);  q = Q_E2M1(fl32(|v| * r)).  S_B == 0 makes the block vanish.
+    Returns (nibbles [..., L], scale bytes [..., L/16]).
+    """
+    L = x.shape[-1]
+    assert L % NV_BLOCK == 0
+    G = np.float32(G)
+    xb = x.reshape(x.shape[:-1] + (L // NV_BLOCK, NV_BLOCK)).astype(np.float32)
+    a = np.abs(xb).max(axis=-1)
+    t = (a * G).astype(np.float32) / np.float32(6.0)
+    sbyte = e4m3_encode_unsigned(t.astype(np.float64))
+    S = e4m3_decode(sbyte).astype(np.float32)
+    with np.errstate(divide="ignore"):
+        r = np.where(S > 0, G / np.where(S > 0, S, np.float32(1)), np.float32(0)).astype(np.float32)
+    scaled = (np.abs(xb) * r[..., None]).astype(np.float32)
+    codes = e2m1_encode(np.copysign(scaled.astype(np.float64), xb.astype(np.float64)))
+    codes = np.where((S > 0)[..., None], codes, 0).astype(np.uint8)
+    return codes.reshape(x.shape), sbyte
+
+
+def nv_dequantize_lastdim(nib: np.ndarray, sbyte: np.ndarray, G=None, hw: bool = False) -> np.ndarray:
+    """S_B*q/G (hw=False) or the tensor-core-facing S_B*q (hw=True)."""
+    L = nib.shape[-1]
+    q = e2m1_decode(nib).reshape(nib.shape[:-1] + (L // NV_BLOCK, NV_BLOCK))
+    v = q * e4m3_decode(sbyte)[..., None]
+    if not hw:
+        v = v / np.float64(G)
+    return v.reshape(nib.shape)
+
+
+# --------------------------------------------------------------------------- roles
+def quantize_qk(bits: np.ndarray, fmt: str):
+    """Q or K, bf16 bit patterns [B,H,N,d] -> dict(nib [B,H,N,d], sf [B,H,N,d/blk], G)."""
+    x = bf16_bits_to_f64(bits)
+    if fmt == "mx":
+        nib, sf = mx_quantize_lastdim(x)
+        return {"nib": nib, "sf": sf, "G": None, "fmt": "mx"}
+    G = nv_tensor_scale(x)
+    nib, sf = nv_quantize_lastdim(x, G)
+    return {"nib": nib, "sf": sf, "G": G, "fmt": "nv"}
+
+
+def quantize_v(bits: np.ndarray):
+    """V bf16 [B,H,N,d] -> MXFP4 of V^T: dict(nib [B,H,d,N], sf [B,H,d,N/32]), blocks of 32 keys."""
+    xt = np.ascontiguousarray(np.swapaxes(bf16_bits_to_f64(bits), -1, -2))
+    nib, sf = mx_quantize_lastdim(xt)
+    return {"nib": nib, "sf": sf, "G": None, "fmt": "mx"}
+
+
+def dequantize(qd: dict, hw: bool = False) -> np.ndarray:
+    if qd["fmt"] == "mx":
+        return mx_dequantize_lastdim(qd["nib"], qd["sf"], hw=hw)
+    return nv_dequantize_lastdim(qd["nib"], qd["sf"], qd["G"], hw=hw)
+
+
+# --------------------------------------------------------------------------- byte layouts
+def pack_nibbles(nib: np.ndarray) -> np.ndarray:
+    """[..., L] nibbles -> [..., L/2] bytes; element 2k in bits 0-3, element 2k+1 in bits 4-7."""
+    return (nib[..., 0::2] | (nib[..., 1::2] << 4)).astype(np.uint8)
+
+
+def strip_negative_zero(packed: np.ndarray) -> np.ndarray:
+    """Map nibble 0x8 (-0) to 0x0 so that byte comparisons ignore the sign of a zero code."""
+    lo = packed & 0x0F
+    hi = packed >> 4
+    lo = np.where(lo == 8, 0, lo)
+    hi = np.where(hi == 8, 0, hi)
+    return (lo | (hi << 4)).astype(np.uint8)
+
+
+def swizzle_scales(sf: np.ndarray) -> np.ndarray:
+    """Scale bytes [B,H,R,C] -> flat atoms [B,H, ceil(R/128)*ceil(C/4)*512].
+
+    Atom (rt, ct) covers rows 128*rt..+127 and scale columns 4*ct..+3 and starts at byte
+    (rt*ceil(C/4) + ct)*512; inside it row r, column c sits at (r%32)*16 + (r%128)//32*4 + c%4.
+    Padding bytes are zero.
+    """
+    B, H, R, C = sf.shape
+    RT, CT = -(-R // 128), -(-C // 4)
+    pad = np.zeros((B, H, RT * 128, CT * 4), dtype=np.uint8)
+    pad[:, :, :R, :C] = sf
+    # [B,H,RT, r_hi(4), r_lo(32), CT, c(4)] -> [B,H,RT,CT, r_lo, r_hi, c]
+    v = pad.reshape(B, H, RT, 4, 32, CT, 4).transpose(0, 1, 2, 5, 4, 3, 6)
+    return np.ascontiguousarray(v).reshape(B, H, RT * CT * 512)

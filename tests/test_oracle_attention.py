@@ -1,0 +1,177 @@
+"""Pins for oracle/attention.py: invariants, special cases with closed-form answers and
+brute-force exact attention."""
+import math
+
+import numpy as np
+
+from oracle import attention as A
+from oracle import formats as F
+from oracle import quantize as Qz
+from paper_2609_04105_b200 import inputs as I
+
+
+def _cfg1(fmt="mx", **kw):
+    w = I.shrink(I.WORKLOADS["cfg1"], **kw)
+    q, k, v = I.make_qkv(w)
+    return w, (q, k, v), Qz.quantize_qk(q, fmt), Qz.quantize_qk(k, fmt), Qz.quantize_v(v)
+
+
+def test_tile_size_and_tile_order_do_not_change_the_result():
+    _, _, qd, kd, vd = _cfg1()
+    O, L = A.direct_p_forward(qd, kd, vd)
+    for tile in (32, 64, 256):
+        O2, L2 = A.direct_p_forward(qd, kd, vd, tile=tile)
+        assert np.abs(O2 - O).max() < 1e-14 and np.abs(L2 - L).max() < 1e-13
+    O3, L3 = A.direct_p_forward(qd, kd, vd, tile=64, tile_order=[3, 0, 2, 1])
+    assert np.abs(O3 - O).max() < 1e-14 and np.abs(L3 - L).max() < 1e-13
+
+
+def test_score_constant_maps_hw_scores_to_log2_domain_logits():
+    for fmt in ("mx", "nv"):
+        w, _, qd, kd, _ = _cfg1(fmt, N=128)
+        c = A.score_constant(qd, kd, w.d)
+        s32 = A.scores_fp32(qd, kd, 0, 1)
+        z = Qz.dequantize(qd)[0, 1] @ Qz.dequantize(kd)[0, 1].T / math.sqrt(w.d)
+        assert np.allclose(s32.astype(np.float64) * float(c), z * math.log2(math.e), rtol=1e-6, atol=1e-6)
+
+
+def _brute_softmax_attention(y, V):
+    """Triple loop, Python floats: p_ij = 2**y_ij / sum_j 2**y_ij, O = p V."""
+    R, N = y.shape
+    O = np.zeros((R, V.shape[1]))
+    lse = np.zeros(R)
+    for i in range(R):
+        m = max(float(v) for v in y[i])
+        den = 0.0
+        for j in range(N):
+            den += 2.0 ** (float(y[i, j]) - m)
+        for j in range(N):
+            p = 2.0 ** (float(y[i, j]) - m) / den
+            for c in range(V.shape[1]):
+                O[i, c] += p * V[j, c]
+        lse[i] = math.log(2.0) * (m + math.log2(den))
+    return O, lse
+
+
+def test_exactly_representable_probabilities_reproduce_exact_attention():
+    """Scores y = E_B - {0,1,2} inside every block give 2**x in {6,3,1.5}: all codes are exact,
+    so Direct-P must equal exact base-2 softmax attention (brute force) to rounding error, across
+    blocks whose exponents differ widely and tiles that raise the running reference."""
+    rng = np.random.default_rng(5)
+    R, N, d = 6, 256, 4
+    EB = rng.integers(-40, 40, size=(R, N // 32))
+    EB[:, 5] = 60                                   # a late block lifts the reference (rescale path)
+    y = np.repeat(EB, 32, axis=1) - rng.integers(0, 3, size=(R, N))
+    y[:, ::32] = np.repeat(EB, 1, axis=1)           # every block attains its maximum
+    V = rng.standard_normal((N, d))
+    O, lse, codes, EBo, mu = A.direct_p_rows(y.astype(np.float32), np.float32(1.0), V, tile=64)
+    Ob, lseb = _brute_softmax_attention(y, V)
+    assert np.array_equal(EBo, EB) and np.all(mu == 60)
+    assert set(np.unique(codes)) <= {3, 5, 7}
+    assert np.abs(O - Ob).max() < 1e-13 and np.abs(lse - lseb).max() < 1e-12
+
+
+def test_zero_block_flush_and_dominant_key():
+    """A key whose score exceeds every other by more than 126 octaves: same-block neighbours
+    round to code 0, later blocks are zero blocks (byte < 1 against the reference in force), and
+    earlier blocks, coded before the reference rose, are scaled by 2**-205: O is that key's V row."""
+    R, N, d = 3, 128, 8
+    y = np.full((R, N), -200.0, dtype=np.float32)
+    y[:, 70] = 5.0
+    V = np.random.default_rng(1).standard_normal((N, d))
+    O, lse, codes, _, mu = A.direct_p_rows(y, np.float32(1.0), V, tile=32)
+    assert np.all(mu == 5) and np.all(codes[:, 70] == 7)
+    assert np.count_nonzero(codes[:, 64:96]) == R and not codes[:, 96:].any()
+    assert np.all(codes[:, :64] == 7)
+    assert np.abs(O - V[70][None]).max() < 1e-15
+    assert np.allclose(lse, 5.0 * math.log(2.0))
+
+
+def test_rows_of_equal_scores_average_v_and_constant_v_is_reproduced():
+    w, (q, k, v), qd, kd, vd = _cfg1(N=128)
+    # constant V: numerator and denominator use the same codes, so O == that constant exactly-ish
+    ones = I.f32_to_bf16_bits(np.full((w.B, w.H, w.N, w.d), 1.0, dtype=np.float32))
+    O, _ = A.direct_p_forward(qd, kd, Qz.quantize_v(ones))
+    assert np.abs(O - 1.0).max() < 1e-14
+    # all keys identical: every score in a row is equal, every code is 6, O = mean of V^
+    kk = Qz.bf16_bits_to_f64(k).copy()
+    kk[:] = kk[:, :, :1, :]
+    kd_same = Qz.quantize_qk(I.f32_to_bf16_bits(kk.astype(np.float32)), "mx")
+    O, lse = A.direct_p_forward(qd, kd_same, vd)
+    Vhat = np.swapaxes(Qz.dequantize(vd), -1, -2)                 # [B,H,N,d]
+    want = Vhat.mean(axis=2).reshape(w.B * w.H, 1, w.d)
+    assert np.abs(O - want).max() < 1e-14
+    # its LSE is log(N) + z up to the E2M1 rounding of the single probability value (<= 25 %)
+    s32 = A.scores_fp32(qd, kd_same, 0, 0)
+    z = s32[:, 0].astype(np.float64) * float(A.score_constant(qd, kd_same, w.d)) * math.log(2.0)
+    assert np.abs(lse[0] - (z + math.log(w.N))).max() <= math.log(1.25) + 1e-9
+
+
+def test_represented_probabilities_define_output_and_stay_within_e2m1_error():
+    """O and LSE equal sum(p~ V^)/sum(p~) and log(sum p~) recomputed from the returned codes, and
+    every p~ is within the E2M1 rounding error of the exact 2**y: |p~ - p| <= max(p/5, alpha_B/24)."""
+    w, _, qd, kd, vd = _cfg1(N=256)
+    c32 = A.score_constant(qd, kd, w.d)
+    s32 = A.scores_fp32(qd, kd, 0, 1)
+    Vhat = np.ascontiguousarray(Qz.dequantize(vd)[0, 1].T)
+    O, lse, codes, EB, mu = A.direct_p_rows(s32, c32, Vhat)
+    alpha = np.repeat(np.ldexp(1.0, EB), 32, axis=1)
+    pt = alpha * F.E2M1_VALUES[codes] / 6.0
+    assert np.abs(O - (pt @ Vhat) / pt.sum(axis=1, keepdims=True)).max() < 1e-13
+    assert np.abs(lse - np.log(pt.sum(axis=1))).max() < 1e-12
+    p = np.exp2(s32.astype(np.float64) * float(c32))
+    assert np.all(np.abs(pt - p) <= np.maximum(p / 5.0, alpha / 24.0) * (1 + 1e-6))
+    assert np.all(pt.max(axis=1) > 0)
+
+
+def test_lossless_inputs_against_bruteforce_exact_attention():
+    """Q, K, V drawn from {0, +-1/4, +-1/2, +-1} with a +-1 in every block are represented
+    without error, so the only approximation left is the E2M1 rounding of P: the output must stay
+    inside the band that rounding allows around triple-loop exact attention."""
+    rng = np.random.default_rng(11)
+    B, H, N, d = 1, 1, 64, 64
+    vals = np.array([0, 0.25, -0.25, 0.5, -0.5, 1, -1])
+    def draw():
+        x = rng.choice(vals, size=(B, H, N, d))
+        x[..., ::32] = 1.0
+        x[:, :, ::32, :] = -1.0
+        return x
+    q, k, v = draw(), draw(), draw()
+    bits = [I.f32_to_bf16_bits(a.astype(np.float32)) for a in (q, k, v)]
+    qd, kd, vd = Qz.quantize_qk(bits[0], "mx"), Qz.quantize_qk(bits[1], "mx"), Qz.quantize_v(bits[2])
+    assert np.array_equal(Qz.dequantize(qd), q) and np.array_equal(Qz.dequantize(kd), k)
+    assert np.array_equal(np.swapaxes(Qz.dequantize(vd), -1, -2), v)
+    O, lse = A.direct_p_forward(qd, kd, vd, tile=32)
+    # brute force exact attention
+    Oe = np.zeros((N, d))
+    for i in range(N):
+        z = [sum(q[0, 0, i, c] * k[0, 0, j, c] for c in range(d)) / math.sqrt(d) for j in range(N)]
+        m = max(z)
+        p = [math.exp(t - m) for t in z]
+        s = sum(p)
+        for j in range(N):
+            Oe[i] += p[j] / s * v[0, 0, j]
+    Oref, lref = A.exact_attention(q[0, 0], k[0, 0], v[0, 0])
+    assert np.abs(Oref - Oe).max() < 1e-13
+    rel = np.linalg.norm(O[0] - Oe) / np.linalg.norm(Oe)
+    cos = (O[0] * Oe).sum() / np.linalg.norm(O[0]) / np.linalg.norm(Oe)
+    assert rel < 0.2 and cos > 0.98
+    assert np.abs(lse[0] - lref).max() < math.log(1.25)      # each p~ is within 20-25 % of p
+
+
+def test_accuracy_band_on_gaussian_inputs():
+    """cos / rel-L2 against unquantised fp64 attention sit where the paper's all-MXFP4 rows do or
+    better (Table "all-formats": cos 0.925-0.941, rel-L2 0.34-0.38 with its affine classifier)."""
+    w, (q, k, v), qd, kd, vd = _cfg1()
+    O, _ = A.direct_p_forward(qd, kd, vd)
+    x = [Qz.bf16_bits_to_f64(a) for a in (q, k, v)]
+    for h in range(w.H):
+        Oe, _ = A.exact_attention(x[0][0, h], x[1][0, h], x[2][0, h])
+        cos = (Oe * O[h]).sum() / np.linalg.norm(Oe) / np.linalg.norm(O[h])
+        rel = np.linalg.norm(Oe - O[h]) / np.linalg.norm(Oe)
+        assert 0.94 < cos < 0.99 and 0.2 < rel < 0.34
+
+
+def test_bf16_round():
+    got = A.bf16_round(np.array([1.0, 1.00390625, 1.01171875, -3.14159, 0.0]))
+    assert list(got) == [1.0, 1.0, 1.015625, -3.140625, 0.0]
