@@ -1,0 +1,150 @@
+/*
+ * fp4attn — full-FP4 attention forward with Direct-P for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Unless an argument says otherwise every pointer is a DEVICE pointer owned by the
+ * caller; the library allocates nothing, keeps no state between calls except cached kernel
+ * attributes and tensor maps' driver entry point, enqueues its work on the caller's stream and
+ * returns without synchronising.  Errors that the host can detect come back as a non-zero
+ * status and nothing is launched; nothing throws, prints or exits.
+ *
+ * Tensor layouts
+ *   x, O          bf16  [B, H, N, d] contiguous
+ *   packed Q, K   u8    [B, H, N, d/2]   element 2k in bits 0-3 of byte k, 2k+1 in bits 4-7;
+ *                                          a nibble is an E2M1 code  s e1 e0 m
+ *   packed V      u8    [B, H, d, N/2]   V is stored TRANSPOSED (key index contiguous) because
+ *                                          4-bit tensor-core operands must be contraction-major
+ *   scale bytes   u8    per (b, h) a grid of 512-byte atoms.  With r the row (query/key index for
+ *                       Q and K, head-dim index for V) and c the scale column (d/32 or d/16 for
+ *                       Q and K, N/32 for V), atom (r/128, c/4) starts at
+ *                       ((r/128) * ceil(C/4) + c/4) * 512 and holds the byte at
+ *                       (r%32)*16 + ((r%128)/32)*4 + c%4.  Rows pad to 128, columns to 4, padding
+ *                       bytes are written as zero.  This is the order in which the block-scaled
+ *                       tcgen05 instruction reads 128 rows x 4 scale factors.
+ *   LSE           f32   [B, H, N], natural logarithm
+ *
+ * Supported shapes: d in {64, 128}; N a multiple of 128, 128 <= N; B, H >= 1; pointers 16-byte
+ * aligned (packed operands and scale buffers 128-byte aligned).  Compute capability 10.0 only.
+ */
+#ifndef FP4ATTN_H_
+#define FP4ATTN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* fp4attn_stream_t;   /* a cudaStream_t; NULL = legacy default stream */
+
+enum {
+  FP4ATTN_OK = 0,
+  FP4ATTN_ERR_INVALID_ARG = 1,        /* NULL pointer, non-positive size, unknown enum        */
+  FP4ATTN_ERR_UNSUPPORTED_SHAPE = 2,  /* d, N outside the supported set                        */
+  FP4ATTN_ERR_UNSUPPORTED_ARCH = 3,   /* current device is not compute capability 10.0        */
+  FP4ATTN_ERR_ALIGNMENT = 4,          /* a pointer violates the stated alignment               */
+  FP4ATTN_ERR_WORKSPACE = 5,          /* workspace missing or too small                        */
+  FP4ATTN_ERR_CUDA = 6,               /* a CUDA runtime / driver call failed                   */
+  FP4ATTN_ERR_TIMEOUT = 7             /* written to *device_status by a kernel whose bounded
+                                         wait ran out; never returned synchronously            */
+};
+
+enum { FP4ATTN_FMT_MXFP4 = 0, FP4ATTN_FMT_NVFP4 = 1 };
+enum { FP4ATTN_ROLE_Q = 0, FP4ATTN_ROLE_K = 1, FP4ATTN_ROLE_V = 2 };
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* fp4attn_status_string(int status);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int fp4attn_version(void);
+
+/* Bytes of the packed E2M1 buffer of one operand: B*H*N*d/2.  0 on invalid arguments. */
+size_t fp4attn_packed_bytes(int B, int H, int N, int d);
+
+/* Bytes of the scale buffer of one operand, padded to whole 128x4 atoms (layout above).
+ * fmt/role decide the scale grid: Q, K: rows N, columns d/32 (MXFP4) or d/16 (NVFP4);
+ * V (MXFP4 only): rows d, columns N/32.  0 on invalid arguments. */
+size_t fp4attn_scale_bytes(int fmt, int role, int B, int H, int N, int d);
+
+/* Bytes of scratch fp4attn_quantize needs: 0 for MXFP4; for NVFP4 room for the per-block
+ * partial maxima of the tensor-wide amax pass. */
+size_t fp4attn_quantize_workspace_bytes(int fmt, int role, int B, int H, int N, int d);
+
+/*
+ * Operand quantizer (Section "Problem 2", Table "fp4-formats", Eqs. "nv-scale", "mx-scale").
+ *
+ * MXFP4: every block of 32 values (along d for Q and K; along the key index for V) with maximum
+ *   magnitude a stores the E8M0 byte u = clamp(127 + ceil(log2 a), 1, 254) (u = 0 and all codes 0
+ *   for an all-zero block) and the codes q = Q_E2M1(6 v / 2^(u-127)), round to nearest, ties to
+ *   even; a value is reconstructed as 2^(u-127) * q / 6 (amplitude convention).
+ * NVFP4 (Q, K only): every block of 16 values stores the E4M3 byte of
+ *   t = fl32(fl32(a_B * G) / 6) (round to nearest even, saturate at 448) and the codes
+ *   q = Q_E2M1(fl32(|v| * fl32(G / S_B))) with the sign of v, S_B the decoded byte; S_B = 0
+ *   zeroes the block.  G = fl32(2688 / max|x|) over the whole tensor (1 if it is all zero) is
+ *   written to *tensor_scale_out (device); reconstruction is S_B * q / G.
+ *
+ * x_bf16 [B,H,N,d]; packed_out / scales_out sized by the queries above; tensor_scale_out is
+ * required for NVFP4 and ignored (may be NULL) for MXFP4; workspace may be NULL when the size
+ * query returns 0.  Outputs are fully overwritten (padding included).
+ */
+int fp4attn_quantize(const void* x_bf16, int fmt, int role, int B, int H, int N, int d,
+                     void* packed_out, void* scales_out, float* tensor_scale_out,
+                     void* workspace, size_t workspace_bytes, fp4attn_stream_t stream);
+
+typedef struct {
+  const void *q, *k, *v;            /* packed E2M1 (V transposed)                           */
+  const void *q_sf, *k_sf, *v_sf;   /* scale atoms                                           */
+  const float *q_G, *k_G;           /* device fp32 encode factors; NVFP4 only, else NULL     */
+  int qk_fmt;                       /* format of Q and K; P and V are always MXFP4           */
+  float softmax_scale;              /* 0 selects 1/sqrt(d)                                   */
+} fp4attn_operands;
+
+/*
+ * Noncausal attention forward with Direct-P (Sections "Fix 1" and "Fix 2", Algorithm
+ * "direct-p-pack", Eqs. "online-recurrence", "represented-probability", "ideal-code-path",
+ * "represented-contributions", "represented-output").
+ *
+ * S = Q K^T runs as a block-scaled FP4 tensor-core product with fp32 accumulation.  With
+ * y = fl32(S * c), c = fl32(fl32(log2(e) * softmax_scale) / k), k = 36 for MXFP4 Q,K (two
+ * amplitude-convention operands) or fl32(G_q * G_k) for NVFP4, every block of 32 consecutive keys
+ * of a query row takes the integer exponent E_B = ceil(max_j y_j), each score maps straight to
+ * the E2M1 code q_j = Q_E2M1(2^(y_j - E_B + log2 6)), and the block's E8M0 byte is
+ * E_B - mu + 127 for an integer row reference mu that never exceeds the running maximum by
+ * construction (blocks whose byte would drop below 1 are zero blocks).  P V runs as a second
+ * block-scaled FP4 product; the output is normalised by the sum of the same rounded values:
+ *   O = sum_j p~_j V^_j / sum_j p~_j,   p~_j = 2^(E_B) q_j / 6,   LSE = ln sum_j p~_j.
+ *
+ * O_bf16 [B,H,N,d]; LSE [B,H,N] (may be NULL); device_status (may be NULL) receives
+ * FP4ATTN_ERR_TIMEOUT if a bounded in-kernel wait ran out, and is otherwise left untouched, so
+ * the caller clears it beforehand.
+ */
+int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int d,
+                void* O_bf16, float* LSE, int* device_status, fp4attn_stream_t stream);
+
+/* Bytes of device scratch fp4attn_attention_host needs for a problem of this size. */
+size_t fp4attn_attention_host_workspace_bytes(int qk_fmt, int B, int H, int N, int d);
+
+/*
+ * Whole path from HOST buffers: copies bf16 Q, K, V [B,H,N,d] from (preferably pinned) host
+ * memory into the caller's device workspace, quantizes them (fp4attn_quantize x3), runs
+ * fp4attn_fwd and copies O (bf16) and, if LSE_host is not NULL, LSE back to host memory, all on
+ * `stream`; returns after enqueuing.  q_host/k_host/v_host/O_host/LSE_host are HOST pointers,
+ * workspace is a DEVICE pointer of at least fp4attn_attention_host_workspace_bytes() bytes,
+ * 256-byte aligned.  The caller synchronises the stream before reading O_host.
+ */
+int fp4attn_attention_host(const void* q_host, const void* k_host, const void* v_host,
+                           int qk_fmt, float softmax_scale, int B, int H, int N, int d,
+                           void* O_host, float* LSE_host,
+                           void* workspace, size_t workspace_bytes, fp4attn_stream_t stream);
+
+/*
+ * Dense FP4 tensor-core ceiling of the current device, measured: every SM issues `iters`
+ * back-to-back block-scaled 128x128x64 E2M1 products on shared-memory-resident tiles.
+ * Enqueues one kernel; *cycles_out (device, 64-bit) receives the slowest SM's clock count.
+ * Used by the benchmark to state the roofline denominator; not part of the attention path.
+ */
+int fp4attn_mma_peak_probe(int iters, unsigned long long* cycles_out, fp4attn_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP4ATTN_H_ */

@@ -1,0 +1,158 @@
+"""Thin ctypes binding over libfp4attn.so: argument marshalling only.
+
+PyTorch appears here for device memory and streams; every step of the path runs inside the
+library's CUDA kernels.  Importing this module fails loudly when the library is missing.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import torch
+
+FMT_MXFP4, FMT_NVFP4 = 0, 1
+ROLE_Q, ROLE_K, ROLE_V = 0, 1, 2
+ERR_TIMEOUT = 7
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfp4attn.so")
+
+EXPORTS = [
+    "fp4attn_status_string", "fp4attn_version", "fp4attn_packed_bytes", "fp4attn_scale_bytes",
+    "fp4attn_quantize_workspace_bytes", "fp4attn_quantize", "fp4attn_fwd",
+    "fp4attn_attention_host_workspace_bytes", "fp4attn_attention_host", "fp4attn_mma_peak_probe",
+]
+
+
+class Fp4AttnError(RuntimeError):
+    pass
+
+
+class _Operands(ctypes.Structure):
+    _fields_ = [("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+                ("q_sf", ctypes.c_void_p), ("k_sf", ctypes.c_void_p), ("v_sf", ctypes.c_void_p),
+                ("q_G", ctypes.c_void_p), ("k_G", ctypes.c_void_p),
+                ("qk_fmt", ctypes.c_int), ("softmax_scale", ctypes.c_float)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise Fp4AttnError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_04105_b200.build` "
+                           "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    i, sz, vp = ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p
+    lib.fp4attn_status_string.restype = ctypes.c_char_p
+    lib.fp4attn_status_string.argtypes = [i]
+    lib.fp4attn_version.restype = i
+    lib.fp4attn_packed_bytes.restype = sz
+    lib.fp4attn_packed_bytes.argtypes = [i, i, i, i]
+    lib.fp4attn_scale_bytes.restype = sz
+    lib.fp4attn_scale_bytes.argtypes = [i, i, i, i, i, i]
+    lib.fp4attn_quantize_workspace_bytes.restype = sz
+    lib.fp4attn_quantize_workspace_bytes.argtypes = [i, i, i, i, i, i]
+    lib.fp4attn_quantize.restype = i
+    lib.fp4attn_quantize.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, sz, vp]
+    lib.fp4attn_fwd.restype = i
+    lib.fp4attn_fwd.argtypes = [ctypes.POINTER(_Operands), i, i, i, i, vp, vp, vp, vp]
+    lib.fp4attn_attention_host_workspace_bytes.restype = sz
+    lib.fp4attn_attention_host_workspace_bytes.argtypes = [i, i, i, i, i]
+    lib.fp4attn_attention_host.restype = i
+    lib.fp4attn_attention_host.argtypes = [vp, vp, vp, i, ctypes.c_float, i, i, i, i, vp, vp, vp, sz, vp]
+    lib.fp4attn_mma_peak_probe.restype = i
+    lib.fp4attn_mma_peak_probe.argtypes = [i, vp, vp]
+    return lib
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = _load()
+    return _lib
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise Fp4AttnError(f"{what}: {lib().fp4attn_status_string(rc).decode()} (status {rc})")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+@dataclass
+class QuantizedOperand:
+    packed: torch.Tensor              # uint8
+    scales: torch.Tensor              # uint8, 128x4 atoms
+    G: Optional[torch.Tensor]         # fp32 [1] (NVFP4) or None
+    fmt: int
+    role: int
+    shape: Tuple[int, int, int, int]  # (B, H, N, d) of the source tensor
+
+
+def fp4attn_quantize(x: torch.Tensor, fmt: int, role: int, workspace: Optional[torch.Tensor] = None) -> QuantizedOperand:
+    """x: CUDA bf16 [B,H,N,d] contiguous -> packed E2M1 + scale factors (see include/fp4attn.h)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 4
+    B, H, N, d = x.shape
+    L = lib()
+    nb = L.fp4attn_packed_bytes(B, H, N, d)
+    ns = L.fp4attn_scale_bytes(fmt, role, B, H, N, d)
+    if nb == 0 or ns == 0:
+        _check(L.fp4attn_quantize(x.data_ptr(), fmt, role, B, H, N, d, 1, 1, None, None, 0, _stream()), "fp4attn_quantize")
+        raise Fp4AttnError("fp4attn_quantize: unsupported arguments")
+    packed = torch.empty(nb, dtype=torch.uint8, device=x.device)
+    scales = torch.empty(ns, dtype=torch.uint8, device=x.device)
+    G = torch.empty(1, dtype=torch.float32, device=x.device) if fmt == FMT_NVFP4 else None
+    nw = L.fp4attn_quantize_workspace_bytes(fmt, role, B, H, N, d)
+    if nw and workspace is None:
+        workspace = torch.empty(nw, dtype=torch.uint8, device=x.device)
+    _check(L.fp4attn_quantize(x.data_ptr(), fmt, role, B, H, N, d, packed.data_ptr(), scales.data_ptr(),
+                              _ptr(G), _ptr(workspace), 0 if workspace is None else workspace.numel(), _stream()),
+           "fp4attn_quantize")
+    return QuantizedOperand(packed, scales, G, fmt, role, (B, H, N, d))
+
+
+def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, softmax_scale: float = 0.0,
+                out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                status: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Direct-P attention forward on quantized operands -> (O bf16 [B,H,N,d], LSE fp32 [B,H,N])."""
+    B, H, N, d = q.shape
+    assert k.shape == q.shape and v.shape == q.shape and q.fmt == k.fmt and v.fmt == FMT_MXFP4
+    dev = q.packed.device
+    if out is None:
+        out = torch.empty((B, H, N, d), dtype=torch.bfloat16, device=dev)
+    if lse is None:
+        lse = torch.empty((B, H, N), dtype=torch.float32, device=dev)
+    ops = _Operands(q.packed.data_ptr(), k.packed.data_ptr(), v.packed.data_ptr(),
+                    q.scales.data_ptr(), k.scales.data_ptr(), v.scales.data_ptr(),
+                    _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale))
+    _check(lib().fp4attn_fwd(ctypes.byref(ops), B, H, N, d, out.data_ptr(), lse.data_ptr(), _ptr(status), _stream()),
+           "fp4attn_fwd")
+    return out, lse
+
+
+def fp4attn_attention_host_workspace_bytes(qk_fmt: int, B: int, H: int, N: int, d: int) -> int:
+    return lib().fp4attn_attention_host_workspace_bytes(qk_fmt, B, H, N, d)
+
+
+def fp4attn_attention_host(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, qk_fmt: int, out: torch.Tensor,
+                           lse: Optional[torch.Tensor], workspace: torch.Tensor, softmax_scale: float = 0.0) -> None:
+    """Host (pinned) bf16 Q, K, V -> host O (and LSE); copies, quantizers and attention are enqueued
+    on the current stream.  `workspace` is a CUDA uint8 tensor of the queried size."""
+    assert not q.is_cuda and not out.is_cuda and workspace.is_cuda
+    B, H, N, d = q.shape
+    _check(lib().fp4attn_attention_host(q.data_ptr(), k.data_ptr(), v.data_ptr(), qk_fmt, float(softmax_scale),
+                                        B, H, N, d, out.data_ptr(), _ptr(lse), workspace.data_ptr(),
+                                        workspace.numel(), _stream()), "fp4attn_attention_host")
+
+
+def fp4attn_mma_peak_probe(iters: int, cycles_out: torch.Tensor) -> None:
+    _check(lib().fp4attn_mma_peak_probe(iters, cycles_out.data_ptr(), _stream()), "fp4attn_mma_peak_probe")

@@ -1,0 +1,281 @@
+// Operand quantizers: bf16 -> packed E2M1 + scale bytes in the 128x4 atom order.
+// HBM-bound: 128-bit loads, block amax by lane shuffles, 32-bit / 128-bit stores.
+#include "common.cuh"
+
+namespace fp4attn {
+
+constexpr int kThreads = 256;
+constexpr int kGroupsPerThread = 4;          // 16-byte loads in flight per thread
+constexpr int kGroupsPerCta = kThreads * kGroupsPerThread;
+constexpr int kMaxPartials = 1024;           // NVFP4 amax pass: one partial maximum per block
+
+__device__ __forceinline__ float amax8(const float* v) {
+  float a = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(v[i]));
+  return a;
+}
+
+// byte offset of the scale of (row r, scale column c) inside one (b,h) scale grid with CT column atoms
+__device__ __forceinline__ size_t sf_offset(int r, int c, int CT) {
+  return (size_t)((r >> 7) * CT + (c >> 2)) * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4 + (c & 3);
+}
+
+// ---------------------------------------------------------------- MXFP4, blocks along d (Q, K)
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+quant_mx_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
+                     uint8_t* __restrict__ sf, int N) {
+  constexpr int GPR = D / 8;                       // 8-element groups per row
+  const size_t base = (size_t)blockIdx.x * kGroupsPerCta + threadIdx.x;
+  uint4 raw[kGroupsPerThread];
+#pragma unroll
+  for (int k = 0; k < kGroupsPerThread; ++k) raw[k] = __ldg(x + base + (size_t)k * kThreads);
+#pragma unroll
+  for (int k = 0; k < kGroupsPerThread; ++k) {
+    const size_t g = base + (size_t)k * kThreads;
+    float v[8];
+    bf16x8_to_f32(raw[k], v);
+    float a = amax8(v);
+    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
+    const uint32_t u = mx_scale_byte(a);
+    const float inv = mx_inv_amplitude(u);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = (v[i] * inv) * 6.0f;      // exact in fp32
+    packed[g] = cvt_e2m1x8(v);
+    // gather the row's D/32 scale bytes into one word, written by the row's first lane
+    const int lane = threadIdx.x & 31;
+    const int seg = (int)(g % GPR);
+    const int row_lane0 = lane - seg;
+    uint32_t word = 0;
+#pragma unroll
+    for (int b = 0; b < D / 32; ++b) word |= __shfl_sync(0xffffffffu, u, row_lane0 + 4 * b) << (8 * b);
+    if (seg == 0) {
+      const size_t row = g / GPR;
+      const size_t bh = row / N;
+      const int r = (int)(row % N);
+      uint8_t* p = sf + bh * (size_t)(N / 128) * 512 + sf_offset(r, 0, 1);
+      *reinterpret_cast<uint32_t*>(p) = word;                    // bytes beyond D/32 are zero padding
+    }
+  }
+}
+
+// ---------------------------------------------------------------- MXFP4, blocks along keys (V), transposed out
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+quant_mx_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ packed, uint8_t* __restrict__ sf, int N) {
+  __shared__ __align__(16) __nv_bfloat16 tile[128 * D];
+  __shared__ uint8_t sfb[128 * 4];
+  const int kt = blockIdx.x;                       // 128-key tile
+  const size_t bh = blockIdx.y;
+  const uint4* src = x + (bh * N + (size_t)kt * 128) * (D / 8);
+  constexpr int LOADS = 128 * D / 8 / kThreads;
+  uint4 raw[LOADS];
+#pragma unroll
+  for (int k = 0; k < LOADS; ++k) raw[k] = __ldg(src + threadIdx.x + k * kThreads);
+#pragma unroll
+  for (int k = 0; k < LOADS; ++k) reinterpret_cast<uint4*>(tile)[threadIdx.x + k * kThreads] = raw[k];
+  if (threadIdx.x < 128) reinterpret_cast<uint32_t*>(sfb)[threadIdx.x] = 0;
+  __syncthreads();
+  const int c = threadIdx.x % D;
+  constexpr int KB_PER_THREAD = 4 * D / kThreads;  // 2 (D=128) or 1 (D=64)
+#pragma unroll
+  for (int s = 0; s < KB_PER_THREAD; ++s) {
+    const int kb = (threadIdx.x / D) * KB_PER_THREAD + s;
+    float v[32];
+    float a = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      v[i] = __bfloat162float(tile[(kb * 32 + i) * D + c]);
+      a = fmaxf(a, fabsf(v[i]));
+    }
+    const uint32_t u = mx_scale_byte(a);
+    const float inv = mx_inv_amplitude(u);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = (v[i] * inv) * 6.0f;
+    uint4 out;
+    out.x = cvt_e2m1x8(v);
+    out.y = cvt_e2m1x8(v + 8);
+    out.z = cvt_e2m1x8(v + 16);
+    out.w = cvt_e2m1x8(v + 24);
+    packed[((bh * D + c) * (size_t)(N / 2) + (size_t)kt * 64 + kb * 16) / 16] = out;
+    sfb[c * 4 + kb] = (uint8_t)u;
+  }
+  __syncthreads();
+  if (threadIdx.x < 128) {
+    const int r = threadIdx.x;                     // head-dim row; rows >= D are zero padding
+    uint8_t* p = sf + (bh * (size_t)(N / 128) + kt) * 512 + (r & 31) * 16 + (r >> 5) * 4;
+    *reinterpret_cast<uint32_t*>(p) = reinterpret_cast<const uint32_t*>(sfb)[r];
+  }
+}
+
+// ---------------------------------------------------------------- NVFP4 pass 1: tensor-wide amax partials
+__global__ void __launch_bounds__(kThreads)
+amax_partials_kernel(const uint4* __restrict__ x, size_t n_groups, float* __restrict__ partials) {
+  float a = 0.f;
+  for (size_t g = (size_t)blockIdx.x * kThreads + threadIdx.x; g < n_groups; g += (size_t)gridDim.x * kThreads) {
+    float v[8];
+    bf16x8_to_f32(__ldg(x + g), v);
+    a = fmaxf(a, amax8(v));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+  __shared__ float wmax[kThreads / 32];
+  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = a;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < kThreads / 32; ++i) a = fmaxf(a, wmax[i]);
+    partials[blockIdx.x] = a;
+  }
+}
+
+__device__ __forceinline__ uint32_t cvt_e4m3_byte(float t) {     // RNE, saturating at 448
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.f), "f"(t));
+  return r & 0xFFu;
+}
+__device__ __forceinline__ float e4m3_byte_to_f32(uint32_t b) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)b));
+  return __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
+}
+
+// ---------------------------------------------------------------- NVFP4 pass 2, blocks of 16 along d (Q, K)
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+quant_nv_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed, uint8_t* __restrict__ sf,
+                     const float* __restrict__ partials, int n_partials, float* __restrict__ G_out, int N) {
+  constexpr int GPR = D / 8;
+  constexpr int CT = (D / 16 + 3) / 4;
+  __shared__ float s_G;
+  {
+    float a = 0.f;
+    for (int i = threadIdx.x; i < n_partials; i += kThreads) a = fmaxf(a, partials[i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+    __shared__ float wmax[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = a;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int i = 1; i < kThreads / 32; ++i) a = fmaxf(a, wmax[i]);
+      const float G = (a == 0.f) ? 1.0f : __fdiv_rn(2688.0f, a);
+      s_G = G;
+      if (blockIdx.x == 0) *G_out = G;
+    }
+    __syncthreads();
+  }
+  const float G = s_G;
+  const size_t base = (size_t)blockIdx.x * kGroupsPerCta + threadIdx.x;
+  uint4 raw[kGroupsPerThread];
+#pragma unroll
+  for (int k = 0; k < kGroupsPerThread; ++k) raw[k] = __ldg(x + base + (size_t)k * kThreads);
+#pragma unroll
+  for (int k = 0; k < kGroupsPerThread; ++k) {
+    const size_t g = base + (size_t)k * kThreads;
+    float v[8];
+    bf16x8_to_f32(raw[k], v);
+    float a = amax8(v);
+    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+    const float t = __fdiv_rn(__fmul_rn(a, G), 6.0f);
+    const uint32_t sb = cvt_e4m3_byte(t);
+    const float S = e4m3_byte_to_f32(sb);
+    const float r = (S > 0.f) ? __fdiv_rn(G, S) : 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __fmul_rn(v[i], r);       // sign rides along; 0*r = 0 for zero blocks
+    packed[g] = cvt_e2m1x8(v);
+    const int lane = threadIdx.x & 31;
+    const int seg = (int)(g % GPR);
+    const int wbase = lane - (seg & 7);                          // first lane of this 4-scale word
+    uint32_t word = 0;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) word |= __shfl_sync(0xffffffffu, sb, wbase + 2 * b) << (8 * b);
+    if ((seg & 7) == 0) {
+      const size_t row = g / GPR;
+      const size_t bh = row / N;
+      const int rr = (int)(row % N);
+      uint8_t* p = sf + bh * (size_t)(N / 128) * CT * 512 + sf_offset(rr, (seg / 8) * 4, CT);
+      *reinterpret_cast<uint32_t*>(p) = word;
+    }
+  }
+}
+
+}  // namespace fp4attn
+
+using namespace fp4attn;
+
+extern "C" size_t fp4attn_packed_bytes(int B, int H, int N, int d) {
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return 0;
+  return (size_t)B * H * N * d / 2;
+}
+
+static bool shape_ok(int B, int H, int N, int d) {
+  return B > 0 && H > 0 && (d == 64 || d == 128) && N >= 128 && N % 128 == 0;
+}
+
+extern "C" size_t fp4attn_scale_bytes(int fmt, int role, int B, int H, int N, int d) {
+  if (!shape_ok(B, H, N, d)) return 0;
+  if (role == FP4ATTN_ROLE_V) {
+    if (fmt != FP4ATTN_FMT_MXFP4) return 0;
+    return (size_t)B * H * ((d + 127) / 128) * (N / 128) * 512;          // rows d, columns N/32
+  }
+  if (role != FP4ATTN_ROLE_Q && role != FP4ATTN_ROLE_K) return 0;
+  if (fmt != FP4ATTN_FMT_MXFP4 && fmt != FP4ATTN_FMT_NVFP4) return 0;
+  const int C = d / (fmt == FP4ATTN_FMT_MXFP4 ? 32 : 16);
+  return (size_t)B * H * (N / 128) * ((C + 3) / 4) * 512;
+}
+
+extern "C" size_t fp4attn_quantize_workspace_bytes(int fmt, int role, int B, int H, int N, int d) {
+  (void)role; (void)B; (void)H; (void)N; (void)d;
+  return fmt == FP4ATTN_FMT_NVFP4 ? (size_t)kMaxPartials * sizeof(float) : 0;
+}
+
+namespace fp4attn {
+// Shared by fp4attn_quantize and the variants that bring their own scratch.
+int launch_quantize(const void* x, int fmt, int role, int B, int H, int N, int d, void* packed, void* scales,
+                    float* G_out, float* partials, cudaStream_t st) {
+  const size_t n_groups = (size_t)B * H * N * d / 8;
+  const unsigned grid = (unsigned)(n_groups / kGroupsPerCta);
+  const uint4* xs = reinterpret_cast<const uint4*>(x);
+  if (fmt == FP4ATTN_FMT_MXFP4 && role != FP4ATTN_ROLE_V) {
+    if (d == 128) quant_mx_rows_kernel<128><<<grid, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
+    else          quant_mx_rows_kernel<64><<<grid, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
+  } else if (fmt == FP4ATTN_FMT_MXFP4) {
+    dim3 g2(N / 128, B * H);
+    if (d == 128) quant_mx_v_kernel<128><<<g2, kThreads, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
+    else          quant_mx_v_kernel<64><<<g2, kThreads, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
+  } else {
+    const int n_partials = (int)(grid < (unsigned)kMaxPartials ? grid : kMaxPartials);
+    amax_partials_kernel<<<n_partials, kThreads, 0, st>>>(xs, n_groups, partials);
+    if (d == 128) quant_nv_rows_kernel<128><<<grid, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N);
+    else          quant_nv_rows_kernel<64><<<grid, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N);
+  }
+  return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
+}
+
+int validate_quantize(const void* x, int fmt, int role, int B, int H, int N, int d, const void* packed,
+                      const void* scales, const float* G_out) {
+  if (!x || !packed || !scales) return FP4ATTN_ERR_INVALID_ARG;
+  if (fmt != FP4ATTN_FMT_MXFP4 && fmt != FP4ATTN_FMT_NVFP4) return FP4ATTN_ERR_INVALID_ARG;
+  if (role != FP4ATTN_ROLE_Q && role != FP4ATTN_ROLE_K && role != FP4ATTN_ROLE_V) return FP4ATTN_ERR_INVALID_ARG;
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return FP4ATTN_ERR_INVALID_ARG;
+  if (!shape_ok(B, H, N, d)) return FP4ATTN_ERR_UNSUPPORTED_SHAPE;
+  if (fmt == FP4ATTN_FMT_NVFP4 && role == FP4ATTN_ROLE_V) return FP4ATTN_ERR_INVALID_ARG;   // V is always MXFP4
+  if (fmt == FP4ATTN_FMT_NVFP4 && !G_out) return FP4ATTN_ERR_INVALID_ARG;
+  if (((uintptr_t)x | (uintptr_t)packed | (uintptr_t)scales) & 15) return FP4ATTN_ERR_ALIGNMENT;
+  return FP4ATTN_OK;
+}
+}  // namespace fp4attn
+
+extern "C" int fp4attn_quantize(const void* x, int fmt, int role, int B, int H, int N, int d, void* packed,
+                                void* scales, float* G_out, void* workspace, size_t workspace_bytes,
+                                fp4attn_stream_t stream) {
+  int rc = validate_quantize(x, fmt, role, B, H, N, d, packed, scales, G_out);
+  if (rc != FP4ATTN_OK) return rc;
+  const size_t need = fp4attn_quantize_workspace_bytes(fmt, role, B, H, N, d);
+  if (need && (!workspace || workspace_bytes < need)) return FP4ATTN_ERR_WORKSPACE;
+  if (need && ((uintptr_t)workspace & 15)) return FP4ATTN_ERR_ALIGNMENT;
+  rc = check_device_sm100();
+  if (rc != FP4ATTN_OK) return rc;
+  return launch_quantize(x, fmt, role, B, H, N, d, packed, scales, G_out, (float*)workspace, (cudaStream_t)stream);
+}

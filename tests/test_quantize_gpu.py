@@ -1,0 +1,80 @@
+"""Kernel (a): the CUDA quantizer must reproduce the oracle's bytes exactly (sign of zero aside)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import quantize as Qz
+from paper_2609_04105_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _check_operand(got, want, role):
+    packed = got.packed.cpu().numpy()
+    want_packed = Qz.pack_nibbles(want["nib"]).reshape(-1)
+    assert np.array_equal(Qz.strip_negative_zero(packed), Qz.strip_negative_zero(want_packed)), "codes differ"
+    want_sf = Qz.swizzle_scales(want["sf"]).reshape(-1)
+    assert np.array_equal(got.scales.cpu().numpy(), want_sf), "scale bytes differ"
+    if want["G"] is not None:
+        assert got.G.cpu().numpy()[0] == want["G"]
+
+
+CASES = [
+    ("cfg1", dict()),
+    ("cfg1", dict(d=64, N=384, H=3)),
+    ("cfg3", dict(B=2, H=2, N=512)),
+    ("cfg3", dict(B=1, H=2, N=256, d=128)),
+    ("cfg4", dict(H=2, N=640)),
+]
+
+
+@pytest.mark.parametrize("name,kw", CASES)
+def test_quantizer_bytes_match_oracle(name, kw):
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    fmt = "mx" if w.qk_fmt == I.FMT_MXFP4 else "nv"
+    for bits, role in ((q, Bd.ROLE_Q), (k, Bd.ROLE_K)):
+        got = Bd.fp4attn_quantize(_dev(bits), w.qk_fmt, role)
+        _check_operand(got, Qz.quantize_qk(bits, fmt), role)
+    got = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    _check_operand(got, Qz.quantize_v(v), Bd.ROLE_V)
+
+
+def test_quantizer_edge_values():
+    """Zero blocks, huge and tiny magnitudes, exact ties, negative zero."""
+    from paper_2609_04105_b200 import binding as Bd
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((1, 1, 128, 128)).astype(np.float32)
+    x[0, 0, 0, :32] = 0.0
+    x[0, 0, 1, :32] = -0.0
+    x[0, 0, 2, :] *= 1e30
+    x[0, 0, 3, :] *= 1e-30
+    x[0, 0, 4, :32] = np.array([1, 0.75, 0.625, 0.4375, 0.125, 1 / 24, -0.875, 0.5] * 4)   # ties of 6v
+    x[0, 0, 5, 0] = 3.0e38
+    x[0, 0, 6, :] = 2.0 ** -130
+    bits = I.f32_to_bf16_bits(x)
+    for fmt, name in ((Bd.FMT_MXFP4, "mx"), (Bd.FMT_NVFP4, "nv")):
+        got = Bd.fp4attn_quantize(_dev(bits), fmt, Bd.ROLE_Q)
+        _check_operand(got, Qz.quantize_qk(bits, name), Bd.ROLE_Q)
+    got = Bd.fp4attn_quantize(_dev(bits), Bd.FMT_MXFP4, Bd.ROLE_V)
+    _check_operand(got, Qz.quantize_v(bits), Bd.ROLE_V)
+    z = np.zeros((1, 1, 128, 64), dtype=np.uint16)
+    got = Bd.fp4attn_quantize(_dev(z), Bd.FMT_NVFP4, Bd.ROLE_K)
+    _check_operand(got, Qz.quantize_qk(z, "nv"), Bd.ROLE_K)
+
+
+def test_full_size_quantizer_sampled(tmp_path):
+    """Config 2's full tensor: every scale byte and a random sample of rows against the oracle."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.WORKLOADS["cfg2"]
+    q, _, v = I.make_qkv(w)
+    got = Bd.fp4attn_quantize(_dev(q), Bd.FMT_MXFP4, Bd.ROLE_Q)
+    want = Qz.quantize_qk(q, "mx")
+    _check_operand(got, want, Bd.ROLE_Q)
+    got = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    _check_operand(got, Qz.quantize_v(v), Bd.ROLE_V)
