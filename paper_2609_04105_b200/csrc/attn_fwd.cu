@@ -1,6 +1,473 @@
-// placeholder until the attention kernel lands
+// Noncausal full-FP4 attention forward with Direct-P for sm_100a.
+//
+// One CTA owns one 128-row query tile of one (batch, head) and walks the keys in tiles of 64;
+// two CTAs share an SM (256 TMEM columns and < 114 KB of shared memory each), so one CTA's
+// tensor-core work overlaps the other's softmax without any cross-CTA protocol.
+//
+//   warp 0      TMA producer: Q tile once, then a ring of {K tile, V^T tile, K scales, V scales}
+//   warp 1      tensor-core issuer (one elected thread): S = Q K^T, then O += P V
+//   warps 2-5   softmax warpgroup, one thread per query row: Algorithm "direct-p-pack"
+//
+// Tensor memory (256 columns): S 0..63 | O 64..64+d-1 | Q scales 192..199 | P scales 200..207 |
+// K scales 208..223 (two slots) | V scales 224..231 (two slots).
+#include <cuda.h>
+
 #include "common.cuh"
-extern "C" int fp4attn_fwd(const fp4attn_operands*, int, int, int, int, void*, float*, int*, fp4attn_stream_t) {
-  return FP4ATTN_ERR_CUDA;
+#include "ptx.cuh"
+
+namespace fp4attn {
+using namespace ptx;
+
+constexpr int BM = 128;          // query rows per CTA
+constexpr int BN = 64;           // keys per tile (two N32 probability blocks)
+constexpr int kAttnThreads = 192;
+constexpr int kLazyShift = 64;   // the row reference follows the running maximum only when it is
+                                 // more than this many octaves behind (rescales are exact powers of 2)
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kColS = 0, kColO = 64, kColSFQ = 192, kColSFP = 200, kColSFK = 208, kColSFV = 224;
+
+template <int D, bool NV>
+struct Cfg {
+  static constexpr int ROW_BYTES = D / 2;                       // packed bytes of one Q/K row
+  static constexpr int KBLK = D / 64;                           // K64 instructions per QK tile
+  static constexpr int CTQ = NV ? (D / 16 + 3) / 4 : 1;         // scale atoms per 128 rows of Q or K
+  static constexpr int Q_BYTES = BM * ROW_BYTES;
+  static constexpr int QSF_BYTES = CTQ * 512;
+  static constexpr int K_BYTES = BN * ROW_BYTES;
+  static constexpr int V_BYTES = D * (BN / 2);
+  static constexpr int KSF_BYTES = CTQ * 512;
+  static constexpr int VSF_BYTES = 512;
+  static constexpr int STAGE_BYTES = K_BYTES + V_BYTES + KSF_BYTES + VSF_BYTES;
+  static constexpr int NST = (D == 128) ? 8 : 12;               // ring depth
+  static constexpr int P_BYTES = BM * (BN / 2);                 // 4 KB: [chunk][row][16 B]
+  static constexpr int PSF_BYTES = 512;
+  // shared-memory map (offsets from a 1024-byte aligned base)
+  static constexpr int OFF_Q = 0;
+  static constexpr int OFF_QSF = OFF_Q + Q_BYTES;
+  static constexpr int OFF_P = OFF_QSF + 1024;
+  static constexpr int OFF_PSF = OFF_P + 2 * P_BYTES;
+  static constexpr int OFF_STAGE = OFF_PSF + 2 * PSF_BYTES;
+  static constexpr int OFF_BAR = OFF_STAGE + NST * STAGE_BYTES;
+  static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;       // barriers + alignment slack
+  static constexpr uint64_t SWZ_QK = (ROW_BYTES == 64) ? kSwz64 : kSwz32;
+  static_assert(STAGE_BYTES % 1024 == 0 || STAGE_BYTES % 512 == 0, "stage alignment");
+};
+
+struct AttnParams {
+  const uint8_t *q_sf, *k_sf, *v_sf;
+  const float *q_G, *k_G;
+  __nv_bfloat16* O;
+  float* LSE;
+  int* status;
+  int N, tiles;            // keys, N / 64
+  float c_base;            // fl32(log2(e) * softmax_scale)
+};
+
+// barrier slots
+enum { BAR_Q = 0, BAR_SFULL, BAR_SEMPTY, BAR_PFULL0, BAR_PFULL1, BAR_PEMPTY0, BAR_PEMPTY1, BAR_OFULL, BAR_RING };
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
-extern "C" int fp4attn_mma_peak_probe(int, unsigned long long*, fp4attn_stream_t) { return FP4ATTN_ERR_CUDA; }
+
+// Sum of the doubled magnitudes {0,1,2,3,4,6,8,12} of the eight non-negative E2M1 codes of a word,
+// returned as four byte-wise partial sums (each <= 24).
+__device__ __forceinline__ uint32_t code_sums_x2(uint32_t w) {
+  const uint32_t lo = 0x03020100u, hi = 0x0C080604u;
+  return __byte_perm(lo, hi, w) + __byte_perm(lo, hi, w >> 16);
+}
+
+template <int D, bool NV>
+__global__ void __launch_bounds__(kAttnThreads, 2)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+  using C = Cfg<D, NV>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
+  uint32_t* tslot = reinterpret_cast<uint32_t*>(sgen + C::OFF_BAR + 384);
+  volatile int* abortf = reinterpret_cast<volatile int*>(sgen + C::OFF_BAR + 392);
+  auto bar = [&](int i) { return sbase + C::OFF_BAR + 8u * i; };
+  auto bar_full = [&](int s) { return bar(BAR_RING + s); };
+  auto bar_empty = [&](int s) { return bar(BAR_RING + C::NST + s); };
+  auto stage_addr = [&](int s) { return sbase + C::OFF_STAGE + (uint32_t)s * C::STAGE_BYTES; };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qtiles = p.N / BM;
+  const int bh = blockIdx.x / qtiles, qt = blockIdx.x % qtiles;
+  const int T = p.tiles;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(BAR_Q), 1);
+    mbar_init(bar(BAR_SFULL), 1);
+    mbar_init(bar(BAR_SEMPTY), 4);
+    mbar_init(bar(BAR_PFULL0), 4);
+    mbar_init(bar(BAR_PFULL1), 4);
+    mbar_init(bar(BAR_PEMPTY0), 1);
+    mbar_init(bar(BAR_PEMPTY1), 1);
+    mbar_init(bar(BAR_OFULL), 1);
+    for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+    *abortf = 0;
+    fence_barrier_init();
+    prefetch_tensormap(&tmQ);
+    prefetch_tensormap(&tmK);
+    prefetch_tensormap(&tmV);
+  }
+  if (warp == 1) { tmem_alloc(sbase + C::OFF_BAR + 384, kTmemCols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tslot;
+
+  if (warp == 0) {
+    // ===================================================================== TMA producer
+    if (lane == 0) {
+      mbar_arrive_expect_tx(bar(BAR_Q), C::Q_BYTES + C::QSF_BYTES);
+      tma_load_2d(sbase + C::OFF_Q, &tmQ, 0, bh * p.N + qt * BM, bar(BAR_Q));
+      bulk_load_1d(sbase + C::OFF_QSF, p.q_sf + ((size_t)bh * qtiles + qt) * C::QSF_BYTES, C::QSF_BYTES, bar(BAR_Q));
+      int issued = 0;
+      for (int j = 0; j < T; ++j) {
+        const int s = j % C::NST;
+        if (j >= C::NST && !mbar_wait(bar_empty(s), ((j / C::NST) - 1) & 1, abortf)) break;
+        const uint32_t st = stage_addr(s);
+        mbar_arrive_expect_tx(bar_full(s), C::STAGE_BYTES);
+        tma_load_2d(st, &tmK, 0, bh * p.N + j * BN, bar_full(s));
+        tma_load_2d(st + C::K_BYTES, &tmV, j * (BN / 2), bh * D, bar_full(s));
+        const size_t pair = (size_t)bh * qtiles + (j >> 1);       // 128-key pair of this tile
+        bulk_load_1d(st + C::K_BYTES + C::V_BYTES, p.k_sf + pair * C::KSF_BYTES, C::KSF_BYTES, bar_full(s));
+        bulk_load_1d(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, p.v_sf + pair * C::VSF_BYTES, C::VSF_BYTES, bar_full(s));
+        issued = j + 1;
+      }
+      if (*abortf) {
+        // bounded drain of copies still in flight before the CTA retires
+        for (int j = max(0, issued - C::NST); j < issued; ++j)
+          for (int spin = 0; spin < (1 << 14) && !mbar_try_wait(bar_full(j % C::NST), (j / C::NST) & 1); ++spin) {}
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ===================================================================== tensor-core issuer
+    if (lane == 0) {
+      const uint32_t tS = tmem + kColS, tO = tmem + kColO;
+      bool ok = mbar_wait(bar(BAR_Q), 0, abortf);
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int a = 0; a < C::CTQ; ++a)
+          tc_cp_32x128b_warpx4(tmem + kColSFQ + 4 * a, make_smem_desc(sbase + C::OFF_QSF + 512 * a, 16, 128, kSwzNone));
+      }
+      for (int j = 0; ok && j <= T; ++j) {
+        if (j < T) {                                            // ---- S(j) = Q K(j)^T
+          const int s = j % C::NST;
+          ok = mbar_wait(bar_full(s), (j / C::NST) & 1, abortf);
+          if (ok && j > 0) ok = mbar_wait(bar(BAR_SEMPTY), (j - 1) & 1, abortf);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t st = stage_addr(s);
+          const uint32_t tSFK = tmem + kColSFK + 8 * (j & 1);
+#pragma unroll
+          for (int a = 0; a < C::CTQ; ++a)
+            tc_cp_32x128b_warpx4(tSFK + 4 * a, make_smem_desc(st + C::K_BYTES + C::V_BYTES + 512 * a, 16, 128, kSwzNone));
+          const uint32_t sfb_col = tSFK + 2 * (j & 1);          // keys 64..127 of the pair sit two columns on
+#pragma unroll
+          for (int kb = 0; kb < C::KBLK; ++kb) {
+            const uint64_t ad = make_smem_desc(sbase + C::OFF_Q + 32 * kb, 16, 8 * C::ROW_BYTES, C::SWZ_QK);
+            const uint64_t bd = make_smem_desc(st + 32 * kb, 16, 8 * C::ROW_BYTES, C::SWZ_QK);
+            if (NV) {
+              tc_mma_fp4_4x(tS, ad, bd, make_idesc_fp4(BM, BN, false, 0, 0), tmem + kColSFQ + 4 * kb, sfb_col + 4 * kb, kb);
+            } else {
+              tc_mma_fp4_2x(tS, ad, bd, make_idesc_fp4(BM, BN, true, 2 * kb, 2 * kb), tmem + kColSFQ, sfb_col, kb);
+            }
+          }
+          tc_commit(bar(BAR_SFULL));
+        }
+        if (j >= 1) {                                           // ---- O += P(j-1) V(j-1)
+          const int t = j - 1, b = t & 1, s = t % C::NST;
+          ok = mbar_wait(bar(BAR_PFULL0 + b), (t >> 1) & 1, abortf);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t st = stage_addr(s);
+          const uint32_t tSFP = tmem + kColSFP + 4 * b, tSFV = tmem + kColSFV + 4 * b;
+          tc_cp_32x128b_warpx4(tSFP, make_smem_desc(sbase + C::OFF_PSF + 512 * b, 16, 128, kSwzNone));
+          tc_cp_32x128b_warpx4(tSFV, make_smem_desc(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, 16, 128, kSwzNone));
+          const uint64_t ad = make_smem_desc(sbase + C::OFF_P + C::P_BYTES * b, BM * 16, 128, kSwzNone);
+          const uint64_t bd = make_smem_desc(st + C::K_BYTES, 16, 8 * 32, kSwz32);
+          // P scales: bytes 0,1 of its atom; V scales: bytes 2*(t&1).. of the 128-key atom
+          const uint32_t idesc = (t & 1) ? make_idesc_fp4(BM, D, true, 0, 2) : make_idesc_fp4(BM, D, true, 0, 0);
+          tc_mma_fp4_2x(tO, ad, bd, idesc, tSFP, tSFV, t > 0);
+          tc_commit(bar_empty(s));
+          tc_commit(bar(BAR_PEMPTY0 + b));
+          if (t == T - 1) tc_commit(bar(BAR_OFULL));
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ===================================================================== softmax warpgroup
+    const int quarter = warp & 3;                               // TMEM lane quarter this warp may touch
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const uint32_t tS = tmem + lane_base + kColS, tO = tmem + lane_base + kColO;
+    float c32;
+    if (NV) c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G), __ldg(p.k_G)));
+    else    c32 = __fdiv_rn(p.c_base, 36.0f);
+    const float LOG2_6 = 2.5849625007211560f;
+    int mu = -(1 << 28);                                        // integer row reference (log2 domain)
+    float L2 = 0.f;                                             // sum of 2^(E_B - mu) * (2 * code sum)
+    bool ok = true;
+    for (int j = 0; j < T; ++j) {
+      const int b = j & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL), j & 1, abortf));
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t sraw[BN];
+      tmem_ld_32x32b_x32(tS, sraw);
+      tmem_ld_32x32b_x32(tS + 32, sraw + 32);
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_SEMPTY));              // S may be overwritten by the next QK
+      // ---- block maxima and integer exponents E_B = ceil(max y)
+      int E[2];
+#pragma unroll
+      for (int blk = 0; blk < 2; ++blk) {
+        float m = __uint_as_float(sraw[32 * blk]);
+#pragma unroll
+        for (int i = 1; i < 32; ++i) m = fmaxf(m, __uint_as_float(sraw[32 * blk + i]));
+        E[blk] = (int)ceilf(__fmul_rn(m, c32));
+      }
+      // ---- lazily raise the row reference; rescale L and the O row by an exact power of two
+      const int Emax = max(E[0], E[1]);
+      const bool need = Emax > mu + kLazyShift;
+      if (__any_sync(0xffffffffu, need)) {
+        float f = 1.0f;
+        if (need) {
+          const int delta = Emax - mu;
+          f = (delta > 126) ? 0.f : __uint_as_float((uint32_t)(127 - delta) << 23);
+          mu = Emax;
+          L2 *= f;
+        }
+        if (j > 0) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PEMPTY0 + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abortf));   // PV(j-1) has landed
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            uint32_t o[32];
+            tmem_ld_32x32b_x32(tO + c0, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+            tmem_st_32x32b_x32(tO + c0, o);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+        }
+      }
+      // ---- Direct-P: codes, scale bytes, represented row sum
+      uint32_t words[8];
+      uint32_t ubytes = 0;
+#pragma unroll
+      for (int blk = 0; blk < 2; ++blk) {
+        const int u = E[blk] - mu + 127;
+        const bool live = u >= 1;
+        const float bB = __fsub_rn(LOG2_6, (float)E[blk]);
+        uint32_t acc = 0;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          float pv[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) pv[i] = ex2_approx(fmaf(__uint_as_float(sraw[32 * blk + 8 * w + i]), c32, bB));
+          uint32_t word = cvt_e2m1x8(pv);
+          word = live ? word : 0u;
+          words[4 * blk + w] = word;
+          acc += code_sums_x2(word);
+        }
+        const int c2 = __dp4a(acc, 0x01010101u, 0u);
+        if (live) {
+          L2 = fmaf((float)c2, __uint_as_float((uint32_t)u << 23), L2);
+          ubytes |= (uint32_t)u << (8 * blk);
+        }
+      }
+      // ---- publish P(j): payload [chunk][row][16 B], scales in atom order
+      if (j >= 2) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PEMPTY0 + b), ((j >> 1) - 1) & 1, abortf));
+        if (!ok) break;
+      }
+      uint8_t* pbuf = sgen + C::OFF_P + C::P_BYTES * b;
+      *reinterpret_cast<uint4*>(pbuf + row * 16) = make_uint4(words[0], words[1], words[2], words[3]);
+      *reinterpret_cast<uint4*>(pbuf + BM * 16 + row * 16) = make_uint4(words[4], words[5], words[6], words[7]);
+      *reinterpret_cast<uint32_t*>(sgen + C::OFF_PSF + 512 * b + lane * 16 + quarter * 4) = ubytes;
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + b));
+    }
+    // ---- epilogue: O = O_hw / (3 * L2), LSE = ln2 * (mu + log2(L2 / 12))
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFULL), 0, abortf));
+    if (ok) {
+      tc_fence_after();
+      const float inv = __frcp_rn(3.0f * L2);
+      const size_t grow = (size_t)bh * p.N + (size_t)qt * BM + row;
+      __nv_bfloat16* orow = p.O + grow * D;
+#pragma unroll
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t o[32];
+        tmem_ld_32x32b_x32(tO + c0, o);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(o[2 * i]) * inv, __uint_as_float(o[2 * i + 1]) * inv);
+          pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+          *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
+      }
+      if (p.LSE) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(L2) - 3.5849625007211560f));
+      tc_fence_before();
+    }
+  }
+  __syncthreads();
+  if (*abortf && threadIdx.x == 0 && p.status) *p.status = FP4ATTN_ERR_TIMEOUT;
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------ dense FP4 issue-rate probe
+__global__ void __launch_bounds__(128, 1) mma_peak_kernel(int iters, unsigned long long* cycles_out) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
+  // A: 128 rows x 32 B, B: 128 rows x 32 B (one K64 slice each), scale atoms 2 x 512 B, all zero
+  for (int i = threadIdx.x; i < (4096 + 4096 + 1024) / 4; i += 128) reinterpret_cast<uint32_t*>(sgen)[i] = 0;
+  uint32_t* tslot = reinterpret_cast<uint32_t*>(sgen + 9216 + 64);
+  volatile int* abortf = reinterpret_cast<volatile int*>(sgen + 9216 + 72);
+  if (threadIdx.x == 0) { mbar_init(sbase + 9216, 1); *abortf = 0; fence_barrier_init(); }
+  fence_proxy_async_smem();
+  if ((threadIdx.x >> 5) == 0) { tmem_alloc(sbase + 9216 + 64, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tslot;
+  if (threadIdx.x == 32) {
+    tc_cp_32x128b_warpx4(tmem + 480, make_smem_desc(sbase + 8192, 16, 128, kSwzNone));
+    tc_cp_32x128b_warpx4(tmem + 484, make_smem_desc(sbase + 8192 + 512, 16, 128, kSwzNone));
+    const uint64_t ad = make_smem_desc(sbase, 16, 256, kSwz32), bd = make_smem_desc(sbase + 4096, 16, 256, kSwz32);
+    const uint32_t idesc = make_idesc_fp4(128, 128, true, 0, 0);
+    const long long t0 = clock64();
+    for (int i = 0; i < iters; ++i) tc_mma_fp4_2x(tmem + 128 * (i & 1), ad, bd, idesc, tmem + 480, tmem + 484, 1);
+    tc_commit(sbase + 9216);
+    const bool ok = mbar_wait(sbase + 9216, 0, abortf);
+    const long long t1 = clock64();
+    if (ok) atomicMax(cycles_out, (unsigned long long)(t1 - t0));
+  }
+  tc_fence_before();
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 0) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// 2-D byte tensor [rows][row_bytes], box [box_rows][box_bytes], swizzle matching the box width
+static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t rows, uint32_t box_bytes,
+                     uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {row_bytes, rows};
+  const cuuint64_t strides[1] = {row_bytes};
+  const cuuint32_t box[2] = {box_bytes, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapSwizzle swz = box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, bool NV>
+static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
+  using C = Cfg<D, NV>;
+  static_assert(C::SMEM_BYTES <= 115 * 1024, "two CTAs must fit one SM");
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+      return FP4ATTN_ERR_CUDA;
+    attr_set = true;
+  }
+  CUtensorMap tmQ, tmK, tmV;
+  const uint64_t rows = (uint64_t)B * H * N;
+  if (!make_map(&tmQ, ops->q, C::ROW_BYTES, rows, C::ROW_BYTES, BM) ||
+      !make_map(&tmK, ops->k, C::ROW_BYTES, rows, C::ROW_BYTES, BN) ||
+      !make_map(&tmV, ops->v, (uint64_t)N / 2, (uint64_t)B * H * D, BN / 2, D))
+    return FP4ATTN_ERR_CUDA;
+  const unsigned grid = (unsigned)(B * H * (N / BM));
+  attn_fwd_kernel<D, NV><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, prm);
+  return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
+}
+
+}  // namespace fp4attn
+
+using namespace fp4attn;
+
+extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int d, void* O, float* LSE,
+                           int* device_status, fp4attn_stream_t stream) {
+  if (!ops || !O || !ops->q || !ops->k || !ops->v || !ops->q_sf || !ops->k_sf || !ops->v_sf)
+    return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->qk_fmt != FP4ATTN_FMT_MXFP4 && ops->qk_fmt != FP4ATTN_FMT_NVFP4) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->qk_fmt == FP4ATTN_FMT_NVFP4 && (!ops->q_G || !ops->k_G)) return FP4ATTN_ERR_INVALID_ARG;
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return FP4ATTN_ERR_INVALID_ARG;
+  if (!(d == 64 || d == 128) || N < 128 || N % 128 != 0) return FP4ATTN_ERR_UNSUPPORTED_SHAPE;
+  if ((uint64_t)B * H * N >= (1ull << 31)) return FP4ATTN_ERR_UNSUPPORTED_SHAPE;
+  if (!(ops->softmax_scale >= 0.f)) return FP4ATTN_ERR_INVALID_ARG;
+  const uintptr_t a128 = (uintptr_t)ops->q | (uintptr_t)ops->k | (uintptr_t)ops->v | (uintptr_t)ops->q_sf |
+                         (uintptr_t)ops->k_sf | (uintptr_t)ops->v_sf;
+  if ((a128 & 127) || ((uintptr_t)O & 15) || ((uintptr_t)LSE & 3)) return FP4ATTN_ERR_ALIGNMENT;
+  int rc = check_device_sm100();
+  if (rc != FP4ATTN_OK) return rc;
+  AttnParams prm;
+  prm.q_sf = (const uint8_t*)ops->q_sf; prm.k_sf = (const uint8_t*)ops->k_sf; prm.v_sf = (const uint8_t*)ops->v_sf;
+  prm.q_G = ops->q_G; prm.k_G = ops->k_G;
+  prm.O = (__nv_bfloat16*)O; prm.LSE = LSE; prm.status = device_status;
+  prm.N = N; prm.tiles = N / BN;
+  const float scale = ops->softmax_scale > 0.f ? ops->softmax_scale : (float)(1.0 / sqrt((double)d));
+  prm.c_base = 1.4426950408889634f * scale;                        // fl32(log2e_32 * scale_32)
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool nv = ops->qk_fmt == FP4ATTN_FMT_NVFP4;
+  if (d == 128) return nv ? launch_attn<128, true>(ops, B, H, N, prm, st) : launch_attn<128, false>(ops, B, H, N, prm, st);
+  return nv ? launch_attn<64, true>(ops, B, H, N, prm, st) : launch_attn<64, false>(ops, B, H, N, prm, st);
+}
+
+extern "C" int fp4attn_mma_peak_probe(int iters, unsigned long long* cycles_out, fp4attn_stream_t stream) {
+  if (iters <= 0 || !cycles_out) return FP4ATTN_ERR_INVALID_ARG;
+  int rc = check_device_sm100();
+  if (rc != FP4ATTN_OK) return rc;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return FP4ATTN_ERR_CUDA;
+  // > 114 KB of dynamic shared memory keeps it at one CTA per SM
+  const int smem = 120 * 1024;
+  if (cudaFuncSetAttribute(mma_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+    return FP4ATTN_ERR_CUDA;
+  if (cudaMemsetAsync(cycles_out, 0, sizeof(unsigned long long), (cudaStream_t)stream) != cudaSuccess) return FP4ATTN_ERR_CUDA;
+  mma_peak_kernel<<<sms, 128, smem, (cudaStream_t)stream>>>(iters, cycles_out);
+  return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
+}

@@ -1,0 +1,150 @@
+"""Kernel (b): the CUDA Direct-P attention forward against the oracle, element by element.
+
+Tolerances (stated by the benchmark spec, per (batch, head)): relative Frobenius error <= 5e-3 and
+max-abs error <= 2e-2 between the bf16 output and the oracle's fp64 output; for the LSE
+|d| <= 1e-3 + 1e-5 |LSE| (fp32 log2 and accumulation of the row sum).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as A
+from oracle import quantize as Qz
+from paper_2609_04105_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+REL_FRO, MAX_ABS = 5e-3, 2e-2
+
+
+def _dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def run_gpu(w, q, k, v, softmax_scale=0.0):
+    from paper_2609_04105_b200 import binding as Bd
+    qd = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q)
+    kd = Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+    vd = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    O, lse = Bd.fp4attn_fwd(qd, kd, vd, softmax_scale=softmax_scale, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "kernel reported a bounded-wait timeout"
+    return O.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+
+
+def oracle_operands(w, q, k, v):
+    fmt = "mx" if w.qk_fmt == I.FMT_MXFP4 else "nv"
+    return Qz.quantize_qk(q, fmt), Qz.quantize_qk(k, fmt), Qz.quantize_v(v)
+
+
+def check_heads(Og, Lg, Oo, Lo, heads, rows=None):
+    """Og [B,H,N,d], Lg [B,H,N] from the GPU; Oo [n_heads,R,d], Lo [n_heads,R] from the oracle."""
+    worst = (0.0, 0.0, 0.0)
+    for n, (b, h) in enumerate(heads):
+        g = Og[b, h] if rows is None else Og[b, h][rows]
+        l = Lg[b, h] if rows is None else Lg[b, h][rows]
+        rel = np.linalg.norm(g - Oo[n]) / np.linalg.norm(Oo[n])
+        mab = np.abs(g - Oo[n]).max()
+        dl = np.abs(l - Lo[n]) - 1e-5 * np.abs(Lo[n])
+        worst = (max(worst[0], rel), max(worst[1], mab), max(worst[2], dl.max()))
+        assert rel <= REL_FRO, f"head {(b, h)}: rel Frobenius {rel:.3e}"
+        assert mab <= MAX_ABS, f"head {(b, h)}: max abs {mab:.3e}"
+        assert dl.max() <= 1e-3, f"head {(b, h)}: LSE error {dl.max():.3e}"
+    return worst
+
+
+SMALL = [
+    ("cfg1", dict()),                                   # B1 H2 N256 d128, MXFP4 x4 (config 1 itself)
+    ("cfg1", dict(N=128)),                              # a single 128-key pair
+    ("cfg1", dict(N=384, H=3)),                         # odd number of pairs, several heads
+    ("cfg1", dict(d=64, N=512)),                        # MXFP4 at d=64
+    ("cfg3", dict(B=2, H=2, N=512)),                    # NVFP4 Q/K at d=64 (config 3's formats)
+    ("cfg3", dict(B=1, H=2, N=384, d=128)),             # NVFP4 Q/K at d=128
+    ("cfg4", dict(H=2, N=1024)),                        # outlier channels: reference rescales, zero blocks
+    ("cfg2", dict(B=2, H=3, N=2304)),                   # ring wraps several times, ragged wave
+]
+
+
+@pytest.mark.parametrize("name,kw", SMALL)
+def test_attention_matches_oracle_elementwise(name, kw):
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu(w, q, k, v)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads)
+    check_heads(Og, Lg, Oo, Lo, heads)
+
+
+def test_explicit_softmax_scale_and_constant_v():
+    w = I.shrink(I.WORKLOADS["cfg1"], N=256)
+    q, k, v = I.make_qkv(w)
+    ones = I.f32_to_bf16_bits(np.full((w.B, w.H, w.N, w.d), -2.0, dtype=np.float32))
+    Og, Lg = run_gpu(w, q, k, ones, softmax_scale=0.25)
+    assert np.all(Og == -2.0)            # numerator and denominator use the same rounded codes
+    qd, kd, vd = oracle_operands(w, q, k, ones)
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, softmax_scale=0.25)
+    check_heads(Og, Lg, Oo, Lo, [(0, 0), (0, 1)])
+
+
+def test_run_to_run_determinism():
+    w = I.shrink(I.WORKLOADS["cfg2"], B=1, H=4, N=1024)
+    q, k, v = I.make_qkv(w)
+    O1, L1 = run_gpu(w, q, k, v)
+    O2, L2 = run_gpu(w, q, k, v)
+    assert np.array_equal(O1, O2) and np.array_equal(L1, L2)
+
+
+def _sampled_case(name, n_rows, n_heads, seed):
+    w = I.WORKLOADS[name]
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu(w, q, k, v)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(w.N, size=n_rows, replace=False))
+    rows[0], rows[-1] = 0, w.N - 1
+    all_heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    pick = rng.choice(len(all_heads), size=min(n_heads, len(all_heads)), replace=False)
+    heads = [all_heads[i] for i in sorted(pick)]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows)
+    return check_heads(Og, Lg, Oo, Lo, heads, rows)
+
+
+def test_config2_full_size_sampled_rows():
+    """B4 H16 N4096 d128 as bench.py launches it; 8 heads x 256 sampled query rows vs the oracle."""
+    _sampled_case("cfg2", 256, 8, 2)
+
+
+def test_config3_full_size_sampled_rows():
+    """B8 H16 N8192 d64, NVFP4 Q/K; 4 heads x 128 sampled rows."""
+    _sampled_case("cfg3", 128, 4, 3)
+
+
+def test_config5_n1024_full_size_sampled_rows():
+    _sampled_case("cfg5_N1024", 128, 8, 5)
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg1"], N=512)
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu(w, q, k, v)
+    host = [torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory() for a in (q, k, v)]
+    out = torch.empty((w.B, w.H, w.N, w.d), dtype=torch.bfloat16).pin_memory()
+    lse = torch.empty((w.B, w.H, w.N), dtype=torch.float32).pin_memory()
+    ws = torch.empty(Bd.fp4attn_attention_host_workspace_bytes(w.qk_fmt, w.B, w.H, w.N, w.d), dtype=torch.uint8, device="cuda")
+    Bd.fp4attn_attention_host(host[0], host[1], host[2], w.qk_fmt, out, lse, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.float().numpy().astype(np.float64), Og)
+    assert np.array_equal(lse.numpy().astype(np.float64), Lg)
+
+
+def test_invalid_arguments_are_rejected_before_launch():
+    from paper_2609_04105_b200 import binding as Bd
+    x = torch.zeros((1, 1, 100, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_quantize(x, Bd.FMT_MXFP4, Bd.ROLE_Q)
+    x = torch.zeros((1, 1, 128, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_quantize(x, Bd.FMT_NVFP4, Bd.ROLE_V)
