@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the FP4 Direct-P attention forward hot path on B200.
+
+One step = one pass of the whole hot path over one batch: quantize Q, K (MXFP4 or NVFP4) and V
+(MXFP4, transposed) + the attention forward.  Prints ONE JSON line on rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+N > 1 is launched with torch.distributed.run (one rank per GPU); every rank runs the same
+workload on its own batch (independent (batch, head) units, no data-path collective), so the
+job is weak-scaled and `value` is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_04105_b200 import inputs as I  # noqa: E402
+
+METRIC = "fp4_attention_fwd_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_FP4_OVER_BF16 = 4.0          # dense 9 PFLOP/s fp4 : 2.25 PFLOP/s bf16
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def _workload_text(w):
+    fmt = "MXFP4 Q,K,P,V" if w.qk_fmt == I.FMT_MXFP4 else "NVFP4 Q,K + MXFP4 P,V"
+    return f"{w.name}: B={w.B},H={w.H},N={w.N},d={w.d}, noncausal, {fmt}" + (", outlier channels x20" if w.outliers else "")
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML (read-only) while running."""
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
+        self.max_mhz, self._stop, self._thr = None, threading.Event(), None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def _nvml_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    ids = [t for t in vis.split(",") if t.strip()]
+    if ids and all(t.strip().isdigit() for t in ids) and local < len(ids):
+        return int(ids[local])
+    return local
+
+
+# ----------------------------------------------------------------------------- oracle legs
+def _blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def oracle_sample(w, q, k, v, heads, rows):
+    """Runs the oracle (as it stands) on a bounded sample: the given (b, h) pairs and query rows.
+    Returns seconds, equivalent TFLOP/s, and its outputs."""
+    from oracle import attention as A
+    from oracle import quantize as Qz
+    fmt = "mx" if w.qk_fmt == I.FMT_MXFP4 else "nv"
+    t0 = time.perf_counter()
+    sub = lambda x: np.ascontiguousarray(np.stack([x[b, h] for b, h in heads])[None])
+    qs, ks, vs = sub(q), sub(k), sub(v)
+    if fmt == "nv":
+        # the tensor-wide encode factor is a property of the whole tensor
+        Gq = Qz.nv_tensor_scale(Qz.bf16_bits_to_f64(q))
+        Gk = Qz.nv_tensor_scale(Qz.bf16_bits_to_f64(k))
+        nq, sq = Qz.nv_quantize_lastdim(Qz.bf16_bits_to_f64(qs), Gq)
+        nk, sk = Qz.nv_quantize_lastdim(Qz.bf16_bits_to_f64(ks), Gk)
+        qd = {"nib": nq, "sf": sq, "G": Gq, "fmt": "nv"}
+        kd = {"nib": nk, "sf": sk, "G": Gk, "fmt": "nv"}
+    else:
+        qd, kd = Qz.quantize_qk(qs, "mx"), Qz.quantize_qk(ks, "mx")
+    vd = Qz.quantize_v(vs)
+    O, lse = A.direct_p_forward(qd, kd, vd, rows=rows, heads=[(0, i) for i in range(len(heads))])
+    dt = time.perf_counter() - t0
+    n_rows = w.N if rows is None else len(rows)
+    flops = 4.0 * len(heads) * n_rows * w.N * w.d
+    return dt, flops / dt / 1e12, O, lse
+
+
+def accuracy_vs_fp64(w, q, k, v, heads, rows, O_gpu, O_oracle):
+    """cos / rel-L2 of the CUDA path and of the oracle against unquantised fp64 attention."""
+    from oracle import attention as A
+    from oracle import quantize as Qz
+    num = {"gpu": [0.0, 0.0, 0.0, 0.0], "oracle": [0.0, 0.0, 0.0, 0.0]}
+    for n, (b, h) in enumerate(heads):
+        x = [Qz.bf16_bits_to_f64(a[b, h]) for a in (q, k, v)]
+        Oe, _ = A.exact_attention(x[0], x[1], x[2], rows=rows)
+        for key, O in (("gpu", O_gpu[n]), ("oracle", O_oracle[n])):
+            acc = num[key]
+            acc[0] += (O * Oe).sum(); acc[1] += (O * O).sum(); acc[2] += (Oe * Oe).sum(); acc[3] += ((O - Oe) ** 2).sum()
+    out = {}
+    for key, (dot, oo, ee, dd) in num.items():
+        out[key] = {"cos": float(dot / np.sqrt(oo * ee)), "rel_l2": float(np.sqrt(dd / ee))}
+    return out
+
+
+def run_reference(args, w):
+    """`--impl reference`: the oracle timed on the host cores, one bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    q, k, v = I.make_qkv(w)
+    rng = np.random.default_rng(7)
+    rows = np.sort(rng.choice(w.N, size=min(w.N, 512), replace=False))
+    heads = [(0, 0)]
+    for _ in range(args.warmup):
+        oracle_sample(w, q, k, v, heads, rows)
+    times = []
+    for _ in range(args.steps):
+        dt, _, _, _ = oracle_sample(w, q, k, v, heads, rows)
+        times.append(dt)
+    flops = 4.0 * len(heads) * len(rows) * w.N * w.d
+    total = sum(times)
+    value = flops * len(times) / total / 1e12
+    cores = _blas_threads()
+    sample = f"{len(heads)} (batch, head) pair x {len(rows)} seeded query rows of {w.name} per step (rows are independent)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": _workload_text(w), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ----------------------------------------------------------------------------- CUDA arm
+def run_cuda(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_04105_b200 import binding as Bd, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    Bd.lib()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    q, k, v = I.make_qkv(w)
+    to_t = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    hq, hk, hv = (to_t(a).pin_memory() for a in (q, k, v))
+    dq, dk, dv = (t.to(dev, non_blocking=True) for t in (hq, hk, hv))
+    B, H, N, d = w.B, w.H, w.N, w.d
+    O = torch.empty((B, H, N, d), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    qws = torch.empty(max(16, Bd.lib().fp4attn_quantize_workspace_bytes(w.qk_fmt, 0, B, H, N, d)), dtype=torch.uint8, device=dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)      # > 126 MB L2
+    launches_per_step = 4 if w.qk_fmt == I.FMT_MXFP4 else 6
+    state = {}
+
+    def step(ev=None):
+        qd = Bd.fp4attn_quantize(dq, w.qk_fmt, Bd.ROLE_Q, qws)
+        kd = Bd.fp4attn_quantize(dk, w.qk_fmt, Bd.ROLE_K, qws)
+        vd = Bd.fp4attn_quantize(dv, Bd.FMT_MXFP4, Bd.ROLE_V)
+        if ev is not None:
+            ev[0].record()
+        Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status)
+        if ev is not None:
+            ev[1].record()
+        state["ops"] = (qd, kd, vd)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    E = lambda: torch.cuda.Event(enable_timing=True)
+    ev_step = [(E(), E()) for _ in range(args.steps)]
+    ev_attn = [(E(), E()) for _ in range(args.steps)]
+    with ClockSampler(_nvml_index(local)) as clk:
+        barrier()
+        for i in range(args.steps):
+            flush.fill_(i & 0xFF)                                   # evict L2 (outside the step's events)
+            ev_step[i][0].record()
+            step(ev_attn[i])
+            ev_step[i][1].record()
+        barrier()
+    assert int(status.item()) == 0, "attention kernel reported a bounded-wait timeout"
+    step_ms = [a.elapsed_time(b) for a, b in ev_step]
+    attn_ms = [a.elapsed_time(b) for a, b in ev_attn]
+    total_ms = sum(step_ms)
+    t = torch.tensor([total_ms, sum(attn_ms)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, attn_total_ms = float(t[0]), float(t[1])
+    value = world * w.flops * args.steps / (total_ms * 1e-3) / 1e12
+    attn_tflops = w.flops * args.steps / (attn_total_ms * 1e-3) / 1e12
+
+    # ---- quantizer alone (kernel a), HBM roofline of its dominant launch (Q rows)
+    qb = [E(), E()]
+    flush.fill_(1)
+    qb[0].record()
+    for _ in range(10):
+        Bd.fp4attn_quantize(dq, Bd.FMT_MXFP4, Bd.ROLE_Q)
+    qb[1].record()
+    torch.cuda.synchronize()
+    q_ms = qb[0].elapsed_time(qb[1]) / 10
+    q_bytes = B * H * N * d * (2 + 0.5 + 1.0 / 32)
+
+    # ---- end to end through the host-buffer entry point (pinned host in, host out)
+    ho = torch.empty((B, H, N, d), dtype=torch.bfloat16).pin_memory()
+    hl = torch.empty((B, H, N), dtype=torch.float32).pin_memory()
+    ws = torch.empty(Bd.fp4attn_attention_host_workspace_bytes(w.qk_fmt, B, H, N, d), dtype=torch.uint8, device=dev)
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        Bd.fp4attn_attention_host(hq, hk, hv, w.qk_fmt, ho, hl, ws)
+    barrier()
+    e0, e1 = E(), E()
+    e0.record()
+    for _ in range(e2e_steps):
+        Bd.fp4attn_attention_host(hq, hk, hv, w.qk_fmt, ho, hl, ws)
+    e1.record()
+    barrier()
+    e2e_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e_value = world * w.flops * e2e_steps / (float(e2e_ms[0]) * 1e-3) / 1e12
+    h2d = 3 * B * H * N * d * 2
+    d2h = B * H * N * d * 2 + B * H * N * 4
+
+    # ---- measured dense FP4 issue rate of this device (context for the roofline)
+    cyc = torch.zeros(1, dtype=torch.int64, device=dev)
+    iters = 20000
+    Bd.fp4attn_mma_peak_probe(iters, cyc)
+    p0, p1 = E(), E()
+    p0.record()
+    Bd.fp4attn_mma_peak_probe(iters, cyc)
+    p1.record()
+    torch.cuda.synchronize()
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    probe_tflops = sms * iters * 2.0 * 128 * 128 * 64 / (p0.elapsed_time(p1) * 1e-3) / 1e12
+    probe_flop_per_clk_sm = iters * 2.0 * 128 * 128 * 64 / max(1, int(cyc.item()))
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = _peaks()
+    fp4_peak = peaks["bf16_tflops"] * NOMINAL_FP4_OVER_BF16
+    attn_launch_ms = statistics.mean(attn_ms)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate)", "data": "synthetic",
+        "config": {"workload": _workload_text(w), "step": "quantize Q,K,V + attention forward",
+                   "l2": "flushed between steps (256 MiB fill, outside the step's events)",
+                   "flops": "4*B*H*N^2*d", "parallelism": f"replica x{world}, (batch, head) units, no collective"},
+        "attn_only": {"value": attn_tflops, "unit": UNIT, "ms": attn_launch_ms,
+                      "note": "attention kernel alone (the paper's timing boundary excludes quantization)"},
+        "roofline": {"kernel": "attn_fwd_kernel", "bound": "tensor", "achieved": w.flops / (attn_launch_ms * 1e-3) / 1e12,
+                     "peak": fp4_peak, "unit": "TFLOP/s",
+                     "frac": w.flops / (attn_launch_ms * 1e-3) / 1e12 / fp4_peak, "traffic": None,
+                     "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x nominal fp4:bf16 ratio 4",
+                     "fp4_issue_probe_tflops": probe_tflops, "fp4_issue_probe_flop_per_clk_per_sm": probe_flop_per_clk_sm},
+        "roofline_quantize": {"kernel": "quant_mx_rows_kernel", "bound": "hbm", "achieved": q_bytes / (q_ms * 1e-3) / 1e9,
+                              "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                              "frac": q_bytes / (q_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                              "bytes_per_element": 2 + 0.5 + 1.0 / 32},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "api": "fp4attn_attention_host (pinned host buffers)"},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clk.summary(),
+    }
+    # ---- oracle on the host cores: bounded sample of the same workload, plus accuracy vs fp64
+    if world == 1 and not args.no_cpu_baseline:
+        rng = np.random.default_rng(7)
+        n_rows = min(N, 2048)
+        rows = np.sort(rng.choice(N, size=n_rows, replace=False))
+        heads = [(0, 0), (B - 1, H - 1)] if B * H > 1 else [(0, 0)]
+        dt, tf, Oo, Lo = oracle_sample(w, q, k, v, heads, rows)
+        Og = np.stack([O[b, h].float().cpu().numpy().astype(np.float64)[rows] for b, h in heads])
+        rel = max(float(np.linalg.norm(Og[i] - Oo[i]) / np.linalg.norm(Oo[i])) for i in range(len(heads)))
+        sample = f"{len(heads)} (batch, head) pairs x {n_rows} seeded query rows of {w.name}, {dt:.1f} s"
+        out["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "sample": sample}
+        out["parity_on_sample"] = {"rel_fro_max": rel, "max_abs": float(np.abs(Og - Oo).max())}
+        out["accuracy_vs_fp64"] = accuracy_vs_fp64(w, q, k, v, heads, rows, Og, Oo)
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg2", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = I.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_cuda(args, w)
+
+
+if __name__ == "__main__":
+    main()
