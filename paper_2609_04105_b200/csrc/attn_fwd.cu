@@ -6,7 +6,8 @@
 //
 //   warp 0      TMA producer: Q tile once, then a ring of {K tile, V^T tile, K scales, V scales}
 //   warp 1      tensor-core issuer (one elected thread): S = Q K^T, then O += P V
-//   warps 2-5   softmax warpgroup, one thread per query row: Algorithm "direct-p-pack"
+//   warps 2-9   softmax, two threads per query row (one per 32-key block of the tile):
+//               Algorithm "direct-p-pack"
 //
 // Tensor memory (256 columns): S 0..63 | O 64..64+d-1 | Q scales 192..199 | P scales 200..207 |
 // K scales 208..223 (two slots) | V scales 224..231 (two slots).
@@ -20,7 +21,8 @@ using namespace ptx;
 
 constexpr int BM = 128;          // query rows per CTA
 constexpr int BN = 64;           // keys per tile (two N32 probability blocks)
-constexpr int kAttnThreads = 192;
+constexpr int kSoftmaxWarps = 8;   // two threads per query row
+constexpr int kAttnThreads = 64 + 32 * kSoftmaxWarps;
 constexpr int kLazyShift = 64;   // the row reference follows the running maximum only when it is
                                  // more than this many octaves behind (rescales are exact powers of 2)
 constexpr uint32_t kTmemCols = 256;
@@ -46,7 +48,8 @@ struct Cfg {
   static constexpr int OFF_QSF = OFF_Q + Q_BYTES;
   static constexpr int OFF_P = OFF_QSF + 1024;
   static constexpr int OFF_PSF = OFF_P + 2 * P_BYTES;
-  static constexpr int OFF_STAGE = OFF_PSF + 2 * PSF_BYTES;
+  static constexpr int OFF_XCH = OFF_PSF + 2 * PSF_BYTES;       // E_B exchange [2][2][128] int + row sums [2][128] float
+  static constexpr int OFF_STAGE = OFF_XCH + 3072;
   static constexpr int OFF_BAR = OFF_STAGE + NST * STAGE_BYTES;
   static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;       // barriers + alignment slack
   static constexpr uint64_t SWZ_QK = (ROW_BYTES == 64) ? kSwz64 : kSwz32;
@@ -64,12 +67,38 @@ struct AttnParams {
 };
 
 // barrier slots
-enum { BAR_Q = 0, BAR_SFULL, BAR_SEMPTY, BAR_PFULL0, BAR_PFULL1, BAR_PEMPTY0, BAR_PEMPTY1, BAR_OFULL, BAR_RING };
+enum { BAR_Q = 0, BAR_SFULL, BAR_SEMPTY, BAR_PFULL0, BAR_PFULL1, BAR_PEMPTY0, BAR_PEMPTY1, BAR_OFULL, BAR_PAIR0,
+       BAR_RING = BAR_PAIR0 + 4 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// maximum of 32 floats held as raw bits, as a depth-4 tree of 3-input maxima
+__device__ __forceinline__ float max32(const uint32_t* r) {
+  float t[12];
+#pragma unroll
+  for (int k = 0; k < 10; ++k)
+    t[k] = max3(__uint_as_float(r[3 * k]), __uint_as_float(r[3 * k + 1]), __uint_as_float(r[3 * k + 2]));
+  t[10] = __uint_as_float(r[30]);
+  t[11] = __uint_as_float(r[31]);
+  const float a = max3(t[0], t[1], t[2]), b = max3(t[3], t[4], t[5]), c = max3(t[6], t[7], t[8]), d = max3(t[9], t[10], t[11]);
+  return fmaxf(max3(a, b, c), d);
+}
+// two fused multiply-adds in one instruction: {x0, x1} = {s0, s1} * {c, c} + {b, b}
+__device__ __forceinline__ void fma2(float s0, float s1, float c, float b, float& x0, float& x1) {
+  asm("{\n\t.reg .b64 s, cc, bb, d;\n\t"
+      "mov.b64 s, {%2, %3};\n\tmov.b64 cc, {%4, %4};\n\tmov.b64 bb, {%5, %5};\n\t"
+      "fma.rn.f32x2 d, s, cc, bb;\n\t"
+      "mov.b64 {%0, %1}, d;\n\t}"
+      : "=f"(x0), "=f"(x1) : "f"(s0), "f"(s1), "f"(c), "f"(b));
 }
 
 // Sum of the doubled magnitudes {0,1,2,3,4,6,8,12} of the eight non-negative E2M1 codes of a word,
@@ -92,7 +121,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   auto bar = [&](int i) { return sbase + C::OFF_BAR + 8u * i; };
   auto bar_full = [&](int s) { return bar(BAR_RING + s); };
   auto bar_empty = [&](int s) { return bar(BAR_RING + C::NST + s); };
-  auto stage_addr = [&](int s) { return sbase + C::OFF_STAGE + (uint32_t)s * C::STAGE_BYTES; };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qtiles = p.N / BM;
@@ -102,12 +130,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (threadIdx.x == 0) {
     mbar_init(bar(BAR_Q), 1);
     mbar_init(bar(BAR_SFULL), 1);
-    mbar_init(bar(BAR_SEMPTY), 4);
-    mbar_init(bar(BAR_PFULL0), 4);
-    mbar_init(bar(BAR_PFULL1), 4);
+    mbar_init(bar(BAR_SEMPTY), kSoftmaxWarps);
+    mbar_init(bar(BAR_PFULL0), kSoftmaxWarps);
+    mbar_init(bar(BAR_PFULL1), kSoftmaxWarps);
     mbar_init(bar(BAR_PEMPTY0), 1);
     mbar_init(bar(BAR_PEMPTY1), 1);
     mbar_init(bar(BAR_OFULL), 1);
+    for (int q = 0; q < 4; ++q) mbar_init(bar(BAR_PAIR0 + q), 2);
     for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
     *abortf = 0;
     fence_barrier_init();
@@ -127,18 +156,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       mbar_arrive_expect_tx(bar(BAR_Q), C::Q_BYTES + C::QSF_BYTES);
       tma_load_2d(sbase + C::OFF_Q, &tmQ, 0, bh * p.N + qt * BM, bar(BAR_Q));
       bulk_load_1d(sbase + C::OFF_QSF, p.q_sf + ((size_t)bh * qtiles + qt) * C::QSF_BYTES, C::QSF_BYTES, bar(BAR_Q));
-      int issued = 0;
+      const uint8_t* ksf = p.k_sf + (size_t)bh * qtiles * C::KSF_BYTES;
+      const uint8_t* vsf = p.v_sf + (size_t)bh * qtiles * C::VSF_BYTES;
+      const int krow0 = bh * p.N, vrow0 = bh * D;
+      int issued = 0, s = 0, ph = 0;
+      uint32_t st = sbase + C::OFF_STAGE;
       for (int j = 0; j < T; ++j) {
-        const int s = j % C::NST;
-        if (j >= C::NST && !mbar_wait(bar_empty(s), ((j / C::NST) - 1) & 1, abortf)) break;
-        const uint32_t st = stage_addr(s);
-        mbar_arrive_expect_tx(bar_full(s), C::STAGE_BYTES);
-        tma_load_2d(st, &tmK, 0, bh * p.N + j * BN, bar_full(s));
-        tma_load_2d(st + C::K_BYTES, &tmV, j * (BN / 2), bh * D, bar_full(s));
-        const size_t pair = (size_t)bh * qtiles + (j >> 1);       // 128-key pair of this tile
-        bulk_load_1d(st + C::K_BYTES + C::V_BYTES, p.k_sf + pair * C::KSF_BYTES, C::KSF_BYTES, bar_full(s));
-        bulk_load_1d(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, p.v_sf + pair * C::VSF_BYTES, C::VSF_BYTES, bar_full(s));
+        if (j >= C::NST && !mbar_wait(bar_empty(s), ph ^ 1, abortf)) break;
+        const uint32_t fb = bar_full(s);
+        mbar_arrive_expect_tx(fb, C::STAGE_BYTES);
+        tma_load_2d(st, &tmK, 0, krow0 + j * BN, fb);
+        tma_load_2d(st + C::K_BYTES, &tmV, j * (BN / 2), vrow0, fb);
+        bulk_load_1d(st + C::K_BYTES + C::V_BYTES, ksf + (size_t)(j >> 1) * C::KSF_BYTES, C::KSF_BYTES, fb);
+        bulk_load_1d(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, vsf + (size_t)(j >> 1) * C::VSF_BYTES, C::VSF_BYTES, fb);
         issued = j + 1;
+        st += C::STAGE_BYTES;
+        if (++s == C::NST) { s = 0; ph ^= 1; st = sbase + C::OFF_STAGE; }
       }
       if (*abortf) {
         // bounded drain of copies still in flight before the CTA retires
@@ -150,96 +183,114 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   } else if (warp == 1) {
     // ===================================================================== tensor-core issuer
     if (lane == 0) {
+      // descriptor templates: everything but the 14 address bits is loop-invariant
+      constexpr uint64_t kDescSF = (uint64_t)(16 >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
+      constexpr uint64_t kDescQK = (uint64_t)(16 >> 4) << 16 | (uint64_t)((8 * C::ROW_BYTES) >> 4) << 32 | 1ull << 46 | C::SWZ_QK << 61;
+      constexpr uint64_t kDescV = (uint64_t)(16 >> 4) << 16 | (uint64_t)(256 >> 4) << 32 | 1ull << 46 | kSwz32 << 61;
+      constexpr uint64_t kDescP = (uint64_t)((BM * 16) >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
+      auto at = [](uint64_t tmpl, uint32_t addr) { return tmpl | (uint64_t)((addr & 0x3FFFFu) >> 4); };
       const uint32_t tS = tmem + kColS, tO = tmem + kColO;
+      const uint64_t dQ0 = at(kDescQK, sbase + C::OFF_Q), dQ1 = at(kDescQK, sbase + C::OFF_Q + 32);
+      const uint64_t dP0 = at(kDescP, sbase + C::OFF_P), dP1 = at(kDescP, sbase + C::OFF_P + C::P_BYTES);
+      const uint64_t dPSF0 = at(kDescSF, sbase + C::OFF_PSF), dPSF1 = at(kDescSF, sbase + C::OFF_PSF + 512);
+      constexpr uint32_t kIdQK0 = NV ? make_idesc_fp4(BM, BN, false, 0, 0) : make_idesc_fp4(BM, BN, true, 0, 0);
+      constexpr uint32_t kIdQK1 = NV ? make_idesc_fp4(BM, BN, false, 0, 0) : make_idesc_fp4(BM, BN, true, 2, 2);
+      constexpr uint32_t kIdPV0 = make_idesc_fp4(BM, D, true, 0, 0), kIdPV1 = make_idesc_fp4(BM, D, true, 0, 2);
       bool ok = mbar_wait(bar(BAR_Q), 0, abortf);
       if (ok) {
         tc_fence_after();
 #pragma unroll
-        for (int a = 0; a < C::CTQ; ++a)
-          tc_cp_32x128b_warpx4(tmem + kColSFQ + 4 * a, make_smem_desc(sbase + C::OFF_QSF + 512 * a, 16, 128, kSwzNone));
+        for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tmem + kColSFQ + 4 * a, at(kDescSF, sbase + C::OFF_QSF + 512 * a));
       }
+      int sq = 0, phq = 0;                       // ring slot / phase of the QK stream
+      int sp = 0;                                // ring slot of the PV stream (one tile behind)
+      uint32_t stq = sbase + C::OFF_STAGE, stp = sbase + C::OFF_STAGE;
       for (int j = 0; ok && j <= T; ++j) {
         if (j < T) {                                            // ---- S(j) = Q K(j)^T
-          const int s = j % C::NST;
-          ok = mbar_wait(bar_full(s), (j / C::NST) & 1, abortf);
+          ok = mbar_wait(bar_full(sq), phq, abortf);
           if (ok && j > 0) ok = mbar_wait(bar(BAR_SEMPTY), (j - 1) & 1, abortf);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t st = stage_addr(s);
-          const uint32_t tSFK = tmem + kColSFK + 8 * (j & 1);
+          // one scale atom covers the 128-key pair: copied by the even tile, reused by the odd one
+          const uint32_t tSFK = tmem + kColSFK + 8 * ((j >> 1) & 1);
+          if (!(j & 1)) {
 #pragma unroll
-          for (int a = 0; a < C::CTQ; ++a)
-            tc_cp_32x128b_warpx4(tSFK + 4 * a, make_smem_desc(st + C::K_BYTES + C::V_BYTES + 512 * a, 16, 128, kSwzNone));
-          const uint32_t sfb_col = tSFK + 2 * (j & 1);          // keys 64..127 of the pair sit two columns on
-#pragma unroll
-          for (int kb = 0; kb < C::KBLK; ++kb) {
-            const uint64_t ad = make_smem_desc(sbase + C::OFF_Q + 32 * kb, 16, 8 * C::ROW_BYTES, C::SWZ_QK);
-            const uint64_t bd = make_smem_desc(st + 32 * kb, 16, 8 * C::ROW_BYTES, C::SWZ_QK);
-            if (NV) {
-              tc_mma_fp4_4x(tS, ad, bd, make_idesc_fp4(BM, BN, false, 0, 0), tmem + kColSFQ + 4 * kb, sfb_col + 4 * kb, kb);
-            } else {
-              tc_mma_fp4_2x(tS, ad, bd, make_idesc_fp4(BM, BN, true, 2 * kb, 2 * kb), tmem + kColSFQ, sfb_col, kb);
-            }
+            for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFK + 4 * a, at(kDescSF, stq + C::K_BYTES + C::V_BYTES + 512 * a));
+          }
+          const uint32_t sfb = tSFK + 2 * (j & 1);              // keys 64..127 of the pair sit two columns on
+          const uint64_t dK0 = at(kDescQK, stq);
+          if (NV) {
+            tc_mma_fp4_4x(tS, dQ0, dK0, kIdQK0, tmem + kColSFQ, sfb, 0);
+            if (C::KBLK == 2) tc_mma_fp4_4x(tS, dQ1, dK0 + 2, kIdQK1, tmem + kColSFQ + 4, sfb + 4, 1);
+          } else {
+            tc_mma_fp4_2x(tS, dQ0, dK0, kIdQK0, tmem + kColSFQ, sfb, 0);
+            if (C::KBLK == 2) tc_mma_fp4_2x(tS, dQ1, dK0 + 2, kIdQK1, tmem + kColSFQ, sfb, 1);
           }
           tc_commit(bar(BAR_SFULL));
+          stq += C::STAGE_BYTES;
+          if (++sq == C::NST) { sq = 0; phq ^= 1; stq = sbase + C::OFF_STAGE; }
         }
         if (j >= 1) {                                           // ---- O += P(j-1) V(j-1)
-          const int t = j - 1, b = t & 1, s = t % C::NST;
+          const int t = j - 1, b = t & 1;
           ok = mbar_wait(bar(BAR_PFULL0 + b), (t >> 1) & 1, abortf);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t st = stage_addr(s);
-          const uint32_t tSFP = tmem + kColSFP + 4 * b, tSFV = tmem + kColSFV + 4 * b;
-          tc_cp_32x128b_warpx4(tSFP, make_smem_desc(sbase + C::OFF_PSF + 512 * b, 16, 128, kSwzNone));
-          tc_cp_32x128b_warpx4(tSFV, make_smem_desc(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, 16, 128, kSwzNone));
-          const uint64_t ad = make_smem_desc(sbase + C::OFF_P + C::P_BYTES * b, BM * 16, 128, kSwzNone);
-          const uint64_t bd = make_smem_desc(st + C::K_BYTES, 16, 8 * 32, kSwz32);
-          // P scales: bytes 0,1 of its atom; V scales: bytes 2*(t&1).. of the 128-key atom
-          const uint32_t idesc = (t & 1) ? make_idesc_fp4(BM, D, true, 0, 2) : make_idesc_fp4(BM, D, true, 0, 0);
-          tc_mma_fp4_2x(tO, ad, bd, idesc, tSFP, tSFV, t > 0);
-          tc_commit(bar_empty(s));
+          const uint32_t tSFP = tmem + kColSFP + 4 * b, tSFV = tmem + kColSFV + 4 * ((t >> 1) & 1);
+          tc_cp_32x128b_warpx4(tSFP, b ? dPSF1 : dPSF0);
+          if (!b) tc_cp_32x128b_warpx4(tSFV, at(kDescSF, stp + C::K_BYTES + C::V_BYTES + C::KSF_BYTES));
+          // P scales: bytes 0,1 of its atom; V scales: bytes 2*(t&1).. of the pair's atom
+          tc_mma_fp4_2x(tO, b ? dP1 : dP0, at(kDescV, stp + C::K_BYTES), b ? kIdPV1 : kIdPV0, tSFP, tSFV, t > 0);
+          tc_commit(bar_empty(sp));
           tc_commit(bar(BAR_PEMPTY0 + b));
           if (t == T - 1) tc_commit(bar(BAR_OFULL));
+          stp += C::STAGE_BYTES;
+          if (++sp == C::NST) { sp = 0; stp = sbase + C::OFF_STAGE; }
         }
       }
     }
     __syncwarp();
   } else {
-    // ===================================================================== softmax warpgroup
-    const int quarter = warp & 3;                               // TMEM lane quarter this warp may touch
+    // ===================================================================== softmax warps
+    // Two threads share a query row: warps 2-5 take the first 32-key block of every tile, warps 6-9
+    // the second.  A warp may only touch the TMEM lane quarter (warp % 4).
+    const int blk = (warp - 2) >> 2;
+    const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const uint32_t tS = tmem + lane_base + kColS, tO = tmem + lane_base + kColO;
+    const uint32_t tS = tmem + lane_base + kColS + 32 * blk;
+    const uint32_t tOh = tmem + lane_base + kColO + blk * (D / 2);     // the half of the O row this thread serves
+    const uint32_t pairbar = bar(BAR_PAIR0 + quarter);
+    int* ebuf = reinterpret_cast<int*>(sgen + C::OFF_XCH);             // [parity][blk][row]
+    float* lbuf = reinterpret_cast<float*>(sgen + C::OFF_XCH + 2048);  // [blk][row]
     float c32;
     if (NV) c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G), __ldg(p.k_G)));
     else    c32 = __fdiv_rn(p.c_base, 36.0f);
     const float LOG2_6 = 2.5849625007211560f;
     int mu = -(1 << 28);                                        // integer row reference (log2 domain)
-    float L2 = 0.f;                                             // sum of 2^(E_B - mu) * (2 * code sum)
+    float L2 = 0.f;                                             // this thread's share of sum 2^(E_B - mu) * (2 * code sum)
+    uint32_t xph = 0;                                           // phase of the pair barrier
     bool ok = true;
     for (int j = 0; j < T; ++j) {
       const int b = j & 1;
       ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL), j & 1, abortf));
       if (!ok) break;
       tc_fence_after();
-      uint32_t sraw[BN];
+      uint32_t sraw[32];
       tmem_ld_32x32b_x32(tS, sraw);
-      tmem_ld_32x32b_x32(tS + 32, sraw + 32);
       tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_SEMPTY));              // S may be overwritten by the next QK
-      // ---- block maxima and integer exponents E_B = ceil(max y)
-      int E[2];
-#pragma unroll
-      for (int blk = 0; blk < 2; ++blk) {
-        float m = __uint_as_float(sraw[32 * blk]);
-#pragma unroll
-        for (int i = 1; i < 32; ++i) m = fmaxf(m, __uint_as_float(sraw[32 * blk + i]));
-        E[blk] = (int)ceilf(__fmul_rn(m, c32));
-      }
+      // ---- block maximum and integer exponent E_B = ceil(max y); swap it with the row's other thread
+      const int E = (int)ceilf(__fmul_rn(max32(sraw), c32));
+      ebuf[(b * 2 + blk) * BM + row] = E;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pairbar);
+      ok = __all_sync(0xffffffffu, mbar_wait(pairbar, xph, abortf));
+      xph ^= 1;
+      if (!ok) break;
+      const int Emax = max(E, ebuf[(b * 2 + (blk ^ 1)) * BM + row]);
       // ---- lazily raise the row reference; rescale L and the O row by an exact power of two
-      const int Emax = max(E[0], E[1]);
       const bool need = Emax > mu + kLazyShift;
       if (__any_sync(0xffffffffu, need)) {
         float f = 1.0f;
@@ -253,68 +304,74 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PEMPTY0 + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abortf));   // PV(j-1) has landed
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int c0 = 0; c0 < D; c0 += 32) {
-            uint32_t o[32];
-            tmem_ld_32x32b_x32(tO + c0, o);
+#pragma unroll 1
+          for (int c0 = 0; c0 < D / 2; c0 += 16) {               // rare path: small chunks keep registers low
+            uint32_t o[16];
+            tmem_ld_32x32b_x16(tOh + c0, o);
             tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-            tmem_st_32x32b_x32(tO + c0, o);
+            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+            tmem_st_32x32b_x16(tOh + c0, o);
           }
           tmem_wait_st();
           tc_fence_before();
         }
       }
-      // ---- Direct-P: codes, scale bytes, represented row sum
-      uint32_t words[8];
-      uint32_t ubytes = 0;
+      // ---- Direct-P: codes, scale byte, represented row sum
+      uint32_t words[4];
+      int u = E - mu + 127;
+      const float bB = __fsub_rn(LOG2_6, (float)E);
+      uint32_t acc = 0;
 #pragma unroll
-      for (int blk = 0; blk < 2; ++blk) {
-        const int u = E[blk] - mu + 127;
-        const bool live = u >= 1;
-        const float bB = __fsub_rn(LOG2_6, (float)E[blk]);
-        uint32_t acc = 0;
+      for (int w = 0; w < 4; ++w) {
+        float pv[8];
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          float pv[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) pv[i] = ex2_approx(fmaf(__uint_as_float(sraw[32 * blk + 8 * w + i]), c32, bB));
-          uint32_t word = cvt_e2m1x8(pv);
-          word = live ? word : 0u;
-          words[4 * blk + w] = word;
-          acc += code_sums_x2(word);
+        for (int i = 0; i < 8; i += 2) {
+          float x0, x1;
+          fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), c32, bB, x0, x1);
+          pv[i] = ex2_approx(x0);
+          pv[i + 1] = ex2_approx(x1);
         }
-        const int c2 = __dp4a(acc, 0x01010101u, 0u);
-        if (live) {
-          L2 = fmaf((float)c2, __uint_as_float((uint32_t)u << 23), L2);
-          ubytes |= (uint32_t)u << (8 * blk);
-        }
+        words[w] = cvt_e2m1x8(pv);
+        acc += code_sums_x2(words[w]);
       }
-      // ---- publish P(j): payload [chunk][row][16 B], scales in atom order
+      int c2 = __dp4a(acc, 0x01010101u, 0u);
+      if (u < 1) {                                              // zero block: no payload, no mass
+        words[0] = words[1] = words[2] = words[3] = 0u;
+        c2 = 0;
+        u = 1;
+      }
+      L2 = fmaf((float)c2, __uint_as_float((uint32_t)u << 23), L2);
+      // ---- publish P(j): payload [block][row][16 B], scale byte in atom order
       if (j >= 2) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PEMPTY0 + b), ((j >> 1) - 1) & 1, abortf));
         if (!ok) break;
       }
-      uint8_t* pbuf = sgen + C::OFF_P + C::P_BYTES * b;
-      *reinterpret_cast<uint4*>(pbuf + row * 16) = make_uint4(words[0], words[1], words[2], words[3]);
-      *reinterpret_cast<uint4*>(pbuf + BM * 16 + row * 16) = make_uint4(words[4], words[5], words[6], words[7]);
-      *reinterpret_cast<uint32_t*>(sgen + C::OFF_PSF + 512 * b + lane * 16 + quarter * 4) = ubytes;
+      *reinterpret_cast<uint4*>(sgen + C::OFF_P + C::P_BYTES * b + blk * (BM * 16) + row * 16) =
+          make_uint4(words[0], words[1], words[2], words[3]);
+      *(sgen + C::OFF_PSF + 512 * b + lane * 16 + quarter * 4 + blk) = (uint8_t)u;
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + b));
     }
-    // ---- epilogue: O = O_hw / (3 * L2), LSE = ln2 * (mu + log2(L2 / 12))
+    // ---- epilogue: O = O_hw / (3 * L2), LSE = ln2 * (mu + log2(L2 / 12)), L2 summed over the pair
+    if (ok) {
+      lbuf[blk * BM + row] = L2;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pairbar);
+      ok = __all_sync(0xffffffffu, mbar_wait(pairbar, xph, abortf));
+    }
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFULL), 0, abortf));
     if (ok) {
       tc_fence_after();
-      const float inv = __frcp_rn(3.0f * L2);
+      const float Lrow = blk ? (lbuf[row] + L2) : (L2 + lbuf[BM + row]);      // same association in both threads
+      const float inv = __frcp_rn(3.0f * Lrow);
       const size_t grow = (size_t)bh * p.N + (size_t)qt * BM + row;
-      __nv_bfloat16* orow = p.O + grow * D;
+      __nv_bfloat16* orow = p.O + grow * D + blk * (D / 2);
 #pragma unroll
-      for (int c0 = 0; c0 < D; c0 += 32) {
+      for (int c0 = 0; c0 < D / 2; c0 += 32) {
         uint32_t o[32];
-        tmem_ld_32x32b_x32(tO + c0, o);
+        tmem_ld_32x32b_x32(tOh + c0, o);
         tmem_wait_ld();
         uint32_t pk[16];
 #pragma unroll
@@ -326,7 +383,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int v = 0; v < 4; ++v)
           *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
       }
-      if (p.LSE) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(L2) - 3.5849625007211560f));
+      if (p.LSE && blk == 0) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(Lrow) - 3.5849625007211560f));
       tc_fence_before();
     }
   }

@@ -19,8 +19,16 @@ __device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi) {
 
 // Eight floats -> one 32-bit word of eight E2M1 codes (element k in nibble k).
 __device__ __forceinline__ uint32_t cvt_e2m1x8(const float* v) {
-  return cvt_e2m1x2(v[0], v[1]) | (cvt_e2m1x2(v[2], v[3]) << 8) |
-         (cvt_e2m1x2(v[4], v[5]) << 16) | (cvt_e2m1x2(v[6], v[7]) << 24);
+  uint32_t w;
+  asm("{\n\t.reg .b8 t0, t1, t2, t3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t2, %6, %5;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t3, %8, %7;\n\t"
+      "mov.b32 %0, {t0, t1, t2, t3};\n\t}"
+      : "=r"(w)
+      : "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]));
+  return w;
 }
 
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& raw, float* v) {
