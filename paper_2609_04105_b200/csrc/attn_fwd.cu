@@ -1,16 +1,23 @@
 // Noncausal full-FP4 attention forward with Direct-P for sm_100a.
 //
-// One CTA owns one 128-row query tile of one (batch, head) and walks the keys in tiles of 64;
-// two CTAs share an SM (256 TMEM columns and < 114 KB of shared memory each), so one CTA's
-// tensor-core work overlaps the other's softmax without any cross-CTA protocol.
+// One CTA per SM owns one 128-row query tile of one (batch, head) and walks the keys in tiles of
+// 64 (two N32 probability blocks).  Score tiles live in a ring of four TMEM slots, each served by its
+// own team of four softmax warps, so four independent score->code streams share every SM
+// sub-partition; everything that is sequential in the key index (row reference, row sum, rescale
+// of O, scale bytes of P) is done by a separate group of correction warps on four numbers per row
+// and tile.
 //
-//   warp 0      TMA producer: Q tile once, then a ring of {K tile, V^T tile, K scales, V scales}
-//   warp 1      tensor-core issuer (one elected thread): S = Q K^T, then O += P V
-//   warps 2-9   softmax, two threads per query row (one per 32-key block of the tile):
-//               Algorithm "direct-p-pack"
+//   warp 0        TMA producer: Q tile once, then a ring of {K tile, V^T tile, K scales, V scales}
+//   warp 1        tensor-core issuer for S(j) = Q K(j)^T into score slot j % 4
+//   warp 2        tensor-core issuer for O += P(j) V(j)
+//   warps 3-6     correction: integer row reference, represented row sum, E8M0 bytes of P,
+//                 exact power-of-two rescale of O, epilogue
+//   warps 7-22    softmax teams 0..3 (team t serves tiles j = t mod 4), one thread per query row:
+//                 Algorithm "direct-p-pack" up to the codes and their sums; codes do not depend on
+//                 the row reference, so teams never wait for one another
 //
-// Tensor memory (256 columns): S 0..63 | O 64..64+d-1 | Q scales 192..199 | P scales 200..207 |
-// K scales 208..223 (two slots) | V scales 224..231 (two slots).
+// Tensor memory (512 columns): S slots 0..255 | O 256..383 | Q scales 384..391 | K scales 392..407
+// (two slots) | V scales 408..415 (two slots) | P scales 416..431 (four slots).
 #include <cuda.h>
 
 #include "common.cuh"
@@ -21,12 +28,13 @@ using namespace ptx;
 
 constexpr int BM = 128;          // query rows per CTA
 constexpr int BN = 64;           // keys per tile (two N32 probability blocks)
-constexpr int kSoftmaxWarps = 8;   // two threads per query row
-constexpr int kAttnThreads = 64 + 32 * kSoftmaxWarps;
+constexpr int kTeams = 4;        // score slots / softmax teams
+constexpr int kFirstCorrWarp = 3, kFirstSoftmaxWarp = 7;
+constexpr int kAttnThreads = 32 * (kFirstSoftmaxWarp + 4 * kTeams);
 constexpr int kLazyShift = 64;   // the row reference follows the running maximum only when it is
                                  // more than this many octaves behind (rescales are exact powers of 2)
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColO = 64, kColSFQ = 192, kColSFP = 200, kColSFK = 208, kColSFV = 224;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256, kColSFQ = 384, kColSFK = 392, kColSFV = 408, kColSFP = 416;
 
 template <int D, bool NV>
 struct Cfg {
@@ -40,20 +48,22 @@ struct Cfg {
   static constexpr int KSF_BYTES = CTQ * 512;
   static constexpr int VSF_BYTES = 512;
   static constexpr int STAGE_BYTES = K_BYTES + V_BYTES + KSF_BYTES + VSF_BYTES;
-  static constexpr int NST = (D == 128) ? 8 : 12;               // ring depth
-  static constexpr int P_BYTES = BM * (BN / 2);                 // 4 KB: [chunk][row][16 B]
+  static constexpr int NST = (D == 128) ? 12 : 16;              // ring depth
+  static constexpr int P_BYTES = BM * (BN / 2);                 // 4 KB: [block][row][16 B]
   static constexpr int PSF_BYTES = 512;
+  static constexpr int META_BYTES = BM * 16;                    // per row {E_0, E_1, 2*c_0, 2*c_1}
   // shared-memory map (offsets from a 1024-byte aligned base)
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_QSF = OFF_Q + Q_BYTES;
   static constexpr int OFF_P = OFF_QSF + 1024;
-  static constexpr int OFF_PSF = OFF_P + 2 * P_BYTES;
-  static constexpr int OFF_XCH = OFF_PSF + 2 * PSF_BYTES;       // E_B exchange [2][2][128] int + row sums [2][128] float
-  static constexpr int OFF_STAGE = OFF_XCH + 3072;
+  static constexpr int OFF_PSF = OFF_P + kTeams * P_BYTES;
+  static constexpr int OFF_META = OFF_PSF + kTeams * PSF_BYTES;
+  static constexpr int OFF_STAGE = OFF_META + kTeams * META_BYTES;
   static constexpr int OFF_BAR = OFF_STAGE + NST * STAGE_BYTES;
-  static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;       // barriers + alignment slack
+  static constexpr int SMEM_BYTES = OFF_BAR + 1024 + 1024;      // barriers + alignment slack
   static constexpr uint64_t SWZ_QK = (ROW_BYTES == 64) ? kSwz64 : kSwz32;
-  static_assert(STAGE_BYTES % 1024 == 0 || STAGE_BYTES % 512 == 0, "stage alignment");
+  static_assert(STAGE_BYTES % 512 == 0, "stage alignment");
+  static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
 };
 
 struct AttnParams {
@@ -66,16 +76,15 @@ struct AttnParams {
   float c_base;            // fl32(log2(e) * softmax_scale)
 };
 
-// barrier slots
-enum { BAR_Q = 0, BAR_SFULL, BAR_SEMPTY, BAR_PFULL0, BAR_PFULL1, BAR_PEMPTY0, BAR_PEMPTY1, BAR_OFULL, BAR_PAIR0,
-       BAR_RING = BAR_PAIR0 + 4 };
+// barrier slots (8 bytes each)
+enum { BAR_Q = 0, BAR_OFULL, BAR_SFULL0, BAR_SEMPTY0 = BAR_SFULL0 + kTeams, BAR_SMDONE0 = BAR_SEMPTY0 + kTeams,
+       BAR_PFULL0 = BAR_SMDONE0 + kTeams, BAR_PFREE0 = BAR_PFULL0 + kTeams, BAR_RING = BAR_PFREE0 + kTeams };
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -100,7 +109,6 @@ __device__ __forceinline__ void fma2(float s0, float s1, float c, float b, float
       "mov.b64 {%0, %1}, d;\n\t}"
       : "=f"(x0), "=f"(x1) : "f"(s0), "f"(s1), "f"(c), "f"(b));
 }
-
 // Sum of the doubled magnitudes {0,1,2,3,4,6,8,12} of the eight non-negative E2M1 codes of a word,
 // returned as four byte-wise partial sums (each <= 24).
 __device__ __forceinline__ uint32_t code_sums_x2(uint32_t w) {
@@ -108,19 +116,48 @@ __device__ __forceinline__ uint32_t code_sums_x2(uint32_t w) {
   return __byte_perm(lo, hi, w) + __byte_perm(lo, hi, w >> 16);
 }
 
+// One N32 score fragment of one row: E_B = ceil(max y), codes q = Q_E2M1(2^(y - E_B + log2 6)),
+// doubled code sum.  Nothing here depends on the row reference.
+__device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, int& E, uint32_t* words, int& c2) {
+  const float LOG2_6 = 2.5849625007211560f;
+  E = (int)ceilf(__fmul_rn(max32(sraw), c32));
+  const float bB = __fsub_rn(LOG2_6, (float)E);
+  uint32_t acc = 0;
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    float pv[8];
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+      float x0, x1;
+      fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), c32, bB, x0, x1);
+      pv[i] = ex2_approx(x0);
+      pv[i + 1] = ex2_approx(x1);
+    }
+    words[w] = cvt_e2m1x8(pv);
+    acc += code_sums_x2(words[w]);
+  }
+  c2 = __dp4a(acc, 0x01010101u, 0u);
+}
+
 template <int D, bool NV>
-__global__ void __launch_bounds__(kAttnThreads, 2)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
   using C = Cfg<D, NV>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
-  uint32_t* tslot = reinterpret_cast<uint32_t*>(sgen + C::OFF_BAR + 384);
-  volatile int* abortf = reinterpret_cast<volatile int*>(sgen + C::OFF_BAR + 392);
+  uint32_t* tslot = reinterpret_cast<uint32_t*>(sgen + C::OFF_BAR + 768);
+  volatile int* abortf = reinterpret_cast<volatile int*>(sgen + C::OFF_BAR + 776);
   auto bar = [&](int i) { return sbase + C::OFF_BAR + 8u * i; };
   auto bar_full = [&](int s) { return bar(BAR_RING + s); };
   auto bar_empty = [&](int s) { return bar(BAR_RING + C::NST + s); };
+  // descriptor templates: everything but the 14 address bits is loop-invariant
+  constexpr uint64_t kDescSF = (uint64_t)(16 >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
+  constexpr uint64_t kDescQK = (uint64_t)(16 >> 4) << 16 | (uint64_t)((8 * C::ROW_BYTES) >> 4) << 32 | 1ull << 46 | C::SWZ_QK << 61;
+  constexpr uint64_t kDescV = (uint64_t)(16 >> 4) << 16 | (uint64_t)(256 >> 4) << 32 | 1ull << 46 | kSwz32 << 61;
+  constexpr uint64_t kDescP = (uint64_t)((BM * 16) >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
+  auto at = [](uint64_t tmpl, uint32_t addr) { return tmpl | (uint64_t)((addr & 0x3FFFFu) >> 4); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qtiles = p.N / BM;
@@ -129,14 +166,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   if (threadIdx.x == 0) {
     mbar_init(bar(BAR_Q), 1);
-    mbar_init(bar(BAR_SFULL), 1);
-    mbar_init(bar(BAR_SEMPTY), kSoftmaxWarps);
-    mbar_init(bar(BAR_PFULL0), kSoftmaxWarps);
-    mbar_init(bar(BAR_PFULL1), kSoftmaxWarps);
-    mbar_init(bar(BAR_PEMPTY0), 1);
-    mbar_init(bar(BAR_PEMPTY1), 1);
     mbar_init(bar(BAR_OFULL), 1);
-    for (int q = 0; q < 4; ++q) mbar_init(bar(BAR_PAIR0 + q), 2);
+    for (int t = 0; t < kTeams; ++t) {
+      mbar_init(bar(BAR_SFULL0 + t), 1);
+      mbar_init(bar(BAR_SEMPTY0 + t), 4);
+      mbar_init(bar(BAR_SMDONE0 + t), 4);
+      mbar_init(bar(BAR_PFULL0 + t), 4);
+      mbar_init(bar(BAR_PFREE0 + t), 1);
+    }
     for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
     *abortf = 0;
     fence_barrier_init();
@@ -144,7 +181,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     prefetch_tensormap(&tmK);
     prefetch_tensormap(&tmV);
   }
-  if (warp == 1) { tmem_alloc(sbase + C::OFF_BAR + 384, kTmemCols); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(sbase + C::OFF_BAR + 768, kTmemCols); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -152,28 +189,33 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   if (warp == 0) {
     // ===================================================================== TMA producer
-    if (lane == 0) {
-      mbar_arrive_expect_tx(bar(BAR_Q), C::Q_BYTES + C::QSF_BYTES);
-      tma_load_2d(sbase + C::OFF_Q, &tmQ, 0, bh * p.N + qt * BM, bar(BAR_Q));
-      bulk_load_1d(sbase + C::OFF_QSF, p.q_sf + ((size_t)bh * qtiles + qt) * C::QSF_BYTES, C::QSF_BYTES, bar(BAR_Q));
+    // The whole warp runs the loop (addresses and waits stay warp-uniform); one elected lane issues.
+    {
+      if (elect_one()) {
+        mbar_arrive_expect_tx(bar(BAR_Q), C::Q_BYTES + C::QSF_BYTES);
+        tma_load_2d(sbase + C::OFF_Q, &tmQ, 0, bh * p.N + qt * BM, bar(BAR_Q));
+        bulk_load_1d(sbase + C::OFF_QSF, p.q_sf + ((size_t)bh * qtiles + qt) * C::QSF_BYTES, C::QSF_BYTES, bar(BAR_Q));
+      }
       const uint8_t* ksf = p.k_sf + (size_t)bh * qtiles * C::KSF_BYTES;
       const uint8_t* vsf = p.v_sf + (size_t)bh * qtiles * C::VSF_BYTES;
       const int krow0 = bh * p.N, vrow0 = bh * D;
       int issued = 0, s = 0, ph = 0;
       uint32_t st = sbase + C::OFF_STAGE;
       for (int j = 0; j < T; ++j) {
-        if (j >= C::NST && !mbar_wait(bar_empty(s), ph ^ 1, abortf)) break;
+        if (j >= C::NST && !__all_sync(0xffffffffu, mbar_wait(bar_empty(s), ph ^ 1, abortf))) break;
         const uint32_t fb = bar_full(s);
-        mbar_arrive_expect_tx(fb, C::STAGE_BYTES);
-        tma_load_2d(st, &tmK, 0, krow0 + j * BN, fb);
-        tma_load_2d(st + C::K_BYTES, &tmV, j * (BN / 2), vrow0, fb);
-        bulk_load_1d(st + C::K_BYTES + C::V_BYTES, ksf + (size_t)(j >> 1) * C::KSF_BYTES, C::KSF_BYTES, fb);
-        bulk_load_1d(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, vsf + (size_t)(j >> 1) * C::VSF_BYTES, C::VSF_BYTES, fb);
+        if (elect_one()) {
+          mbar_arrive_expect_tx(fb, C::STAGE_BYTES);
+          tma_load_2d(st, &tmK, 0, krow0 + j * BN, fb);
+          tma_load_2d(st + C::K_BYTES, &tmV, j * (BN / 2), vrow0, fb);
+          bulk_load_1d(st + C::K_BYTES + C::V_BYTES, ksf + (size_t)(j >> 1) * C::KSF_BYTES, C::KSF_BYTES, fb);
+          bulk_load_1d(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, vsf + (size_t)(j >> 1) * C::VSF_BYTES, C::VSF_BYTES, fb);
+        }
         issued = j + 1;
         st += C::STAGE_BYTES;
         if (++s == C::NST) { s = 0; ph ^= 1; st = sbase + C::OFF_STAGE; }
       }
-      if (*abortf) {
+      if (*abortf && lane == 0) {
         // bounded drain of copies still in flight before the CTA retires
         for (int j = max(0, issued - C::NST); j < issued; ++j)
           for (int spin = 0; spin < (1 << 14) && !mbar_try_wait(bar_full(j % C::NST), (j / C::NST) & 1); ++spin) {}
@@ -181,44 +223,38 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ===================================================================== tensor-core issuer
-    if (lane == 0) {
-      // descriptor templates: everything but the 14 address bits is loop-invariant
-      constexpr uint64_t kDescSF = (uint64_t)(16 >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
-      constexpr uint64_t kDescQK = (uint64_t)(16 >> 4) << 16 | (uint64_t)((8 * C::ROW_BYTES) >> 4) << 32 | 1ull << 46 | C::SWZ_QK << 61;
-      constexpr uint64_t kDescV = (uint64_t)(16 >> 4) << 16 | (uint64_t)(256 >> 4) << 32 | 1ull << 46 | kSwz32 << 61;
-      constexpr uint64_t kDescP = (uint64_t)((BM * 16) >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
-      auto at = [](uint64_t tmpl, uint32_t addr) { return tmpl | (uint64_t)((addr & 0x3FFFFu) >> 4); };
-      const uint32_t tS = tmem + kColS, tO = tmem + kColO;
+    // ===================================================================== QK issuer: S(j) = Q K(j)^T
+    // Warp-uniform control flow; tcgen05 instructions are issued by one elected lane.
+    {
       const uint64_t dQ0 = at(kDescQK, sbase + C::OFF_Q), dQ1 = at(kDescQK, sbase + C::OFF_Q + 32);
-      const uint64_t dP0 = at(kDescP, sbase + C::OFF_P), dP1 = at(kDescP, sbase + C::OFF_P + C::P_BYTES);
-      const uint64_t dPSF0 = at(kDescSF, sbase + C::OFF_PSF), dPSF1 = at(kDescSF, sbase + C::OFF_PSF + 512);
       constexpr uint32_t kIdQK0 = NV ? make_idesc_fp4(BM, BN, false, 0, 0) : make_idesc_fp4(BM, BN, true, 0, 0);
       constexpr uint32_t kIdQK1 = NV ? make_idesc_fp4(BM, BN, false, 0, 0) : make_idesc_fp4(BM, BN, true, 2, 2);
-      constexpr uint32_t kIdPV0 = make_idesc_fp4(BM, D, true, 0, 0), kIdPV1 = make_idesc_fp4(BM, D, true, 0, 2);
-      bool ok = mbar_wait(bar(BAR_Q), 0, abortf);
+      bool ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_Q), 0, abortf));
       if (ok) {
         tc_fence_after();
+        if (elect_one()) {
 #pragma unroll
-        for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tmem + kColSFQ + 4 * a, at(kDescSF, sbase + C::OFF_QSF + 512 * a));
+          for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tmem + kColSFQ + 4 * a, at(kDescSF, sbase + C::OFF_QSF + 512 * a));
+        }
       }
-      int sq = 0, phq = 0;                       // ring slot / phase of the QK stream
-      int sp = 0;                                // ring slot of the PV stream (one tile behind)
-      uint32_t stq = sbase + C::OFF_STAGE, stp = sbase + C::OFF_STAGE;
-      for (int j = 0; ok && j <= T; ++j) {
-        if (j < T) {                                            // ---- S(j) = Q K(j)^T
-          ok = mbar_wait(bar_full(sq), phq, abortf);
-          if (ok && j > 0) ok = mbar_wait(bar(BAR_SEMPTY), (j - 1) & 1, abortf);
-          if (!ok) break;
-          tc_fence_after();
-          // one scale atom covers the 128-key pair: copied by the even tile, reused by the odd one
-          const uint32_t tSFK = tmem + kColSFK + 8 * ((j >> 1) & 1);
+      int sq = 0, phq = 0;
+      uint32_t stq = sbase + C::OFF_STAGE;
+      for (int j = 0; ok && j < T; ++j) {
+        const int slot = j & (kTeams - 1), k = j >> 2;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_full(sq), phq, abortf));
+        if (ok && k > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SEMPTY0 + slot), (k - 1) & 1, abortf));   // team has read S(j-4)
+        if (!ok) break;
+        tc_fence_after();
+        // one scale atom covers the 128-key pair: copied by the even tile, reused by the odd one
+        const uint32_t tSFK = tmem + kColSFK + 8 * ((j >> 1) & 1);
+        const uint32_t sfb = tSFK + 2 * (j & 1);                // keys 64..127 of the pair sit two columns on
+        const uint32_t tS = tmem + kColS + BN * slot;
+        const uint64_t dK0 = at(kDescQK, stq);
+        if (elect_one()) {
           if (!(j & 1)) {
 #pragma unroll
             for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFK + 4 * a, at(kDescSF, stq + C::K_BYTES + C::V_BYTES + 512 * a));
           }
-          const uint32_t sfb = tSFK + 2 * (j & 1);              // keys 64..127 of the pair sit two columns on
-          const uint64_t dK0 = at(kDescQK, stq);
           if (NV) {
             tc_mma_fp4_4x(tS, dQ0, dK0, kIdQK0, tmem + kColSFQ, sfb, 0);
             if (C::KBLK == 2) tc_mma_fp4_4x(tS, dQ1, dK0 + 2, kIdQK1, tmem + kColSFQ + 4, sfb + 4, 1);
@@ -226,71 +262,61 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tc_mma_fp4_2x(tS, dQ0, dK0, kIdQK0, tmem + kColSFQ, sfb, 0);
             if (C::KBLK == 2) tc_mma_fp4_2x(tS, dQ1, dK0 + 2, kIdQK1, tmem + kColSFQ, sfb, 1);
           }
-          tc_commit(bar(BAR_SFULL));
-          stq += C::STAGE_BYTES;
-          if (++sq == C::NST) { sq = 0; phq ^= 1; stq = sbase + C::OFF_STAGE; }
+          tc_commit(bar(BAR_SFULL0 + slot));
         }
-        if (j >= 1) {                                           // ---- O += P(j-1) V(j-1)
-          const int t = j - 1, b = t & 1;
-          ok = mbar_wait(bar(BAR_PFULL0 + b), (t >> 1) & 1, abortf);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t tSFP = tmem + kColSFP + 4 * b, tSFV = tmem + kColSFV + 4 * ((t >> 1) & 1);
-          tc_cp_32x128b_warpx4(tSFP, b ? dPSF1 : dPSF0);
-          if (!b) tc_cp_32x128b_warpx4(tSFV, at(kDescSF, stp + C::K_BYTES + C::V_BYTES + C::KSF_BYTES));
-          // P scales: bytes 0,1 of its atom; V scales: bytes 2*(t&1).. of the pair's atom
-          tc_mma_fp4_2x(tO, b ? dP1 : dP0, at(kDescV, stp + C::K_BYTES), b ? kIdPV1 : kIdPV0, tSFP, tSFV, t > 0);
-          tc_commit(bar_empty(sp));
-          tc_commit(bar(BAR_PEMPTY0 + b));
-          if (t == T - 1) tc_commit(bar(BAR_OFULL));
-          stp += C::STAGE_BYTES;
-          if (++sp == C::NST) { sp = 0; stp = sbase + C::OFF_STAGE; }
-        }
+        __syncwarp();
+        stq += C::STAGE_BYTES;
+        if (++sq == C::NST) { sq = 0; phq ^= 1; stq = sbase + C::OFF_STAGE; }
       }
     }
     __syncwarp();
-  } else {
-    // ===================================================================== softmax warps
-    // Two threads share a query row: warps 2-5 take the first 32-key block of every tile, warps 6-9
-    // the second.  A warp may only touch the TMEM lane quarter (warp % 4).
-    const int blk = (warp - 2) >> 2;
+  } else if (warp == 2) {
+    // ===================================================================== PV issuer: O += P(j) V(j)
+    {
+      constexpr uint32_t kIdPV0 = make_idesc_fp4(BM, D, true, 0, 0), kIdPV1 = make_idesc_fp4(BM, D, true, 0, 2);
+      const uint32_t tO = tmem + kColO;
+      int sp = 0;
+      uint32_t stp = sbase + C::OFF_STAGE;
+      bool ok = true;
+      for (int j = 0; ok && j < T; ++j) {
+        const int slot = j & (kTeams - 1), k = j >> 2;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFULL0 + slot), k & 1, abortf));  // codes and scale bytes of P(j) are in smem
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tSFP = tmem + kColSFP + 4 * slot, tSFV = tmem + kColSFV + 4 * ((j >> 1) & 1);
+        if (elect_one()) {
+          tc_cp_32x128b_warpx4(tSFP, at(kDescSF, sbase + C::OFF_PSF + 512 * slot));
+          if (!(j & 1)) tc_cp_32x128b_warpx4(tSFV, at(kDescSF, stp + C::K_BYTES + C::V_BYTES + C::KSF_BYTES));
+          // P scales: bytes 0,1 of its atom; V scales: bytes 2*(j&1).. of the pair's atom
+          tc_mma_fp4_2x(tO, at(kDescP, sbase + C::OFF_P + C::P_BYTES * slot), at(kDescV, stp + C::K_BYTES),
+                        (j & 1) ? kIdPV1 : kIdPV0, tSFP, tSFV, j > 0);
+          tc_commit(bar_empty(sp));                               // K(j), V(j) stage back to the producer
+          tc_commit(bar(BAR_PFREE0 + slot));                      // P slot reusable; O holds tiles <= j
+          if (j == T - 1) tc_commit(bar(BAR_OFULL));
+        }
+        __syncwarp();
+        stp += C::STAGE_BYTES;
+        if (++sp == C::NST) { sp = 0; stp = sbase + C::OFF_STAGE; }
+      }
+    }
+    __syncwarp();
+  } else if (warp < kFirstSoftmaxWarp) {
+    // ===================================================================== correction warps
+    // One thread per query row, tiles in key order.  Owns the integer row reference mu, the
+    // represented row sum and the O accumulator's scale; turns the teams' absolute block exponents
+    // into the E8M0 bytes the PV instruction reads.
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
-    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const uint32_t tS = tmem + lane_base + kColS + 32 * blk;
-    const uint32_t tOh = tmem + lane_base + kColO + blk * (D / 2);     // the half of the O row this thread serves
-    const uint32_t pairbar = bar(BAR_PAIR0 + quarter);
-    int* ebuf = reinterpret_cast<int*>(sgen + C::OFF_XCH);             // [parity][blk][row]
-    float* lbuf = reinterpret_cast<float*>(sgen + C::OFF_XCH + 2048);  // [blk][row]
-    float c32;
-    if (NV) c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G), __ldg(p.k_G)));
-    else    c32 = __fdiv_rn(p.c_base, 36.0f);
-    const float LOG2_6 = 2.5849625007211560f;
-    int mu = -(1 << 28);                                        // integer row reference (log2 domain)
-    float L2 = 0.f;                                             // this thread's share of sum 2^(E_B - mu) * (2 * code sum)
-    uint32_t xph = 0;                                           // phase of the pair barrier
+    const uint32_t tO = tmem + ((uint32_t)(quarter * 32) << 16) + kColO;
+    int mu = -(1 << 28);
+    float L2 = 0.f;                                             // sum of 2^(E_B - mu) * (2 * code sum)
     bool ok = true;
     for (int j = 0; j < T; ++j) {
-      const int b = j & 1;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL), j & 1, abortf));
+      const int slot = j & (kTeams - 1), k = j >> 2;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + slot), k & 1, abortf));
       if (!ok) break;
-      tc_fence_after();
-      uint32_t sraw[32];
-      tmem_ld_32x32b_x32(tS, sraw);
-      tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_SEMPTY));              // S may be overwritten by the next QK
-      // ---- block maximum and integer exponent E_B = ceil(max y); swap it with the row's other thread
-      const int E = (int)ceilf(__fmul_rn(max32(sraw), c32));
-      ebuf[(b * 2 + blk) * BM + row] = E;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(pairbar);
-      ok = __all_sync(0xffffffffu, mbar_wait(pairbar, xph, abortf));
-      xph ^= 1;
-      if (!ok) break;
-      const int Emax = max(E, ebuf[(b * 2 + (blk ^ 1)) * BM + row]);
-      // ---- lazily raise the row reference; rescale L and the O row by an exact power of two
+      const int4 m = *reinterpret_cast<const int4*>(sgen + C::OFF_META + C::META_BYTES * slot + row * 16);
+      const int Emax = max(m.x, m.y);
       const bool need = Emax > mu + kLazyShift;
       if (__any_sync(0xffffffffu, need)) {
         float f = 1.0f;
@@ -301,77 +327,44 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           L2 *= f;
         }
         if (j > 0) {
-          ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PEMPTY0 + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abortf));   // PV(j-1) has landed
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFREE0 + ((j - 1) & 3)), ((j - 1) >> 2) & 1, abortf));   // PV(j-1) has landed
           if (!ok) break;
           tc_fence_after();
 #pragma unroll 1
-          for (int c0 = 0; c0 < D / 2; c0 += 16) {               // rare path: small chunks keep registers low
+          for (int c0 = 0; c0 < D; c0 += 16) {
             uint32_t o[16];
-            tmem_ld_32x32b_x16(tOh + c0, o);
+            tmem_ld_32x32b_x16(tO + c0, o);
             tmem_wait_ld();
 #pragma unroll
             for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-            tmem_st_32x32b_x16(tOh + c0, o);
+            tmem_st_32x32b_x16(tO + c0, o);
           }
           tmem_wait_st();
           tc_fence_before();
         }
       }
-      // ---- Direct-P: codes, scale byte, represented row sum
-      uint32_t words[4];
-      int u = E - mu + 127;
-      const float bB = __fsub_rn(LOG2_6, (float)E);
-      uint32_t acc = 0;
-#pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        float pv[8];
-#pragma unroll
-        for (int i = 0; i < 8; i += 2) {
-          float x0, x1;
-          fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), c32, bB, x0, x1);
-          pv[i] = ex2_approx(x0);
-          pv[i + 1] = ex2_approx(x1);
-        }
-        words[w] = cvt_e2m1x8(pv);
-        acc += code_sums_x2(words[w]);
-      }
-      int c2 = __dp4a(acc, 0x01010101u, 0u);
-      if (u < 1) {                                              // zero block: no payload, no mass
-        words[0] = words[1] = words[2] = words[3] = 0u;
-        c2 = 0;
-        u = 1;
-      }
-      L2 = fmaf((float)c2, __uint_as_float((uint32_t)u << 23), L2);
-      // ---- publish P(j): payload [block][row][16 B], scale byte in atom order
-      if (j >= 2) {
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PEMPTY0 + b), ((j >> 1) - 1) & 1, abortf));
-        if (!ok) break;
-      }
-      *reinterpret_cast<uint4*>(sgen + C::OFF_P + C::P_BYTES * b + blk * (BM * 16) + row * 16) =
-          make_uint4(words[0], words[1], words[2], words[3]);
-      *(sgen + C::OFF_PSF + 512 * b + lane * 16 + quarter * 4 + blk) = (uint8_t)u;
+      // A block more than 126 octaves below the reference is a zero block: it gets the smallest
+      // byte (2^-127, below 2^-60 of the row's mass by construction) and no share of the row sum.
+      const int u0 = m.x - mu + 127, u1 = m.y - mu + 127;
+      if (u0 >= 1) L2 = fmaf((float)m.z, __uint_as_float((uint32_t)u0 << 23), L2);
+      if (u1 >= 1) L2 = fmaf((float)m.w, __uint_as_float((uint32_t)u1 << 23), L2);
+      *reinterpret_cast<uint32_t*>(sgen + C::OFF_PSF + 512 * slot + lane * 16 + quarter * 4) =
+          (uint32_t)max(u0, 0) | ((uint32_t)max(u1, 0) << 8);
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + b));
+      if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + slot));
     }
-    // ---- epilogue: O = O_hw / (3 * L2), LSE = ln2 * (mu + log2(L2 / 12)), L2 summed over the pair
-    if (ok) {
-      lbuf[blk * BM + row] = L2;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(pairbar);
-      ok = __all_sync(0xffffffffu, mbar_wait(pairbar, xph, abortf));
-    }
+    // ---- epilogue: O = O_hw / (3 * L2), LSE = ln2 * (mu + log2(L2 / 12))
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFULL), 0, abortf));
     if (ok) {
       tc_fence_after();
-      const float Lrow = blk ? (lbuf[row] + L2) : (L2 + lbuf[BM + row]);      // same association in both threads
-      const float inv = __frcp_rn(3.0f * Lrow);
+      const float inv = __frcp_rn(3.0f * L2);
       const size_t grow = (size_t)bh * p.N + (size_t)qt * BM + row;
-      __nv_bfloat16* orow = p.O + grow * D + blk * (D / 2);
-#pragma unroll
-      for (int c0 = 0; c0 < D / 2; c0 += 32) {
+      __nv_bfloat16* orow = p.O + grow * D;
+#pragma unroll 1
+      for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t o[32];
-        tmem_ld_32x32b_x32(tOh + c0, o);
+        tmem_ld_32x32b_x32(tO + c0, o);
         tmem_wait_ld();
         uint32_t pk[16];
 #pragma unroll
@@ -383,8 +376,44 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int v = 0; v < 4; ++v)
           *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
       }
-      if (p.LSE && blk == 0) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(Lrow) - 3.5849625007211560f));
+      if (p.LSE) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(L2) - 3.5849625007211560f));
       tc_fence_before();
+    }
+  } else {
+    // ===================================================================== softmax teams
+    const int team = (warp - kFirstSoftmaxWarp) >> 2;
+    const int quarter = warp & 3;                               // TMEM lane quarter this warp may touch
+    const int row = quarter * 32 + lane;
+    const uint32_t tS = tmem + ((uint32_t)(quarter * 32) << 16) + kColS + BN * team;
+    const uint32_t sfull = bar(BAR_SFULL0 + team), sempty = bar(BAR_SEMPTY0 + team);
+    const uint32_t smdone = bar(BAR_SMDONE0 + team), pfree = bar(BAR_PFREE0 + team);
+    uint8_t* pbuf = sgen + C::OFF_P + C::P_BYTES * team + row * 16;
+    int4* meta = reinterpret_cast<int4*>(sgen + C::OFF_META + C::META_BYTES * team + row * 16);
+    float c32;
+    if (NV) c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G), __ldg(p.k_G)));
+    else    c32 = __fdiv_rn(p.c_base, 36.0f);
+    uint32_t ph = 0;
+    for (int j = team; j < T; j += kTeams, ph ^= 1) {
+      if (!__all_sync(0xffffffffu, mbar_wait(sfull, ph, abortf))) break;
+      tc_fence_after();
+      uint32_t sraw[32], w0[4], w1[4];
+      int E0, E1, c0, c1;
+      tmem_ld_32x32b_x32(tS, sraw);
+      tmem_wait_ld();
+      direct_p_block(sraw, c32, E0, w0, c0);
+      tmem_ld_32x32b_x32(tS + 32, sraw);
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sempty);                       // slot may take S(j+4)
+      direct_p_block(sraw, c32, E1, w1, c1);
+      if (j >= kTeams && !__all_sync(0xffffffffu, mbar_wait(pfree, ph ^ 1, abortf))) break;   // PV(j-4) consumed the slot
+      *reinterpret_cast<uint4*>(pbuf) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
+      *reinterpret_cast<uint4*>(pbuf + BM * 16) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+      *meta = make_int4(E0, E1, c0, c1);
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smdone);
     }
   }
   __syncthreads();
@@ -463,7 +492,6 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint6
 template <int D, bool NV>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
   using C = Cfg<D, NV>;
-  static_assert(C::SMEM_BYTES <= 115 * 1024, "two CTAs must fit one SM");
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
