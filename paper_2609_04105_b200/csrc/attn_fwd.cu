@@ -1,23 +1,25 @@
 // Noncausal full-FP4 attention forward with Direct-P for sm_100a.
 //
-// One CTA per SM owns one 128-row query tile of one (batch, head) and walks the keys in tiles of
-// 64 (two N32 probability blocks).  Score tiles live in a ring of four TMEM slots, each served by its
-// own team of four softmax warps, so four independent score->code streams share every SM
-// sub-partition; everything that is sequential in the key index (row reference, row sum, rescale
-// of O, scale bytes of P) is done by a separate group of correction warps on four numbers per row
-// and tile.
+// Persistent kernel, one CTA per SM.  A CTA takes work items (one 128-row query tile of one
+// (batch, head)) round-robin and walks the keys of an item in stages of 128 (two 64-key tiles, four
+// N32 probability blocks).  Score tiles live in a ring of four 64-column TMEM slots (two per stage),
+// each served by its own team of four softmax warps, so four independent score->code streams share
+// every SM sub-partition; everything that is sequential in the key index (row reference, row sum,
+// rescale of O, scale bytes of P) is done by separate correction warps on four numbers per row and
+// tile.  All roles keep running counters across items, so the next item's loads, QK products and
+// softmax overlap the previous item's epilogue.
 //
-//   warp 0        TMA producer: Q tile once, then a ring of {K tile, V^T tile, K scales, V scales}
-//   warp 1        tensor-core issuer for S(j) = Q K(j)^T into score slot j % 4
-//   warp 2        tensor-core issuer for O += P(j) V(j)
+//   warp 0        TMA producer: Q tile per item (two buffers), ring of {K, V^T, K scales, V scales}
+//   warp 1        tensor-core issuer for S = Q K^T, one 128-key stage (two score slots) per issue
+//   warp 2        tensor-core issuer for O += P V, one stage (two K64 products) per issue
 //   warps 3-6     correction: integer row reference, represented row sum, E8M0 bytes of P,
 //                 exact power-of-two rescale of O, epilogue
-//   warps 7-22    softmax teams 0..3 (team t serves tiles j = t mod 4), one thread per query row:
-//                 Algorithm "direct-p-pack" up to the codes and their sums; codes do not depend on
-//                 the row reference, so teams never wait for one another
+//   warps 7-22    softmax teams 0..3, one thread per query row; team 2p+h serves the h-th 64 keys of
+//                 the stages with parity p: Algorithm "direct-p-pack" up to the codes and their
+//                 sums; codes do not depend on the row reference, so teams never wait for one another
 //
-// Tensor memory (512 columns): S slots 0..255 | O 256..383 | Q scales 384..391 | K scales 392..407
-// (two slots) | V scales 408..415 (two slots) | P scales 416..431 (four slots).
+// Tensor memory (512 columns): S slots 0..255 | O 256..383 | Q scales 384..399 (two buffers) |
+// K scales 400..415 (two slots) | V scales 416..423 (two slots) | P scales 424..431 (two slots).
 #include <cuda.h>
 
 #include "common.cuh"
@@ -26,43 +28,44 @@
 namespace fp4attn {
 using namespace ptx;
 
-constexpr int BM = 128;          // query rows per CTA
-constexpr int BN = 64;           // keys per tile (two N32 probability blocks)
+constexpr int BM = 128;          // query rows per work item
+constexpr int BN = 64;           // keys per score tile (two N32 probability blocks)
+constexpr int BS = 128;          // keys per stage
 constexpr int kTeams = 4;        // score slots / softmax teams
 constexpr int kFirstCorrWarp = 3, kFirstSoftmaxWarp = 7;
 constexpr int kAttnThreads = 32 * (kFirstSoftmaxWarp + 4 * kTeams);
 constexpr int kLazyShift = 64;   // the row reference follows the running maximum only when it is
                                  // more than this many octaves behind (rescales are exact powers of 2)
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256, kColSFQ = 384, kColSFK = 392, kColSFV = 408, kColSFP = 416;
+constexpr uint32_t kColS = 0, kColO = 256, kColSFQ = 384, kColSFK = 400, kColSFV = 416, kColSFP = 424;
 
 template <int D, bool NV>
 struct Cfg {
   static constexpr int ROW_BYTES = D / 2;                       // packed bytes of one Q/K row
-  static constexpr int KBLK = D / 64;                           // K64 instructions per QK tile
+  static constexpr int KBLK = D / 64;                           // K64 instructions per QK stage
   static constexpr int CTQ = NV ? (D / 16 + 3) / 4 : 1;         // scale atoms per 128 rows of Q or K
   static constexpr int Q_BYTES = BM * ROW_BYTES;
   static constexpr int QSF_BYTES = CTQ * 512;
-  static constexpr int K_BYTES = BN * ROW_BYTES;
-  static constexpr int V_BYTES = D * (BN / 2);
+  static constexpr int K_BYTES = BS * ROW_BYTES;                // 128 keys
+  static constexpr int V_BYTES = D * (BS / 2);                  // V^T: d rows x 64 bytes
   static constexpr int KSF_BYTES = CTQ * 512;
   static constexpr int VSF_BYTES = 512;
   static constexpr int STAGE_BYTES = K_BYTES + V_BYTES + KSF_BYTES + VSF_BYTES;
-  static constexpr int NST = (D == 128) ? 12 : 16;              // ring depth
-  static constexpr int P_BYTES = BM * (BN / 2);                 // 4 KB: [block][row][16 B]
-  static constexpr int PSF_BYTES = 512;
+  static constexpr int NST = (D == 128) ? 6 : 8;                // ring depth (stages of 128 keys)
+  static constexpr int P_BYTES = BM * (BN / 2);                 // 4 KB per 64-key tile: [block][row][16 B]
+  static constexpr int PSF_BYTES = 512;                         // one atom per stage: bytes {0,1} tile 0, {2,3} tile 1
   static constexpr int META_BYTES = BM * 16;                    // per row {E_0, E_1, 2*c_0, 2*c_1}
   // shared-memory map (offsets from a 1024-byte aligned base)
-  static constexpr int OFF_Q = 0;
-  static constexpr int OFF_QSF = OFF_Q + Q_BYTES;
-  static constexpr int OFF_P = OFF_QSF + 1024;
+  static constexpr int OFF_Q = 0;                               // two buffers
+  static constexpr int OFF_QSF = OFF_Q + 2 * Q_BYTES;           // two buffers of 1 KB
+  static constexpr int OFF_P = OFF_QSF + 2048;
   static constexpr int OFF_PSF = OFF_P + kTeams * P_BYTES;
-  static constexpr int OFF_META = OFF_PSF + kTeams * PSF_BYTES;
+  static constexpr int OFF_META = OFF_PSF + 2 * PSF_BYTES;
   static constexpr int OFF_STAGE = OFF_META + kTeams * META_BYTES;
   static constexpr int OFF_BAR = OFF_STAGE + NST * STAGE_BYTES;
   static constexpr int SMEM_BYTES = OFF_BAR + 1024 + 1024;      // barriers + alignment slack
   static constexpr uint64_t SWZ_QK = (ROW_BYTES == 64) ? kSwz64 : kSwz32;
-  static_assert(STAGE_BYTES % 512 == 0, "stage alignment");
+  static_assert(STAGE_BYTES % 512 == 0 && OFF_STAGE % 1024 == 0, "stage alignment");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
 };
 
@@ -72,13 +75,14 @@ struct AttnParams {
   __nv_bfloat16* O;
   float* LSE;
   int* status;
-  int N, tiles;            // keys, N / 64
+  int N, stages;           // keys, N / 128
+  int n_items;             // B * H * N / 128
   float c_base;            // fl32(log2(e) * softmax_scale)
 };
 
 // barrier slots (8 bytes each)
-enum { BAR_Q = 0, BAR_OFULL, BAR_SFULL0, BAR_SEMPTY0 = BAR_SFULL0 + kTeams, BAR_SMDONE0 = BAR_SEMPTY0 + kTeams,
-       BAR_PFULL0 = BAR_SMDONE0 + kTeams, BAR_PFREE0 = BAR_PFULL0 + kTeams, BAR_RING = BAR_PFREE0 + kTeams };
+enum { BAR_QFULL0 = 0, BAR_QFREE0 = 2, BAR_OFULL = 4, BAR_OFREE = 5, BAR_SFULL0 = 6, BAR_SEMPTY0 = 8,
+       BAR_PFULL0 = 10, BAR_PFREE0 = 12, BAR_SMDONE0 = 14, BAR_RING = BAR_SMDONE0 + kTeams };
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -155,25 +159,26 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   // descriptor templates: everything but the 14 address bits is loop-invariant
   constexpr uint64_t kDescSF = (uint64_t)(16 >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
   constexpr uint64_t kDescQK = (uint64_t)(16 >> 4) << 16 | (uint64_t)((8 * C::ROW_BYTES) >> 4) << 32 | 1ull << 46 | C::SWZ_QK << 61;
-  constexpr uint64_t kDescV = (uint64_t)(16 >> 4) << 16 | (uint64_t)(256 >> 4) << 32 | 1ull << 46 | kSwz32 << 61;
+  constexpr uint64_t kDescV = (uint64_t)(16 >> 4) << 16 | (uint64_t)(512 >> 4) << 32 | 1ull << 46 | kSwz64 << 61;
   constexpr uint64_t kDescP = (uint64_t)((BM * 16) >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
   auto at = [](uint64_t tmpl, uint32_t addr) { return tmpl | (uint64_t)((addr & 0x3FFFFu) >> 4); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qtiles = p.N / BM;
-  const int bh = blockIdx.x / qtiles, qt = blockIdx.x % qtiles;
-  const int T = p.tiles;
+  const int T2 = p.stages;
 
   if (threadIdx.x == 0) {
-    mbar_init(bar(BAR_Q), 1);
-    mbar_init(bar(BAR_OFULL), 1);
-    for (int t = 0; t < kTeams; ++t) {
-      mbar_init(bar(BAR_SFULL0 + t), 1);
-      mbar_init(bar(BAR_SEMPTY0 + t), 4);
-      mbar_init(bar(BAR_SMDONE0 + t), 4);
-      mbar_init(bar(BAR_PFULL0 + t), 4);
-      mbar_init(bar(BAR_PFREE0 + t), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar(BAR_QFULL0 + b), 1);
+      mbar_init(bar(BAR_QFREE0 + b), 1);
+      mbar_init(bar(BAR_SFULL0 + b), 1);
+      mbar_init(bar(BAR_SEMPTY0 + b), 8);      // both teams of the pair, four warps each
+      mbar_init(bar(BAR_PFULL0 + b), 8);       // four correction warps, two tiles
+      mbar_init(bar(BAR_PFREE0 + b), 1);
     }
+    mbar_init(bar(BAR_OFULL), 1);
+    mbar_init(bar(BAR_OFREE), 4);
+    for (int t = 0; t < kTeams; ++t) mbar_init(bar(BAR_SMDONE0 + t), 4);
     for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
     *abortf = 0;
     fence_barrier_init();
@@ -190,79 +195,88 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (warp == 0) {
     // ===================================================================== TMA producer
     // The whole warp runs the loop (addresses and waits stay warp-uniform); one elected lane issues.
-    {
+    int s = 0, ph = 0;
+    uint32_t gs = 0;                                            // stages issued so far (all items)
+    uint32_t st = sbase + C::OFF_STAGE;
+    bool ok = true;
+    int i = 0;
+    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
+      const int bh = item / qtiles, qt = item - bh * qtiles;
+      const int qb = i & 1;
+      if (i >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_QFREE0 + qb), ((i >> 1) - 1) & 1, abortf));
+      if (!ok) break;
       if (elect_one()) {
-        mbar_arrive_expect_tx(bar(BAR_Q), C::Q_BYTES + C::QSF_BYTES);
-        tma_load_2d(sbase + C::OFF_Q, &tmQ, 0, bh * p.N + qt * BM, bar(BAR_Q));
-        bulk_load_1d(sbase + C::OFF_QSF, p.q_sf + ((size_t)bh * qtiles + qt) * C::QSF_BYTES, C::QSF_BYTES, bar(BAR_Q));
+        mbar_arrive_expect_tx(bar(BAR_QFULL0 + qb), C::Q_BYTES + C::QSF_BYTES);
+        tma_load_2d(sbase + C::OFF_Q + qb * C::Q_BYTES, &tmQ, 0, bh * p.N + qt * BM, bar(BAR_QFULL0 + qb));
+        bulk_load_1d(sbase + C::OFF_QSF + qb * 1024, p.q_sf + (size_t)item * C::QSF_BYTES, C::QSF_BYTES, bar(BAR_QFULL0 + qb));
       }
       const uint8_t* ksf = p.k_sf + (size_t)bh * qtiles * C::KSF_BYTES;
       const uint8_t* vsf = p.v_sf + (size_t)bh * qtiles * C::VSF_BYTES;
       const int krow0 = bh * p.N, vrow0 = bh * D;
-      int issued = 0, s = 0, ph = 0;
-      uint32_t st = sbase + C::OFF_STAGE;
-      for (int j = 0; j < T; ++j) {
-        if (j >= C::NST && !__all_sync(0xffffffffu, mbar_wait(bar_empty(s), ph ^ 1, abortf))) break;
+      for (int s2 = 0; s2 < T2; ++s2, ++gs) {
+        if (gs >= (uint32_t)C::NST) ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(s), ph ^ 1, abortf));
+        if (!ok) break;
         const uint32_t fb = bar_full(s);
         if (elect_one()) {
           mbar_arrive_expect_tx(fb, C::STAGE_BYTES);
-          tma_load_2d(st, &tmK, 0, krow0 + j * BN, fb);
-          tma_load_2d(st + C::K_BYTES, &tmV, j * (BN / 2), vrow0, fb);
-          bulk_load_1d(st + C::K_BYTES + C::V_BYTES, ksf + (size_t)(j >> 1) * C::KSF_BYTES, C::KSF_BYTES, fb);
-          bulk_load_1d(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, vsf + (size_t)(j >> 1) * C::VSF_BYTES, C::VSF_BYTES, fb);
+          tma_load_2d(st, &tmK, 0, krow0 + s2 * BS, fb);
+          tma_load_2d(st + C::K_BYTES, &tmV, s2 * (BS / 2), vrow0, fb);
+          bulk_load_1d(st + C::K_BYTES + C::V_BYTES, ksf + (size_t)s2 * C::KSF_BYTES, C::KSF_BYTES, fb);
+          bulk_load_1d(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, vsf + (size_t)s2 * C::VSF_BYTES, C::VSF_BYTES, fb);
         }
-        issued = j + 1;
         st += C::STAGE_BYTES;
         if (++s == C::NST) { s = 0; ph ^= 1; st = sbase + C::OFF_STAGE; }
       }
-      if (*abortf && lane == 0) {
-        // bounded drain of copies still in flight before the CTA retires
-        for (int j = max(0, issued - C::NST); j < issued; ++j)
-          for (int spin = 0; spin < (1 << 14) && !mbar_try_wait(bar_full(j % C::NST), (j / C::NST) & 1); ++spin) {}
-      }
+    }
+    if (*abortf && lane == 0) {
+      // bounded drain: give copies still in flight time to land before the CTA retires
+      for (int r = 0; r < C::NST; ++r)
+        for (int spin = 0; spin < (1 << 12) && !mbar_try_wait(bar_full(r), 0) && !mbar_try_wait(bar_full(r), 1); ++spin) {}
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ===================================================================== QK issuer: S(j) = Q K(j)^T
+    // ===================================================================== QK issuer: S = Q K^T, one stage per issue
     // Warp-uniform control flow; tcgen05 instructions are issued by one elected lane.
-    {
-      const uint64_t dQ0 = at(kDescQK, sbase + C::OFF_Q), dQ1 = at(kDescQK, sbase + C::OFF_Q + 32);
-      constexpr uint32_t kIdQK0 = NV ? make_idesc_fp4(BM, BN, false, 0, 0) : make_idesc_fp4(BM, BN, true, 0, 0);
-      constexpr uint32_t kIdQK1 = NV ? make_idesc_fp4(BM, BN, false, 0, 0) : make_idesc_fp4(BM, BN, true, 2, 2);
-      bool ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_Q), 0, abortf));
-      if (ok) {
-        tc_fence_after();
-        if (elect_one()) {
+    constexpr uint32_t kIdQK0 = NV ? make_idesc_fp4(BM, BS, false, 0, 0) : make_idesc_fp4(BM, BS, true, 0, 0);
+    constexpr uint32_t kIdQK1 = NV ? make_idesc_fp4(BM, BS, false, 0, 0) : make_idesc_fp4(BM, BS, true, 2, 2);
+    int sq = 0, phq = 0;
+    uint32_t stq = sbase + C::OFF_STAGE;
+    uint32_t g = 0;                                             // stages issued so far (all items)
+    bool ok = true;
+    int i = 0;
+    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
+      const int qb = i & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_QFULL0 + qb), (i >> 1) & 1, abortf));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t tSFQ = tmem + kColSFQ + 8 * qb;
+      if (elect_one()) {
 #pragma unroll
-          for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tmem + kColSFQ + 4 * a, at(kDescSF, sbase + C::OFF_QSF + 512 * a));
-        }
+        for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFQ + 4 * a, at(kDescSF, sbase + C::OFF_QSF + qb * 1024 + 512 * a));
       }
-      int sq = 0, phq = 0;
-      uint32_t stq = sbase + C::OFF_STAGE;
-      for (int j = 0; ok && j < T; ++j) {
-        const int slot = j & (kTeams - 1), k = j >> 2;
+      const uint64_t dQ0 = at(kDescQK, sbase + C::OFF_Q + qb * C::Q_BYTES);
+      for (int s2 = 0; s2 < T2; ++s2, ++g) {
+        const int pr = g & 1;
+        const uint32_t m = g >> 1;
         ok = __all_sync(0xffffffffu, mbar_wait(bar_full(sq), phq, abortf));
-        if (ok && k > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SEMPTY0 + slot), (k - 1) & 1, abortf));   // team has read S(j-4)
+        if (ok && m > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SEMPTY0 + pr), (m - 1) & 1, abortf));   // both teams have read the pair
         if (!ok) break;
         tc_fence_after();
-        // one scale atom covers the 128-key pair: copied by the even tile, reused by the odd one
-        const uint32_t tSFK = tmem + kColSFK + 8 * ((j >> 1) & 1);
-        const uint32_t sfb = tSFK + 2 * (j & 1);                // keys 64..127 of the pair sit two columns on
-        const uint32_t tS = tmem + kColS + BN * slot;
+        const uint32_t tSFK = tmem + kColSFK + 8 * pr;
+        const uint32_t tS = tmem + kColS + BS * pr;
         const uint64_t dK0 = at(kDescQK, stq);
         if (elect_one()) {
-          if (!(j & 1)) {
 #pragma unroll
-            for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFK + 4 * a, at(kDescSF, stq + C::K_BYTES + C::V_BYTES + 512 * a));
-          }
+          for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFK + 4 * a, at(kDescSF, stq + C::K_BYTES + C::V_BYTES + 512 * a));
           if (NV) {
-            tc_mma_fp4_4x(tS, dQ0, dK0, kIdQK0, tmem + kColSFQ, sfb, 0);
-            if (C::KBLK == 2) tc_mma_fp4_4x(tS, dQ1, dK0 + 2, kIdQK1, tmem + kColSFQ + 4, sfb + 4, 1);
+            tc_mma_fp4_4x(tS, dQ0, dK0, kIdQK0, tSFQ, tSFK, 0);
+            if (C::KBLK == 2) tc_mma_fp4_4x(tS, dQ0 + 2, dK0 + 2, kIdQK1, tSFQ + 4, tSFK + 4, 1);
           } else {
-            tc_mma_fp4_2x(tS, dQ0, dK0, kIdQK0, tmem + kColSFQ, sfb, 0);
-            if (C::KBLK == 2) tc_mma_fp4_2x(tS, dQ1, dK0 + 2, kIdQK1, tmem + kColSFQ, sfb, 1);
+            tc_mma_fp4_2x(tS, dQ0, dK0, kIdQK0, tSFQ, tSFK, 0);
+            if (C::KBLK == 2) tc_mma_fp4_2x(tS, dQ0 + 2, dK0 + 2, kIdQK1, tSFQ, tSFK, 1);
           }
-          tc_commit(bar(BAR_SFULL0 + slot));
+          tc_commit(bar(BAR_SFULL0 + pr));
+          if (s2 == T2 - 1) tc_commit(bar(BAR_QFREE0 + qb));    // Q buffer may take the item after next
         }
         __syncwarp();
         stq += C::STAGE_BYTES;
@@ -271,28 +285,34 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     __syncwarp();
   } else if (warp == 2) {
-    // ===================================================================== PV issuer: O += P(j) V(j)
-    {
-      constexpr uint32_t kIdPV0 = make_idesc_fp4(BM, D, true, 0, 0), kIdPV1 = make_idesc_fp4(BM, D, true, 0, 2);
-      const uint32_t tO = tmem + kColO;
-      int sp = 0;
-      uint32_t stp = sbase + C::OFF_STAGE;
-      bool ok = true;
-      for (int j = 0; ok && j < T; ++j) {
-        const int slot = j & (kTeams - 1), k = j >> 2;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFULL0 + slot), k & 1, abortf));  // codes and scale bytes of P(j) are in smem
+    // ===================================================================== PV issuer: O += P V, one stage per issue
+    constexpr uint32_t kIdPV0 = make_idesc_fp4(BM, D, true, 0, 0), kIdPV1 = make_idesc_fp4(BM, D, true, 2, 2);
+    const uint32_t tO = tmem + kColO;
+    int sp = 0;
+    uint32_t stp = sbase + C::OFF_STAGE;
+    uint32_t g = 0;
+    bool ok = true;
+    int i = 0;
+    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
+      if (i >= 1) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFREE), (i - 1) & 1, abortf));   // epilogue has read O
+      for (int s2 = 0; ok && s2 < T2; ++s2, ++g) {
+        const int pr = g & 1;
+        const uint32_t m = g >> 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFULL0 + pr), m & 1, abortf));   // codes and scale bytes of both tiles are in smem
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tSFP = tmem + kColSFP + 4 * slot, tSFV = tmem + kColSFV + 4 * ((j >> 1) & 1);
+        const uint32_t tSFP = tmem + kColSFP + 4 * pr, tSFV = tmem + kColSFV + 4 * pr;
+        const uint64_t dV = at(kDescV, stp + C::K_BYTES);
+        const uint64_t dP = at(kDescP, sbase + C::OFF_P + C::P_BYTES * 2 * pr);
         if (elect_one()) {
-          tc_cp_32x128b_warpx4(tSFP, at(kDescSF, sbase + C::OFF_PSF + 512 * slot));
-          if (!(j & 1)) tc_cp_32x128b_warpx4(tSFV, at(kDescSF, stp + C::K_BYTES + C::V_BYTES + C::KSF_BYTES));
-          // P scales: bytes 0,1 of its atom; V scales: bytes 2*(j&1).. of the pair's atom
-          tc_mma_fp4_2x(tO, at(kDescP, sbase + C::OFF_P + C::P_BYTES * slot), at(kDescV, stp + C::K_BYTES),
-                        (j & 1) ? kIdPV1 : kIdPV0, tSFP, tSFV, j > 0);
-          tc_commit(bar_empty(sp));                               // K(j), V(j) stage back to the producer
-          tc_commit(bar(BAR_PFREE0 + slot));                      // P slot reusable; O holds tiles <= j
-          if (j == T - 1) tc_commit(bar(BAR_OFULL));
+          tc_cp_32x128b_warpx4(tSFP, at(kDescSF, sbase + C::OFF_PSF + 512 * pr));
+          tc_cp_32x128b_warpx4(tSFV, at(kDescSF, stp + C::K_BYTES + C::V_BYTES + C::KSF_BYTES));
+          // tile h of the stage: P slot 2*pr+h, keys 64h..64h+63 of V^T (32 bytes on), scale bytes {2h, 2h+1}
+          tc_mma_fp4_2x(tO, dP, dV, kIdPV0, tSFP, tSFV, s2 > 0);
+          tc_mma_fp4_2x(tO, dP + (C::P_BYTES >> 4), dV + 2, kIdPV1, tSFP, tSFV, 1);
+          tc_commit(bar_empty(sp));                             // stage back to the producer
+          tc_commit(bar(BAR_PFREE0 + pr));                      // P slots reusable; O holds this stage
+          if (s2 == T2 - 1) tc_commit(bar(BAR_OFULL));
         }
         __syncwarp();
         stp += C::STAGE_BYTES;
@@ -308,112 +328,140 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const uint32_t tO = tmem + ((uint32_t)(quarter * 32) << 16) + kColO;
-    int mu = -(1 << 28);
-    float L2 = 0.f;                                             // sum of 2^(E_B - mu) * (2 * code sum)
+    uint32_t g0 = 0;                                            // stages completed in earlier items
     bool ok = true;
-    for (int j = 0; j < T; ++j) {
-      const int slot = j & (kTeams - 1), k = j >> 2;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + slot), k & 1, abortf));
-      if (!ok) break;
-      const int4 m = *reinterpret_cast<const int4*>(sgen + C::OFF_META + C::META_BYTES * slot + row * 16);
-      const int Emax = max(m.x, m.y);
-      const bool need = Emax > mu + kLazyShift;
-      if (__any_sync(0xffffffffu, need)) {
-        float f = 1.0f;
-        if (need) {
-          const int delta = Emax - mu;
-          f = (delta > 126) ? 0.f : __uint_as_float((uint32_t)(127 - delta) << 23);
-          mu = Emax;
-          L2 *= f;
-        }
-        if (j > 0) {
-          ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFREE0 + ((j - 1) & 3)), ((j - 1) >> 2) & 1, abortf));   // PV(j-1) has landed
-          if (!ok) break;
-          tc_fence_after();
-#pragma unroll 1
-          for (int c0 = 0; c0 < D; c0 += 16) {
-            uint32_t o[16];
-            tmem_ld_32x32b_x16(tO + c0, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-            tmem_st_32x32b_x16(tO + c0, o);
+    int i = 0;
+    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i, g0 += T2) {
+      int mu = -(1 << 28);
+      float L2 = 0.f;                                           // sum of 2^(E_B - mu) * (2 * code sum)
+      int pu0 = 0, pu1 = 0;                                     // bytes written for the previous tile
+      for (int j = 0; j < 2 * T2; ++j) {
+        const uint32_t g = g0 + (j >> 1);
+        const int h = j & 1, pr = g & 1, slot = 2 * pr + h;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + slot), (g >> 1) & 1, abortf));
+        if (!ok) break;
+        const int4 mt = *reinterpret_cast<const int4*>(sgen + C::OFF_META + C::META_BYTES * slot + row * 16);
+        uint8_t* psf = sgen + C::OFF_PSF + 512 * pr + lane * 16 + quarter * 4;
+        const int Emax = max(mt.x, mt.y);
+        const bool need = Emax > mu + kLazyShift;
+        if (__any_sync(0xffffffffu, need)) {
+          float f = 1.0f;
+          if (need) {
+            const int delta = Emax - mu;
+            f = (delta > 126) ? 0.f : __uint_as_float((uint32_t)(127 - delta) << 23);
+            mu = Emax;
+            L2 *= f;
+            if (h) {
+              // the stage's first tile is not in O yet (both tiles are issued together): move its bytes
+              pu0 = max(pu0 - delta, 0);
+              pu1 = max(pu1 - delta, 0);
+              *reinterpret_cast<uint16_t*>(psf) = (uint16_t)(pu0 | (pu1 << 8));
+            }
           }
-          tmem_wait_st();
-          tc_fence_before();
+          if (j >= 2) {
+            // O holds the item's earlier stages once their PV has landed
+            const uint32_t gprev = g - 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFREE0 + (gprev & 1)), (gprev >> 1) & 1, abortf));
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int c0 = 0; c0 < D; c0 += 16) {
+              uint32_t o[16];
+              tmem_ld_32x32b_x16(tO + c0, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int q = 0; q < 16; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * f);
+              tmem_st_32x32b_x16(tO + c0, o);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+          }
         }
+        // A block more than 126 octaves below the reference is a zero block: it gets the smallest
+        // byte (2^-127, below 2^-60 of the row's mass by construction) and no share of the row sum.
+        const int u0 = mt.x - mu + 127, u1 = mt.y - mu + 127;
+        if (u0 >= 1) L2 = fmaf((float)mt.z, __uint_as_float((uint32_t)u0 << 23), L2);
+        if (u1 >= 1) L2 = fmaf((float)mt.w, __uint_as_float((uint32_t)u1 << 23), L2);
+        pu0 = max(u0, 0);
+        pu1 = max(u1, 0);
+        *reinterpret_cast<uint16_t*>(psf + 2 * h) = (uint16_t)(pu0 | (pu1 << 8));
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + pr));
       }
-      // A block more than 126 octaves below the reference is a zero block: it gets the smallest
-      // byte (2^-127, below 2^-60 of the row's mass by construction) and no share of the row sum.
-      const int u0 = m.x - mu + 127, u1 = m.y - mu + 127;
-      if (u0 >= 1) L2 = fmaf((float)m.z, __uint_as_float((uint32_t)u0 << 23), L2);
-      if (u1 >= 1) L2 = fmaf((float)m.w, __uint_as_float((uint32_t)u1 << 23), L2);
-      *reinterpret_cast<uint32_t*>(sgen + C::OFF_PSF + 512 * slot + lane * 16 + quarter * 4) =
-          (uint32_t)max(u0, 0) | ((uint32_t)max(u1, 0) << 8);
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + slot));
-    }
-    // ---- epilogue: O = O_hw / (3 * L2), LSE = ln2 * (mu + log2(L2 / 12))
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFULL), 0, abortf));
-    if (ok) {
+      if (!ok) break;
+      // ---- epilogue: O = O_hw / (3 * L2), LSE = ln2 * (mu + log2(L2 / 12))
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFULL), i & 1, abortf));
+      if (!ok) break;
       tc_fence_after();
       const float inv = __frcp_rn(3.0f * L2);
-      const size_t grow = (size_t)bh * p.N + (size_t)qt * BM + row;
+      const size_t grow = (size_t)item * BM + row;
       __nv_bfloat16* orow = p.O + grow * D;
 #pragma unroll 1
       for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t o[32];
         tmem_ld_32x32b_x32(tO + c0, o);
         tmem_wait_ld();
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(o[2 * i]) * inv, __uint_as_float(o[2 * i + 1]) * inv);
-          pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+        if (c0 + 32 == D) {                                     // last read of O: the next item's PV may overwrite it
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(BAR_OFREE));
         }
 #pragma unroll
-        for (int v = 0; v < 4; ++v)
-          *reinterpret_cast<uint4*>(orow + c0 + 8 * v) = make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
+        for (int c = 0; c < 32; c += 8) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[c + 2 * q]) * inv, __uint_as_float(o[c + 2 * q + 1]) * inv);
+            pk[q] = *reinterpret_cast<const uint32_t*>(&hh);
+          }
+          *reinterpret_cast<uint4*>(orow + c0 + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
       }
       if (p.LSE) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(L2) - 3.5849625007211560f));
-      tc_fence_before();
     }
   } else {
     // ===================================================================== softmax teams
     const int team = (warp - kFirstSoftmaxWarp) >> 2;
+    const int pr = team >> 1, h = team & 1;
     const int quarter = warp & 3;                               // TMEM lane quarter this warp may touch
     const int row = quarter * 32 + lane;
     const uint32_t tS = tmem + ((uint32_t)(quarter * 32) << 16) + kColS + BN * team;
-    const uint32_t sfull = bar(BAR_SFULL0 + team), sempty = bar(BAR_SEMPTY0 + team);
-    const uint32_t smdone = bar(BAR_SMDONE0 + team), pfree = bar(BAR_PFREE0 + team);
+    const uint32_t sfull = bar(BAR_SFULL0 + pr), sempty = bar(BAR_SEMPTY0 + pr);
+    const uint32_t smdone = bar(BAR_SMDONE0 + team), pfree = bar(BAR_PFREE0 + pr);
     uint8_t* pbuf = sgen + C::OFF_P + C::P_BYTES * team + row * 16;
     int4* meta = reinterpret_cast<int4*>(sgen + C::OFF_META + C::META_BYTES * team + row * 16);
     float c32;
     if (NV) c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G), __ldg(p.k_G)));
     else    c32 = __fdiv_rn(p.c_base, 36.0f);
-    uint32_t ph = 0;
-    for (int j = team; j < T; j += kTeams, ph ^= 1) {
-      if (!__all_sync(0xffffffffu, mbar_wait(sfull, ph, abortf))) break;
-      tc_fence_after();
-      uint32_t sraw[32], w0[4], w1[4];
-      int E0, E1, c0, c1;
-      tmem_ld_32x32b_x32(tS, sraw);
-      tmem_wait_ld();
-      direct_p_block(sraw, c32, E0, w0, c0);
-      tmem_ld_32x32b_x32(tS + 32, sraw);
-      tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(sempty);                       // slot may take S(j+4)
-      direct_p_block(sraw, c32, E1, w1, c1);
-      if (j >= kTeams && !__all_sync(0xffffffffu, mbar_wait(pfree, ph ^ 1, abortf))) break;   // PV(j-4) consumed the slot
-      *reinterpret_cast<uint4*>(pbuf) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
-      *reinterpret_cast<uint4*>(pbuf + BM * 16) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
-      *meta = make_int4(E0, E1, c0, c1);
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smdone);
+    uint32_t g0 = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, g0 += T2) {
+      for (uint32_t g = g0 + ((g0 & 1) != (uint32_t)pr); g < g0 + T2; g += 2) {   // this team's stages of the item
+        const uint32_t m = g >> 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(sfull, m & 1, abortf));
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t sraw[32], w0[4], w1[4];
+        int E0, E1, c0, c1;
+        tmem_ld_32x32b_x32(tS, sraw);
+        tmem_wait_ld();
+        direct_p_block(sraw, c32, E0, w0, c0);
+        tmem_ld_32x32b_x32(tS + 32, sraw);
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sempty);                     // pair may take the stage after next
+        direct_p_block(sraw, c32, E1, w1, c1);
+        if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
+        if (!ok) break;
+        *reinterpret_cast<uint4*>(pbuf) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
+        *reinterpret_cast<uint4*>(pbuf + BM * 16) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+        *meta = make_int4(E0, E1, c0, c1);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smdone);
+      }
     }
   }
   __syncthreads();
@@ -501,10 +549,13 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
   CUtensorMap tmQ, tmK, tmV;
   const uint64_t rows = (uint64_t)B * H * N;
   if (!make_map(&tmQ, ops->q, C::ROW_BYTES, rows, C::ROW_BYTES, BM) ||
-      !make_map(&tmK, ops->k, C::ROW_BYTES, rows, C::ROW_BYTES, BN) ||
-      !make_map(&tmV, ops->v, (uint64_t)N / 2, (uint64_t)B * H * D, BN / 2, D))
+      !make_map(&tmK, ops->k, C::ROW_BYTES, rows, C::ROW_BYTES, BS) ||
+      !make_map(&tmV, ops->v, (uint64_t)N / 2, (uint64_t)B * H * D, BS / 2, D))
     return FP4ATTN_ERR_CUDA;
-  const unsigned grid = (unsigned)(B * H * (N / BM));
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return FP4ATTN_ERR_CUDA;
+  const unsigned grid = (unsigned)(prm.n_items < sms ? prm.n_items : sms);     // persistent: one CTA per SM
   attn_fwd_kernel<D, NV><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, prm);
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
@@ -532,7 +583,7 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.q_sf = (const uint8_t*)ops->q_sf; prm.k_sf = (const uint8_t*)ops->k_sf; prm.v_sf = (const uint8_t*)ops->v_sf;
   prm.q_G = ops->q_G; prm.k_G = ops->k_G;
   prm.O = (__nv_bfloat16*)O; prm.LSE = LSE; prm.status = device_status;
-  prm.N = N; prm.tiles = N / BN;
+  prm.N = N; prm.stages = N / BS; prm.n_items = B * H * (N / BM);
   const float scale = ops->softmax_scale > 0.f ? ops->softmax_scale : (float)(1.0 / sqrt((double)d));
   prm.c_base = 1.4426950408889634f * scale;                        // fl32(log2e_32 * scale_32)
   cudaStream_t st = (cudaStream_t)stream;
