@@ -90,6 +90,38 @@ int fp4attn_quantize(const void* x_bf16, int fmt, int role, int B, int H, int N,
                      void* packed_out, void* scales_out, float* tensor_scale_out,
                      void* workspace, size_t workspace_bytes, fp4attn_stream_t stream);
 
+/* Largest tensor fp4attn_quantize_nvfp4_noalloc accepts: 2^27 elements. */
+#define FP4ATTN_NOALLOC_MAX_ELEMENTS (1ull << 27)
+
+/*
+ * NVFP4 quantizer for callers that cannot allocate device memory.  (The paper has no counterpart;
+ * this is a packaging variant of fp4attn_quantize with fmt = FP4ATTN_FMT_NVFP4, same bytes out.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a region whose memory
+ * budget is fixed up front, under a framework whose allocator must not be bypassed, or in a
+ * latency-critical loop where an allocation would synchronise the device.  fp4attn_quantize asks
+ * such callers for a workspace they have no means to provide.
+ *
+ * What it does instead: the tensor-wide amax pass keeps its per-block partial maxima in a 4 KB
+ * array that lives inside the library image (a file-scope __device__ array), so every GPU that
+ * loads the library carries those 4 KB until the process exits.  The array is sized for 1024
+ * partial maxima of at most 2^17 elements each; tensors with more than
+ * FP4ATTN_NOALLOC_MAX_ELEMENTS elements are rejected with FP4ATTN_ERR_WORKSPACE and nothing is
+ * launched.  The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ *
+ * The first call on each device looks up the array's device address (once per device, with that
+ * device current) before launching; make that first call outside any stream capture.
+ * All calls share the one array: its contents are whatever the previous call left (every slot a
+ * call reads it has first overwritten, so nothing needs clearing), and two calls whose kernels
+ * overlap on the GPU - different streams, or different host threads - race on it.  Serialise them.
+ *
+ * x_bf16 [B,H,N,d]; role is FP4ATTN_ROLE_Q or FP4ATTN_ROLE_K; packed_out, scales_out and
+ * tensor_scale_out as for fp4attn_quantize.
+ */
+int fp4attn_quantize_nvfp4_noalloc(const void* x_bf16, int role, int B, int H, int N, int d,
+                                   void* packed_out, void* scales_out, float* tensor_scale_out,
+                                   fp4attn_stream_t stream);
+
 typedef struct {
   const void *q, *k, *v;            /* packed E2M1 (V transposed)                           */
   const void *q_sf, *k_sf, *v_sf;   /* scale atoms                                           */

@@ -23,6 +23,7 @@ EXPORTS = [
     "fp4attn_status_string", "fp4attn_version", "fp4attn_packed_bytes", "fp4attn_scale_bytes",
     "fp4attn_quantize_workspace_bytes", "fp4attn_quantize", "fp4attn_fwd",
     "fp4attn_attention_host_workspace_bytes", "fp4attn_attention_host", "fp4attn_mma_peak_probe",
+    "fp4attn_quantize_nvfp4_noalloc",
 ]
 
 
@@ -60,6 +61,8 @@ def _load() -> ctypes.CDLL:
     lib.fp4attn_attention_host_workspace_bytes.argtypes = [i, i, i, i, i]
     lib.fp4attn_attention_host.restype = i
     lib.fp4attn_attention_host.argtypes = [vp, vp, vp, i, ctypes.c_float, i, i, i, i, vp, vp, vp, sz, vp]
+    lib.fp4attn_quantize_nvfp4_noalloc.restype = i
+    lib.fp4attn_quantize_nvfp4_noalloc.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp]
     lib.fp4attn_mma_peak_probe.restype = i
     lib.fp4attn_mma_peak_probe.argtypes = [i, vp, vp]
     return lib
@@ -118,6 +121,17 @@ def fp4attn_quantize(x: torch.Tensor, fmt: int, role: int, workspace: Optional[t
                               _ptr(G), _ptr(workspace), 0 if workspace is None else workspace.numel(), _stream()),
            "fp4attn_quantize")
     return QuantizedOperand(packed, scales, G, fmt, role, (B, H, N, d))
+
+
+def fp4attn_quantize_nvfp4_noalloc(x: torch.Tensor, role: int, packed: torch.Tensor, scales: torch.Tensor,
+                                   G: torch.Tensor) -> QuantizedOperand:
+    """NVFP4 quantizer that allocates nothing: the caller passes every output buffer and the library
+    uses its built-in 4 KB scratch.  For callers that must not touch the CUDA allocator."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 4
+    B, H, N, d = x.shape
+    _check(lib().fp4attn_quantize_nvfp4_noalloc(x.data_ptr(), role, B, H, N, d, packed.data_ptr(), scales.data_ptr(),
+                                                G.data_ptr(), _stream()), "fp4attn_quantize_nvfp4_noalloc")
+    return QuantizedOperand(packed, scales, G, FMT_NVFP4, role, (B, H, N, d))
 
 
 def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, softmax_scale: float = 0.0,

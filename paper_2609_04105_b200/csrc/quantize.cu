@@ -279,3 +279,29 @@ extern "C" int fp4attn_quantize(const void* x, int fmt, int role, int B, int H, 
   if (rc != FP4ATTN_OK) return rc;
   return launch_quantize(x, fmt, role, B, H, N, d, packed, scales, G_out, (float*)workspace, (cudaStream_t)stream);
 }
+
+// ---------------------------------------------------------------- allocation-free NVFP4 variant
+// Scratch for the amax pass lives in the library image.  In host code the symbol below is only a
+// handle; the device address is fetched once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) float g_noalloc_partials[kMaxPartials];
+
+extern "C" int fp4attn_quantize_nvfp4_noalloc(const void* x, int role, int B, int H, int N, int d, void* packed,
+                                              void* scales, float* G_out, fp4attn_stream_t stream) {
+  int rc = validate_quantize(x, FP4ATTN_FMT_NVFP4, role, B, H, N, d, packed, scales, G_out);
+  if (rc != FP4ATTN_OK) return rc;
+  if ((unsigned long long)B * H * N * d > FP4ATTN_NOALLOC_MAX_ELEMENTS) return FP4ATTN_ERR_WORKSPACE;
+  rc = check_device_sm100();
+  if (rc != FP4ATTN_OK) return rc;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FP4ATTN_ERR_CUDA;
+  constexpr int kMaxDevices = 64;
+  static float* scratch_addr[kMaxDevices] = {};          // per-device address of g_noalloc_partials
+  if (dev < 0 || dev >= kMaxDevices) return FP4ATTN_ERR_INVALID_ARG;
+  if (!scratch_addr[dev]) {
+    float* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_noalloc_partials) != cudaSuccess || !ptr) return FP4ATTN_ERR_CUDA;
+    scratch_addr[dev] = ptr;
+  }
+  return launch_quantize(x, FP4ATTN_FMT_NVFP4, role, B, H, N, d, packed, scales, G_out, scratch_addr[dev],
+                         (cudaStream_t)stream);
+}
