@@ -32,7 +32,7 @@ constexpr int BM = 128;          // query rows per work item
 constexpr int BN = 64;           // keys per score tile (two N32 probability blocks)
 constexpr int BS = 128;          // keys per stage
 constexpr int kTeams = 4;        // score slots / softmax teams
-constexpr int kFirstCorrWarp = 3, kFirstSoftmaxWarp = 7;
+constexpr int kFirstSoftmaxWarp = 7;     // warps 3..6 are the correction warps
 constexpr int kAttnThreads = 32 * (kFirstSoftmaxWarp + 4 * kTeams);
 constexpr int kLazyShift = 64;   // the row reference follows the running maximum only when it is
                                  // more than this many octaves behind (rescales are exact powers of 2)
@@ -423,7 +423,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   } else {
     // ===================================================================== softmax teams
     const int team = (warp - kFirstSoftmaxWarp) >> 2;
-    const int pr = team >> 1, h = team & 1;
+    const int pr = team >> 1;                                   // stage parity this team serves (keys 64*(team&1)..)
     const int quarter = warp & 3;                               // TMEM lane quarter this warp may touch
     const int row = quarter * 32 + lane;
     const uint32_t tS = tmem + ((uint32_t)(quarter * 32) << 16) + kColS + BN * team;

@@ -16,48 +16,59 @@ __device__ __forceinline__ float amax8(const float* v) {
   return a;
 }
 
-// byte offset of the scale of (row r, scale column c) inside one (b,h) scale grid with CT column atoms
-__device__ __forceinline__ size_t sf_offset(int r, int c, int CT) {
-  return (size_t)((r >> 7) * CT + (c >> 2)) * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4 + (c & 3);
+// ---------------------------------------------------------------- MXFP4, blocks along d (Q, K)
+// |bf16| bit patterns order like the magnitudes, so the block maximum is taken on packed 16-bit
+// integers; 6 v / alpha = v * (1.5 * 2^(129-u)) is one exact fp32 multiply.
+__device__ __forceinline__ uint32_t absmax_bf16x8(const uint4& r) {
+  const uint32_t m = __vmaxu2(__vmaxu2(r.x & 0x7FFF7FFFu, r.y & 0x7FFF7FFFu), __vmaxu2(r.z & 0x7FFF7FFFu, r.w & 0x7FFF7FFFu));
+  return max(m & 0xFFFFu, m >> 16);
+}
+// E8M0 byte from the bf16 bit pattern of the block maximum (see mx_scale_byte)
+__device__ __forceinline__ uint32_t mx_scale_byte_bf16(uint32_t a16) {
+  if (a16 == 0) return 0;
+  const uint32_t u = (a16 >> 7) + ((a16 & 0x7Fu) != 0 ? 1u : 0u);
+  return min(max(u, 1u), 254u);
+}
+__device__ __forceinline__ uint32_t mx_codes_x8(const uint4& raw, uint32_t u) {
+  float v[8];
+  bf16x8_to_f32(raw, v);
+  if (u >= 2u) {
+    const float s6 = __uint_as_float(((256u - u) << 23) | 0x400000u);   // 1.5 * 2^(129-u) = 6 / alpha
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] *= s6;
+  } else {                                                              // alpha = 2^-126: 6/alpha overflows fp32
+    const float inv = mx_inv_amplitude(u);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = (v[i] * inv) * 6.0f;
+  }
+  return cvt_e2m1x8(v);
 }
 
-// ---------------------------------------------------------------- MXFP4, blocks along d (Q, K)
+// grid (N * D/8 / kGroupsPerCta, B*H)
 template <int D>
 __global__ void __launch_bounds__(kThreads)
 quant_mx_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
                      uint8_t* __restrict__ sf, int N) {
   constexpr int GPR = D / 8;                       // 8-element groups per row
-  const size_t base = (size_t)blockIdx.x * kGroupsPerCta + threadIdx.x;
+  const uint32_t bh = blockIdx.y;
+  const uint32_t gl = blockIdx.x * kGroupsPerCta + threadIdx.x;
+  const size_t gbase = (size_t)bh * N * GPR;
+  uint8_t* sfb = sf + (size_t)bh * (N / 128) * 512;
   uint4 raw[kGroupsPerThread];
 #pragma unroll
-  for (int k = 0; k < kGroupsPerThread; ++k) raw[k] = __ldg(x + base + (size_t)k * kThreads);
+  for (int k = 0; k < kGroupsPerThread; ++k) raw[k] = __ldg(x + gbase + gl + k * kThreads);
 #pragma unroll
   for (int k = 0; k < kGroupsPerThread; ++k) {
-    const size_t g = base + (size_t)k * kThreads;
-    float v[8];
-    bf16x8_to_f32(raw[k], v);
-    float a = amax8(v);
-    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
-    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
-    const uint32_t u = mx_scale_byte(a);
-    const float inv = mx_inv_amplitude(u);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = (v[i] * inv) * 6.0f;      // exact in fp32
-    packed[g] = cvt_e2m1x8(v);
-    // gather the row's D/32 scale bytes into one word, written by the row's first lane
-    const int lane = threadIdx.x & 31;
-    const int seg = (int)(g % GPR);
-    const int row_lane0 = lane - seg;
-    uint32_t word = 0;
-#pragma unroll
-    for (int b = 0; b < D / 32; ++b) word |= __shfl_sync(0xffffffffu, u, row_lane0 + 4 * b) << (8 * b);
-    if (seg == 0) {
-      const size_t row = g / GPR;
-      const size_t bh = row / N;
-      const int r = (int)(row % N);
-      uint8_t* p = sf + bh * (size_t)(N / 128) * 512 + sf_offset(r, 0, 1);
-      *reinterpret_cast<uint32_t*>(p) = word;                    // bytes beyond D/32 are zero padding
-    }
+    const uint32_t g = gl + k * kThreads;
+    uint32_t a = absmax_bf16x8(raw[k]);
+    a = max(a, __shfl_xor_sync(0xffffffffu, a, 1));
+    a = max(a, __shfl_xor_sync(0xffffffffu, a, 2));
+    const uint32_t u = mx_scale_byte_bf16(a);
+    packed[gbase + g] = mx_codes_x8(raw[k], u);
+    const uint32_t row = g / GPR, seg = g % GPR;
+    uint8_t* p = sfb + (row >> 7) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4;
+    if ((seg & 3) == 0) p[seg >> 2] = (uint8_t)u;                    // one lane per 32-block
+    if (D == 64 && (seg & 3) == 1) p[2 + (seg >> 2)] = 0;            // padding columns
   }
 }
 
@@ -142,6 +153,7 @@ __device__ __forceinline__ float e4m3_byte_to_f32(uint32_t b) {
 }
 
 // ---------------------------------------------------------------- NVFP4 pass 2, blocks of 16 along d (Q, K)
+// grid (N * D/8 / kGroupsPerCta, B*H)
 template <int D>
 __global__ void __launch_bounds__(kThreads)
 quant_nv_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed, uint8_t* __restrict__ sf,
@@ -161,41 +173,37 @@ quant_nv_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
       for (int i = 1; i < kThreads / 32; ++i) a = fmaxf(a, wmax[i]);
       const float G = (a == 0.f) ? 1.0f : __fdiv_rn(2688.0f, a);
       s_G = G;
-      if (blockIdx.x == 0) *G_out = G;
+      if (blockIdx.x == 0 && blockIdx.y == 0) *G_out = G;
     }
     __syncthreads();
   }
   const float G = s_G;
-  const size_t base = (size_t)blockIdx.x * kGroupsPerCta + threadIdx.x;
+  const uint32_t bh = blockIdx.y;
+  const uint32_t gl = blockIdx.x * kGroupsPerCta + threadIdx.x;
+  const size_t gbase = (size_t)bh * N * GPR;
+  uint8_t* sfb = sf + (size_t)bh * (N / 128) * CT * 512;
   uint4 raw[kGroupsPerThread];
 #pragma unroll
-  for (int k = 0; k < kGroupsPerThread; ++k) raw[k] = __ldg(x + base + (size_t)k * kThreads);
+  for (int k = 0; k < kGroupsPerThread; ++k) raw[k] = __ldg(x + gbase + gl + k * kThreads);
 #pragma unroll
   for (int k = 0; k < kGroupsPerThread; ++k) {
-    const size_t g = base + (size_t)k * kThreads;
-    float v[8];
-    bf16x8_to_f32(raw[k], v);
-    float a = amax8(v);
-    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+    const uint32_t g = gl + k * kThreads;
+    uint32_t a16 = absmax_bf16x8(raw[k]);
+    a16 = max(a16, __shfl_xor_sync(0xffffffffu, a16, 1));
+    const float a = __uint_as_float(a16 << 16);
     const float t = __fdiv_rn(__fmul_rn(a, G), 6.0f);
     const uint32_t sb = cvt_e4m3_byte(t);
     const float S = e4m3_byte_to_f32(sb);
     const float r = (S > 0.f) ? __fdiv_rn(G, S) : 0.f;
+    float v[8];
+    bf16x8_to_f32(raw[k], v);
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = __fmul_rn(v[i], r);       // sign rides along; 0*r = 0 for zero blocks
-    packed[g] = cvt_e2m1x8(v);
-    const int lane = threadIdx.x & 31;
-    const int seg = (int)(g % GPR);
-    const int wbase = lane - (seg & 7);                          // first lane of this 4-scale word
-    uint32_t word = 0;
-#pragma unroll
-    for (int b = 0; b < 4; ++b) word |= __shfl_sync(0xffffffffu, sb, wbase + 2 * b) << (8 * b);
-    if ((seg & 7) == 0) {
-      const size_t row = g / GPR;
-      const size_t bh = row / N;
-      const int rr = (int)(row % N);
-      uint8_t* p = sf + bh * (size_t)(N / 128) * CT * 512 + sf_offset(rr, (seg / 8) * 4, CT);
-      *reinterpret_cast<uint32_t*>(p) = word;
+    packed[gbase + g] = cvt_e2m1x8(v);
+    const uint32_t row = g / GPR, seg = g % GPR;
+    if ((seg & 1) == 0) {                                        // one lane per 16-block
+      const uint32_t c = seg >> 1;                               // scale column
+      sfb[((row >> 7) * CT + (c >> 2)) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4 + (c & 3)] = (uint8_t)sb;
     }
   }
 }
@@ -236,10 +244,11 @@ int launch_quantize(const void* x, int fmt, int role, int B, int H, int N, int d
                     float* G_out, float* partials, cudaStream_t st) {
   const size_t n_groups = (size_t)B * H * N * d / 8;
   const unsigned grid = (unsigned)(n_groups / kGroupsPerCta);
+  const dim3 grid2((unsigned)((size_t)N * d / 8 / kGroupsPerCta), (unsigned)(B * H));   // N % 128 == 0 makes this exact
   const uint4* xs = reinterpret_cast<const uint4*>(x);
   if (fmt == FP4ATTN_FMT_MXFP4 && role != FP4ATTN_ROLE_V) {
-    if (d == 128) quant_mx_rows_kernel<128><<<grid, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
-    else          quant_mx_rows_kernel<64><<<grid, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
+    if (d == 128) quant_mx_rows_kernel<128><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
+    else          quant_mx_rows_kernel<64><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
   } else if (fmt == FP4ATTN_FMT_MXFP4) {
     dim3 g2(N / 128, B * H);
     if (d == 128) quant_mx_v_kernel<128><<<g2, kThreads, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
@@ -247,8 +256,8 @@ int launch_quantize(const void* x, int fmt, int role, int B, int H, int N, int d
   } else {
     const int n_partials = (int)(grid < (unsigned)kMaxPartials ? grid : kMaxPartials);
     amax_partials_kernel<<<n_partials, kThreads, 0, st>>>(xs, n_groups, partials);
-    if (d == 128) quant_nv_rows_kernel<128><<<grid, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N);
-    else          quant_nv_rows_kernel<64><<<grid, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N);
+    if (d == 128) quant_nv_rows_kernel<128><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N);
+    else          quant_nv_rows_kernel<64><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N);
   }
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
