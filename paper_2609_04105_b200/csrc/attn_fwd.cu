@@ -18,8 +18,12 @@
 //                 the stages with parity p: Algorithm "direct-p-pack" up to the codes and their
 //                 sums; codes do not depend on the row reference, so teams never wait for one another
 //
-// Tensor memory (512 columns): S slots 0..255 | O 256..383 | Q scales 384..399 (two buffers) |
-// K scales 400..415 (two slots) | V scales 416..423 (two slots) | P scales 424..431 (two slots).
+// The represented row sum (the denominator of Eq. "represented-output") is produced by the same PV
+// instruction as the numerator: sixteen constant rows of ones follow V^T in every stage, so column d
+// of the accumulator is sum_j 2^(u_B-127) q_j over exactly the codes and scale bytes PV consumed.
+//
+// Tensor memory (512 columns): S slots 0..255 | O 256..399 (d + 16 columns) | Q scales 400..415 (two
+// buffers) | K scales 416..431 (two slots) | V scales 432..447 (two slots of 8) | P scales 448..455.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -37,7 +41,8 @@ constexpr int kAttnThreads = 32 * (kFirstSoftmaxWarp + 4 * kTeams);
 constexpr int kLazyShift = 64;   // the row reference follows the running maximum only when it is
                                  // more than this many octaves behind (rescales are exact powers of 2)
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256, kColSFQ = 384, kColSFK = 400, kColSFV = 416, kColSFP = 424;
+constexpr uint32_t kColS = 0, kColO = 256, kColSFQ = 400, kColSFK = 416, kColSFV = 432, kColSFP = 448;
+constexpr int kOnesRows = 16;    // rows of ones appended to V^T (the MMA's N must be a multiple of 16)
 
 template <int D, bool NV>
 struct Cfg {
@@ -48,20 +53,25 @@ struct Cfg {
   static constexpr int QSF_BYTES = CTQ * 512;
   static constexpr int K_BYTES = BS * ROW_BYTES;                // 128 keys
   static constexpr int V_BYTES = D * (BS / 2);                  // V^T: d rows x 64 bytes
+  static constexpr int ONES_BYTES = kOnesRows * (BS / 2);       // constant rows of E2M1 1.0, written once
+  static constexpr int DN = D + kOnesRows;                      // N of the PV instruction
   static constexpr int KSF_BYTES = CTQ * 512;
   static constexpr int VSF_BYTES = 512;
-  static constexpr int STAGE_BYTES = K_BYTES + V_BYTES + KSF_BYTES + VSF_BYTES;
+  static constexpr int OFF_KSF = K_BYTES + V_BYTES + ONES_BYTES;   // within a stage
+  static constexpr int OFF_VSF = OFF_KSF + KSF_BYTES;
+  static constexpr int STAGE_BYTES = OFF_VSF + VSF_BYTES;
   static constexpr int NST = (D == 128) ? 6 : 8;                // ring depth (stages of 128 keys)
   static constexpr int P_BYTES = BM * (BN / 2);                 // 4 KB per 64-key tile: [block][row][16 B]
   static constexpr int PSF_BYTES = 512;                         // one atom per stage: bytes {0,1} tile 0, {2,3} tile 1
-  static constexpr int META_BYTES = BM * 16;                    // per row {E_0, E_1, 2*c_0, 2*c_1}
+  static constexpr int META_BYTES = BM * 8;                     // per row {E_0, E_1}
   // shared-memory map (offsets from a 1024-byte aligned base)
   static constexpr int OFF_Q = 0;                               // two buffers
   static constexpr int OFF_QSF = OFF_Q + 2 * Q_BYTES;           // two buffers of 1 KB
   static constexpr int OFF_P = OFF_QSF + 2048;
   static constexpr int OFF_PSF = OFF_P + kTeams * P_BYTES;
-  static constexpr int OFF_META = OFF_PSF + 2 * PSF_BYTES;
-  static constexpr int OFF_STAGE = OFF_META + kTeams * META_BYTES;
+  static constexpr int OFF_ONESF = OFF_PSF + 2 * PSF_BYTES;     // scale atom of 1.0 for the rows of ones
+  static constexpr int OFF_META = OFF_ONESF + 512;
+  static constexpr int OFF_STAGE = (OFF_META + kTeams * META_BYTES + 1023) / 1024 * 1024;
   static constexpr int OFF_BAR = OFF_STAGE + NST * STAGE_BYTES;
   static constexpr int SMEM_BYTES = OFF_BAR + 1024 + 1024;      // barriers + alignment slack
   static constexpr uint64_t SWZ_QK = (ROW_BYTES == 64) ? kSwz64 : kSwz32;
@@ -113,20 +123,12 @@ __device__ __forceinline__ void fma2(float s0, float s1, float c, float b, float
       "mov.b64 {%0, %1}, d;\n\t}"
       : "=f"(x0), "=f"(x1) : "f"(s0), "f"(s1), "f"(c), "f"(b));
 }
-// Sum of the doubled magnitudes {0,1,2,3,4,6,8,12} of the eight non-negative E2M1 codes of a word,
-// returned as four byte-wise partial sums (each <= 24).
-__device__ __forceinline__ uint32_t code_sums_x2(uint32_t w) {
-  const uint32_t lo = 0x03020100u, hi = 0x0C080604u;
-  return __byte_perm(lo, hi, w) + __byte_perm(lo, hi, w >> 16);
-}
-
-// One N32 score fragment of one row: E_B = ceil(max y), codes q = Q_E2M1(2^(y - E_B + log2 6)),
-// doubled code sum.  Nothing here depends on the row reference.
-__device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, int& E, uint32_t* words, int& c2) {
+// One N32 score fragment of one row: E_B = ceil(max y) and the codes q = Q_E2M1(2^(y - E_B + log2 6)).
+// Nothing here depends on the row reference.
+__device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, int& E, uint32_t* words) {
   const float LOG2_6 = 2.5849625007211560f;
   E = (int)ceilf(__fmul_rn(max32(sraw), c32));
   const float bB = __fsub_rn(LOG2_6, (float)E);
-  uint32_t acc = 0;
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
     float pv[8];
@@ -138,9 +140,7 @@ __device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, 
       pv[i + 1] = ex2_approx(x1);
     }
     words[w] = cvt_e2m1x8(pv);
-    acc += code_sums_x2(words[w]);
   }
-  c2 = __dp4a(acc, 0x01010101u, 0u);
 }
 
 template <int D, bool NV>
@@ -187,6 +187,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     prefetch_tensormap(&tmV);
   }
   if (warp == 1) { tmem_alloc(sbase + C::OFF_BAR + 768, kTmemCols); tmem_relinquish(); }
+  // constant operand rows: E2M1 code 2 (= 1.0) in every nibble, E8M0 byte 127 (= 2^0) as their scale
+  for (int i = threadIdx.x; i < C::NST * (C::ONES_BYTES / 4); i += kAttnThreads)
+    reinterpret_cast<uint32_t*>(sgen + C::OFF_STAGE + (i / (C::ONES_BYTES / 4)) * C::STAGE_BYTES + C::K_BYTES + C::V_BYTES)[i % (C::ONES_BYTES / 4)] = 0x22222222u;
+  for (int i = threadIdx.x; i < 128; i += kAttnThreads) reinterpret_cast<uint32_t*>(sgen + C::OFF_ONESF)[i] = 0x7F7F7F7Fu;
+  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -218,11 +223,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         const uint32_t fb = bar_full(s);
         if (elect_one()) {
-          mbar_arrive_expect_tx(fb, C::STAGE_BYTES);
+          mbar_arrive_expect_tx(fb, C::K_BYTES + C::V_BYTES + C::KSF_BYTES + C::VSF_BYTES);
           tma_load_2d(st, &tmK, 0, krow0 + s2 * BS, fb);
           tma_load_2d(st + C::K_BYTES, &tmV, s2 * (BS / 2), vrow0, fb);
-          bulk_load_1d(st + C::K_BYTES + C::V_BYTES, ksf + (size_t)s2 * C::KSF_BYTES, C::KSF_BYTES, fb);
-          bulk_load_1d(st + C::K_BYTES + C::V_BYTES + C::KSF_BYTES, vsf + (size_t)s2 * C::VSF_BYTES, C::VSF_BYTES, fb);
+          bulk_load_1d(st + C::OFF_KSF, ksf + (size_t)s2 * C::KSF_BYTES, C::KSF_BYTES, fb);
+          bulk_load_1d(st + C::OFF_VSF, vsf + (size_t)s2 * C::VSF_BYTES, C::VSF_BYTES, fb);
         }
         st += C::STAGE_BYTES;
         if (++s == C::NST) { s = 0; ph ^= 1; st = sbase + C::OFF_STAGE; }
@@ -267,7 +272,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint64_t dK0 = at(kDescQK, stq);
         if (elect_one()) {
 #pragma unroll
-          for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFK + 4 * a, at(kDescSF, stq + C::K_BYTES + C::V_BYTES + 512 * a));
+          for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFK + 4 * a, at(kDescSF, stq + C::OFF_KSF + 512 * a));
           if (NV) {
             tc_mma_fp4_4x(tS, dQ0, dK0, kIdQK0, tSFQ, tSFK, 0);
             if (C::KBLK == 2) tc_mma_fp4_4x(tS, dQ0 + 2, dK0 + 2, kIdQK1, tSFQ + 4, tSFK + 4, 1);
@@ -286,8 +291,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     __syncwarp();
   } else if (warp == 2) {
     // ===================================================================== PV issuer: O += P V, one stage per issue
-    constexpr uint32_t kIdPV0 = make_idesc_fp4(BM, D, true, 0, 0), kIdPV1 = make_idesc_fp4(BM, D, true, 2, 2);
+    constexpr uint32_t kIdPV0 = make_idesc_fp4(BM, C::DN, true, 0, 0), kIdPV1 = make_idesc_fp4(BM, C::DN, true, 2, 2);
     const uint32_t tO = tmem + kColO;
+    if (D == 128) {
+      // B rows 128..143 (the ones) read their scales from a fifth column group: constant, set once per slot
+      if (elect_one()) {
+        tc_cp_32x128b_warpx4(tmem + kColSFV + 4, at(kDescSF, sbase + C::OFF_ONESF));
+        tc_cp_32x128b_warpx4(tmem + kColSFV + 12, at(kDescSF, sbase + C::OFF_ONESF));
+      }
+      __syncwarp();
+    }
     int sp = 0;
     uint32_t stp = sbase + C::OFF_STAGE;
     uint32_t g = 0;
@@ -301,12 +314,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFULL0 + pr), m & 1, abortf));   // codes and scale bytes of both tiles are in smem
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tSFP = tmem + kColSFP + 4 * pr, tSFV = tmem + kColSFV + 4 * pr;
+        const uint32_t tSFP = tmem + kColSFP + 4 * pr, tSFV = tmem + kColSFV + 8 * pr;
+        if (D == 64) {
+          // B rows 64..79 (the ones) take their scales from the V atom's padding rows: set them to 2^0
+          if (lane < kOnesRows) *reinterpret_cast<uint32_t*>(sgen + (stp - sbase) + C::OFF_VSF + lane * 16 + 8) = 0x7F7F7F7Fu;
+          fence_proxy_async_smem();
+          __syncwarp();
+        }
         const uint64_t dV = at(kDescV, stp + C::K_BYTES);
         const uint64_t dP = at(kDescP, sbase + C::OFF_P + C::P_BYTES * 2 * pr);
         if (elect_one()) {
           tc_cp_32x128b_warpx4(tSFP, at(kDescSF, sbase + C::OFF_PSF + 512 * pr));
-          tc_cp_32x128b_warpx4(tSFV, at(kDescSF, stp + C::K_BYTES + C::V_BYTES + C::KSF_BYTES));
+          tc_cp_32x128b_warpx4(tSFV, at(kDescSF, stp + C::OFF_VSF));
           // tile h of the stage: P slot 2*pr+h, keys 64h..64h+63 of V^T (32 bytes on), scale bytes {2h, 2h+1}
           tc_mma_fp4_2x(tO, dP, dV, kIdPV0, tSFP, tSFV, s2 > 0);
           tc_mma_fp4_2x(tO, dP + (C::P_BYTES >> 4), dV + 2, kIdPV1, tSFP, tSFV, 1);
@@ -333,14 +352,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     int i = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i, g0 += T2) {
       int mu = -(1 << 28);
-      float L2 = 0.f;                                           // sum of 2^(E_B - mu) * (2 * code sum)
       int pu0 = 0, pu1 = 0;                                     // bytes written for the previous tile
       for (int j = 0; j < 2 * T2; ++j) {
         const uint32_t g = g0 + (j >> 1);
         const int h = j & 1, pr = g & 1, slot = 2 * pr + h;
         ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + slot), (g >> 1) & 1, abortf));
         if (!ok) break;
-        const int4 mt = *reinterpret_cast<const int4*>(sgen + C::OFF_META + C::META_BYTES * slot + row * 16);
+        const int2 mt = *reinterpret_cast<const int2*>(sgen + C::OFF_META + C::META_BYTES * slot + row * 8);
         uint8_t* psf = sgen + C::OFF_PSF + 512 * pr + lane * 16 + quarter * 4;
         const int Emax = max(mt.x, mt.y);
         const bool need = Emax > mu + kLazyShift;
@@ -350,7 +368,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const int delta = Emax - mu;
             f = (delta > 126) ? 0.f : __uint_as_float((uint32_t)(127 - delta) << 23);
             mu = Emax;
-            L2 *= f;
             if (h) {
               // the stage's first tile is not in O yet (both tiles are issued together): move its bytes
               pu0 = max(pu0 - delta, 0);
@@ -365,7 +382,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (!ok) break;
             tc_fence_after();
 #pragma unroll 1
-            for (int c0 = 0; c0 < D; c0 += 16) {
+            for (int c0 = 0; c0 < C::DN; c0 += 16) {             // numerator columns and the row-sum columns
               uint32_t o[16];
               tmem_ld_32x32b_x16(tO + c0, o);
               tmem_wait_ld();
@@ -378,10 +395,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
         // A block more than 126 octaves below the reference is a zero block: it gets the smallest
-        // byte (2^-127, below 2^-60 of the row's mass by construction) and no share of the row sum.
+        // byte (2^-127, below 2^-60 of the row's mass by construction) in numerator and row sum alike.
         const int u0 = mt.x - mu + 127, u1 = mt.y - mu + 127;
-        if (u0 >= 1) L2 = fmaf((float)mt.z, __uint_as_float((uint32_t)u0 << 23), L2);
-        if (u1 >= 1) L2 = fmaf((float)mt.w, __uint_as_float((uint32_t)u1 << 23), L2);
         pu0 = max(u0, 0);
         pu1 = max(u1, 0);
         *reinterpret_cast<uint16_t*>(psf + 2 * h) = (uint16_t)(pu0 | (pu1 << 8));
@@ -390,11 +405,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + pr));
       }
       if (!ok) break;
-      // ---- epilogue: O = O_hw / (3 * L2), LSE = ln2 * (mu + log2(L2 / 12))
+      // ---- epilogue: with L_hw = column d of the accumulator, O = O_hw / (6 L_hw), LSE = ln2 (mu + log2(L_hw / 6))
       ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFULL), i & 1, abortf));
       if (!ok) break;
       tc_fence_after();
-      const float inv = __frcp_rn(3.0f * L2);
+      float Lhw;
+      {
+        uint32_t r16[16];
+        tmem_ld_32x32b_x16(tO + D, r16);
+        tmem_wait_ld();
+        Lhw = __uint_as_float(r16[0]);
+      }
+      const float inv = __frcp_rn(6.0f * Lhw);
       const size_t grow = (size_t)item * BM + row;
       __nv_bfloat16* orow = p.O + grow * D;
 #pragma unroll 1
@@ -418,7 +440,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           *reinterpret_cast<uint4*>(orow + c0 + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
       }
-      if (p.LSE) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(L2) - 3.5849625007211560f));
+      if (p.LSE) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(Lhw) - 2.5849625007211560f));
     }
   } else {
     // ===================================================================== softmax teams
@@ -430,7 +452,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t sfull = bar(BAR_SFULL0 + pr), sempty = bar(BAR_SEMPTY0 + pr);
     const uint32_t smdone = bar(BAR_SMDONE0 + team), pfree = bar(BAR_PFREE0 + pr);
     uint8_t* pbuf = sgen + C::OFF_P + C::P_BYTES * team + row * 16;
-    int4* meta = reinterpret_cast<int4*>(sgen + C::OFF_META + C::META_BYTES * team + row * 16);
+    int2* meta = reinterpret_cast<int2*>(sgen + C::OFF_META + C::META_BYTES * team + row * 8);
     float c32;
     if (NV) c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G), __ldg(p.k_G)));
     else    c32 = __fdiv_rn(p.c_base, 36.0f);
@@ -443,21 +465,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         tc_fence_after();
         uint32_t sraw[32], w0[4], w1[4];
-        int E0, E1, c0, c1;
+        int E0, E1;
         tmem_ld_32x32b_x32(tS, sraw);
         tmem_wait_ld();
-        direct_p_block(sraw, c32, E0, w0, c0);
+        direct_p_block(sraw, c32, E0, w0);
         tmem_ld_32x32b_x32(tS + 32, sraw);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(sempty);                     // pair may take the stage after next
-        direct_p_block(sraw, c32, E1, w1, c1);
+        direct_p_block(sraw, c32, E1, w1);
         if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
         if (!ok) break;
         *reinterpret_cast<uint4*>(pbuf) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
         *reinterpret_cast<uint4*>(pbuf + BM * 16) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
-        *meta = make_int4(E0, E1, c0, c1);
+        *meta = make_int2(E0, E1);
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(smdone);
