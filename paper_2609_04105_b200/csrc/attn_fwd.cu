@@ -123,6 +123,41 @@ __device__ __forceinline__ void fma2(float s0, float s1, float c, float b, float
       "mov.b64 {%0, %1}, d;\n\t}"
       : "=f"(x0), "=f"(x1) : "f"(s0), "f"(s1), "f"(c), "f"(b));
 }
+// ---- 2^x on the FMA pipe for a share of the elements (the SFU's 16 ex2/clk/SM is the tightest unit).
+// Only the E2M1 code of 2^x matters, and codes change only where the significand of 2^x crosses
+// 1, 1.25, 1.5 or 1.75.  With x = n + f (n = floor x), 2^f is replaced by the degree-4 polynomial
+// through (0,1), (log2 1.25, 1.25), (log2 1.5, 1.5), (log2 1.75, 1.75), (1,2): monotone, equal to 2^f
+// at every point where a code can change, so the codes are those of the exact exponential (a
+// 4-million-point sweep plus dense sweeps around the seven boundaries differ only within one fp32
+// ulp of x at a boundary - the same class as ex2.approx).  n enters through the exponent field.
+#ifndef FP4ATTN_POLY_MASK
+#define FP4ATTN_POLY_MASK 0x0842u      // which of a block's 16 element pairs take the polynomial path
+#endif
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float& p1) {
+  const float M = 12582912.0f;                       // 1.5 * 2^23: x + M rounded down holds floor(x) in its low bits
+  const uint64_t x = pack2(fmaxf(x0, -40.0f), fmaxf(x1, -40.0f));
+  const uint64_t m = pack2(M, M);
+  uint64_t t, nb, f, q;
+  asm("add.rm.f32x2 %0, %1, %2;" : "=l"(t) : "l"(x), "l"(m));
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(nb) : "l"(m), "l"(t));          // -floor(x), exact
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(f) : "l"(x), "l"(nb));          // x - floor(x) in [0,1), exact
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(pack2(0.014081917703151703f, 0.014081917703151703f)), "l"(f),
+      "l"(pack2(0.05088741332292557f, 0.05088741332292557f)));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(f), "l"(pack2(0.24216225743293762f, 0.24216225743293762f)));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(f), "l"(pack2(0.6928684115409851f, 0.6928684115409851f)));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(f), "l"(pack2(1.0f, 1.0f)));
+  uint32_t tl, th, ql, qh;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(tl), "=r"(th) : "l"(t));
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(ql), "=r"(qh) : "l"(q));
+  p0 = __uint_as_float(tl * 0x800000u + ql);         // significand bits + (floor(x) << 23)
+  p1 = __uint_as_float(th * 0x800000u + qh);
+}
+
 // One N32 score fragment of one row: E_B = ceil(max y) and the codes q = Q_E2M1(2^(y - E_B + log2 6)).
 // Nothing here depends on the row reference.
 __device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, int& E, uint32_t* words) {
@@ -136,8 +171,12 @@ __device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, 
     for (int i = 0; i < 8; i += 2) {
       float x0, x1;
       fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), c32, bB, x0, x1);
-      pv[i] = ex2_approx(x0);
-      pv[i + 1] = ex2_approx(x1);
+      if ((FP4ATTN_POLY_MASK >> (4 * w + i / 2)) & 1u) {
+        exp2_poly2(x0, x1, pv[i], pv[i + 1]);
+      } else {
+        pv[i] = ex2_approx(x0);
+        pv[i + 1] = ex2_approx(x1);
+      }
     }
     words[w] = cvt_e2m1x8(pv);
   }
