@@ -121,8 +121,16 @@ def test_config3_full_size_sampled_rows():
     _sampled_case("cfg3", 128, 4, 3)
 
 
-def test_config5_n1024_full_size_sampled_rows():
-    _sampled_case("cfg5_N1024", 128, 8, 5)
+def test_config4_full_size_sampled_rows():
+    """B1 H32 N16384 d128 with x20 outlier channels (|y| ~ 300: moving reference, zero blocks);
+    3 heads x 96 sampled rows."""
+    _sampled_case("cfg4", 96, 3, 4)
+
+
+@pytest.mark.parametrize("N", [1024, 8192, 32768])
+def test_config5_sweep_full_size_sampled_rows(N):
+    """Sequence sweep at B*N = 32768 tokens, H=16, d=128: shortest, middle and longest point."""
+    _sampled_case(f"cfg5_N{N}", 128 if N < 32768 else 64, 8 if N < 32768 else 2, 5)
 
 
 def test_host_buffer_entry_point_matches_device_path():
