@@ -27,6 +27,10 @@ sys.path.insert(0, ROOT)
 
 from paper_2609_04105_b200 import inputs as I  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised in profiles/
+# (attention: profiles/attn_fwd_cfg2.md, quantizer: profiles/quantizers_cfg2.md); other workloads: not captured.
+NCU_TRAFFIC_BYTES = {"cfg2": {"attn": 53.55e6 + 20.36e6, "quant_rows": 67.12e6 + 2.39e6}}
+
 METRIC = "fp4_attention_fwd_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_FP4_OVER_BF16 = 4.0          # dense 9 PFLOP/s fp4 : 2.25 PFLOP/s bf16
@@ -332,12 +336,14 @@ def run_cuda(args, w):
                       "note": "attention kernel alone (the paper's timing boundary excludes quantization)"},
         "roofline": {"kernel": "attn_fwd_kernel", "bound": "tensor", "achieved": w.flops / (attn_launch_ms * 1e-3) / 1e12,
                      "peak": fp4_peak, "unit": "TFLOP/s",
-                     "frac": w.flops / (attn_launch_ms * 1e-3) / 1e12 / fp4_peak, "traffic": None,
+                     "frac": w.flops / (attn_launch_ms * 1e-3) / 1e12 / fp4_peak,
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get("attn"),
                      "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x nominal fp4:bf16 ratio 4",
                      "fp4_issue_probe_tflops": probe_tflops, "fp4_issue_probe_flop_per_clk_per_sm": probe_flop_per_clk_sm},
         "roofline_quantize": {"kernel": "quant_mx_rows_kernel", "bound": "hbm", "achieved": q_bytes / (q_ms * 1e-3) / 1e9,
                               "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                              "frac": q_bytes / (q_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                              "frac": q_bytes / (q_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                              "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get("quant_rows"),
                               "bytes_per_element": 2 + 0.5 + 1.0 / 32},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "api": "fp4attn_attention_host (pinned host buffers)"},
