@@ -38,8 +38,11 @@ constexpr int BS = 128;          // keys per stage
 constexpr int kTeams = 4;        // score slots / softmax teams
 constexpr int kFirstSoftmaxWarp = 7;     // warps 3..6 are the correction warps
 constexpr int kAttnThreads = 32 * (kFirstSoftmaxWarp + 4 * kTeams);
-constexpr int kLazyShift = 64;   // the row reference follows the running maximum only when it is
-                                 // more than this many octaves behind (rescales are exact powers of 2)
+constexpr int kLazyShift = 64;   // the row reference is raised only when a block exponent exceeds it by more
+                                 // than this many octaves (rescales are exact powers of 2) ...
+constexpr int kRefHeadroom = 60; // ... and is then set this far ABOVE that exponent, so that a later raise
+                                 // needs a jump of 124 octaves: E8M0 bytes stay within 1..191, blocks weaker
+                                 // than 2^-66 of the row maximum become zero blocks
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256, kColSFQ = 400, kColSFK = 416, kColSFV = 432, kColSFP = 448;
 constexpr int kOnesRows = 16;    // rows of ones appended to V^T (the MMA's N must be a multiple of 16)
@@ -72,10 +75,12 @@ struct Cfg {
   static constexpr int OFF_ONESF = OFF_PSF + 2 * PSF_BYTES;     // scale atom of 1.0 for the rows of ones
   static constexpr int OFF_META = OFF_ONESF + 512;
   static constexpr int OFF_STAGE = (OFF_META + kTeams * META_BYTES + 1023) / 1024 * 1024;
-  static constexpr int OFF_BAR = OFF_STAGE + NST * STAGE_BYTES;
+  static constexpr int OFF_OUT = OFF_STAGE + NST * STAGE_BYTES; // bf16 O tile staged for TMA stores: D/64 halves of [128 rows][128 B]
+  static constexpr int OUT_BYTES = (D / 64) * BM * 128;
+  static constexpr int OFF_BAR = OFF_OUT + OUT_BYTES;
   static constexpr int SMEM_BYTES = OFF_BAR + 1024 + 1024;      // barriers + alignment slack
   static constexpr uint64_t SWZ_QK = (ROW_BYTES == 64) ? kSwz64 : kSwz32;
-  static_assert(STAGE_BYTES % 512 == 0 && OFF_STAGE % 1024 == 0, "stage alignment");
+  static_assert(STAGE_BYTES % 512 == 0 && OFF_STAGE % 1024 == 0 && OFF_OUT % 1024 == 0, "stage alignment");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
 };
 
@@ -185,7 +190,8 @@ __device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, 
 template <int D, bool NV>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                const AttnParams p) {
   using C = Cfg<D, NV>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -224,6 +230,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     prefetch_tensormap(&tmQ);
     prefetch_tensormap(&tmK);
     prefetch_tensormap(&tmV);
+    prefetch_tensormap(&tmO);
   }
   if (warp == 1) { tmem_alloc(sbase + C::OFF_BAR + 768, kTmemCols); tmem_relinquish(); }
   // constant operand rows: E2M1 code 2 (= 1.0) in every nibble, E8M0 byte 127 (= 2^0) as their scale
@@ -404,12 +411,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (__any_sync(0xffffffffu, need)) {
           float f = 1.0f;
           if (need) {
-            const int delta = Emax - mu;
+            // new reference: kRefHeadroom above the offending exponent, but never more than 126 octaves
+            // above the old one while the old contributions can still matter (they reach up to
+            // mu + kLazyShift); only when even that is out of reach are they dropped (f = 0)
+            int delta = Emax + kRefHeadroom - mu;
+            if (delta > 126 && Emax <= mu + 126 + kLazyShift) delta = 126;
             f = (delta > 126) ? 0.f : __uint_as_float((uint32_t)(127 - delta) << 23);
-            mu = Emax;
+            mu = (delta > 126) ? Emax + kRefHeadroom : mu + delta;
             if (h) {
               // the stage's first tile is not in O yet (both tiles are issued together): move its bytes
-              pu0 = max(pu0 - delta, 0);
+              pu0 = max(pu0 - delta, 0);                        // (delta as computed above: new reference - old)
               pu1 = max(pu1 - delta, 0);
               *reinterpret_cast<uint16_t*>(psf) = (uint16_t)(pu0 | (pu1 << 8));
             }
@@ -457,7 +468,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       const float inv = __frcp_rn(6.0f * Lhw);
       const size_t grow = (size_t)item * BM + row;
-      __nv_bfloat16* orow = p.O + grow * D;
+      // stage the bf16 tile in shared memory (128-byte rows, 128B-swizzled like the tensor map) and
+      // let TMA write it out, so O is released after four TMEM reads instead of after 16 global stores
+      if (lane == 0) bulk_wait_read_all();                      // this warp's previous stores have read the buffer
+      __syncwarp();
 #pragma unroll 1
       for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t o[32];
@@ -468,6 +482,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           __syncwarp();
           if (lane == 0) mbar_arrive(bar(BAR_OFREE));
         }
+        uint8_t* half = sgen + C::OFF_OUT + (c0 >> 6) * (BM * 128) + row * 128;
 #pragma unroll
         for (int c = 0; c < 32; c += 8) {
           uint32_t pk[4];
@@ -476,8 +491,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[c + 2 * q]) * inv, __uint_as_float(o[c + 2 * q + 1]) * inv);
             pk[q] = *reinterpret_cast<const uint32_t*>(&hh);
           }
-          *reinterpret_cast<uint4*>(orow + c0 + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          const int chunk = ((c0 & 63) + c) >> 3;               // 16-byte chunk of the 128-byte row
+          *reinterpret_cast<uint4*>(half + ((chunk ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {                                          // this warp's 32 rows, one box per 128-byte half
+#pragma unroll
+        for (int hf = 0; hf < D / 64; ++hf)
+          tma_store_2d(&tmO, hf * 128, item * BM + quarter * 32, sbase + C::OFF_OUT + hf * (BM * 128) + quarter * 32 * 128);
+        bulk_commit_group();
       }
       if (p.LSE) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(Lhw) - 2.5849625007211560f));
     }
@@ -525,6 +549,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
     }
   }
+  if (warp >= 3 && warp < kFirstSoftmaxWarp && lane == 0) bulk_wait_all();
   __syncthreads();
   if (*abortf && threadIdx.x == 0 && p.status) *p.status = FP4ATTN_ERR_TIMEOUT;
   if (warp == 1) {
@@ -592,7 +617,7 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint6
   const cuuint64_t strides[1] = {row_bytes};
   const cuuint32_t box[2] = {box_bytes, box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  const CUtensorMapSwizzle swz = box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+  const CUtensorMapSwizzle swz = box_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -607,17 +632,18 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
       return FP4ATTN_ERR_CUDA;
     attr_set = true;
   }
-  CUtensorMap tmQ, tmK, tmV;
+  CUtensorMap tmQ, tmK, tmV, tmO;
   const uint64_t rows = (uint64_t)B * H * N;
   if (!make_map(&tmQ, ops->q, C::ROW_BYTES, rows, C::ROW_BYTES, BM) ||
       !make_map(&tmK, ops->k, C::ROW_BYTES, rows, C::ROW_BYTES, BS) ||
-      !make_map(&tmV, ops->v, (uint64_t)N / 2, (uint64_t)B * H * D, BS / 2, D))
+      !make_map(&tmV, ops->v, (uint64_t)N / 2, (uint64_t)B * H * D, BS / 2, D) ||
+      !make_map(&tmO, prm.O, (uint64_t)D * 2, rows, 128, 32))
     return FP4ATTN_ERR_CUDA;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return FP4ATTN_ERR_CUDA;
   const unsigned grid = (unsigned)(prm.n_items < sms ? prm.n_items : sms);     // persistent: one CTA per SM
-  attn_fwd_kernel<D, NV><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, prm);
+  attn_fwd_kernel<D, NV><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, tmO, prm);
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
 
