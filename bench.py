@@ -317,6 +317,43 @@ def run_cuda(args, w):
     probe_tflops = sms * iters * 2.0 * 128 * 128 * 64 / (p0.elapsed_time(p1) * 1e-3) / 1e12
     probe_flop_per_clk_sm = iters * 2.0 * 128 * 128 * 64 / max(1, int(cyc.item()))
 
+    # ---- attention kernel alone on the other configurations (quick; context for the headline line)
+    sweep = {}
+    if world == 1 and not args.no_sweep:
+        del dq, dk, dv, hq, hk, hv, ws, ho, hl
+        torch.cuda.empty_cache()
+        for name in ("cfg5_N1024", "cfg5_N8192", "cfg5_N32768", "cfg3", "cfg4"):
+            if name == w.name:
+                continue
+            ww = I.WORKLOADS[name]
+            g = torch.Generator(device=dev).manual_seed(1)
+            mk = lambda: torch.randn((ww.B, ww.H, ww.N, ww.d), device=dev, generator=g).to(torch.bfloat16)
+            xq, xk, xv = mk(), mk(), mk()
+            if ww.outliers:                                          # 3 channels x20 in Q and K, as in the seeded recipe
+                ch = torch.from_numpy(I.outlier_channels(ww)).to(dev)
+                for h in range(ww.H):
+                    xq[:, h, :, ch[h]] *= 20
+                    xk[:, h, :, ch[h]] *= 20
+            sq = Bd.fp4attn_quantize(xq, ww.qk_fmt, Bd.ROLE_Q)
+            sk = Bd.fp4attn_quantize(xk, ww.qk_fmt, Bd.ROLE_K)
+            sv = Bd.fp4attn_quantize(xv, Bd.FMT_MXFP4, Bd.ROLE_V)
+            del xq, xk, xv
+            so = torch.empty((ww.B, ww.H, ww.N, ww.d), dtype=torch.bfloat16, device=dev)
+            for _ in range(3):
+                Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status)
+            torch.cuda.synchronize()
+            a, b = E(), E()
+            n_it = 10
+            a.record()
+            for _ in range(n_it):
+                Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / n_it
+            sweep[name] = {"workload": _workload_text(ww), "attn_ms": ms, "attn_tflops": ww.flops / (ms * 1e-3) / 1e12}
+            del sq, sk, sv, so
+            torch.cuda.empty_cache()
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -347,15 +384,19 @@ def run_cuda(args, w):
                               "bytes_per_element": 2 + 0.5 + 1.0 / 32},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "api": "fp4attn_attention_host (pinned host buffers)"},
+        "attn_other_workloads": sweep,
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clk.summary(),
     }
     # ---- oracle on the host cores: bounded sample of the same workload, plus accuracy vs fp64
     if world == 1 and not args.no_cpu_baseline:
         rng = np.random.default_rng(7)
-        n_rows = min(N, 2048)
+        # sized for roughly 10-30 s of host work: cost ~ heads * rows * N * d
+        n_rows = min(N, 4096)
+        n_heads = max(1, min(B * H, int(8 * (4096.0 / N) ** 1)))
         rows = np.sort(rng.choice(N, size=n_rows, replace=False))
-        heads = [(0, 0), (B - 1, H - 1)] if B * H > 1 else [(0, 0)]
+        all_heads = [(b, h) for b in range(B) for h in range(H)]
+        heads = [all_heads[i] for i in np.linspace(0, len(all_heads) - 1, n_heads).astype(int)]
         dt, tf, Oo, Lo = oracle_sample(w, q, k, v, heads, rows)
         Og = np.stack([O[b, h].float().cpu().numpy().astype(np.float64)[rows] for b, h in heads])
         rel = max(float(np.linalg.norm(Og[i] - Oo[i]) / np.linalg.norm(Oo[i])) for i in range(len(heads)))
@@ -376,6 +417,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(I.WORKLOADS))
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the attention-only timings of the other configurations")
     args = ap.parse_args()
     w = I.WORKLOADS[args.workload]
     if args.impl == "reference":

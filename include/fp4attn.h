@@ -176,6 +176,15 @@ int fp4attn_attention_host(const void* q_host, const void* k_host, const void* v
  */
 int fp4attn_mma_peak_probe(int iters, unsigned long long* cycles_out, fp4attn_stream_t stream);
 
+/*
+ * Self-test of the bounded in-kernel waits (the failure-detection path; the paper has no
+ * counterpart).  Launches one warp that waits on a barrier nothing completes, with a limit of
+ * `limit_cycles` SM clocks (1 .. 2^31), and writes to *device_status what the attention kernel
+ * would: FP4ATTN_ERR_TIMEOUT once the limit has run out (expected), FP4ATTN_OK otherwise.  The warp
+ * returns normally; the context stays usable.
+ */
+int fp4attn_selftest_bounded_wait(long long limit_cycles, int* device_status, fp4attn_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,7 @@ EXPORTS = [
     "fp4attn_status_string", "fp4attn_version", "fp4attn_packed_bytes", "fp4attn_scale_bytes",
     "fp4attn_quantize_workspace_bytes", "fp4attn_quantize", "fp4attn_fwd",
     "fp4attn_attention_host_workspace_bytes", "fp4attn_attention_host", "fp4attn_mma_peak_probe",
-    "fp4attn_quantize_nvfp4_noalloc",
+    "fp4attn_quantize_nvfp4_noalloc", "fp4attn_selftest_bounded_wait",
 ]
 
 
@@ -63,6 +63,8 @@ def _load() -> ctypes.CDLL:
     lib.fp4attn_attention_host.argtypes = [vp, vp, vp, i, ctypes.c_float, i, i, i, i, vp, vp, vp, sz, vp]
     lib.fp4attn_quantize_nvfp4_noalloc.restype = i
     lib.fp4attn_quantize_nvfp4_noalloc.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp]
+    lib.fp4attn_selftest_bounded_wait.restype = i
+    lib.fp4attn_selftest_bounded_wait.argtypes = [ctypes.c_longlong, vp, vp]
     lib.fp4attn_mma_peak_probe.restype = i
     lib.fp4attn_mma_peak_probe.argtypes = [i, vp, vp]
     return lib
@@ -170,3 +172,8 @@ def fp4attn_attention_host(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, qk
 
 def fp4attn_mma_peak_probe(iters: int, cycles_out: torch.Tensor) -> None:
     _check(lib().fp4attn_mma_peak_probe(iters, cycles_out.data_ptr(), _stream()), "fp4attn_mma_peak_probe")
+
+
+def fp4attn_selftest_bounded_wait(limit_cycles: int, status: torch.Tensor) -> None:
+    """One warp waits (bounded) on a barrier nothing completes; `status` (int32 CUDA) receives the time-out code."""
+    _check(lib().fp4attn_selftest_bounded_wait(int(limit_cycles), status.data_ptr(), _stream()), "fp4attn_selftest_bounded_wait")

@@ -591,6 +591,18 @@ __global__ void __launch_bounds__(128, 1) mma_peak_kernel(int iters, unsigned lo
   if ((threadIdx.x >> 5) == 0) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
+// ------------------------------------------------------------------ bounded-wait self-test
+// One warp waits on an mbarrier that nothing will ever complete, with a short limit, and must come
+// back through the same time-out path the attention kernel uses (abort flag -> status word).
+__global__ void __launch_bounds__(32, 1) bounded_wait_selftest_kernel(long long limit_cycles, int* status) {
+  __shared__ __align__(8) uint64_t never;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) { mbar_init(smem_u32(&never), 1); abort_flag = 0; fence_barrier_init(); }
+  __syncwarp();
+  const bool ok = __all_sync(0xffffffffu, mbar_wait_limit(smem_u32(&never), 0, &abort_flag, limit_cycles));
+  if (threadIdx.x == 0) *status = (!ok && abort_flag) ? FP4ATTN_ERR_TIMEOUT : FP4ATTN_OK;
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -692,5 +704,13 @@ extern "C" int fp4attn_mma_peak_probe(int iters, unsigned long long* cycles_out,
     return FP4ATTN_ERR_CUDA;
   if (cudaMemsetAsync(cycles_out, 0, sizeof(unsigned long long), (cudaStream_t)stream) != cudaSuccess) return FP4ATTN_ERR_CUDA;
   mma_peak_kernel<<<sms, 128, smem, (cudaStream_t)stream>>>(iters, cycles_out);
+  return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
+}
+
+extern "C" int fp4attn_selftest_bounded_wait(long long limit_cycles, int* device_status, fp4attn_stream_t stream) {
+  if (!device_status || limit_cycles <= 0 || limit_cycles > (1ll << 31)) return FP4ATTN_ERR_INVALID_ARG;
+  int rc = check_device_sm100();
+  if (rc != FP4ATTN_OK) return rc;
+  bounded_wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_cycles, device_status);
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }

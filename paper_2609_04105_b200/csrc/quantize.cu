@@ -73,45 +73,58 @@ quant_mx_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
 }
 
 // ---------------------------------------------------------------- MXFP4, blocks along keys (V), transposed out
+// A [128 keys x D] tile goes through shared memory; a thread owns two adjacent head-dim columns and
+// one 32-key block, reads them as bf16x2 words (conflict-free) and writes two 16-byte code groups.
+// grid (N / 128, B*H), 2*D threads
 template <int D>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(2 * D)
 quant_mx_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ packed, uint8_t* __restrict__ sf, int N) {
-  __shared__ __align__(16) __nv_bfloat16 tile[128 * D];
+  constexpr int T = 2 * D;                         // threads: D/2 column pairs x 4 key blocks
+  __shared__ __align__(16) uint32_t tile[128 * D / 2];
   __shared__ uint8_t sfb[128 * 4];
   const int kt = blockIdx.x;                       // 128-key tile
   const size_t bh = blockIdx.y;
   const uint4* src = x + (bh * N + (size_t)kt * 128) * (D / 8);
-  constexpr int LOADS = 128 * D / 8 / kThreads;
+  constexpr int LOADS = 128 * D / 8 / T;           // 8
   uint4 raw[LOADS];
 #pragma unroll
-  for (int k = 0; k < LOADS; ++k) raw[k] = __ldg(src + threadIdx.x + k * kThreads);
+  for (int k = 0; k < LOADS; ++k) raw[k] = __ldg(src + threadIdx.x + k * T);
 #pragma unroll
-  for (int k = 0; k < LOADS; ++k) reinterpret_cast<uint4*>(tile)[threadIdx.x + k * kThreads] = raw[k];
+  for (int k = 0; k < LOADS; ++k) reinterpret_cast<uint4*>(tile)[threadIdx.x + k * T] = raw[k];
   if (threadIdx.x < 128) reinterpret_cast<uint32_t*>(sfb)[threadIdx.x] = 0;
   __syncthreads();
-  const int c = threadIdx.x % D;
-  constexpr int KB_PER_THREAD = 4 * D / kThreads;  // 2 (D=128) or 1 (D=64)
+  const int cp = threadIdx.x % (D / 2);            // column pair: columns 2cp, 2cp+1
+  const int kb = threadIdx.x / (D / 2);            // key block 0..3
+  uint32_t w[32];
+  uint32_t m = 0;
 #pragma unroll
-  for (int s = 0; s < KB_PER_THREAD; ++s) {
-    const int kb = (threadIdx.x / D) * KB_PER_THREAD + s;
+  for (int i = 0; i < 32; ++i) {
+    w[i] = tile[(kb * 32 + i) * (D / 2) + cp];
+    m = __vmaxu2(m, w[i] & 0x7FFF7FFFu);
+  }
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {                    // low half = column 2cp, high half = column 2cp+1
+    const uint32_t u = mx_scale_byte_bf16(c ? (m >> 16) : (m & 0xFFFFu));
     float v[32];
-    float a = 0.f;
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      v[i] = __bfloat162float(tile[(kb * 32 + i) * D + c]);
-      a = fmaxf(a, fabsf(v[i]));
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(c ? (w[i] & 0xFFFF0000u) : (w[i] << 16));
+    if (u >= 2u) {
+      const float s6 = __uint_as_float(((256u - u) << 23) | 0x400000u);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] *= s6;
+    } else {
+      const float inv = mx_inv_amplitude(u);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = (v[i] * inv) * 6.0f;
     }
-    const uint32_t u = mx_scale_byte(a);
-    const float inv = mx_inv_amplitude(u);
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = (v[i] * inv) * 6.0f;
     uint4 out;
     out.x = cvt_e2m1x8(v);
     out.y = cvt_e2m1x8(v + 8);
     out.z = cvt_e2m1x8(v + 16);
     out.w = cvt_e2m1x8(v + 24);
-    packed[((bh * D + c) * (size_t)(N / 2) + (size_t)kt * 64 + kb * 16) / 16] = out;
-    sfb[c * 4 + kb] = (uint8_t)u;
+    const int col = 2 * cp + c;
+    packed[((bh * D + col) * (size_t)(N / 2) + (size_t)kt * 64 + kb * 16) / 16] = out;
+    sfb[col * 4 + kb] = (uint8_t)u;
   }
   __syncthreads();
   if (threadIdx.x < 128) {
@@ -251,8 +264,8 @@ int launch_quantize(const void* x, int fmt, int role, int B, int H, int N, int d
     else          quant_mx_rows_kernel<64><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
   } else if (fmt == FP4ATTN_FMT_MXFP4) {
     dim3 g2(N / 128, B * H);
-    if (d == 128) quant_mx_v_kernel<128><<<g2, kThreads, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
-    else          quant_mx_v_kernel<64><<<g2, kThreads, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
+    if (d == 128) quant_mx_v_kernel<128><<<g2, 256, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
+    else          quant_mx_v_kernel<64><<<g2, 128, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
   } else {
     const int n_partials = (int)(grid < (unsigned)kMaxPartials ? grid : kMaxPartials);
     amax_partials_kernel<<<n_partials, kThreads, 0, st>>>(xs, n_groups, partials);

@@ -156,3 +156,20 @@ def test_invalid_arguments_are_rejected_before_launch():
     x = torch.zeros((1, 1, 128, 128), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(Bd.Fp4AttnError):
         Bd.fp4attn_quantize(x, Bd.FMT_NVFP4, Bd.ROLE_V)
+
+
+def test_bounded_wait_times_out_and_reports_status():
+    """Failure detection without a GPU fault: a wait that nothing satisfies runs out after its
+    limit, the warp returns normally with the time-out status, and the context keeps working."""
+    import time
+    from paper_2609_04105_b200 import binding as Bd
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t0 = time.perf_counter()
+    Bd.fp4attn_selftest_bounded_wait(1 << 26, status)          # ~35 ms at 1.9 GHz
+    torch.cuda.synchronize()
+    assert int(status.item()) == Bd.ERR_TIMEOUT
+    assert time.perf_counter() - t0 < 5.0
+    x = torch.ones(8, device="cuda")                            # the context is still usable
+    assert float((x + 1).sum()) == 16.0
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_selftest_bounded_wait(0, status)
