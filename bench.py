@@ -124,7 +124,7 @@ def _blas_threads():
         return len(os.sched_getaffinity(0))
 
 
-def oracle_sample(w, q, k, v, heads, rows):
+def oracle_sample(w, q, k, v, heads, rows, p_map="ideal"):
     """Runs the oracle (as it stands) on a bounded sample: the given (b, h) pairs and query rows.
     Returns seconds, equivalent TFLOP/s, and its outputs."""
     from oracle import attention as A
@@ -144,7 +144,7 @@ def oracle_sample(w, q, k, v, heads, rows):
     else:
         qd, kd = Qz.quantize_qk(qs, "mx"), Qz.quantize_qk(ks, "mx")
     vd = Qz.quantize_v(vs)
-    O, lse = A.direct_p_forward(qd, kd, vd, rows=rows, heads=[(0, i) for i in range(len(heads))])
+    O, lse = A.direct_p_forward(qd, kd, vd, rows=rows, heads=[(0, i) for i in range(len(heads))], p_map=p_map)
     dt = time.perf_counter() - t0
     n_rows = w.N if rows is None else len(rows)
     flops = 4.0 * len(heads) * n_rows * w.N * w.d
@@ -234,6 +234,7 @@ def run_cuda(args, w):
     qws = torch.empty(max(16, Bd.lib().fp4attn_quantize_workspace_bytes(w.qk_fmt, 0, B, H, N, d)), dtype=torch.uint8, device=dev)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)      # > 126 MB L2
     launches_per_step = 4 if w.qk_fmt == I.FMT_MXFP4 else 6
+    pmap = Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_IDEAL
     state = {}
 
     def step(ev=None):
@@ -242,7 +243,7 @@ def run_cuda(args, w):
         vd = Bd.fp4attn_quantize(dv, Bd.FMT_MXFP4, Bd.ROLE_V)
         if ev is not None:
             ev[0].record()
-        Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status)
+        Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status, p_map=pmap)
         if ev is not None:
             ev[1].record()
         state["ops"] = (qd, kd, vd)
@@ -351,6 +352,17 @@ def run_cuda(args, w):
             torch.cuda.synchronize()
             ms = a.elapsed_time(b) / n_it
             sweep[name] = {"workload": _workload_text(ww), "attn_ms": ms, "attn_tflops": ww.flops / (ms * 1e-3) / 1e12}
+            # the same operands through the affine classifier (the paper's `fast` code map)
+            for _ in range(2):
+                Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status, p_map=Bd.PMAP_AFFINE)
+            a.record()
+            for _ in range(n_it):
+                Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status, p_map=Bd.PMAP_AFFINE)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / n_it
+            sweep[name]["affine_attn_ms"] = ms
+            sweep[name]["affine_attn_tflops"] = ww.flops / (ms * 1e-3) / 1e12
             del sq, sk, sv, so
             torch.cuda.empty_cache()
 
@@ -366,7 +378,7 @@ def run_cuda(args, w):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate)", "data": "synthetic",
-        "config": {"workload": _workload_text(w), "step": "quantize Q,K,V + attention forward",
+        "config": {"workload": _workload_text(w), "step": "quantize Q,K,V + attention forward", "p_map": args.p_map,
                    "l2": "flushed between steps (256 MiB fill, outside the step's events)",
                    "flops": "4*B*H*N^2*d", "parallelism": f"replica x{world}, (batch, head) units, no collective"},
         "attn_only": {"value": attn_tflops, "unit": UNIT, "ms": attn_launch_ms,
@@ -393,11 +405,11 @@ def run_cuda(args, w):
         rng = np.random.default_rng(7)
         # sized for roughly 10-30 s of host work: cost ~ heads * rows * N * d
         n_rows = min(N, 4096)
-        n_heads = max(1, min(B * H, int(8 * (4096.0 / N) ** 1)))
+        n_heads = max(1, min(B * H, int(24 * (4096.0 / N) ** 1)))
         rows = np.sort(rng.choice(N, size=n_rows, replace=False))
         all_heads = [(b, h) for b in range(B) for h in range(H)]
         heads = [all_heads[i] for i in np.linspace(0, len(all_heads) - 1, n_heads).astype(int)]
-        dt, tf, Oo, Lo = oracle_sample(w, q, k, v, heads, rows)
+        dt, tf, Oo, Lo = oracle_sample(w, q, k, v, heads, rows, args.p_map)
         Og = np.stack([O[b, h].float().cpu().numpy().astype(np.float64)[rows] for b, h in heads])
         rel = max(float(np.linalg.norm(Og[i] - Oo[i]) / np.linalg.norm(Oo[i])) for i in range(len(heads)))
         sample = f"{len(heads)} (batch, head) pairs x {n_rows} seeded query rows of {w.name}, {dt:.1f} s"
@@ -418,6 +430,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the attention-only timings of the other configurations")
+    ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine"],
+                    help="score->code map of the timed path: exact codes (default) or the paper's affine classifier")
     args = ap.parse_args()
     w = I.WORKLOADS[args.workload]
     if args.impl == "reference":

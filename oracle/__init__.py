@@ -11,5 +11,8 @@ Pinned by tests/test_oracle_*.py (run with -m "not gpu"):
   quantize.py   MXFP4 / NVFP4 operand quantizers -> closed forms, brute force, error bounds
   attention.py  tiled Direct-P forward          -> tile-size / tile-order invariance, V == 1,
                                                   equal keys, dominant key, brute-force exact
-                                                  attention on losslessly representable inputs
+                                                  attention on losslessly representable inputs;
+                                                  affine code map -> its printed decision boundaries
+                                                  (t_j - B)/A, the same invariants, the paper's
+                                                  all-MXFP4 accuracy band
 """

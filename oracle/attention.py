@@ -22,6 +22,13 @@ Readings where the paper leaves a choice (listed in the design notes of the repo
   * LSE is the natural log of the represented denominator.
 
 Everything else is float64.
+
+Second code map (p_map="affine", Eq. "affine-code-map"): q = Q_E2M1(max(0, A x + B)) with the paper's
+generic `fast` fit A = 1.50, B = 1.20 by default.  The paper folds the score transform, e_B and the
+log2 6 term into the coefficients of one fused multiply-add; that arithmetic is fixed here in
+float32 so that a GPU reproduces the codes bit for bit:
+    cA = fl32(A * c32),  bA = fl32(A * fl32(log2 6 - E_B) + B)  (one fma),  u = fl32(s32 * cA + bA)  (one fma).
+Block exponents, reference, denominator and output are unchanged.
 """
 from __future__ import annotations
 
@@ -60,7 +67,15 @@ def scores_fp32(qd: dict, kd: dict, b: int, h: int, rows=None) -> np.ndarray:
     return (A @ Bm.T).astype(np.float32)
 
 
-def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int = 128, tile_order=None):
+def _fma32(a, b, c):
+    """fl32(a*b + c) for float32 inputs: the product is exact in float64, the sum is rounded once more
+    only when it needs more than 53 bits (not the case for the magnitudes used here)."""
+    return (np.asarray(a, np.float32).astype(np.float64) * np.asarray(b, np.float32).astype(np.float64)
+            + np.asarray(c, np.float32).astype(np.float64)).astype(np.float32)
+
+
+def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int = 128, tile_order=None,
+                  p_map: str = "ideal", affine=(1.5, 1.2)):
     """Direct-P online softmax + PV for a set of query rows of one (batch, head).
 
     s32  [R, N] float32 tensor-core-facing scores;  Vhat [N, d] float64 reconstructed V.
@@ -76,6 +91,9 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
     O = np.zeros((R, Vhat.shape[1]))
     codes_all = np.zeros((R, N), dtype=np.uint8)
     EB_all = np.zeros((R, N // P_BLOCK), dtype=np.int64)
+    assert p_map in ("ideal", "affine")
+    A32, B32 = np.float32(affine[0]), np.float32(affine[1])
+    cA = np.float32(A32 * np.float32(c32))
     order = range(N // tile) if tile_order is None else tile_order
     for t in order:
         j0 = t * tile
@@ -89,9 +107,14 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
             E_B = np.ceil(y32[:, bj:bj + P_BLOCK].max(axis=1).astype(np.float64))
             e_B = E_B - mu
             live = (e_B + 127) >= 1
-            b_B = np.float32(LOG2_6_32 - E_B.astype(np.float32)).astype(np.float64)
-            x = yx[:, bj:bj + P_BLOCK] + b_B[:, None]
-            code = e2m1_encode_mag(np.exp2(x))
+            b_B32 = np.float32(LOG2_6_32 - E_B.astype(np.float32))
+            if p_map == "ideal":
+                x = yx[:, bj:bj + P_BLOCK] + b_B32.astype(np.float64)[:, None]
+                code = e2m1_encode_mag(np.exp2(x))
+            else:
+                bA = _fma32(A32, b_B32, B32)
+                u = _fma32(s32[:, bj:bj + P_BLOCK], cA, bA[:, None])
+                code = e2m1_encode_mag(np.maximum(u, np.float32(0)).astype(np.float64))
             code = np.where(live[:, None], code, 0).astype(np.uint8)
             q = E2M1_VALUES[code]
             alpha = np.where(live, np.exp2(e_B), 0.0)
@@ -106,7 +129,7 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
 
 
 def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int = 128,
-                     rows=None, heads=None, tile_order=None):
+                     rows=None, heads=None, tile_order=None, p_map: str = "ideal", affine=(1.5, 1.2)):
     """Whole-operator oracle.  qd/kd/vd come from oracle.quantize.quantize_qk / quantize_v.
 
     rows : optional 1-D index array of query rows evaluated for every (b, h) (rows are
@@ -120,7 +143,7 @@ def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int
     for (b, h) in heads:
         s32 = scores_fp32(qd, kd, b, h, rows)
         Vhat = dequantize({**vd, "nib": vd["nib"][b, h][None, None], "sf": vd["sf"][b, h][None, None]})[0, 0].T
-        O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order)
+        O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order, p_map, affine)
         Os.append(O)
         Ls.append(lse)
     return np.stack(Os), np.stack(Ls)

@@ -14,6 +14,7 @@ import torch
 
 FMT_MXFP4, FMT_NVFP4 = 0, 1
 ROLE_Q, ROLE_K, ROLE_V = 0, 1, 2
+PMAP_IDEAL, PMAP_AFFINE = 0, 1
 ERR_TIMEOUT = 7
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -35,7 +36,8 @@ class _Operands(ctypes.Structure):
     _fields_ = [("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
                 ("q_sf", ctypes.c_void_p), ("k_sf", ctypes.c_void_p), ("v_sf", ctypes.c_void_p),
                 ("q_G", ctypes.c_void_p), ("k_G", ctypes.c_void_p),
-                ("qk_fmt", ctypes.c_int), ("softmax_scale", ctypes.c_float)]
+                ("qk_fmt", ctypes.c_int), ("softmax_scale", ctypes.c_float),
+                ("p_map", ctypes.c_int), ("affine_a", ctypes.c_float), ("affine_b", ctypes.c_float)]
 
 
 def _load() -> ctypes.CDLL:
@@ -138,8 +140,10 @@ def fp4attn_quantize_nvfp4_noalloc(x: torch.Tensor, role: int, packed: torch.Ten
 
 def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, softmax_scale: float = 0.0,
                 out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
-                status: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
-    """Direct-P attention forward on quantized operands -> (O bf16 [B,H,N,d], LSE fp32 [B,H,N])."""
+                status: Optional[torch.Tensor] = None, p_map: int = PMAP_IDEAL, affine_a: float = 0.0,
+                affine_b: float = 0.0) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Direct-P attention forward on quantized operands -> (O bf16 [B,H,N,d], LSE fp32 [B,H,N]).
+    p_map selects the exact code map or the affine classifier (affine_a = 0: A = 1.5, B = 1.2)."""
     B, H, N, d = q.shape
     assert k.shape == q.shape and v.shape == q.shape and q.fmt == k.fmt and v.fmt == FMT_MXFP4
     dev = q.packed.device
@@ -149,7 +153,7 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
         lse = torch.empty((B, H, N), dtype=torch.float32, device=dev)
     ops = _Operands(q.packed.data_ptr(), k.packed.data_ptr(), v.packed.data_ptr(),
                     q.scales.data_ptr(), k.scales.data_ptr(), v.scales.data_ptr(),
-                    _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale))
+                    _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b))
     _check(lib().fp4attn_fwd(ctypes.byref(ops), B, H, N, d, out.data_ptr(), lse.data_ptr(), _ptr(status), _stream()),
            "fp4attn_fwd")
     return out, lse

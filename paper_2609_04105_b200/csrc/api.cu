@@ -92,7 +92,7 @@ extern "C" int fp4attn_attention_host(const void* q_host, const void* k_host, co
                               i < 2 ? G + i : nullptr, ws + p.qws, workspace_bytes - p.qws, stream);
     if (rc != FP4ATTN_OK) return rc;
   }
-  fp4attn_operands ops;
+  fp4attn_operands ops = {};
   ops.q = ws + p.packed[0]; ops.k = ws + p.packed[1]; ops.v = ws + p.packed[2];
   ops.q_sf = ws + p.sf[0]; ops.k_sf = ws + p.sf[1]; ops.v_sf = ws + p.sf[2];
   ops.q_G = qk_fmt == FP4ATTN_FMT_NVFP4 ? G : nullptr;

@@ -93,6 +93,7 @@ struct AttnParams {
   int N, stages;           // keys, N / 128
   int n_items;             // B * H * N / 128
   float c_base;            // fl32(log2(e) * softmax_scale)
+  float aff_a, aff_b;      // affine classifier u = max(0, A x + B) (only read by the affine variant)
 };
 
 // barrier slots (8 bytes each)
@@ -163,31 +164,50 @@ __device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float&
   p1 = __uint_as_float(th * 0x800000u + qh);
 }
 
-// One N32 score fragment of one row: E_B = ceil(max y) and the codes q = Q_E2M1(2^(y - E_B + log2 6)).
-// Nothing here depends on the row reference.
-__device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, int& E, uint32_t* words) {
+// One N32 score fragment of one row: E_B = ceil(max y) and the codes.  Nothing here depends on the
+// row reference.
+//   ideal map  (Eq. "ideal-code-path"):  q = Q_E2M1(2^x),            x = y - E_B + log2 6
+//   affine map (Eq. "affine-code-map"):  q = Q_E2M1(max(0, A x + B)), folded into one fused multiply-add
+//                                        per element: u = s * fl32(A c) + fma(A, log2 6 - E_B, B)
+template <bool AFFINE>
+__device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, float A, float B, int& E, uint32_t* words) {
   const float LOG2_6 = 2.5849625007211560f;
   E = (int)ceilf(__fmul_rn(max32(sraw), c32));
   const float bB = __fsub_rn(LOG2_6, (float)E);
+  if (AFFINE) {
+    const float cA = __fmul_rn(A, c32), bA = __fmaf_rn(A, bB, B);
 #pragma unroll
-  for (int w = 0; w < 4; ++w) {
-    float pv[8];
+    for (int w = 0; w < 4; ++w) {
+      float pv[8];
 #pragma unroll
-    for (int i = 0; i < 8; i += 2) {
-      float x0, x1;
-      fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), c32, bB, x0, x1);
-      if ((FP4ATTN_POLY_MASK >> (4 * w + i / 2)) & 1u) {
-        exp2_poly2(x0, x1, pv[i], pv[i + 1]);
-      } else {
-        pv[i] = ex2_approx(x0);
-        pv[i + 1] = ex2_approx(x1);
-      }
+      for (int i = 0; i < 8; i += 2)
+        fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), cA, bA, pv[i], pv[i + 1]);
+      words[w] = cvt_e2m1x8_relu(pv);                            // the conversion clamps negative inputs to +0
     }
-    words[w] = cvt_e2m1x8(pv);
+  } else {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      float pv[8];
+#pragma unroll
+      for (int i = 0; i < 8; i += 2) {
+        float x0, x1;
+        fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), c32, bB, x0, x1);
+        if ((FP4ATTN_POLY_MASK >> (4 * w + i / 2)) & 1u) {
+          exp2_poly2(x0, x1, pv[i], pv[i + 1]);
+        } else {
+          pv[i] = ex2_approx(x0);
+          pv[i + 1] = ex2_approx(x1);
+        }
+      }
+      words[w] = cvt_e2m1x8(pv);
+    }
   }
 }
 
-template <int D, bool NV>
+// AFFINE selects the affine classifier and, with it, stage-wise correction (both 64-key tiles of a stage
+// per pass): without the SFU work the teams outrun a tile-by-tile correction chain, while the exact
+// map runs ~2 % faster with the tile-by-tile chain, which staggers the teams.
+template <int D, bool NV, bool AFFINE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -218,7 +238,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       mbar_init(bar(BAR_QFREE0 + b), 1);
       mbar_init(bar(BAR_SFULL0 + b), 1);
       mbar_init(bar(BAR_SEMPTY0 + b), 8);      // both teams of the pair, four warps each
-      mbar_init(bar(BAR_PFULL0 + b), 8);       // four correction warps, two tiles
+      mbar_init(bar(BAR_PFULL0 + b), AFFINE ? 4 : 8);   // four correction warps, once per tile (per stage if AFFINE)
       mbar_init(bar(BAR_PFREE0 + b), 1);
     }
     mbar_init(bar(BAR_OFULL), 1);
@@ -398,15 +418,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     int i = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i, g0 += T2) {
       int mu = -(1 << 28);
-      int pu0 = 0, pu1 = 0;                                     // bytes written for the previous tile
-      for (int j = 0; j < 2 * T2; ++j) {
-        const uint32_t g = g0 + (j >> 1);
-        const int h = j & 1, pr = g & 1, slot = 2 * pr + h;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + slot), (g >> 1) & 1, abortf));
+      int pu0 = 0, pu1 = 0;                                     // bytes written for the previous tile (tile-by-tile mode)
+      // one pass per 64-key tile, or (AFFINE) one pass per 128-key stage covering both of its tiles
+      const int n_pass = AFFINE ? T2 : 2 * T2;
+      for (int j = 0; j < n_pass; ++j) {
+        const uint32_t g = g0 + (AFFINE ? j : (j >> 1));
+        const int h = AFFINE ? 0 : (j & 1), pr = g & 1;
+        const uint32_t par = (g >> 1) & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + 2 * pr + h), par, abortf));
+        if (AFFINE && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + 2 * pr + 1), par, abortf));
         if (!ok) break;
-        const int2 mt = *reinterpret_cast<const int2*>(sgen + C::OFF_META + C::META_BYTES * slot + row * 8);
+        const int2 ma = *reinterpret_cast<const int2*>(sgen + C::OFF_META + C::META_BYTES * (2 * pr + h) + row * 8);
+        const int2 mb = AFFINE ? *reinterpret_cast<const int2*>(sgen + C::OFF_META + C::META_BYTES * (2 * pr + 1) + row * 8) : ma;
         uint8_t* psf = sgen + C::OFF_PSF + 512 * pr + lane * 16 + quarter * 4;
-        const int Emax = max(mt.x, mt.y);
+        const int Emax = max(max(ma.x, ma.y), max(mb.x, mb.y));
         const bool need = Emax > mu + kLazyShift;
         if (__any_sync(0xffffffffu, need)) {
           float f = 1.0f;
@@ -418,14 +443,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (delta > 126 && Emax <= mu + 126 + kLazyShift) delta = 126;
             f = (delta > 126) ? 0.f : __uint_as_float((uint32_t)(127 - delta) << 23);
             mu = (delta > 126) ? Emax + kRefHeadroom : mu + delta;
-            if (h) {
+            if (!AFFINE && h) {
               // the stage's first tile is not in O yet (both tiles are issued together): move its bytes
-              pu0 = max(pu0 - delta, 0);                        // (delta as computed above: new reference - old)
+              pu0 = max(pu0 - delta, 0);
               pu1 = max(pu1 - delta, 0);
               *reinterpret_cast<uint16_t*>(psf) = (uint16_t)(pu0 | (pu1 << 8));
             }
           }
-          if (j >= 2) {
+          if (AFFINE ? (j >= 1) : (j >= 2)) {
             // O holds the item's earlier stages once their PV has landed
             const uint32_t gprev = g - 1;
             ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFREE0 + (gprev & 1)), (gprev >> 1) & 1, abortf));
@@ -446,10 +471,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         // A block more than 126 octaves below the reference is a zero block: it gets the smallest
         // byte (2^-127, below 2^-60 of the row's mass by construction) in numerator and row sum alike.
-        const int u0 = mt.x - mu + 127, u1 = mt.y - mu + 127;
-        pu0 = max(u0, 0);
-        pu1 = max(u1, 0);
-        *reinterpret_cast<uint16_t*>(psf + 2 * h) = (uint16_t)(pu0 | (pu1 << 8));
+        pu0 = max(ma.x - mu + 127, 0);
+        pu1 = max(ma.y - mu + 127, 0);
+        if (AFFINE) {
+          const uint32_t u2 = (uint32_t)max(mb.x - mu + 127, 0), u3 = (uint32_t)max(mb.y - mu + 127, 0);
+          *reinterpret_cast<uint32_t*>(psf) = (uint32_t)pu0 | ((uint32_t)pu1 << 8) | (u2 << 16) | (u3 << 24);
+        } else {
+          *reinterpret_cast<uint16_t*>(psf + 2 * h) = (uint16_t)(pu0 | (pu1 << 8));
+        }
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + pr));
@@ -531,13 +560,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         int E0, E1;
         tmem_ld_32x32b_x32(tS, sraw);
         tmem_wait_ld();
-        direct_p_block(sraw, c32, E0, w0);
+        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, E0, w0);
         tmem_ld_32x32b_x32(tS + 32, sraw);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(sempty);                     // pair may take the stage after next
-        direct_p_block(sraw, c32, E1, w1);
+        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, E1, w1);
         if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
         if (!ok) break;
         *reinterpret_cast<uint4*>(pbuf) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
@@ -635,12 +664,12 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint6
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool NV>
+template <int D, bool NV, bool AFFINE>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
   using C = Cfg<D, NV>;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV, AFFINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
       return FP4ATTN_ERR_CUDA;
     attr_set = true;
   }
@@ -655,7 +684,7 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return FP4ATTN_ERR_CUDA;
   const unsigned grid = (unsigned)(prm.n_items < sms ? prm.n_items : sms);     // persistent: one CTA per SM
-  attn_fwd_kernel<D, NV><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, tmO, prm);
+  attn_fwd_kernel<D, NV, AFFINE><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, tmO, prm);
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
 
@@ -673,6 +702,9 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   if (!(d == 64 || d == 128) || N < 128 || N % 128 != 0) return FP4ATTN_ERR_UNSUPPORTED_SHAPE;
   if ((uint64_t)B * H * N >= (1ull << 31)) return FP4ATTN_ERR_UNSUPPORTED_SHAPE;
   if (!(ops->softmax_scale >= 0.f)) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->p_map != FP4ATTN_PMAP_IDEAL && ops->p_map != FP4ATTN_PMAP_AFFINE) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->p_map == FP4ATTN_PMAP_AFFINE && !(ops->affine_a >= 0.f && ops->affine_a < 16.f && fabsf(ops->affine_b) < 16.f))
+    return FP4ATTN_ERR_INVALID_ARG;
   const uintptr_t a128 = (uintptr_t)ops->q | (uintptr_t)ops->k | (uintptr_t)ops->v | (uintptr_t)ops->q_sf |
                          (uintptr_t)ops->k_sf | (uintptr_t)ops->v_sf;
   if ((a128 & 127) || ((uintptr_t)O & 15) || ((uintptr_t)LSE & 3)) return FP4ATTN_ERR_ALIGNMENT;
@@ -687,8 +719,20 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.c_base = 1.4426950408889634f * scale;                        // fl32(log2e_32 * scale_32)
   cudaStream_t st = (cudaStream_t)stream;
   const bool nv = ops->qk_fmt == FP4ATTN_FMT_NVFP4;
-  if (d == 128) return nv ? launch_attn<128, true>(ops, B, H, N, prm, st) : launch_attn<128, false>(ops, B, H, N, prm, st);
-  return nv ? launch_attn<64, true>(ops, B, H, N, prm, st) : launch_attn<64, false>(ops, B, H, N, prm, st);
+  const bool affine = ops->p_map == FP4ATTN_PMAP_AFFINE;
+  prm.aff_a = ops->affine_a != 0.f ? ops->affine_a : 1.5f;         // the paper's generic `fast` fit
+  prm.aff_b = ops->affine_a != 0.f ? ops->affine_b : 1.2f;
+  const int variant = (d == 128 ? 4 : 0) | (nv ? 2 : 0) | (affine ? 1 : 0);
+  switch (variant) {
+    case 0: return launch_attn<64, false, false>(ops, B, H, N, prm, st);
+    case 1: return launch_attn<64, false, true>(ops, B, H, N, prm, st);
+    case 2: return launch_attn<64, true, false>(ops, B, H, N, prm, st);
+    case 3: return launch_attn<64, true, true>(ops, B, H, N, prm, st);
+    case 4: return launch_attn<128, false, false>(ops, B, H, N, prm, st);
+    case 5: return launch_attn<128, false, true>(ops, B, H, N, prm, st);
+    case 6: return launch_attn<128, true, false>(ops, B, H, N, prm, st);
+    default: return launch_attn<128, true, true>(ops, B, H, N, prm, st);
+  }
 }
 
 extern "C" int fp4attn_mma_peak_probe(int iters, unsigned long long* cycles_out, fp4attn_stream_t stream) {

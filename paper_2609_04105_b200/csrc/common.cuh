@@ -31,6 +31,20 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float* v) {
   return w;
 }
 
+// same, with negative inputs clamped to +0 by the conversion itself
+__device__ __forceinline__ uint32_t cvt_e2m1x8_relu(const float* v) {
+  uint32_t w;
+  asm("{\n\t.reg .b8 t0, t1, t2, t3;\n\t"
+      "cvt.rn.satfinite.relu.e2m1x2.f32 t0, %2, %1;\n\t"
+      "cvt.rn.satfinite.relu.e2m1x2.f32 t1, %4, %3;\n\t"
+      "cvt.rn.satfinite.relu.e2m1x2.f32 t2, %6, %5;\n\t"
+      "cvt.rn.satfinite.relu.e2m1x2.f32 t3, %8, %7;\n\t"
+      "mov.b32 %0, {t0, t1, t2, t3};\n\t}"
+      : "=r"(w)
+      : "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]));
+  return w;
+}
+
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& raw, float* v) {
   const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll

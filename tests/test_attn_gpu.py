@@ -173,3 +173,64 @@ def test_bounded_wait_times_out_and_reports_status():
     assert float((x + 1).sum()) == 16.0
     with pytest.raises(Bd.Fp4AttnError):
         Bd.fp4attn_selftest_bounded_wait(0, status)
+
+
+# ------------------------------------------------------------------ affine classifier (p_map = AFFINE)
+def run_gpu_affine(w, q, k, v, a=0.0, b=0.0):
+    from paper_2609_04105_b200 import binding as Bd
+    qd = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q)
+    kd = Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+    vd = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    O, lse = Bd.fp4attn_fwd(qd, kd, vd, status=status, p_map=Bd.PMAP_AFFINE, affine_a=a, affine_b=b)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return O.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+
+
+AFFINE_CASES = [
+    ("cfg1", dict(), (0.0, 0.0)),
+    ("cfg1", dict(N=384, H=3), (1.6, 0.95)),                 # the paper's second constant pair
+    ("cfg1", dict(d=64, N=512), (0.0, 0.0)),
+    ("cfg3", dict(B=2, H=2, N=512), (0.0, 0.0)),
+    ("cfg3", dict(B=1, H=2, N=384, d=128), (0.0, 0.0)),
+    ("cfg4", dict(H=2, N=1024), (0.0, 0.0)),
+    ("cfg2", dict(B=2, H=3, N=2304), (0.0, 0.0)),
+]
+
+
+@pytest.mark.parametrize("name,kw,ab", AFFINE_CASES)
+def test_affine_map_matches_oracle_elementwise(name, kw, ab):
+    """Same tolerances as the exact map: the classifier's arithmetic is fixed in fp32 on both sides,
+    so the codes agree bit for bit and only accumulation order and bf16 rounding differ."""
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu_affine(w, q, k, v, *ab)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    aff = ab if ab[0] else (1.5, 1.2)
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, p_map="affine", affine=aff)
+    check_heads(Og, Lg, Oo, Lo, heads)
+
+
+def test_affine_map_config2_full_size_sampled_rows():
+    w = I.WORKLOADS["cfg2"]
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu_affine(w, q, k, v)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    rng = np.random.default_rng(12)
+    rows = np.sort(rng.choice(w.N, size=192, replace=False))
+    heads = [(0, 0), (1, 7), (3, 15)]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows, p_map="affine")
+    check_heads(Og, Lg, Oo, Lo, heads, rows)
+
+
+def test_unknown_p_map_is_rejected():
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg1"], N=128)
+    q, k, v = I.make_qkv(w)
+    qd = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q)
+    kd = Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+    vd = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_fwd(qd, kd, vd, p_map=7)
