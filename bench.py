@@ -124,7 +124,7 @@ def _blas_threads():
         return len(os.sched_getaffinity(0))
 
 
-def oracle_sample(w, q, k, v, heads, rows, p_map="ideal"):
+def oracle_sample(w, q, k, v, heads, rows, p_map="ideal", p_scale="ceil"):
     """Runs the oracle (as it stands) on a bounded sample: the given (b, h) pairs and query rows.
     Returns seconds, equivalent TFLOP/s, and its outputs."""
     from oracle import attention as A
@@ -144,7 +144,7 @@ def oracle_sample(w, q, k, v, heads, rows, p_map="ideal"):
     else:
         qd, kd = Qz.quantize_qk(qs, "mx"), Qz.quantize_qk(ks, "mx")
     vd = Qz.quantize_v(vs)
-    O, lse = A.direct_p_forward(qd, kd, vd, rows=rows, heads=[(0, i) for i in range(len(heads))], p_map=p_map)
+    O, lse = A.direct_p_forward(qd, kd, vd, rows=rows, heads=[(0, i) for i in range(len(heads))], p_map=p_map, p_scale=p_scale)
     dt = time.perf_counter() - t0
     n_rows = w.N if rows is None else len(rows)
     flops = 4.0 * len(heads) * n_rows * w.N * w.d
@@ -235,6 +235,7 @@ def run_cuda(args, w):
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)      # > 126 MB L2
     launches_per_step = 4 if w.qk_fmt == I.FMT_MXFP4 else 6
     pmap = Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_IDEAL
+    pscale = Bd.PSCALE_THR16 if args.p_scale == "thr16" else Bd.PSCALE_CEIL
     state = {}
 
     def step(ev=None):
@@ -243,7 +244,7 @@ def run_cuda(args, w):
         vd = Bd.fp4attn_quantize(dv, Bd.FMT_MXFP4, Bd.ROLE_V)
         if ev is not None:
             ev[0].record()
-        Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status, p_map=pmap)
+        Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status, p_map=pmap, p_scale_rule=pscale)
         if ev is not None:
             ev[1].record()
         state["ops"] = (qd, kd, vd)
@@ -378,7 +379,7 @@ def run_cuda(args, w):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate)", "data": "synthetic",
-        "config": {"workload": _workload_text(w), "step": "quantize Q,K,V + attention forward", "p_map": args.p_map,
+        "config": {"workload": _workload_text(w), "step": "quantize Q,K,V + attention forward", "p_map": args.p_map, "p_scale": args.p_scale,
                    "l2": "flushed between steps (256 MiB fill, outside the step's events)",
                    "flops": "4*B*H*N^2*d", "parallelism": f"replica x{world}, (batch, head) units, no collective"},
         "attn_only": {"value": attn_tflops, "unit": UNIT, "ms": attn_launch_ms,
@@ -409,7 +410,7 @@ def run_cuda(args, w):
         rows = np.sort(rng.choice(N, size=n_rows, replace=False))
         all_heads = [(b, h) for b in range(B) for h in range(H)]
         heads = [all_heads[i] for i in np.linspace(0, len(all_heads) - 1, n_heads).astype(int)]
-        dt, tf, Oo, Lo = oracle_sample(w, q, k, v, heads, rows, args.p_map)
+        dt, tf, Oo, Lo = oracle_sample(w, q, k, v, heads, rows, args.p_map, args.p_scale)
         Og = np.stack([O[b, h].float().cpu().numpy().astype(np.float64)[rows] for b, h in heads])
         rel = max(float(np.linalg.norm(Og[i] - Oo[i]) / np.linalg.norm(Oo[i])) for i in range(len(heads)))
         sample = f"{len(heads)} (batch, head) pairs x {n_rows} seeded query rows of {w.name}, {dt:.1f} s"
@@ -430,6 +431,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the attention-only timings of the other configurations")
+    ap.add_argument("--p-scale", default="ceil", choices=["ceil", "thr16"],
+                    help="block-exponent rule of P: ceiling (default) or floor(max y + log2 1.6)")
     ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine"],
                     help="score->code map of the timed path: exact codes (default) or the paper's affine classifier")
     args = ap.parse_args()

@@ -125,6 +125,12 @@ int fp4attn_quantize_nvfp4_noalloc(const void* x_bf16, int role, int B, int H, i
                                    void* packed_out, void* scales_out, float* tensor_scale_out,
                                    fp4attn_stream_t stream);
 
+/* how the integer exponent E_B of a 32-key probability block follows from its maximum y (Eq. "mx-scale"
+ * allows either neighbouring power of two as the amplitude) */
+enum { FP4ATTN_PSCALE_CEIL = 0,    /* E_B = ceil(max y): nothing saturates                              */
+       FP4ATTN_PSCALE_THR16 = 1 }; /* E_B = floor(fl32(max y + fl32(log2 1.6))): the block maximum lands in
+                                      [3.75, 7.5) code units, values above 6 saturate; lower P error    */
+
 typedef struct {
   const void *q, *k, *v;            /* packed E2M1 (V transposed)                           */
   const void *q_sf, *k_sf, *v_sf;   /* scale atoms                                           */
@@ -134,6 +140,7 @@ typedef struct {
   int p_map;                        /* FP4ATTN_PMAP_IDEAL or FP4ATTN_PMAP_AFFINE             */
   float affine_a, affine_b;         /* classifier constants; affine_a == 0 selects the
                                        paper's generic fit A = 1.50, B = 1.20                */
+  int p_scale_rule;                 /* FP4ATTN_PSCALE_CEIL or FP4ATTN_PSCALE_THR16           */
 } fp4attn_operands;
 
 /*

@@ -14,5 +14,6 @@ Pinned by tests/test_oracle_*.py (run with -m "not gpu"):
                                                   attention on losslessly representable inputs;
                                                   affine code map -> its printed decision boundaries
                                                   (t_j - B)/A, the same invariants, the paper's
-                                                  all-MXFP4 accuracy band
+                                                  all-MXFP4 accuracy band; threshold amplitude rule
+                                                  -> closed form, Table "p-range" MXFP4 row
 """

@@ -29,6 +29,12 @@ log2 6 term into the coefficients of one fused multiply-add; that arithmetic is 
 float32 so that a GPU reproduces the codes bit for bit:
     cA = fl32(A * c32),  bA = fl32(A * fl32(log2 6 - E_B) + B)  (one fma),  u = fl32(s32 * cA + bA)  (one fma).
 Block exponents, reference, denominator and output are unchanged.
+
+Second block-exponent rule (p_scale="thr16"): Eq. "mx-scale" allows either neighbouring power of two
+as the amplitude; besides the ceiling (default) the oracle offers the threshold rule
+E_B = floor(fl32(max y + fl32(log2 1.6))), i.e. alpha_B = 2^floor(log2(1.6 a_B)): the block maximum then
+lands in [3.75, 7.5) code units and values above 6 saturate.  It reproduces the MXFP4 rows of Table
+"p-range" (pinned in the tests) and lowers the P error.
 """
 from __future__ import annotations
 
@@ -41,7 +47,16 @@ from .quantize import dequantize
 
 LOG2E_32 = np.float32(1.4426950408889634)
 LOG2_6_32 = np.float32(math.log2(6.0))
+LOG2_1P6_32 = np.float32(math.log2(1.6))
 P_BLOCK = 32
+
+
+def block_exponent(ymax32: np.ndarray, p_scale: str = "ceil") -> np.ndarray:
+    """Integer block exponent E_B from the block maximum of y (float32), as float64 integers."""
+    if p_scale == "ceil":
+        return np.ceil(np.asarray(ymax32, np.float32).astype(np.float64))
+    assert p_scale == "thr16"
+    return np.floor((np.asarray(ymax32, np.float32) + LOG2_1P6_32).astype(np.float32).astype(np.float64))
 
 
 def score_constant(qd: dict, kd: dict, d: int, softmax_scale=None) -> np.float32:
@@ -75,7 +90,7 @@ def _fma32(a, b, c):
 
 
 def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int = 128, tile_order=None,
-                  p_map: str = "ideal", affine=(1.5, 1.2)):
+                  p_map: str = "ideal", affine=(1.5, 1.2), p_scale: str = "ceil"):
     """Direct-P online softmax + PV for a set of query rows of one (batch, head).
 
     s32  [R, N] float32 tensor-core-facing scores;  Vhat [N, d] float64 reconstructed V.
@@ -97,14 +112,15 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
     order = range(N // tile) if tile_order is None else tile_order
     for t in order:
         j0 = t * tile
-        m_tile = np.ceil(y32[:, j0:j0 + tile].max(axis=1).astype(np.float64))
+        m_tile = np.max(np.stack([block_exponent(y32[:, bj:bj + P_BLOCK].max(axis=1), p_scale)
+                                  for bj in range(j0, j0 + tile, P_BLOCK)]), axis=0)
         mu_new = np.maximum(mu, m_tile)
         f = np.where(np.isinf(mu), 0.0, np.exp2(mu - mu_new))     # exact power of two
         L *= f
         O *= f[:, None]
         mu = mu_new
         for bj in range(j0, j0 + tile, P_BLOCK):
-            E_B = np.ceil(y32[:, bj:bj + P_BLOCK].max(axis=1).astype(np.float64))
+            E_B = block_exponent(y32[:, bj:bj + P_BLOCK].max(axis=1), p_scale)
             e_B = E_B - mu
             live = (e_B + 127) >= 1
             b_B32 = np.float32(LOG2_6_32 - E_B.astype(np.float32))
@@ -129,7 +145,8 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
 
 
 def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int = 128,
-                     rows=None, heads=None, tile_order=None, p_map: str = "ideal", affine=(1.5, 1.2)):
+                     rows=None, heads=None, tile_order=None, p_map: str = "ideal", affine=(1.5, 1.2),
+                     p_scale: str = "ceil"):
     """Whole-operator oracle.  qd/kd/vd come from oracle.quantize.quantize_qk / quantize_v.
 
     rows : optional 1-D index array of query rows evaluated for every (b, h) (rows are
@@ -143,7 +160,7 @@ def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int
     for (b, h) in heads:
         s32 = scores_fp32(qd, kd, b, h, rows)
         Vhat = dequantize({**vd, "nib": vd["nib"][b, h][None, None], "sf": vd["sf"][b, h][None, None]})[0, 0].T
-        O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order, p_map, affine)
+        O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order, p_map, affine, p_scale)
         Os.append(O)
         Ls.append(lse)
     return np.stack(Os), np.stack(Ls)

@@ -15,6 +15,7 @@ import torch
 FMT_MXFP4, FMT_NVFP4 = 0, 1
 ROLE_Q, ROLE_K, ROLE_V = 0, 1, 2
 PMAP_IDEAL, PMAP_AFFINE = 0, 1
+PSCALE_CEIL, PSCALE_THR16 = 0, 1
 ERR_TIMEOUT = 7
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -37,7 +38,8 @@ class _Operands(ctypes.Structure):
                 ("q_sf", ctypes.c_void_p), ("k_sf", ctypes.c_void_p), ("v_sf", ctypes.c_void_p),
                 ("q_G", ctypes.c_void_p), ("k_G", ctypes.c_void_p),
                 ("qk_fmt", ctypes.c_int), ("softmax_scale", ctypes.c_float),
-                ("p_map", ctypes.c_int), ("affine_a", ctypes.c_float), ("affine_b", ctypes.c_float)]
+                ("p_map", ctypes.c_int), ("affine_a", ctypes.c_float), ("affine_b", ctypes.c_float),
+                ("p_scale_rule", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:
@@ -141,7 +143,7 @@ def fp4attn_quantize_nvfp4_noalloc(x: torch.Tensor, role: int, packed: torch.Ten
 def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, softmax_scale: float = 0.0,
                 out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
                 status: Optional[torch.Tensor] = None, p_map: int = PMAP_IDEAL, affine_a: float = 0.0,
-                affine_b: float = 0.0) -> Tuple[torch.Tensor, torch.Tensor]:
+                affine_b: float = 0.0, p_scale_rule: int = PSCALE_CEIL) -> Tuple[torch.Tensor, torch.Tensor]:
     """Direct-P attention forward on quantized operands -> (O bf16 [B,H,N,d], LSE fp32 [B,H,N]).
     p_map selects the exact code map or the affine classifier (affine_a = 0: A = 1.5, B = 1.2)."""
     B, H, N, d = q.shape
@@ -153,7 +155,7 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
         lse = torch.empty((B, H, N), dtype=torch.float32, device=dev)
     ops = _Operands(q.packed.data_ptr(), k.packed.data_ptr(), v.packed.data_ptr(),
                     q.scales.data_ptr(), k.scales.data_ptr(), v.scales.data_ptr(),
-                    _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b))
+                    _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b), int(p_scale_rule))
     _check(lib().fp4attn_fwd(ctypes.byref(ops), B, H, N, d, out.data_ptr(), lse.data_ptr(), _ptr(status), _stream()),
            "fp4attn_fwd")
     return out, lse

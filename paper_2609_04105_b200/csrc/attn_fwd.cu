@@ -94,6 +94,7 @@ struct AttnParams {
   int n_items;             // B * H * N / 128
   float c_base;            // fl32(log2(e) * softmax_scale)
   float aff_a, aff_b;      // affine classifier u = max(0, A x + B) (only read by the affine variant)
+  int thr16;               // block exponent rule: 0 = ceil(max y), 1 = floor(max y + log2 1.6)
 };
 
 // barrier slots (8 bytes each)
@@ -170,9 +171,13 @@ __device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float&
 //   affine map (Eq. "affine-code-map"):  q = Q_E2M1(max(0, A x + B)), folded into one fused multiply-add
 //                                        per element: u = s * fl32(A c) + fma(A, log2 6 - E_B, B)
 template <bool AFFINE>
-__device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, float A, float B, int& E, uint32_t* words) {
+__device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, float A, float B, int thr16, int& E,
+                                               uint32_t* words) {
   const float LOG2_6 = 2.5849625007211560f;
-  E = (int)ceilf(__fmul_rn(max32(sraw), c32));
+  const float ymax = __fmul_rn(max32(sraw), c32);
+  // amplitude rule (Eq. "mx-scale" allows either neighbouring power of two): ceiling, or the threshold
+  // rule alpha = 2^floor(log2(1.6 a)) under which values above the amplitude saturate at code 6
+  E = thr16 ? (int)floorf(__fadd_rn(ymax, 0.6780719161033630f)) : (int)ceilf(ymax);
   const float bB = __fsub_rn(LOG2_6, (float)E);
   if (AFFINE) {
     const float cA = __fmul_rn(A, c32), bA = __fmaf_rn(A, bB, B);
@@ -560,13 +565,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         int E0, E1;
         tmem_ld_32x32b_x32(tS, sraw);
         tmem_wait_ld();
-        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, E0, w0);
+        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, p.thr16, E0, w0);
         tmem_ld_32x32b_x32(tS + 32, sraw);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(sempty);                     // pair may take the stage after next
-        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, E1, w1);
+        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, p.thr16, E1, w1);
         if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
         if (!ok) break;
         *reinterpret_cast<uint4*>(pbuf) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
@@ -703,6 +708,7 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   if ((uint64_t)B * H * N >= (1ull << 31)) return FP4ATTN_ERR_UNSUPPORTED_SHAPE;
   if (!(ops->softmax_scale >= 0.f)) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->p_map != FP4ATTN_PMAP_IDEAL && ops->p_map != FP4ATTN_PMAP_AFFINE) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->p_scale_rule != FP4ATTN_PSCALE_CEIL && ops->p_scale_rule != FP4ATTN_PSCALE_THR16) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->p_map == FP4ATTN_PMAP_AFFINE && !(ops->affine_a >= 0.f && ops->affine_a < 16.f && fabsf(ops->affine_b) < 16.f))
     return FP4ATTN_ERR_INVALID_ARG;
   const uintptr_t a128 = (uintptr_t)ops->q | (uintptr_t)ops->k | (uintptr_t)ops->v | (uintptr_t)ops->q_sf |
@@ -722,6 +728,7 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   const bool affine = ops->p_map == FP4ATTN_PMAP_AFFINE;
   prm.aff_a = ops->affine_a != 0.f ? ops->affine_a : 1.5f;         // the paper's generic `fast` fit
   prm.aff_b = ops->affine_a != 0.f ? ops->affine_b : 1.2f;
+  prm.thr16 = ops->p_scale_rule == FP4ATTN_PSCALE_THR16;
   const int variant = (d == 128 ? 4 : 0) | (nv ? 2 : 0) | (affine ? 1 : 0);
   switch (variant) {
     case 0: return launch_attn<64, false, false>(ops, B, H, N, prm, st);

@@ -234,3 +234,28 @@ def test_unknown_p_map_is_rejected():
     vd = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
     with pytest.raises(Bd.Fp4AttnError):
         Bd.fp4attn_fwd(qd, kd, vd, p_map=7)
+
+
+# ------------------------------------------------------------------ threshold block-exponent rule
+@pytest.mark.parametrize("name,kw,p_map", [
+    ("cfg1", dict(), "ideal"), ("cfg1", dict(), "affine"),
+    ("cfg3", dict(B=2, H=2, N=512), "ideal"), ("cfg4", dict(H=2, N=1024), "ideal"),
+    ("cfg2", dict(B=1, H=2, N=2048), "affine"),
+])
+def test_threshold_scale_rule_matches_oracle_elementwise(name, kw, p_map):
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    qg = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q)
+    kg = Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+    vg = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    O, lse = Bd.fp4attn_fwd(qg, kg, vg, status=status, p_scale_rule=Bd.PSCALE_THR16,
+                            p_map=Bd.PMAP_AFFINE if p_map == "affine" else Bd.PMAP_IDEAL)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    Og, Lg = O.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, p_map=p_map, p_scale="thr16")
+    check_heads(Og, Lg, Oo, Lo, heads)

@@ -3,6 +3,7 @@ brute-force exact attention."""
 import math
 
 import numpy as np
+import pytest
 
 from oracle import attention as A
 from oracle import formats as F
@@ -236,3 +237,65 @@ def test_affine_and_ideal_codes_never_differ_by_more_than_one_code():
     assert np.abs(ci.astype(int) - ca.astype(int)).max() <= 1
     assert np.mean(ci == ca) > 0.35
     assert np.mean(ca == 0) > np.mean(ci == 0)
+
+
+# ------------------------------------------------------------------ threshold block-exponent rule
+def test_threshold_rule_closed_form_and_saturation():
+    """E_B = floor(max y + log2 1.6): the block maximum lands in [3.75, 7.5) code units."""
+    ym = np.array([0.0, 0.3219, 0.3220, 1.0, -0.678, -0.679, 5.5], dtype=np.float32)   # log2(1.25) = 0.32193
+    E = A.block_exponent(ym, "thr16")
+    assert list(E) == [0, 0, 1, 1, 0, -1, 6]
+    top = 6.0 * np.exp2(ym.astype(np.float64) - E)
+    assert np.all((top >= 3.75 - 1e-3) & (top < 7.5 + 1e-3))
+    assert list(A.block_exponent(ym, "ceil")) == [0, 1, 1, 1, 0, 0, 6]
+    # a block whose maximum exceeds the amplitude saturates at code 6, neighbours keep their codes
+    y = np.full((1, 32), -40.0, dtype=np.float32)
+    y[0, 0], y[0, 1] = 0.30, -0.70            # E_B = 0: 6*2^0.30 = 7.39 -> 6 ; 6*2^-0.70 = 3.69 -> 4
+    _, _, codes, EB, _ = A.direct_p_rows(y, np.float32(1.0), np.ones((32, 1)), tile=32, p_scale="thr16")
+    assert EB[0, 0] == 0 and codes[0, 0] == 7 and codes[0, 1] == 6
+
+
+def test_threshold_rule_reproduces_table_p_range_mxfp4_row():
+    """Exact Gaussian softmax -> N32 blocks coded with the threshold rule (through the oracle's own
+    block_exponent and code map) -> zero payload / lost mass / P rel-L2 / PV cosine of the printed
+    MXFP4 row at S = 1024 (Table "p-range": 0.188683 / 0.040178 / 0.146380 / 0.989846)."""
+    rng = np.random.default_rng(4)
+    S, d, R = 1024, 128, 192
+    q, k, V = rng.standard_normal((R, d)), rng.standard_normal((S, d)), rng.standard_normal((S, d))
+    z = q @ k.T / math.sqrt(d)
+    p = np.exp(z - z.max(axis=1, keepdims=True))
+    p /= p.sum(axis=1, keepdims=True)
+    y = np.log2(p).astype(np.float32)                           # absolute log2 probabilities as "scores"
+    _, _, codes, EB, _ = A.direct_p_rows(y, np.float32(1.0), V, tile=128, p_scale="thr16")
+    phat = np.repeat(np.ldexp(1.0, EB), 32, axis=1) * F.E2M1_VALUES[codes] / 6.0
+    zero_payload = np.mean(phat == 0)
+    lost = np.mean((p * (phat == 0)).sum(axis=1))
+    pn = phat / phat.sum(axis=1, keepdims=True)
+    rel = np.linalg.norm(pn - p) / np.linalg.norm(p)
+    o, oh = p @ V, pn @ V
+    cos = (o * oh).sum() / np.linalg.norm(o) / np.linalg.norm(oh)
+    assert zero_payload == pytest.approx(0.188683, rel=0.04)
+    assert lost == pytest.approx(0.040178, rel=0.06)
+    assert rel == pytest.approx(0.146380, rel=0.03)
+    assert cos == pytest.approx(0.989846, abs=2e-3)
+    # the default ceiling rule is measurably coarser on the same data
+    _, _, codes_c, EB_c, _ = A.direct_p_rows(y, np.float32(1.0), V, tile=128)
+    ph_c = np.repeat(np.ldexp(1.0, EB_c), 32, axis=1) * F.E2M1_VALUES[codes_c] / 6.0
+    pn_c = ph_c / ph_c.sum(axis=1, keepdims=True)
+    assert np.linalg.norm(pn_c - p) / np.linalg.norm(p) > rel * 1.08
+
+
+def test_threshold_rule_brings_the_affine_map_into_the_papers_band():
+    """Table "all-formats", all-MXFP4 rows: cos 0.925-0.941, rel-L2 0.344-0.381 (vs a BF16 kernel)."""
+    w, (q, k, v), qd, kd, vd = _cfg1(N=1024, H=1)
+    x = [Qz.bf16_bits_to_f64(a)[0, 0] for a in (q, k, v)]
+    Oe, _ = A.exact_attention(*x)
+    O, _ = A.direct_p_forward(qd, kd, vd, p_map="affine", p_scale="thr16")
+    cos = (Oe * O[0]).sum() / np.linalg.norm(Oe) / np.linalg.norm(O[0])
+    rel = np.linalg.norm(Oe - O[0]) / np.linalg.norm(Oe)
+    assert 0.925 < cos < 0.955 and 0.33 < rel < 0.42
+    Oi, _ = A.direct_p_forward(qd, kd, vd, p_scale="thr16")
+    Oc, _ = A.direct_p_forward(qd, kd, vd)
+    reli = np.linalg.norm(Oe - Oi[0]) / np.linalg.norm(Oe)
+    relc = np.linalg.norm(Oe - Oc[0]) / np.linalg.norm(Oe)
+    assert reli < relc                                          # and it helps the exact map too
