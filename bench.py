@@ -364,6 +364,17 @@ def run_cuda(args, w):
             ms = a.elapsed_time(b) / n_it
             sweep[name]["affine_attn_ms"] = ms
             sweep[name]["affine_attn_tflops"] = ww.flops / (ms * 1e-3) / 1e12
+            # causal mask, exact map: flops counted as half of the full product (the usual convention)
+            for _ in range(2):
+                Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status, causal=True)
+            a.record()
+            for _ in range(n_it):
+                Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status, causal=True)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / n_it
+            sweep[name]["causal_attn_ms"] = ms
+            sweep[name]["causal_attn_tflops"] = 0.5 * ww.flops / (ms * 1e-3) / 1e12
             del sq, sk, sv, so
             torch.cuda.empty_cache()
 

@@ -141,6 +141,10 @@ typedef struct {
   float affine_a, affine_b;         /* classifier constants; affine_a == 0 selects the
                                        paper's generic fit A = 1.50, B = 1.20                */
   int p_scale_rule;                 /* FP4ATTN_PSCALE_CEIL or FP4ATTN_PSCALE_THR16           */
+  int causal;                       /* 1: query row i attends keys 0..i only; 0: all keys     */
+  int kv_heads;                     /* K and V hold this many heads ([B, kv_heads, N, d]);
+                                       H query heads share them in groups of H / kv_heads
+                                       (grouped-query attention).  0 selects H               */
 } fp4attn_operands;
 
 /*
@@ -159,6 +163,11 @@ typedef struct {
  * construction (blocks whose byte would drop below 1 are zero blocks).  P V runs as a second
  * block-scaled FP4 product; the output is normalised by the sum of the same rounded values:
  *   O = sum_j p~_j V^_j / sum_j p~_j,   p~_j = 2^(E_B) q_j / 6,   LSE = ln sum_j p~_j.
+ *
+ * With causal = 1 (the forward the paper's training section starts from, Section "Causal backward")
+ * keys j > i are removed from row i before anything else: they never raise a block maximum, always
+ * code to 0, and a block without a visible key contributes nothing.  B, H, N, d describe Q and O;
+ * K and V have kv_heads heads.
  *
  * O_bf16 [B,H,N,d]; LSE [B,H,N] (may be NULL); device_status (may be NULL) receives
  * FP4ATTN_ERR_TIMEOUT if a bounded in-kernel wait ran out, and is otherwise left untouched, so

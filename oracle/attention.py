@@ -35,6 +35,11 @@ as the amplitude; besides the ceiling (default) the oracle offers the threshold 
 E_B = floor(fl32(max y + fl32(log2 1.6))), i.e. alpha_B = 2^floor(log2(1.6 a_B)): the block maximum then
 lands in [3.75, 7.5) code units and values above 6 saturate.  It reproduces the MXFP4 rows of Table
 "p-range" (pinned in the tests) and lowers the P error.
+
+Causal mask and grouped-query attention (the forward the paper's training section builds on,
+Section "Causal backward ..."): causal=True removes keys j > i from query row i before anything else
+(their score is -inf: they never raise a block maximum and always code to 0; a block with no visible
+key contributes nothing); kv_group = g lets g consecutive query heads share one K/V head.
 """
 from __future__ import annotations
 
@@ -73,10 +78,11 @@ def score_constant(qd: dict, kd: dict, d: int, softmax_scale=None) -> np.float32
     return np.float32(base / np.float32(np.float32(qd["G"]) * np.float32(kd["G"])))
 
 
-def scores_fp32(qd: dict, kd: dict, b: int, h: int, rows=None) -> np.ndarray:
+def scores_fp32(qd: dict, kd: dict, b: int, h: int, rows=None, hk=None) -> np.ndarray:
     """S_hw[i, j] = sum_k (scale*code)_Q[i,k] * (scale*code)_K[j,k], exact, rounded once to fp32."""
     A = dequantize({**qd, "nib": qd["nib"][b, h][None, None], "sf": qd["sf"][b, h][None, None]}, hw=True)[0, 0]
-    Bm = dequantize({**kd, "nib": kd["nib"][b, h][None, None], "sf": kd["sf"][b, h][None, None]}, hw=True)[0, 0]
+    hk = h if hk is None else hk
+    Bm = dequantize({**kd, "nib": kd["nib"][b, hk][None, None], "sf": kd["sf"][b, hk][None, None]}, hw=True)[0, 0]
     if rows is not None:
         A = A[rows]
     return (A @ Bm.T).astype(np.float32)
@@ -90,7 +96,7 @@ def _fma32(a, b, c):
 
 
 def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int = 128, tile_order=None,
-                  p_map: str = "ideal", affine=(1.5, 1.2), p_scale: str = "ceil"):
+                  p_map: str = "ideal", affine=(1.5, 1.2), p_scale: str = "ceil", row_index=None):
     """Direct-P online softmax + PV for a set of query rows of one (batch, head).
 
     s32  [R, N] float32 tensor-core-facing scores;  Vhat [N, d] float64 reconstructed V.
@@ -99,6 +105,8 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
     """
     R, N = s32.shape
     assert N % P_BLOCK == 0 and tile % P_BLOCK == 0 and N % tile == 0
+    if row_index is not None:                                    # causal: query row i sees keys 0..i
+        s32 = np.where(np.arange(N)[None, :] > np.asarray(row_index)[:, None], np.float32(-np.inf), s32).astype(np.float32)
     y32 = (s32 * np.float32(c32)).astype(np.float32)             # decision variable, fp32
     yx = s32.astype(np.float64) * np.float64(c32)                # converter input, fp64
     mu = np.full(R, -np.inf)
@@ -121,7 +129,9 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
         mu = mu_new
         for bj in range(j0, j0 + tile, P_BLOCK):
             E_B = block_exponent(y32[:, bj:bj + P_BLOCK].max(axis=1), p_scale)
-            e_B = E_B - mu
+            seen = np.isfinite(E_B)                              # False: every key of the block is masked
+            E_B = np.where(seen, E_B, 0.0)
+            e_B = np.where(seen, E_B - mu, -np.inf)
             live = (e_B + 127) >= 1
             b_B32 = np.float32(LOG2_6_32 - E_B.astype(np.float32))
             if p_map == "ideal":
@@ -133,12 +143,12 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
                 code = e2m1_encode_mag(np.maximum(u, np.float32(0)).astype(np.float64))
             code = np.where(live[:, None], code, 0).astype(np.uint8)
             q = E2M1_VALUES[code]
-            alpha = np.where(live, np.exp2(e_B), 0.0)
+            alpha = np.where(live, np.exp2(np.where(live, e_B, 0.0)), 0.0)
             c_B = q.sum(axis=1)
             L += alpha * (c_B / 6.0)
             O += (alpha / 6.0)[:, None] * (q @ Vhat[bj:bj + P_BLOCK])
             codes_all[:, bj:bj + P_BLOCK] = code
-            EB_all[:, bj // P_BLOCK] = E_B.astype(np.int64)
+            EB_all[:, bj // P_BLOCK] = np.where(seen, E_B, -(1 << 40)).astype(np.int64)
     Oout = O / L[:, None]
     lse = math.log(2.0) * (mu + np.log2(L))
     return Oout, lse, codes_all, EB_all, mu
@@ -146,7 +156,7 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
 
 def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int = 128,
                      rows=None, heads=None, tile_order=None, p_map: str = "ideal", affine=(1.5, 1.2),
-                     p_scale: str = "ceil"):
+                     p_scale: str = "ceil", causal: bool = False, kv_group: int = 1):
     """Whole-operator oracle.  qd/kd/vd come from oracle.quantize.quantize_qk / quantize_v.
 
     rows : optional 1-D index array of query rows evaluated for every (b, h) (rows are
@@ -154,24 +164,31 @@ def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int
            float64 and LSE [n_heads, R] float64 in the order of `heads`.
     """
     B, H, N, d = qd["nib"].shape
+    assert H % kv_group == 0 and kd["nib"].shape[1] == H // kv_group and vd["nib"].shape[1] == H // kv_group
     heads = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
     c32 = score_constant(qd, kd, d, softmax_scale)
+    ridx = np.arange(N) if rows is None else np.asarray(rows)
     Os, Ls = [], []
     for (b, h) in heads:
-        s32 = scores_fp32(qd, kd, b, h, rows)
-        Vhat = dequantize({**vd, "nib": vd["nib"][b, h][None, None], "sf": vd["sf"][b, h][None, None]})[0, 0].T
-        O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order, p_map, affine, p_scale)
+        hk = h // kv_group                                       # K/V head shared by the group
+        s32 = scores_fp32(qd, kd, b, h, rows, hk)
+        Vhat = dequantize({**vd, "nib": vd["nib"][b, hk][None, None], "sf": vd["sf"][b, hk][None, None]})[0, 0].T
+        O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order, p_map, affine, p_scale,
+                                        ridx if causal else None)
         Os.append(O)
         Ls.append(lse)
     return np.stack(Os), np.stack(Ls)
 
 
-def exact_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray, softmax_scale=None, rows=None):
+def exact_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray, softmax_scale=None, rows=None, causal=False):
     """Eq. "exact-attention" in float64 for one head: Q [N,d], K [N,d], V [N,d] -> O, LSE."""
     d = Q.shape[1]
     scale = 1.0 / math.sqrt(d) if softmax_scale is None else float(softmax_scale)
     Qr = Q if rows is None else Q[rows]
     z = (Qr @ K.T) * scale
+    if causal:
+        ridx = np.arange(Q.shape[0]) if rows is None else np.asarray(rows)
+        z = np.where(np.arange(K.shape[0])[None, :] > ridx[:, None], -np.inf, z)
     m = z.max(axis=1, keepdims=True)
     p = np.exp(z - m)
     l = p.sum(axis=1, keepdims=True)

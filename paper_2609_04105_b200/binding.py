@@ -39,7 +39,7 @@ class _Operands(ctypes.Structure):
                 ("q_G", ctypes.c_void_p), ("k_G", ctypes.c_void_p),
                 ("qk_fmt", ctypes.c_int), ("softmax_scale", ctypes.c_float),
                 ("p_map", ctypes.c_int), ("affine_a", ctypes.c_float), ("affine_b", ctypes.c_float),
-                ("p_scale_rule", ctypes.c_int)]
+                ("p_scale_rule", ctypes.c_int), ("causal", ctypes.c_int), ("kv_heads", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:
@@ -143,11 +143,12 @@ def fp4attn_quantize_nvfp4_noalloc(x: torch.Tensor, role: int, packed: torch.Ten
 def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, softmax_scale: float = 0.0,
                 out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
                 status: Optional[torch.Tensor] = None, p_map: int = PMAP_IDEAL, affine_a: float = 0.0,
-                affine_b: float = 0.0, p_scale_rule: int = PSCALE_CEIL) -> Tuple[torch.Tensor, torch.Tensor]:
+                affine_b: float = 0.0, p_scale_rule: int = PSCALE_CEIL, causal: bool = False) -> Tuple[torch.Tensor, torch.Tensor]:
     """Direct-P attention forward on quantized operands -> (O bf16 [B,H,N,d], LSE fp32 [B,H,N]).
     p_map selects the exact code map or the affine classifier (affine_a = 0: A = 1.5, B = 1.2)."""
     B, H, N, d = q.shape
-    assert k.shape == q.shape and v.shape == q.shape and q.fmt == k.fmt and v.fmt == FMT_MXFP4
+    Hkv = k.shape[1]                                   # grouped-query attention when Hkv < H
+    assert k.shape == v.shape and k.shape == (B, Hkv, N, d) and H % Hkv == 0 and q.fmt == k.fmt and v.fmt == FMT_MXFP4
     dev = q.packed.device
     if out is None:
         out = torch.empty((B, H, N, d), dtype=torch.bfloat16, device=dev)
@@ -155,7 +156,7 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
         lse = torch.empty((B, H, N), dtype=torch.float32, device=dev)
     ops = _Operands(q.packed.data_ptr(), k.packed.data_ptr(), v.packed.data_ptr(),
                     q.scales.data_ptr(), k.scales.data_ptr(), v.scales.data_ptr(),
-                    _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b), int(p_scale_rule))
+                    _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b), int(p_scale_rule), int(bool(causal)), int(Hkv))
     _check(lib().fp4attn_fwd(ctypes.byref(ops), B, H, N, d, out.data_ptr(), lse.data_ptr(), _ptr(status), _stream()),
            "fp4attn_fwd")
     return out, lse

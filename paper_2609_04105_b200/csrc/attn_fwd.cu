@@ -95,7 +95,36 @@ struct AttnParams {
   float c_base;            // fl32(log2(e) * softmax_scale)
   float aff_a, aff_b;      // affine classifier u = max(0, A x + B) (only read by the affine variant)
   int thr16;               // block exponent rule: 0 = ceil(max y), 1 = floor(max y + log2 1.6)
+  int causal;              // 1: query row i sees keys 0..i
+  int H, Hkv;              // query heads, K/V heads (H % Hkv == 0: grouped-query attention)
 };
+
+// One work item = one 128-row query tile of one (batch, query head).
+struct WorkItem {
+  int qt;                  // query tile within the head
+  int qrow0;               // first row of the tile in the [B*H*N] row space of Q, O, LSE
+  int qtile_lin;           // (b*H + h) * qtiles + qt: index of the tile's Q scale atom(s)
+  int kvh;                 // b*Hkv + h / (H/Hkv): the K/V head this query head reads
+  int T2;                  // 128-key stages to walk (causal: up to and including the diagonal)
+};
+__device__ __forceinline__ WorkItem decode_item(int item, const AttnParams& p, int qtiles) {
+  WorkItem w;
+  int bh;
+  if (p.causal) {           // longest items first, so the persistent CTAs finish together
+    const int BH = p.n_items / qtiles;
+    w.qt = qtiles - 1 - item / BH;
+    bh = item % BH;
+  } else {                  // consecutive items share K/V in L2
+    bh = item / qtiles;
+    w.qt = item - bh * qtiles;
+  }
+  w.qrow0 = bh * p.N + w.qt * BM;
+  w.qtile_lin = bh * qtiles + w.qt;
+  const int b = bh / p.H, h = bh - b * p.H;
+  w.kvh = b * p.Hkv + h / (p.H / p.Hkv);
+  w.T2 = p.causal ? w.qt + 1 : p.stages;
+  return w;
+}
 
 // barrier slots (8 bytes each)
 enum { BAR_QFULL0 = 0, BAR_QFREE0 = 2, BAR_OFULL = 4, BAR_OFREE = 5, BAR_SFULL0 = 6, BAR_SEMPTY0 = 8,
@@ -171,13 +200,18 @@ __device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float&
 //   affine map (Eq. "affine-code-map"):  q = Q_E2M1(max(0, A x + B)), folded into one fused multiply-add
 //                                        per element: u = s * fl32(A c) + fma(A, log2 6 - E_B, B)
 template <bool AFFINE>
-__device__ __forceinline__ void direct_p_block(const uint32_t* sraw, float c32, float A, float B, int thr16, int& E,
+__device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float A, float B, int thr16, int visible, int& E,
                                                uint32_t* words) {
   const float LOG2_6 = 2.5849625007211560f;
+  if (visible < 32) {                                           // causal diagonal: keys beyond the query get -inf
+#pragma unroll
+    for (int i = 0; i < 32; ++i) sraw[i] = (i < visible) ? sraw[i] : 0xFF800000u;
+  }
   const float ymax = __fmul_rn(max32(sraw), c32);
   // amplitude rule (Eq. "mx-scale" allows either neighbouring power of two): ceiling, or the threshold
   // rule alpha = 2^floor(log2(1.6 a)) under which values above the amplitude saturate at code 6
   E = thr16 ? (int)floorf(__fadd_rn(ymax, 0.6780719161033630f)) : (int)ceilf(ymax);
+  E = max(E, -(1 << 24));                                       // a fully masked block (ymax = -inf) stays finite
   const float bB = __fsub_rn(LOG2_6, (float)E);
   if (AFFINE) {
     const float cA = __fmul_rn(A, c32), bA = __fmaf_rn(A, bB, B);
@@ -235,7 +269,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qtiles = p.N / BM;
-  const int T2 = p.stages;
 
   if (threadIdx.x == 0) {
     for (int b = 0; b < 2; ++b) {
@@ -277,18 +310,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     bool ok = true;
     int i = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
-      const int bh = item / qtiles, qt = item - bh * qtiles;
+      const WorkItem wi = decode_item(item, p, qtiles);
+      const int T2 = wi.T2;
       const int qb = i & 1;
       if (i >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_QFREE0 + qb), ((i >> 1) - 1) & 1, abortf));
       if (!ok) break;
       if (elect_one()) {
         mbar_arrive_expect_tx(bar(BAR_QFULL0 + qb), C::Q_BYTES + C::QSF_BYTES);
-        tma_load_2d(sbase + C::OFF_Q + qb * C::Q_BYTES, &tmQ, 0, bh * p.N + qt * BM, bar(BAR_QFULL0 + qb));
-        bulk_load_1d(sbase + C::OFF_QSF + qb * 1024, p.q_sf + (size_t)item * C::QSF_BYTES, C::QSF_BYTES, bar(BAR_QFULL0 + qb));
+        tma_load_2d(sbase + C::OFF_Q + qb * C::Q_BYTES, &tmQ, 0, wi.qrow0, bar(BAR_QFULL0 + qb));
+        bulk_load_1d(sbase + C::OFF_QSF + qb * 1024, p.q_sf + (size_t)wi.qtile_lin * C::QSF_BYTES, C::QSF_BYTES, bar(BAR_QFULL0 + qb));
       }
-      const uint8_t* ksf = p.k_sf + (size_t)bh * qtiles * C::KSF_BYTES;
-      const uint8_t* vsf = p.v_sf + (size_t)bh * qtiles * C::VSF_BYTES;
-      const int krow0 = bh * p.N, vrow0 = bh * D;
+      const uint8_t* ksf = p.k_sf + (size_t)wi.kvh * qtiles * C::KSF_BYTES;
+      const uint8_t* vsf = p.v_sf + (size_t)wi.kvh * qtiles * C::VSF_BYTES;
+      const int krow0 = wi.kvh * p.N, vrow0 = wi.kvh * D;
       for (int s2 = 0; s2 < T2; ++s2, ++gs) {
         if (gs >= (uint32_t)C::NST) ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(s), ph ^ 1, abortf));
         if (!ok) break;
@@ -321,6 +355,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     bool ok = true;
     int i = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
+      const int T2 = decode_item(item, p, qtiles).T2;
       const int qb = i & 1;
       ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_QFULL0 + qb), (i >> 1) & 1, abortf));
       if (!ok) break;
@@ -378,6 +413,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     bool ok = true;
     int i = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
+      const int T2 = decode_item(item, p, qtiles).T2;
       if (i >= 1) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFREE), (i - 1) & 1, abortf));   // epilogue has read O
       for (int s2 = 0; ok && s2 < T2; ++s2, ++g) {
         const int pr = g & 1;
@@ -421,7 +457,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     uint32_t g0 = 0;                                            // stages completed in earlier items
     bool ok = true;
     int i = 0;
+    int T2 = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i, g0 += T2) {
+      const WorkItem wi = decode_item(item, p, qtiles);
+      T2 = wi.T2;
       int mu = -(1 << 28);
       int pu0 = 0, pu1 = 0;                                     // bytes written for the previous tile (tile-by-tile mode)
       // one pass per 64-key tile, or (AFFINE) one pass per 128-key stage covering both of its tiles
@@ -501,7 +540,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         Lhw = __uint_as_float(r16[0]);
       }
       const float inv = __frcp_rn(6.0f * Lhw);
-      const size_t grow = (size_t)item * BM + row;
+      const size_t grow = (size_t)wi.qrow0 + row;
       // stage the bf16 tile in shared memory (128-byte rows, 128B-swizzled like the tensor map) and
       // let TMA write it out, so O is released after four TMEM reads instead of after 16 global stores
       if (lane == 0) bulk_wait_read_all();                      // this warp's previous stores have read the buffer
@@ -534,7 +573,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (lane == 0) {                                          // this warp's 32 rows, one box per 128-byte half
 #pragma unroll
         for (int hf = 0; hf < D / 64; ++hf)
-          tma_store_2d(&tmO, hf * 128, item * BM + quarter * 32, sbase + C::OFF_OUT + hf * (BM * 128) + quarter * 32 * 128);
+          tma_store_2d(&tmO, hf * 128, wi.qrow0 + quarter * 32, sbase + C::OFF_OUT + hf * (BM * 128) + quarter * 32 * 128);
         bulk_commit_group();
       }
       if (p.LSE) p.LSE[grow] = 0.69314718055994531f * ((float)mu + (log2f(Lhw) - 2.5849625007211560f));
@@ -555,9 +594,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     else    c32 = __fdiv_rn(p.c_base, 36.0f);
     uint32_t g0 = 0;
     bool ok = true;
+    int T2 = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, g0 += T2) {
+      const WorkItem wi = decode_item(item, p, qtiles);
+      T2 = wi.T2;
       for (uint32_t g = g0 + ((g0 & 1) != (uint32_t)pr); g < g0 + T2; g += 2) {   // this team's stages of the item
         const uint32_t m = g >> 1;
+        // causal diagonal stage: this row sees keys 0..row of the stage; the team's tile starts at key 64*(team&1)
+        const bool diag = p.causal && (int)(g - g0) == wi.qt;
+        const int vis0 = diag ? min(max(row - 64 * (team & 1) + 1, 0), 32) : 32;
+        const int vis1 = diag ? min(max(row - 64 * (team & 1) - 31, 0), 32) : 32;
         ok = __all_sync(0xffffffffu, mbar_wait(sfull, m & 1, abortf));
         if (!ok) break;
         tc_fence_after();
@@ -565,13 +611,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         int E0, E1;
         tmem_ld_32x32b_x32(tS, sraw);
         tmem_wait_ld();
-        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, p.thr16, E0, w0);
+        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, p.thr16, vis0, E0, w0);
         tmem_ld_32x32b_x32(tS + 32, sraw);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(sempty);                     // pair may take the stage after next
-        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, p.thr16, E1, w1);
+        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, p.thr16, vis1, E1, w1);
         if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
         if (!ok) break;
         *reinterpret_cast<uint4*>(pbuf) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
@@ -671,6 +717,7 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint6
 
 template <int D, bool NV, bool AFFINE>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
+  const int Hkv = prm.Hkv;
   using C = Cfg<D, NV>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -679,10 +726,10 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
     attr_set = true;
   }
   CUtensorMap tmQ, tmK, tmV, tmO;
-  const uint64_t rows = (uint64_t)B * H * N;
+  const uint64_t rows = (uint64_t)B * H * N, kv_rows = (uint64_t)B * Hkv * N;
   if (!make_map(&tmQ, ops->q, C::ROW_BYTES, rows, C::ROW_BYTES, BM) ||
-      !make_map(&tmK, ops->k, C::ROW_BYTES, rows, C::ROW_BYTES, BS) ||
-      !make_map(&tmV, ops->v, (uint64_t)N / 2, (uint64_t)B * H * D, BS / 2, D) ||
+      !make_map(&tmK, ops->k, C::ROW_BYTES, kv_rows, C::ROW_BYTES, BS) ||
+      !make_map(&tmV, ops->v, (uint64_t)N / 2, (uint64_t)B * Hkv * D, BS / 2, D) ||
       !make_map(&tmO, prm.O, (uint64_t)D * 2, rows, 128, 32))
     return FP4ATTN_ERR_CUDA;
   int dev = 0, sms = 0;
@@ -709,6 +756,8 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   if (!(ops->softmax_scale >= 0.f)) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->p_map != FP4ATTN_PMAP_IDEAL && ops->p_map != FP4ATTN_PMAP_AFFINE) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->p_scale_rule != FP4ATTN_PSCALE_CEIL && ops->p_scale_rule != FP4ATTN_PSCALE_THR16) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->kv_heads < 0 || (ops->kv_heads > 0 && H % ops->kv_heads != 0) || (ops->causal != 0 && ops->causal != 1))
+    return FP4ATTN_ERR_INVALID_ARG;
   if (ops->p_map == FP4ATTN_PMAP_AFFINE && !(ops->affine_a >= 0.f && ops->affine_a < 16.f && fabsf(ops->affine_b) < 16.f))
     return FP4ATTN_ERR_INVALID_ARG;
   const uintptr_t a128 = (uintptr_t)ops->q | (uintptr_t)ops->k | (uintptr_t)ops->v | (uintptr_t)ops->q_sf |
@@ -721,6 +770,9 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.q_G = ops->q_G; prm.k_G = ops->k_G;
   prm.O = (__nv_bfloat16*)O; prm.LSE = LSE; prm.status = device_status;
   prm.N = N; prm.stages = N / BS; prm.n_items = B * H * (N / BM);
+  prm.causal = ops->causal ? 1 : 0;
+  prm.H = H;
+  prm.Hkv = ops->kv_heads > 0 ? ops->kv_heads : H;
   const float scale = ops->softmax_scale > 0.f ? ops->softmax_scale : (float)(1.0 / sqrt((double)d));
   prm.c_base = 1.4426950408889634f * scale;                        // fl32(log2e_32 * scale_32)
   cudaStream_t st = (cudaStream_t)stream;

@@ -259,3 +259,66 @@ def test_threshold_scale_rule_matches_oracle_elementwise(name, kw, p_map):
     heads = [(b, h) for b in range(w.B) for h in range(w.H)]
     Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, p_map=p_map, p_scale="thr16")
     check_heads(Og, Lg, Oo, Lo, heads)
+
+
+# ------------------------------------------------------------------ causal mask and grouped-query attention
+def run_gpu_general(w, q, k, v, **kw):
+    from paper_2609_04105_b200 import binding as Bd
+    qg = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q)
+    kg = Bd.fp4attn_quantize(_dev(np.ascontiguousarray(k)), w.qk_fmt, Bd.ROLE_K)
+    vg = Bd.fp4attn_quantize(_dev(np.ascontiguousarray(v)), Bd.FMT_MXFP4, Bd.ROLE_V)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    O, lse = Bd.fp4attn_fwd(qg, kg, vg, status=status, **kw)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return O.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+
+
+CAUSAL_CASES = [
+    ("cfg1", dict(), 1, "ideal"),
+    ("cfg1", dict(N=128), 1, "ideal"),
+    ("cfg1", dict(N=640, H=3), 1, "ideal"),
+    ("cfg1", dict(N=512, H=4), 2, "ideal"),                 # grouped-query: 4 query heads on 2 K/V heads
+    ("cfg1", dict(d=64, N=512, H=4), 4, "affine"),          # multi-query, affine map
+    ("cfg3", dict(B=2, H=2, N=512), 1, "ideal"),            # NVFP4 Q/K, d = 64
+    ("cfg4", dict(H=2, N=1024), 1, "ideal"),
+    ("cfg2", dict(B=2, H=3, N=2304), 1, "affine"),
+]
+
+
+@pytest.mark.parametrize("name,kw,group,p_map", CAUSAL_CASES)
+def test_causal_and_gqa_match_oracle_elementwise(name, kw, group, p_map):
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    k, v = k[:, : w.H // group], v[:, : w.H // group]
+    Og, Lg = run_gpu_general(w, q, k, v, causal=True, p_map=Bd.PMAP_AFFINE if p_map == "affine" else Bd.PMAP_IDEAL)
+    fmt = "mx" if w.qk_fmt == I.FMT_MXFP4 else "nv"
+    qd, kd, vd = Qz.quantize_qk(q, fmt), Qz.quantize_qk(np.ascontiguousarray(k), fmt), Qz.quantize_v(np.ascontiguousarray(v))
+    heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, causal=True, kv_group=group, p_map=p_map)
+    check_heads(Og, Lg, Oo, Lo, heads)
+
+
+def test_gqa_noncausal_matches_oracle():
+    w = I.shrink(I.WORKLOADS["cfg1"], N=384, H=6)
+    q, k, v = I.make_qkv(w)
+    k, v = k[:, :2], v[:, :2]
+    Og, Lg = run_gpu_general(w, q, k, v)
+    qd, kd, vd = Qz.quantize_qk(q, "mx"), Qz.quantize_qk(np.ascontiguousarray(k), "mx"), Qz.quantize_v(np.ascontiguousarray(v))
+    heads = [(0, h) for h in range(6)]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, kv_group=3)
+    check_heads(Og, Lg, Oo, Lo, heads)
+
+
+def test_causal_config2_full_size_sampled_rows():
+    w = I.WORKLOADS["cfg2"]
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu_general(w, q, k, v, causal=True)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    rng = np.random.default_rng(31)
+    rows = np.sort(np.concatenate([rng.choice(w.N, size=160, replace=False), [0, 1, 63, 64, 127, 128, w.N - 1]]))
+    rows = np.unique(rows)
+    heads = [(0, 3), (2, 9), (3, 15)]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows, causal=True)
+    check_heads(Og, Lg, Oo, Lo, heads, rows)

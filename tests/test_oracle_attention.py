@@ -299,3 +299,58 @@ def test_threshold_rule_brings_the_affine_map_into_the_papers_band():
     reli = np.linalg.norm(Oe - Oi[0]) / np.linalg.norm(Oe)
     relc = np.linalg.norm(Oe - Oc[0]) / np.linalg.norm(Oe)
     assert reli < relc                                          # and it helps the exact map too
+
+
+# ------------------------------------------------------------------ causal mask and grouped-query attention
+def test_causal_rows_equal_noncausal_attention_over_their_visible_prefix():
+    """Row i of the causal operator attends keys 0..i.  When i + 1 is a multiple of the tile it must
+    equal the noncausal operator run on the first i + 1 keys; row 0 returns V^_0; masked keys never
+    carry a code."""
+    w, _, qd, kd, vd = _cfg1(N=512, H=1)
+    O, L = A.direct_p_forward(qd, kd, vd, causal=True)
+    Vhat = np.swapaxes(Qz.dequantize(vd), -1, -2)[0, 0]
+    assert np.abs(O[0][0] - Vhat[0]).max() < 1e-15
+    c32 = A.score_constant(qd, kd, w.d)
+    s32 = A.scores_fp32(qd, kd, 0, 0)
+    for i in (127, 255, 383, 511):
+        Oi, Li, codes, _, _ = A.direct_p_rows(s32[i:i + 1, :i + 1], c32, np.ascontiguousarray(Vhat[:i + 1]), tile=128)
+        assert np.abs(O[0][i] - Oi[0]).max() < 1e-14 and abs(L[0][i] - Li[0]) < 1e-13
+    _, _, codes, _, _ = A.direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), row_index=np.arange(512))
+    assert not np.triu(codes, k=1).any()
+
+
+def test_causal_lossless_inputs_stay_in_the_rounding_band_of_bruteforce_causal_attention():
+    rng = np.random.default_rng(21)
+    B, H, N, d = 1, 1, 96, 64
+    vals = np.array([0, 0.25, -0.25, 0.5, -0.5, 1, -1])
+    def draw():
+        x = rng.choice(vals, size=(B, H, N, d))
+        x[..., ::32] = 1.0
+        x[:, :, ::32, :] = -1.0
+        return x
+    q, k, v = draw(), draw(), draw()
+    bits = [I.f32_to_bf16_bits(a.astype(np.float32)) for a in (q, k, v)]
+    qd, kd, vd = Qz.quantize_qk(bits[0], "mx"), Qz.quantize_qk(bits[1], "mx"), Qz.quantize_v(bits[2])
+    O, lse = A.direct_p_forward(qd, kd, vd, tile=32, causal=True)
+    Oe = np.zeros((N, d))
+    for i in range(N):
+        z = [sum(q[0, 0, i, c] * k[0, 0, j, c] for c in range(d)) / math.sqrt(d) for j in range(i + 1)]
+        m = max(z)
+        pz = [math.exp(t - m) for t in z]
+        for j in range(i + 1):
+            Oe[i] += pz[j] / sum(pz) * v[0, 0, j]
+    Oref, _ = A.exact_attention(q[0, 0], k[0, 0], v[0, 0], causal=True)
+    assert np.abs(Oref - Oe).max() < 1e-13
+    rel = np.linalg.norm(O[0] - Oe) / np.linalg.norm(Oe)
+    assert rel < 0.2 and np.abs(O[0][0] - v[0, 0, 0]).max() < 1e-15
+
+
+def test_grouped_query_attention_equals_repeating_the_kv_heads():
+    w = I.shrink(I.WORKLOADS["cfg1"], H=4, N=128)
+    q, k, v = I.make_qkv(w)
+    qd = Qz.quantize_qk(q, "mx")
+    kd2, vd2 = Qz.quantize_qk(k[:, :2], "mx"), Qz.quantize_v(v[:, :2])          # two K/V heads, group of 2
+    O, L = A.direct_p_forward(qd, kd2, vd2, kv_group=2, causal=True)
+    krep, vrep = np.repeat(k[:, :2], 2, axis=1), np.repeat(v[:, :2], 2, axis=1)
+    O2, L2 = A.direct_p_forward(qd, Qz.quantize_qk(krep, "mx"), Qz.quantize_v(vrep), causal=True)
+    assert np.array_equal(O, O2) and np.array_equal(L, L2)
