@@ -199,11 +199,11 @@ __device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float&
 //   ideal map  (Eq. "ideal-code-path"):  q = Q_E2M1(2^x),            x = y - E_B + log2 6
 //   affine map (Eq. "affine-code-map"):  q = Q_E2M1(max(0, A x + B)), folded into one fused multiply-add
 //                                        per element: u = s * fl32(A c) + fma(A, log2 6 - E_B, B)
-template <bool AFFINE>
+template <bool AFFINE, bool MASKED>
 __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float A, float B, int thr16, int visible, int& E,
                                                uint32_t* words) {
   const float LOG2_6 = 2.5849625007211560f;
-  if (visible < 32) {                                           // causal diagonal: keys beyond the query get -inf
+  if (MASKED) {                                                 // causal diagonal: keys beyond the query get -inf
 #pragma unroll
     for (int i = 0; i < 32; ++i) sraw[i] = (i < visible) ? sraw[i] : 0xFF800000u;
   }
@@ -211,7 +211,7 @@ __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float 
   // amplitude rule (Eq. "mx-scale" allows either neighbouring power of two): ceiling, or the threshold
   // rule alpha = 2^floor(log2(1.6 a)) under which values above the amplitude saturate at code 6
   E = thr16 ? (int)floorf(__fadd_rn(ymax, 0.6780719161033630f)) : (int)ceilf(ymax);
-  E = max(E, -(1 << 24));                                       // a fully masked block (ymax = -inf) stays finite
+  if (MASKED) E = max(E, -(1 << 24));                           // a fully masked block (ymax = -inf) stays finite
   const float bB = __fsub_rn(LOG2_6, (float)E);
   if (AFFINE) {
     const float cA = __fmul_rn(A, c32), bA = __fmaf_rn(A, bB, B);
@@ -596,14 +596,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     bool ok = true;
     int T2 = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, g0 += T2) {
-      const WorkItem wi = decode_item(item, p, qtiles);
-      T2 = wi.T2;
+      uint32_t gdiag;                                           // global index of the causal diagonal stage (none: ~0)
+      {
+        const WorkItem wi = decode_item(item, p, qtiles);
+        T2 = wi.T2;
+        gdiag = p.causal ? g0 + (uint32_t)wi.qt : 0xFFFFFFFFu;
+      }
       for (uint32_t g = g0 + ((g0 & 1) != (uint32_t)pr); g < g0 + T2; g += 2) {   // this team's stages of the item
         const uint32_t m = g >> 1;
-        // causal diagonal stage: this row sees keys 0..row of the stage; the team's tile starts at key 64*(team&1)
-        const bool diag = p.causal && (int)(g - g0) == wi.qt;
-        const int vis0 = diag ? min(max(row - 64 * (team & 1) + 1, 0), 32) : 32;
-        const int vis1 = diag ? min(max(row - 64 * (team & 1) - 31, 0), 32) : 32;
         ok = __all_sync(0xffffffffu, mbar_wait(sfull, m & 1, abortf));
         if (!ok) break;
         tc_fence_after();
@@ -611,13 +611,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         int E0, E1;
         tmem_ld_32x32b_x32(tS, sraw);
         tmem_wait_ld();
-        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, p.thr16, vis0, E0, w0);
-        tmem_ld_32x32b_x32(tS + 32, sraw);
-        tmem_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(sempty);                     // pair may take the stage after next
-        direct_p_block<AFFINE>(sraw, c32, p.aff_a, p.aff_b, p.thr16, vis1, E1, w1);
+        if (g != gdiag) {
+          direct_p_block<AFFINE, false>(sraw, c32, p.aff_a, p.aff_b, p.thr16, 32, E0, w0);
+          tmem_ld_32x32b_x32(tS + 32, sraw);
+          tmem_wait_ld();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(sempty);                   // pair may take the stage after next
+          direct_p_block<AFFINE, false>(sraw, c32, p.aff_a, p.aff_b, p.thr16, 32, E1, w1);
+        } else {
+          // causal diagonal stage: this row sees keys 0..row of the stage; the team's tile starts at key 64*(team&1)
+          const int v0 = row - 64 * (team & 1) + 1;
+          direct_p_block<AFFINE, true>(sraw, c32, p.aff_a, p.aff_b, p.thr16, v0, E0, w0);
+          tmem_ld_32x32b_x32(tS + 32, sraw);
+          tmem_wait_ld();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(sempty);
+          direct_p_block<AFFINE, true>(sraw, c32, p.aff_a, p.aff_b, p.thr16, v0 - 32, E1, w1);
+        }
         if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
         if (!ok) break;
         *reinterpret_cast<uint4*>(pbuf) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
