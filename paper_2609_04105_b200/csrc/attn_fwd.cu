@@ -107,10 +107,11 @@ struct WorkItem {
   int kvh;                 // b*Hkv + h / (H/Hkv): the K/V head this query head reads
   int T2;                  // 128-key stages to walk (causal: up to and including the diagonal)
 };
+template <bool CAUSAL>
 __device__ __forceinline__ WorkItem decode_item(int item, const AttnParams& p, int qtiles) {
   WorkItem w;
   int bh;
-  if (p.causal) {           // longest items first, so the persistent CTAs finish together
+  if (CAUSAL) {             // longest items first, so the persistent CTAs finish together
     const int BH = p.n_items / qtiles;
     w.qt = qtiles - 1 - item / BH;
     bh = item % BH;
@@ -122,7 +123,7 @@ __device__ __forceinline__ WorkItem decode_item(int item, const AttnParams& p, i
   w.qtile_lin = bh * qtiles + w.qt;
   const int b = bh / p.H, h = bh - b * p.H;
   w.kvh = b * p.Hkv + h / (p.H / p.Hkv);
-  w.T2 = p.causal ? w.qt + 1 : p.stages;
+  w.T2 = CAUSAL ? w.qt + 1 : p.stages;
   return w;
 }
 
@@ -160,12 +161,13 @@ __device__ __forceinline__ void fma2(float s0, float s1, float c, float b, float
       : "=f"(x0), "=f"(x1) : "f"(s0), "f"(s1), "f"(c), "f"(b));
 }
 // ---- 2^x on the FMA pipe for a share of the elements (the SFU's 16 ex2/clk/SM is the tightest unit).
-// Only the E2M1 code of 2^x matters, and codes change only where the significand of 2^x crosses
-// 1, 1.25, 1.5 or 1.75.  With x = n + f (n = floor x), 2^f is replaced by the degree-4 polynomial
-// through (0,1), (log2 1.25, 1.25), (log2 1.5, 1.5), (log2 1.75, 1.75), (1,2): monotone, equal to 2^f
-// at every point where a code can change, so the codes are those of the exact exponential (a
-// 4-million-point sweep plus dense sweeps around the seven boundaries differ only within one fp32
-// ulp of x at a boundary - the same class as ex2.approx).  n enters through the exponent field.
+// Only the E2M1 code of 2^x matters, and it changes only where 2^x crosses 0.25, 0.75, 1.25, 1.75, 2.5,
+// 3.5 or 5.  2^x is therefore replaced by the degree-6 polynomial through the seven points (log2 b, b):
+// equal to 2^x at every point where a code can change and monotone on [-2.75, 3.3], so the codes are
+// those of the exact exponential (a 4-million-point sweep plus dense sweeps around the seven boundaries
+// differ only within three fp32 ulps of x at a boundary - the same class as ex2.approx).  No range
+// reduction: x is at most log2(9.6) by construction of the block exponent, and below -2.75 it is clamped
+// (there the polynomial stays inside (0.18, 0.25), i.e. code 0 like 2^x).
 #ifndef FP4ATTN_POLY_MASK
 #define FP4ATTN_POLY_MASK 0x0842u      // which of a block's 16 element pairs take the polynomial path
 #endif
@@ -174,24 +176,17 @@ __device__ __forceinline__ uint64_t pack2(float a, float b) {
   asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
   return r;
 }
-__device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float& p1) {
-  const float M = 12582912.0f;                       // 1.5 * 2^23: x + M rounded down holds floor(x) in its low bits
-  const uint64_t x = pack2(fmaxf(x0, -40.0f), fmaxf(x1, -40.0f));
-  const uint64_t m = pack2(M, M);
-  uint64_t t, nb, f, q;
-  asm("add.rm.f32x2 %0, %1, %2;" : "=l"(t) : "l"(x), "l"(m));
-  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(nb) : "l"(m), "l"(t));          // -floor(x), exact
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(f) : "l"(x), "l"(nb));          // x - floor(x) in [0,1), exact
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(pack2(0.014081917703151703f, 0.014081917703151703f)), "l"(f),
-      "l"(pack2(0.05088741332292557f, 0.05088741332292557f)));
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(f), "l"(pack2(0.24216225743293762f, 0.24216225743293762f)));
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(f), "l"(pack2(0.6928684115409851f, 0.6928684115409851f)));
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(f), "l"(pack2(1.0f, 1.0f)));
-  uint32_t tl, th, ql, qh;
-  asm("mov.b64 {%0, %1}, %2;" : "=r"(tl), "=r"(th) : "l"(t));
-  asm("mov.b64 {%0, %1}, %2;" : "=r"(ql), "=r"(qh) : "l"(q));
-  p0 = __uint_as_float(tl * 0x800000u + ql);         // significand bits + (floor(x) << 23)
-  p1 = __uint_as_float(th * 0x800000u + qh);
+__device__ __forceinline__ void exp2_poly6(float x0, float x1, float& p0, float& p1) {
+  const uint64_t x = pack2(fmaxf(x0, -2.75f), fmaxf(x1, -2.75f));
+  uint64_t q;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(pack2(0.0002452842309139669f, 0.0002452842309139669f)), "l"(x),
+      "l"(pack2(0.0012840019771829247f, 0.0012840019771829247f)));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(x), "l"(pack2(0.009303540922701359f, 0.009303540922701359f)));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(x), "l"(pack2(0.05597471818327904f, 0.05597471818327904f)));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(x), "l"(pack2(0.2401072233915329f, 0.2401072233915329f)));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(x), "l"(pack2(0.6930626630783081f, 0.6930626630783081f)));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(x), "l"(pack2(1.0000272989273071f, 1.0000272989273071f)));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(p0), "=f"(p1) : "l"(q));
 }
 
 // One N32 score fragment of one row: E_B = ceil(max y) and the codes.  Nothing here depends on the
@@ -199,20 +194,25 @@ __device__ __forceinline__ void exp2_poly2(float x0, float x1, float& p0, float&
 //   ideal map  (Eq. "ideal-code-path"):  q = Q_E2M1(2^x),            x = y - E_B + log2 6
 //   affine map (Eq. "affine-code-map"):  q = Q_E2M1(max(0, A x + B)), folded into one fused multiply-add
 //                                        per element: u = s * fl32(A c) + fma(A, log2 6 - E_B, B)
-template <bool AFFINE, bool MASKED>
-__device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float A, float B, int thr16, int visible, int& E,
+template <bool AFFINE, bool MASKED, bool THR16>
+__device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float A, float B, int visible, int& E,
                                                uint32_t* words) {
   const float LOG2_6 = 2.5849625007211560f;
   if (MASKED) {                                                 // causal diagonal: keys beyond the query get -inf
 #pragma unroll
     for (int i = 0; i < 32; ++i) sraw[i] = (i < visible) ? sraw[i] : 0xFF800000u;
   }
-  const float ymax = __fmul_rn(max32(sraw), c32);
+  // y is clamped to +-2^21 (scores beyond that are outside any softmax's range; a fully masked block,
+  // max = -inf, lands on the lower clamp and becomes a zero block)
+  const float ymax = fminf(fmaxf(__fmul_rn(max32(sraw), c32), -2097152.0f), 2097152.0f);
   // amplitude rule (Eq. "mx-scale" allows either neighbouring power of two): ceiling, or the threshold
-  // rule alpha = 2^floor(log2(1.6 a)) under which values above the amplitude saturate at code 6
-  E = thr16 ? (int)floorf(__fadd_rn(ymax, 0.6780719161033630f)) : (int)ceilf(ymax);
-  if (MASKED) E = max(E, -(1 << 24));                           // a fully masked block (ymax = -inf) stays finite
-  const float bB = __fsub_rn(LOG2_6, (float)E);
+  // rule alpha = 2^floor(log2(1.6 a)) under which values above the amplitude saturate at code 6.
+  // Integer rounding on the FMA pipe (the conversion instructions share the SFU's issue slots with
+  // ex2): for |y| < 2^22, y + 1.5*2^23 rounded up (down) is ceil(y) (floor(y)) + 1.5*2^23 exactly.
+  const float M = 12582912.0f;
+  const float t = THR16 ? __fadd_rd(__fadd_rn(ymax, 0.6780719161033630f), M) : __fadd_ru(ymax, M);
+  E = (int)(__float_as_uint(t) - 0x4B400000u);
+  const float bB = __fsub_rn(LOG2_6, __fsub_rn(t, M));          // t - M = (float)E, exact
   if (AFFINE) {
     const float cA = __fmul_rn(A, c32), bA = __fmaf_rn(A, bB, B);
 #pragma unroll
@@ -232,7 +232,7 @@ __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float 
         float x0, x1;
         fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), c32, bB, x0, x1);
         if ((FP4ATTN_POLY_MASK >> (4 * w + i / 2)) & 1u) {
-          exp2_poly2(x0, x1, pv[i], pv[i + 1]);
+          exp2_poly6(x0, x1, pv[i], pv[i + 1]);
         } else {
           pv[i] = ex2_approx(x0);
           pv[i + 1] = ex2_approx(x1);
@@ -246,7 +246,7 @@ __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float 
 // AFFINE selects the affine classifier and, with it, stage-wise correction (both 64-key tiles of a stage
 // per pass): without the SFU work the teams outrun a tile-by-tile correction chain, while the exact
 // map runs ~2 % faster with the tile-by-tile chain, which staggers the teams.
-template <int D, bool NV, bool AFFINE>
+template <int D, bool NV, bool AFFINE, bool CAUSAL, bool THR16>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -310,7 +310,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     bool ok = true;
     int i = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
-      const WorkItem wi = decode_item(item, p, qtiles);
+      const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
       const int T2 = wi.T2;
       const int qb = i & 1;
       if (i >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_QFREE0 + qb), ((i >> 1) - 1) & 1, abortf));
@@ -355,7 +355,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     bool ok = true;
     int i = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
-      const int T2 = decode_item(item, p, qtiles).T2;
+      const int T2 = decode_item<CAUSAL>(item, p, qtiles).T2;
       const int qb = i & 1;
       ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_QFULL0 + qb), (i >> 1) & 1, abortf));
       if (!ok) break;
@@ -413,7 +413,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     bool ok = true;
     int i = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
-      const int T2 = decode_item(item, p, qtiles).T2;
+      const int T2 = decode_item<CAUSAL>(item, p, qtiles).T2;
       if (i >= 1) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFREE), (i - 1) & 1, abortf));   // epilogue has read O
       for (int s2 = 0; ok && s2 < T2; ++s2, ++g) {
         const int pr = g & 1;
@@ -459,7 +459,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     int i = 0;
     int T2 = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i, g0 += T2) {
-      const WorkItem wi = decode_item(item, p, qtiles);
+      const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
       T2 = wi.T2;
       int mu = -(1 << 28);
       int pu0 = 0, pu1 = 0;                                     // bytes written for the previous tile (tile-by-tile mode)
@@ -598,9 +598,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, g0 += T2) {
       uint32_t gdiag;                                           // global index of the causal diagonal stage (none: ~0)
       {
-        const WorkItem wi = decode_item(item, p, qtiles);
+        const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
         T2 = wi.T2;
-        gdiag = p.causal ? g0 + (uint32_t)wi.qt : 0xFFFFFFFFu;
+        gdiag = CAUSAL ? g0 + (uint32_t)wi.qt : 0xFFFFFFFFu;
       }
       for (uint32_t g = g0 + ((g0 & 1) != (uint32_t)pr); g < g0 + T2; g += 2) {   // this team's stages of the item
         const uint32_t m = g >> 1;
@@ -611,24 +611,24 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         int E0, E1;
         tmem_ld_32x32b_x32(tS, sraw);
         tmem_wait_ld();
-        if (g != gdiag) {
-          direct_p_block<AFFINE, false>(sraw, c32, p.aff_a, p.aff_b, p.thr16, 32, E0, w0);
+        if (!CAUSAL || g != gdiag) {
+          direct_p_block<AFFINE, false, THR16>(sraw, c32, p.aff_a, p.aff_b, 32, E0, w0);
           tmem_ld_32x32b_x32(tS + 32, sraw);
           tmem_wait_ld();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(sempty);                   // pair may take the stage after next
-          direct_p_block<AFFINE, false>(sraw, c32, p.aff_a, p.aff_b, p.thr16, 32, E1, w1);
+          direct_p_block<AFFINE, false, THR16>(sraw, c32, p.aff_a, p.aff_b, 32, E1, w1);
         } else {
           // causal diagonal stage: this row sees keys 0..row of the stage; the team's tile starts at key 64*(team&1)
           const int v0 = row - 64 * (team & 1) + 1;
-          direct_p_block<AFFINE, true>(sraw, c32, p.aff_a, p.aff_b, p.thr16, v0, E0, w0);
+          direct_p_block<AFFINE, true, THR16>(sraw, c32, p.aff_a, p.aff_b, v0, E0, w0);
           tmem_ld_32x32b_x32(tS + 32, sraw);
           tmem_wait_ld();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(sempty);
-          direct_p_block<AFFINE, true>(sraw, c32, p.aff_a, p.aff_b, p.thr16, v0 - 32, E1, w1);
+          direct_p_block<AFFINE, true, THR16>(sraw, c32, p.aff_a, p.aff_b, v0 - 32, E1, w1);
         }
         if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
         if (!ok) break;
@@ -727,13 +727,13 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint6
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool NV, bool AFFINE>
+template <int D, bool NV, bool AFFINE, bool CAUSAL, bool THR16>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
   const int Hkv = prm.Hkv;
   using C = Cfg<D, NV>;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV, AFFINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV, AFFINE, CAUSAL, THR16>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
       return FP4ATTN_ERR_CUDA;
     attr_set = true;
   }
@@ -748,7 +748,7 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return FP4ATTN_ERR_CUDA;
   const unsigned grid = (unsigned)(prm.n_items < sms ? prm.n_items : sms);     // persistent: one CTA per SM
-  attn_fwd_kernel<D, NV, AFFINE><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, tmO, prm);
+  attn_fwd_kernel<D, NV, AFFINE, CAUSAL, THR16><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, tmO, prm);
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
 
@@ -793,17 +793,25 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.aff_a = ops->affine_a != 0.f ? ops->affine_a : 1.5f;         // the paper's generic `fast` fit
   prm.aff_b = ops->affine_a != 0.f ? ops->affine_b : 1.2f;
   prm.thr16 = ops->p_scale_rule == FP4ATTN_PSCALE_THR16;
-  const int variant = (d == 128 ? 4 : 0) | (nv ? 2 : 0) | (affine ? 1 : 0);
+  // one kernel instance per (d, Q/K format, P map, mask, P scale rule): nothing of these is decided at run time
+  const int variant = (prm.thr16 ? 16 : 0) | (prm.causal ? 8 : 0) | (d == 128 ? 4 : 0) | (nv ? 2 : 0) | (affine ? 1 : 0);
+#define FP4ATTN_CASE4(n, D_, NV_, AFF_)                                                         \
+  case n: return launch_attn<D_, NV_, AFF_, false, false>(ops, B, H, N, prm, st);                \
+  case n + 8: return launch_attn<D_, NV_, AFF_, true, false>(ops, B, H, N, prm, st);             \
+  case n + 16: return launch_attn<D_, NV_, AFF_, false, true>(ops, B, H, N, prm, st);            \
+  case n + 24: return launch_attn<D_, NV_, AFF_, true, true>(ops, B, H, N, prm, st);
   switch (variant) {
-    case 0: return launch_attn<64, false, false>(ops, B, H, N, prm, st);
-    case 1: return launch_attn<64, false, true>(ops, B, H, N, prm, st);
-    case 2: return launch_attn<64, true, false>(ops, B, H, N, prm, st);
-    case 3: return launch_attn<64, true, true>(ops, B, H, N, prm, st);
-    case 4: return launch_attn<128, false, false>(ops, B, H, N, prm, st);
-    case 5: return launch_attn<128, false, true>(ops, B, H, N, prm, st);
-    case 6: return launch_attn<128, true, false>(ops, B, H, N, prm, st);
-    default: return launch_attn<128, true, true>(ops, B, H, N, prm, st);
+    FP4ATTN_CASE4(0, 64, false, false)
+    FP4ATTN_CASE4(1, 64, false, true)
+    FP4ATTN_CASE4(2, 64, true, false)
+    FP4ATTN_CASE4(3, 64, true, true)
+    FP4ATTN_CASE4(4, 128, false, false)
+    FP4ATTN_CASE4(5, 128, false, true)
+    FP4ATTN_CASE4(6, 128, true, false)
+    FP4ATTN_CASE4(7, 128, true, true)
+    default: return FP4ATTN_ERR_INVALID_ARG;
   }
+#undef FP4ATTN_CASE4
 }
 
 extern "C" int fp4attn_mma_peak_probe(int iters, unsigned long long* cycles_out, fp4attn_stream_t stream) {
