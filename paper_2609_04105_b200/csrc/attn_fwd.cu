@@ -4,16 +4,15 @@
 // (batch, head)) round-robin and walks the keys of an item in stages of 128 (two 64-key tiles, four
 // N32 probability blocks).  Score tiles live in a ring of four 64-column TMEM slots (two per stage),
 // each served by its own team of four softmax warps, so four independent score->code streams share
-// every SM sub-partition; everything that is sequential in the key index (row reference, row sum,
-// rescale of O, scale bytes of P) is done by separate correction warps on four numbers per row and
-// tile.  All roles keep running counters across items, so the next item's loads, QK products and
+// every SM sub-partition; everything that is sequential in the key index (row reference, rescale of O,
+// scale bytes of P) is done by separate correction warps on four numbers per row and stage.  All roles keep running counters across items, so the next item's loads, QK products and
 // softmax overlap the previous item's epilogue.
 //
 //   warp 0        TMA producer: Q tile per item (two buffers), ring of {K, V^T, K scales, V scales}
 //   warp 1        tensor-core issuer for S = Q K^T, one 128-key stage (two score slots) per issue
 //   warp 2        tensor-core issuer for O += P V, one stage (two K64 products) per issue
-//   warps 3-6     correction: integer row reference, represented row sum, E8M0 bytes of P,
-//                 exact power-of-two rescale of O, epilogue
+//   warps 3-6     correction: integer row reference, E8M0 bytes of P, exact power-of-two rescale of
+//                 O, epilogue; one pass per stage
 //   warps 7-22    softmax teams 0..3, one thread per query row; team 2p+h serves the h-th 64 keys of
 //                 the stages with parity p: Algorithm "direct-p-pack" up to the codes and their
 //                 sums; codes do not depend on the row reference, so teams never wait for one another
@@ -66,7 +65,7 @@ struct Cfg {
   static constexpr int NST = (D == 128) ? 6 : 8;                // ring depth (stages of 128 keys)
   static constexpr int P_BYTES = BM * (BN / 2);                 // 4 KB per 64-key tile: [block][row][16 B]
   static constexpr int PSF_BYTES = 512;                         // one atom per stage: bytes {0,1} tile 0, {2,3} tile 1
-  static constexpr int META_BYTES = BM * 8;                     // per row {E_0, E_1}
+  static constexpr int META_BYTES = BM * 16;                    // per stage parity and row: {E_0, E_1} of tile 0, of tile 1
   // shared-memory map (offsets from a 1024-byte aligned base)
   static constexpr int OFF_Q = 0;                               // two buffers
   static constexpr int OFF_QSF = OFF_Q + 2 * Q_BYTES;           // two buffers of 1 KB
@@ -74,7 +73,7 @@ struct Cfg {
   static constexpr int OFF_PSF = OFF_P + kTeams * P_BYTES;
   static constexpr int OFF_ONESF = OFF_PSF + 2 * PSF_BYTES;     // scale atom of 1.0 for the rows of ones
   static constexpr int OFF_META = OFF_ONESF + 512;
-  static constexpr int OFF_STAGE = (OFF_META + kTeams * META_BYTES + 1023) / 1024 * 1024;
+  static constexpr int OFF_STAGE = (OFF_META + 2 * META_BYTES + 1023) / 1024 * 1024;
   static constexpr int OFF_OUT = OFF_STAGE + NST * STAGE_BYTES; // bf16 O tile staged for TMA stores: D/64 halves of [128 rows][128 B]
   static constexpr int OUT_BYTES = (D / 64) * BM * 128;
   static constexpr int OFF_BAR = OFF_OUT + OUT_BYTES;
@@ -129,7 +128,7 @@ __device__ __forceinline__ WorkItem decode_item(int item, const AttnParams& p, i
 
 // barrier slots (8 bytes each)
 enum { BAR_QFULL0 = 0, BAR_QFREE0 = 2, BAR_OFULL = 4, BAR_OFREE = 5, BAR_SFULL0 = 6, BAR_SEMPTY0 = 8,
-       BAR_PFULL0 = 10, BAR_PFREE0 = 12, BAR_SMDONE0 = 14, BAR_RING = BAR_SMDONE0 + kTeams };
+       BAR_PFULL0 = 10, BAR_PFREE0 = 12, BAR_SMDONE0 = 14, BAR_RING = 16 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -169,7 +168,7 @@ __device__ __forceinline__ void fma2(float s0, float s1, float c, float b, float
 // reduction: x is at most log2(9.6) by construction of the block exponent, and below -2.75 it is clamped
 // (there the polynomial stays inside (0.18, 0.25), i.e. code 0 like 2^x).
 #ifndef FP4ATTN_POLY_MASK
-#define FP4ATTN_POLY_MASK 0x0842u      // which of a block's 16 element pairs take the polynomial path
+#define FP4ATTN_POLY_MASK 0x8421u      // which of a block's 16 element pairs take the polynomial path
 #endif
 __device__ __forceinline__ uint64_t pack2(float a, float b) {
   uint64_t r;
@@ -243,9 +242,6 @@ __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float 
   }
 }
 
-// AFFINE selects the affine classifier and, with it, stage-wise correction (both 64-key tiles of a stage
-// per pass): without the SFU work the teams outrun a tile-by-tile correction chain, while the exact
-// map runs ~2 % faster with the tile-by-tile chain, which staggers the teams.
 template <int D, bool NV, bool AFFINE, bool CAUSAL, bool THR16>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -276,12 +272,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       mbar_init(bar(BAR_QFREE0 + b), 1);
       mbar_init(bar(BAR_SFULL0 + b), 1);
       mbar_init(bar(BAR_SEMPTY0 + b), 8);      // both teams of the pair, four warps each
-      mbar_init(bar(BAR_PFULL0 + b), AFFINE ? 4 : 8);   // four correction warps, once per tile (per stage if AFFINE)
+      mbar_init(bar(BAR_PFULL0 + b), 4);       // the four correction warps, once per stage
+      mbar_init(bar(BAR_SMDONE0 + b), 8);      // both teams of the pair, four warps each
       mbar_init(bar(BAR_PFREE0 + b), 1);
     }
     mbar_init(bar(BAR_OFULL), 1);
     mbar_init(bar(BAR_OFREE), 4);
-    for (int t = 0; t < kTeams; ++t) mbar_init(bar(BAR_SMDONE0 + t), 4);
     for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
     *abortf = 0;
     fence_barrier_init();
@@ -462,20 +458,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
       T2 = wi.T2;
       int mu = -(1 << 28);
-      int pu0 = 0, pu1 = 0;                                     // bytes written for the previous tile (tile-by-tile mode)
-      // one pass per 64-key tile, or (AFFINE) one pass per 128-key stage covering both of its tiles
-      const int n_pass = AFFINE ? T2 : 2 * T2;
-      for (int j = 0; j < n_pass; ++j) {
-        const uint32_t g = g0 + (AFFINE ? j : (j >> 1));
-        const int h = AFFINE ? 0 : (j & 1), pr = g & 1;
-        const uint32_t par = (g >> 1) & 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + 2 * pr + h), par, abortf));
-        if (AFFINE && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + 2 * pr + 1), par, abortf));
+      for (uint32_t g = g0; g < g0 + T2; ++g) {                  // one pass per 128-key stage (both of its tiles)
+        const int pr = g & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + pr), (g >> 1) & 1, abortf));
         if (!ok) break;
-        const int2 ma = *reinterpret_cast<const int2*>(sgen + C::OFF_META + C::META_BYTES * (2 * pr + h) + row * 8);
-        const int2 mb = AFFINE ? *reinterpret_cast<const int2*>(sgen + C::OFF_META + C::META_BYTES * (2 * pr + 1) + row * 8) : ma;
-        uint8_t* psf = sgen + C::OFF_PSF + 512 * pr + lane * 16 + quarter * 4;
-        const int Emax = max(max(ma.x, ma.y), max(mb.x, mb.y));
+        const int4 me = *reinterpret_cast<const int4*>(sgen + C::OFF_META + C::META_BYTES * pr + row * 16);
+        const int Emax = max(max(me.x, me.y), max(me.z, me.w));
         const bool need = Emax > mu + kLazyShift;
         if (__any_sync(0xffffffffu, need)) {
           float f = 1.0f;
@@ -487,14 +475,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (delta > 126 && Emax <= mu + 126 + kLazyShift) delta = 126;
             f = (delta > 126) ? 0.f : __uint_as_float((uint32_t)(127 - delta) << 23);
             mu = (delta > 126) ? Emax + kRefHeadroom : mu + delta;
-            if (!AFFINE && h) {
-              // the stage's first tile is not in O yet (both tiles are issued together): move its bytes
-              pu0 = max(pu0 - delta, 0);
-              pu1 = max(pu1 - delta, 0);
-              *reinterpret_cast<uint16_t*>(psf) = (uint16_t)(pu0 | (pu1 << 8));
-            }
           }
-          if (AFFINE ? (j >= 1) : (j >= 2)) {
+          if (g > g0) {
             // O holds the item's earlier stages once their PV has landed
             const uint32_t gprev = g - 1;
             ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFREE0 + (gprev & 1)), (gprev >> 1) & 1, abortf));
@@ -515,14 +497,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         // A block more than 126 octaves below the reference is a zero block: it gets the smallest
         // byte (2^-127, below 2^-60 of the row's mass by construction) in numerator and row sum alike.
-        pu0 = max(ma.x - mu + 127, 0);
-        pu1 = max(ma.y - mu + 127, 0);
-        if (AFFINE) {
-          const uint32_t u2 = (uint32_t)max(mb.x - mu + 127, 0), u3 = (uint32_t)max(mb.y - mu + 127, 0);
-          *reinterpret_cast<uint32_t*>(psf) = (uint32_t)pu0 | ((uint32_t)pu1 << 8) | (u2 << 16) | (u3 << 24);
-        } else {
-          *reinterpret_cast<uint16_t*>(psf + 2 * h) = (uint16_t)(pu0 | (pu1 << 8));
-        }
+        const uint32_t u0 = (uint32_t)max(me.x - mu + 127, 0), u1 = (uint32_t)max(me.y - mu + 127, 0);
+        const uint32_t u2 = (uint32_t)max(me.z - mu + 127, 0), u3 = (uint32_t)max(me.w - mu + 127, 0);
+        *reinterpret_cast<uint32_t*>(sgen + C::OFF_PSF + 512 * pr + lane * 16 + quarter * 4) = u0 | (u1 << 8) | (u2 << 16) | (u3 << 24);
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + pr));
@@ -586,9 +563,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int row = quarter * 32 + lane;
     const uint32_t tS = tmem + ((uint32_t)(quarter * 32) << 16) + kColS + BN * team;
     const uint32_t sfull = bar(BAR_SFULL0 + pr), sempty = bar(BAR_SEMPTY0 + pr);
-    const uint32_t smdone = bar(BAR_SMDONE0 + team), pfree = bar(BAR_PFREE0 + pr);
+    const uint32_t smdone = bar(BAR_SMDONE0 + pr), pfree = bar(BAR_PFREE0 + pr);
     uint8_t* pbuf = sgen + C::OFF_P + C::P_BYTES * team + row * 16;
-    int2* meta = reinterpret_cast<int2*>(sgen + C::OFF_META + C::META_BYTES * team + row * 8);
+    int2* meta = reinterpret_cast<int2*>(sgen + C::OFF_META + C::META_BYTES * pr + row * 16 + 8 * (team & 1));
     float c32;
     if (NV) c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G), __ldg(p.k_G)));
     else    c32 = __fdiv_rn(p.c_base, 36.0f);
