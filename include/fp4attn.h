@@ -93,6 +93,23 @@ int fp4attn_quantize(const void* x_bf16, int fmt, int role, int B, int H, int N,
                      void* packed_out, void* scales_out, float* tensor_scale_out,
                      void* workspace, size_t workspace_bytes, fp4attn_stream_t stream);
 
+/* Which of the two powers of two that Eq. "mx-scale" allows becomes the amplitude of an MXFP4 block with
+ * maximum magnitude a (the paper fixes none; Section "Problem 2" names both neighbours). */
+enum { FP4ATTN_QSCALE_CEIL = 0,    /* alpha = 2^ceil(log2 a): the maximum lands in (3, 6], nothing saturates      */
+       FP4ATTN_QSCALE_THR16 = 1,   /* alpha = 2^floor(log2(1.6 a)): maxima up to 1.25 alpha saturate at code 6    */
+       FP4ATTN_QSCALE_FLOOR = 2 }; /* alpha = 2^floor(log2 a): the maximum always saturates at code 6             */
+
+/*
+ * MXFP4 operand quantizer with a selectable amplitude rule (Eq. "mx-scale"): as fp4attn_quantize with
+ * fmt = FP4ATTN_FMT_MXFP4, except that the E8M0 byte is u = clamp(127 + e, 1, 254) with e the exponent
+ * the rule picks, and that codes are q = Q_E2M1(6 v / 2^(u-127)) saturating at +-6.  FP4ATTN_QSCALE_CEIL
+ * gives the bytes of fp4attn_quantize.  The decision is taken on the bf16 bit pattern of the block
+ * maximum (significand >= 1.25 for the threshold rule), so it is exact.  Same buffers, layouts,
+ * alignment and status codes as fp4attn_quantize; no workspace.
+ */
+int fp4attn_quantize_mxfp4_rule(const void* x_bf16, int role, int scale_rule, int B, int H, int N, int d,
+                                void* packed_out, void* scales_out, fp4attn_stream_t stream);
+
 /* Largest tensor fp4attn_quantize_nvfp4_noalloc accepts: 2^27 elements. */
 #define FP4ATTN_NOALLOC_MAX_ELEMENTS (1ull << 27)
 

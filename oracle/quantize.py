@@ -4,7 +4,8 @@ MXFP4 (Eq. "mx-scale", amplitude convention): a block of 32 values with maximum
 magnitude a stores the power-of-two amplitude alpha = 2**ceil(log2 a) as the E8M0 byte
 u = 127 + ceil(log2 a) and the codes q = Q_E2M1(6 v / alpha); a value is reconstructed
 as alpha * q / 6.  Reading taken here: the ceiling of the two powers the paper allows,
-so the block maximum lands in (3, 6] and never saturates.
+so the block maximum lands in (3, 6] and never saturates; the floor and the threshold rule
+alpha = 2**floor(log2(1.6 a)) are selectable (`rule`), and then maxima above alpha saturate.
 
 NVFP4 (Table "fp4-formats", Eq. "nv-scale"): a block of 16 values stores
 S_B = Q_E4M3(G a_B / 6) and q = Q_E2M1(G v / S_B); reconstruction S_B q / G.  Reading
@@ -35,17 +36,33 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- MXFP4
-def mx_quantize_lastdim(x: np.ndarray):
+def mx_amplitude_exponent(a: np.ndarray, rule: str) -> np.ndarray:
+    """Exponent e of the amplitude alpha = 2**e for block maxima a > 0 (Eq. "mx-scale" allows either
+    power of two next to a):  "ceil"  ceil(log2 a);  "floor"  floor(log2 a);
+    "thr16"  floor(log2(1.6 a)), i.e. round up exactly when a / 2**floor(log2 a) >= 1.25."""
+    m, k = np.frexp(a)                      # a = m 2**k, m in [0.5, 1): exact
+    fl = k.astype(np.int64) - 1             # floor(log2 a)
+    if rule == "floor":
+        return fl
+    if rule == "ceil":
+        return fl + (m != 0.5)
+    if rule == "thr16":
+        return fl + (2.0 * m >= 1.25)
+    raise ValueError(rule)
+
+
+def mx_quantize_lastdim(x: np.ndarray, rule: str = "ceil"):
     """x float64 [..., L], L % 32 == 0, blocks of 32 along the last axis.
 
-    Returns (nibbles uint8 [..., L], scale bytes uint8 [..., L/32]).
+    Returns (nibbles uint8 [..., L], scale bytes uint8 [..., L/32]).  `rule` picks the amplitude
+    (see mx_amplitude_exponent); values above it saturate at code 6.
     """
     L = x.shape[-1]
     assert L % MX_BLOCK == 0
     xb = x.reshape(x.shape[:-1] + (L // MX_BLOCK, MX_BLOCK))
     a = np.abs(xb).max(axis=-1)
     nz = a > 0
-    e = ceil_log2(np.where(nz, a, 1.0))
+    e = ceil_log2(np.where(nz, a, 1.0)) if rule == "ceil" else mx_amplitude_exponent(np.where(nz, a, 1.0), rule)
     u = np.clip(e + 127, 1, 254)
     u = np.where(nz, u, 0).astype(np.uint8)
     alpha = e8m0_decode(u)
@@ -108,21 +125,21 @@ def nv_dequantize_lastdim(nib: np.ndarray, sbyte: np.ndarray, G=None, hw: bool =
 
 
 # --------------------------------------------------------------------------- roles
-def quantize_qk(bits: np.ndarray, fmt: str):
+def quantize_qk(bits: np.ndarray, fmt: str, rule: str = "ceil"):
     """Q or K, bf16 bit patterns [B,H,N,d] -> dict(nib [B,H,N,d], sf [B,H,N,d/blk], G)."""
     x = bf16_bits_to_f64(bits)
     if fmt == "mx":
-        nib, sf = mx_quantize_lastdim(x)
+        nib, sf = mx_quantize_lastdim(x, rule)
         return {"nib": nib, "sf": sf, "G": None, "fmt": "mx"}
     G = nv_tensor_scale(x)
     nib, sf = nv_quantize_lastdim(x, G)
     return {"nib": nib, "sf": sf, "G": G, "fmt": "nv"}
 
 
-def quantize_v(bits: np.ndarray):
+def quantize_v(bits: np.ndarray, rule: str = "ceil"):
     """V bf16 [B,H,N,d] -> MXFP4 of V^T: dict(nib [B,H,d,N], sf [B,H,d,N/32]), blocks of 32 keys."""
     xt = np.ascontiguousarray(np.swapaxes(bf16_bits_to_f64(bits), -1, -2))
-    nib, sf = mx_quantize_lastdim(xt)
+    nib, sf = mx_quantize_lastdim(xt, rule)
     return {"nib": nib, "sf": sf, "G": None, "fmt": "mx"}
 
 

@@ -16,6 +16,7 @@ FMT_MXFP4, FMT_NVFP4 = 0, 1
 ROLE_Q, ROLE_K, ROLE_V = 0, 1, 2
 PMAP_IDEAL, PMAP_AFFINE = 0, 1
 PSCALE_CEIL, PSCALE_THR16 = 0, 1
+QSCALE_CEIL, QSCALE_THR16, QSCALE_FLOOR = 0, 1, 2
 ERR_TIMEOUT = 7
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -25,7 +26,7 @@ EXPORTS = [
     "fp4attn_status_string", "fp4attn_version", "fp4attn_packed_bytes", "fp4attn_scale_bytes",
     "fp4attn_quantize_workspace_bytes", "fp4attn_quantize", "fp4attn_fwd",
     "fp4attn_attention_host_workspace_bytes", "fp4attn_attention_host", "fp4attn_mma_peak_probe",
-    "fp4attn_quantize_nvfp4_noalloc", "fp4attn_selftest_bounded_wait",
+    "fp4attn_quantize_nvfp4_noalloc", "fp4attn_selftest_bounded_wait", "fp4attn_quantize_mxfp4_rule",
 ]
 
 
@@ -65,6 +66,8 @@ def _load() -> ctypes.CDLL:
     lib.fp4attn_attention_host_workspace_bytes.argtypes = [i, i, i, i, i]
     lib.fp4attn_attention_host.restype = i
     lib.fp4attn_attention_host.argtypes = [vp, vp, vp, i, ctypes.c_float, i, i, i, i, vp, vp, vp, sz, vp]
+    lib.fp4attn_quantize_mxfp4_rule.restype = i
+    lib.fp4attn_quantize_mxfp4_rule.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp]
     lib.fp4attn_quantize_nvfp4_noalloc.restype = i
     lib.fp4attn_quantize_nvfp4_noalloc.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp]
     lib.fp4attn_selftest_bounded_wait.restype = i
@@ -127,6 +130,24 @@ def fp4attn_quantize(x: torch.Tensor, fmt: int, role: int, workspace: Optional[t
                               _ptr(G), _ptr(workspace), 0 if workspace is None else workspace.numel(), _stream()),
            "fp4attn_quantize")
     return QuantizedOperand(packed, scales, G, fmt, role, (B, H, N, d))
+
+
+def fp4attn_quantize_mxfp4_rule(x: torch.Tensor, role: int, scale_rule: int) -> QuantizedOperand:
+    """MXFP4 quantizer with a selectable amplitude rule (QSCALE_CEIL / QSCALE_THR16 / QSCALE_FLOOR)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 4
+    B, H, N, d = x.shape
+    L = lib()
+    nb = L.fp4attn_packed_bytes(B, H, N, d)
+    ns = L.fp4attn_scale_bytes(FMT_MXFP4, role, B, H, N, d)
+    if nb == 0 or ns == 0:
+        _check(L.fp4attn_quantize_mxfp4_rule(x.data_ptr(), role, scale_rule, B, H, N, d, 1, 1, _stream()),
+               "fp4attn_quantize_mxfp4_rule")
+        raise Fp4AttnError("fp4attn_quantize_mxfp4_rule: unsupported arguments")
+    packed = torch.empty(nb, dtype=torch.uint8, device=x.device)
+    scales = torch.empty(ns, dtype=torch.uint8, device=x.device)
+    _check(L.fp4attn_quantize_mxfp4_rule(x.data_ptr(), role, scale_rule, B, H, N, d, packed.data_ptr(),
+                                         scales.data_ptr(), _stream()), "fp4attn_quantize_mxfp4_rule")
+    return QuantizedOperand(packed, scales, None, FMT_MXFP4, role, (B, H, N, d))
 
 
 def fp4attn_quantize_nvfp4_noalloc(x: torch.Tensor, role: int, packed: torch.Tensor, scales: torch.Tensor,

@@ -23,11 +23,16 @@ __device__ __forceinline__ uint32_t absmax_bf16x8(const uint4& r) {
   const uint32_t m = __vmaxu2(__vmaxu2(r.x & 0x7FFF7FFFu, r.y & 0x7FFF7FFFu), __vmaxu2(r.z & 0x7FFF7FFFu, r.w & 0x7FFF7FFFu));
   return max(m & 0xFFFFu, m >> 16);
 }
-// E8M0 byte from the bf16 bit pattern of the block maximum (see mx_scale_byte)
+// E8M0 byte from the bf16 bit pattern of the block maximum a = (1 + m/128) 2^(e-127): the biased exponent
+// e, plus one where the rule rounds the amplitude up (Eq. "mx-scale" allows either neighbouring power of
+// two): ceiling - whenever a is not a power of two; threshold - alpha = 2^floor(log2(1.6 a)), i.e. when
+// 1 + m/128 >= 1.25; floor - never.  Values above the amplitude saturate at code 6 in the conversion.
+template <int RULE>
 __device__ __forceinline__ uint32_t mx_scale_byte_bf16(uint32_t a16) {
   if (a16 == 0) return 0;
-  const uint32_t u = (a16 >> 7) + ((a16 & 0x7Fu) != 0 ? 1u : 0u);
-  return min(max(u, 1u), 254u);
+  const uint32_t m = a16 & 0x7Fu;
+  const uint32_t up = RULE == FP4ATTN_QSCALE_CEIL ? (m != 0) : RULE == FP4ATTN_QSCALE_THR16 ? (m >= 32u) : 0u;
+  return min(max((a16 >> 7) + up, 1u), 254u);
 }
 __device__ __forceinline__ uint32_t mx_codes_x8(const uint4& raw, uint32_t u) {
   float v[8];
@@ -45,7 +50,7 @@ __device__ __forceinline__ uint32_t mx_codes_x8(const uint4& raw, uint32_t u) {
 }
 
 // grid (N * D/8 / kGroupsPerCta, B*H)
-template <int D>
+template <int D, int RULE>
 __global__ void __launch_bounds__(kThreads)
 quant_mx_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
                      uint8_t* __restrict__ sf, int N) {
@@ -63,7 +68,7 @@ quant_mx_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
     uint32_t a = absmax_bf16x8(raw[k]);
     a = max(a, __shfl_xor_sync(0xffffffffu, a, 1));
     a = max(a, __shfl_xor_sync(0xffffffffu, a, 2));
-    const uint32_t u = mx_scale_byte_bf16(a);
+    const uint32_t u = mx_scale_byte_bf16<RULE>(a);
     packed[gbase + g] = mx_codes_x8(raw[k], u);
     const uint32_t row = g / GPR, seg = g % GPR;
     uint8_t* p = sfb + (row >> 7) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4;
@@ -76,7 +81,7 @@ quant_mx_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
 // A [128 keys x D] tile goes through shared memory; a thread owns two adjacent head-dim columns and
 // one 32-key block, reads them as bf16x2 words (conflict-free) and writes two 16-byte code groups.
 // grid (N / 128, B*H), 2*D threads
-template <int D>
+template <int D, int RULE>
 __global__ void __launch_bounds__(2 * D)
 quant_mx_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ packed, uint8_t* __restrict__ sf, int N) {
   constexpr int T = 2 * D;                         // threads: D/2 column pairs x 4 key blocks
@@ -104,7 +109,7 @@ quant_mx_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ packed, uint8
   }
 #pragma unroll
   for (int c = 0; c < 2; ++c) {                    // low half = column 2cp, high half = column 2cp+1
-    const uint32_t u = mx_scale_byte_bf16(c ? (m >> 16) : (m & 0xFFFFu));
+    const uint32_t u = mx_scale_byte_bf16<RULE>(c ? (m >> 16) : (m & 0xFFFFu));
     float v[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(c ? (w[i] & 0xFFFF0000u) : (w[i] << 16));
@@ -253,19 +258,29 @@ extern "C" size_t fp4attn_quantize_workspace_bytes(int fmt, int role, int B, int
 
 namespace fp4attn {
 // Shared by fp4attn_quantize and the variants that bring their own scratch.
+template <int RULE>
+static void launch_mx(const uint4* xs, int role, int B, int H, int N, int d, void* packed, void* scales, cudaStream_t st) {
+  if (role != FP4ATTN_ROLE_V) {
+    const dim3 grid2((unsigned)((size_t)N * d / 8 / kGroupsPerCta), (unsigned)(B * H));   // N % 128 == 0 makes this exact
+    if (d == 128) quant_mx_rows_kernel<128, RULE><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
+    else          quant_mx_rows_kernel<64, RULE><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
+  } else {
+    dim3 g2(N / 128, B * H);
+    if (d == 128) quant_mx_v_kernel<128, RULE><<<g2, 256, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
+    else          quant_mx_v_kernel<64, RULE><<<g2, 128, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
+  }
+}
+
 int launch_quantize(const void* x, int fmt, int role, int B, int H, int N, int d, void* packed, void* scales,
-                    float* G_out, float* partials, cudaStream_t st) {
+                    float* G_out, float* partials, cudaStream_t st, int mx_rule) {
   const size_t n_groups = (size_t)B * H * N * d / 8;
   const unsigned grid = (unsigned)(n_groups / kGroupsPerCta);
   const dim3 grid2((unsigned)((size_t)N * d / 8 / kGroupsPerCta), (unsigned)(B * H));   // N % 128 == 0 makes this exact
   const uint4* xs = reinterpret_cast<const uint4*>(x);
-  if (fmt == FP4ATTN_FMT_MXFP4 && role != FP4ATTN_ROLE_V) {
-    if (d == 128) quant_mx_rows_kernel<128><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
-    else          quant_mx_rows_kernel<64><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
-  } else if (fmt == FP4ATTN_FMT_MXFP4) {
-    dim3 g2(N / 128, B * H);
-    if (d == 128) quant_mx_v_kernel<128><<<g2, 256, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
-    else          quant_mx_v_kernel<64><<<g2, 128, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
+  if (fmt == FP4ATTN_FMT_MXFP4) {
+    if (mx_rule == FP4ATTN_QSCALE_THR16)      launch_mx<FP4ATTN_QSCALE_THR16>(xs, role, B, H, N, d, packed, scales, st);
+    else if (mx_rule == FP4ATTN_QSCALE_FLOOR) launch_mx<FP4ATTN_QSCALE_FLOOR>(xs, role, B, H, N, d, packed, scales, st);
+    else                                      launch_mx<FP4ATTN_QSCALE_CEIL>(xs, role, B, H, N, d, packed, scales, st);
   } else {
     const int n_partials = (int)(grid < (unsigned)kMaxPartials ? grid : kMaxPartials);
     amax_partials_kernel<<<n_partials, kThreads, 0, st>>>(xs, n_groups, partials);
@@ -299,7 +314,20 @@ extern "C" int fp4attn_quantize(const void* x, int fmt, int role, int B, int H, 
   if (need && ((uintptr_t)workspace & 15)) return FP4ATTN_ERR_ALIGNMENT;
   rc = check_device_sm100();
   if (rc != FP4ATTN_OK) return rc;
-  return launch_quantize(x, fmt, role, B, H, N, d, packed, scales, G_out, (float*)workspace, (cudaStream_t)stream);
+  return launch_quantize(x, fmt, role, B, H, N, d, packed, scales, G_out, (float*)workspace, (cudaStream_t)stream,
+                         FP4ATTN_QSCALE_CEIL);
+}
+
+extern "C" int fp4attn_quantize_mxfp4_rule(const void* x, int role, int scale_rule, int B, int H, int N, int d,
+                                           void* packed, void* scales, fp4attn_stream_t stream) {
+  if (scale_rule != FP4ATTN_QSCALE_CEIL && scale_rule != FP4ATTN_QSCALE_THR16 && scale_rule != FP4ATTN_QSCALE_FLOOR)
+    return FP4ATTN_ERR_INVALID_ARG;
+  int rc = validate_quantize(x, FP4ATTN_FMT_MXFP4, role, B, H, N, d, packed, scales, nullptr);
+  if (rc != FP4ATTN_OK) return rc;
+  rc = check_device_sm100();
+  if (rc != FP4ATTN_OK) return rc;
+  return launch_quantize(x, FP4ATTN_FMT_MXFP4, role, B, H, N, d, packed, scales, nullptr, nullptr, (cudaStream_t)stream,
+                         scale_rule);
 }
 
 // ---------------------------------------------------------------- allocation-free NVFP4 variant
@@ -325,5 +353,5 @@ extern "C" int fp4attn_quantize_nvfp4_noalloc(const void* x, int role, int B, in
     scratch_addr[dev] = ptr;
   }
   return launch_quantize(x, FP4ATTN_FMT_NVFP4, role, B, H, N, d, packed, scales, G_out, scratch_addr[dev],
-                         (cudaStream_t)stream);
+                         (cudaStream_t)stream, FP4ATTN_QSCALE_CEIL);
 }

@@ -98,3 +98,60 @@ def test_byte_layouts():
         off = ((r // 128) * 2 + c // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + c % 4
         assert sw[0, 1, off] == sf[0, 1, r, c]
     assert sw[0, 0].astype(int).sum() == sf[0, 0].astype(int).sum()      # padding is zero
+
+
+def test_mx_amplitude_rules_against_exact_rational_arithmetic():
+    """Eq. "mx-scale": alpha is one of the two powers of two next to the block maximum.  The three rules'
+    exponents are checked against their definitions in exact integer arithmetic on every positive normal
+    bf16 value with exponent -20..20: ceil(log2 a), floor(log2 a), floor(log2(1.6 a)) (8 a >= 5 2^j)."""
+    from fractions import Fraction
+    pats = np.array([(e << 7) | m for e in range(107, 148) for m in range(128)], dtype=np.uint16)
+    a = Qz.bf16_bits_to_f64(pats)
+    got = {r: Qz.mx_amplitude_exponent(a, r) for r in ("ceil", "floor", "thr16")}
+    for i, v in enumerate(a):
+        f = Fraction(float(v))
+        fl = f.numerator.bit_length() - f.denominator.bit_length()
+        if Fraction(2) ** fl > f:
+            fl -= 1
+        assert Fraction(2) ** fl <= f < Fraction(2) ** (fl + 1)
+        assert got["floor"][i] == fl
+        assert got["ceil"][i] == (fl if f == Fraction(2) ** fl else fl + 1)
+        j = fl + 1 if 8 * f >= 5 * Fraction(2) ** (fl + 1) else fl      # 1.6 a >= 2^(fl+1)
+        assert got["thr16"][i] == j
+    # the default quantizer is the ceiling rule
+    x = np.random.default_rng(0).standard_normal((3, 64)) * 3
+    xb = Qz.bf16_bits_to_f64(I.f32_to_bf16_bits(x.astype(np.float32)))
+    n0, u0 = Qz.mx_quantize_lastdim(xb)
+    n1, u1 = Qz.mx_quantize_lastdim(xb, "ceil")
+    assert np.array_equal(n0, n1) and np.array_equal(u0, u1)
+
+
+def test_mx_amplitude_rules_closed_forms_and_saturation():
+    """Hand-computed blocks.  Maximum 1.25: ceil -> alpha 2 (6v/alpha = 3.75 -> value 4, code index 6), thr16 -> alpha 2,
+    floor -> alpha 1 (7.5 saturates at 6).  Maximum 1.2421875: thr16 keeps alpha 1 and saturates.  The block
+    maximum's code is 6 for every block under floor, never saturated under ceil, and reconstruction error on
+    Gaussian blocks orders thr16 < ceil < floor (the threshold rule is the paper's lower-error choice)."""
+    blk = np.zeros((1, 32)); blk[0, 0] = 1.25; blk[0, 1] = -0.5
+    for rule, u, c0 in (("ceil", 128, 6), ("thr16", 128, 6), ("floor", 127, 7)):
+        nib, ub = Qz.mx_quantize_lastdim(blk, rule)
+        assert ub[0, 0] == u and nib[0, 0] == c0, rule
+    blk[0, 0] = 1.2421875
+    for rule, u, c0 in (("ceil", 128, 6), ("thr16", 127, 7), ("floor", 127, 7)):
+        nib, ub = Qz.mx_quantize_lastdim(blk, rule)
+        assert ub[0, 0] == u and nib[0, 0] == c0, rule
+    assert Qz.mx_quantize_lastdim(blk, "thr16")[0][0, 1] == 8 + 5          # -0.5 * 6 / 1 = -3 -> code index 5 (value 3), sign bit
+    rng = np.random.default_rng(2)
+    x = Qz.bf16_bits_to_f64(I.f32_to_bf16_bits(rng.standard_normal((64, 256)).astype(np.float32)))
+    err = {}
+    for rule in ("ceil", "thr16", "floor"):
+        nib, u = Qz.mx_quantize_lastdim(x, rule)
+        xr = Qz.mx_dequantize_lastdim(nib, u)
+        err[rule] = np.linalg.norm(xr - x) / np.linalg.norm(x)
+        top = (nib & 7).reshape(64, 8, 32).max(axis=-1)
+        if rule == "floor":
+            assert np.all(top == 7)
+        if rule == "ceil":
+            xb = np.abs(x).reshape(64, 8, 32)
+            assert np.all(np.abs(xr).reshape(64, 8, 32).max(axis=-1) <= 2.0 ** np.ceil(np.log2(xb.max(axis=-1))))
+    assert err["thr16"] < err["ceil"] < err["floor"]
+    assert 0.10 < err["thr16"] < 0.12 and 0.17 < err["floor"] < 0.19

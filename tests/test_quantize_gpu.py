@@ -78,3 +78,52 @@ def test_full_size_quantizer_sampled(tmp_path):
     _check_operand(got, want, Bd.ROLE_Q)
     got = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
     _check_operand(got, Qz.quantize_v(v), Bd.ROLE_V)
+
+
+RULES = [("ceil", 0), ("thr16", 1), ("floor", 2)]
+
+
+@pytest.mark.parametrize("rule,code", RULES)
+@pytest.mark.parametrize("name,kw", [("cfg1", dict()), ("cfg1", dict(d=64, N=384, H=3)), ("cfg4", dict(H=2, N=640))])
+def test_mx_amplitude_rules_match_oracle(name, kw, rule, code):
+    """Eq. "mx-scale" with either neighbouring power of two: bytes and codes bit for bit, all three roles."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    for bits, role in ((q, Bd.ROLE_Q), (k, Bd.ROLE_K)):
+        got = Bd.fp4attn_quantize_mxfp4_rule(_dev(bits), role, code)
+        _check_operand(got, Qz.quantize_qk(bits, "mx", rule), role)
+    got = Bd.fp4attn_quantize_mxfp4_rule(_dev(v), Bd.ROLE_V, code)
+    _check_operand(got, Qz.quantize_v(v, rule), Bd.ROLE_V)
+    if rule == "ceil":                                      # the default entry point writes the same bytes
+        ref = Bd.fp4attn_quantize(_dev(q), Bd.FMT_MXFP4, Bd.ROLE_Q)
+        again = Bd.fp4attn_quantize_mxfp4_rule(_dev(q), Bd.ROLE_Q, code)
+        assert torch.equal(ref.packed, again.packed) and torch.equal(ref.scales, again.scales)
+
+
+@pytest.mark.parametrize("rule,code", RULES)
+def test_mx_amplitude_rules_edge_values(rule, code):
+    """Maxima exactly on the threshold (significand 1.25), just below it, powers of two, saturating values."""
+    from paper_2609_04105_b200 import binding as Bd
+    rng = np.random.default_rng(5)
+    x = (rng.standard_normal((1, 1, 128, 128)) * 0.1).astype(np.float32)
+    x[0, 0, 0, 0] = 1.25          # threshold: rounds up under thr16
+    x[0, 0, 1, 0] = 1.2421875     # largest bf16 below it: stays
+    x[0, 0, 2, 0] = -2.0          # power of two: amplitude 2 under every rule
+    x[0, 0, 3, 0] = 1.9921875     # largest significand
+    x[0, 0, 4, :32] = 0.0
+    x[0, 0, 5, :] *= 1e30
+    x[0, 0, 6, :] = 2.0 ** -130
+    x[0, 0, 7, 0] = 3.0e38
+    bits = I.f32_to_bf16_bits(x)
+    got = Bd.fp4attn_quantize_mxfp4_rule(_dev(bits), Bd.ROLE_Q, code)
+    _check_operand(got, Qz.quantize_qk(bits, "mx", rule), Bd.ROLE_Q)
+    got = Bd.fp4attn_quantize_mxfp4_rule(_dev(bits), Bd.ROLE_V, code)
+    _check_operand(got, Qz.quantize_v(bits, rule), Bd.ROLE_V)
+
+
+def test_mx_amplitude_rule_rejects_unknown_rule():
+    from paper_2609_04105_b200 import binding as Bd
+    x = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_quantize_mxfp4_rule(x, Bd.ROLE_Q, 7)
