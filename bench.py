@@ -124,6 +124,9 @@ def _blas_threads():
         return len(os.sched_getaffinity(0))
 
 
+HYBRID_PATTERNS = {"hybrid4": 0x1111, "hybrid8": 0x5555, "hybrid12": 0x7777}     # exact element pairs of 16
+
+
 def oracle_sample(w, q, k, v, heads, rows, p_map="ideal", p_scale="ceil"):
     """Runs the oracle (as it stands) on a bounded sample: the given (b, h) pairs and query rows.
     Returns seconds, equivalent TFLOP/s, and its outputs."""
@@ -144,7 +147,8 @@ def oracle_sample(w, q, k, v, heads, rows, p_map="ideal", p_scale="ceil"):
     else:
         qd, kd = Qz.quantize_qk(qs, "mx"), Qz.quantize_qk(ks, "mx")
     vd = Qz.quantize_v(vs)
-    O, lse = A.direct_p_forward(qd, kd, vd, rows=rows, heads=[(0, i) for i in range(len(heads))], p_map=p_map, p_scale=p_scale)
+    okw = dict(p_map="hybrid", exact_pairs=HYBRID_PATTERNS[p_map]) if p_map in HYBRID_PATTERNS else dict(p_map=p_map)
+    O, lse = A.direct_p_forward(qd, kd, vd, rows=rows, heads=[(0, i) for i in range(len(heads))], p_scale=p_scale, **okw)
     dt = time.perf_counter() - t0
     n_rows = w.N if rows is None else len(rows)
     flops = 4.0 * len(heads) * n_rows * w.N * w.d
@@ -234,7 +238,8 @@ def run_cuda(args, w):
     qws = torch.empty(max(16, Bd.lib().fp4attn_quantize_workspace_bytes(w.qk_fmt, 0, B, H, N, d)), dtype=torch.uint8, device=dev)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)      # > 126 MB L2
     launches_per_step = 4 if w.qk_fmt == I.FMT_MXFP4 else 6
-    pmap = Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_IDEAL
+    pmap = Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_HYBRID if args.p_map in HYBRID_PATTERNS else Bd.PMAP_IDEAL
+    pairs = HYBRID_PATTERNS.get(args.p_map, 0)
     pscale = Bd.PSCALE_THR16 if args.p_scale == "thr16" else Bd.PSCALE_CEIL
     state = {}
 
@@ -244,7 +249,7 @@ def run_cuda(args, w):
         vd = Bd.fp4attn_quantize(dv, Bd.FMT_MXFP4, Bd.ROLE_V)
         if ev is not None:
             ev[0].record()
-        Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status, p_map=pmap, p_scale_rule=pscale)
+        Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status, p_map=pmap, p_scale_rule=pscale, exact_pairs=pairs)
         if ev is not None:
             ev[1].record()
         state["ops"] = (qd, kd, vd)
@@ -456,8 +461,9 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the attention-only timings of the other configurations")
     ap.add_argument("--p-scale", default="ceil", choices=["ceil", "thr16"],
                     help="block-exponent rule of P: ceiling (default) or floor(max y + log2 1.6)")
-    ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine"],
-                    help="score->code map of the timed path: exact codes (default) or the paper's affine classifier")
+    ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine", "hybrid4", "hybrid8", "hybrid12"],
+                    help="score->code map of the timed path: exact codes (default), the paper's affine classifier, or "
+                         "4 / 8 / 12 of every 16 element pairs exact and the rest affine (EX2-density control)")
     args = ap.parse_args()
     w = I.WORKLOADS[args.workload]
     if args.impl == "reference":

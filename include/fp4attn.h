@@ -52,7 +52,9 @@ enum { FP4ATTN_FMT_MXFP4 = 0, FP4ATTN_FMT_NVFP4 = 1 };
 enum { FP4ATTN_ROLE_Q = 0, FP4ATTN_ROLE_K = 1, FP4ATTN_ROLE_V = 2 };
 /* how a normalised score x = y - E_B + log2 6 becomes an E2M1 probability code */
 enum { FP4ATTN_PMAP_IDEAL = 0,    /* q = Q_E2M1(2^x)              (Eq. "ideal-code-path")  */
-       FP4ATTN_PMAP_AFFINE = 1 }; /* q = Q_E2M1(max(0, A x + B))  (Eq. "affine-code-map")  */
+       FP4ATTN_PMAP_AFFINE = 1,   /* q = Q_E2M1(max(0, A x + B))  (Eq. "affine-code-map")  */
+       FP4ATTN_PMAP_HYBRID = 2 }; /* per element pair one of the two: the EX2-density control of
+                                     Appendix "SM103 launch and EX2 controls"; see exact_pairs     */
 
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* fp4attn_status_string(int status);
@@ -154,7 +156,7 @@ typedef struct {
   const float *q_G, *k_G;           /* device fp32 encode factors; NVFP4 only, else NULL     */
   int qk_fmt;                       /* format of Q and K; P and V are always MXFP4           */
   float softmax_scale;              /* 0 selects 1/sqrt(d)                                   */
-  int p_map;                        /* FP4ATTN_PMAP_IDEAL or FP4ATTN_PMAP_AFFINE             */
+  int p_map;                        /* FP4ATTN_PMAP_IDEAL, _AFFINE or _HYBRID                */
   float affine_a, affine_b;         /* classifier constants; affine_a == 0 selects the
                                        paper's generic fit A = 1.50, B = 1.20                */
   int p_scale_rule;                 /* FP4ATTN_PSCALE_CEIL or FP4ATTN_PSCALE_THR16           */
@@ -162,6 +164,11 @@ typedef struct {
   int kv_heads;                     /* K and V hold this many heads ([B, kv_heads, N, d]);
                                        H query heads share them in groups of H / kv_heads
                                        (grouped-query attention).  0 selects H               */
+  int exact_pairs;                  /* p_map = FP4ATTN_PMAP_HYBRID only: element pair k of every
+                                       32-key block (keys 2k, 2k+1) takes the ideal map where bit k
+                                       is set, the affine map elsewhere.  Supported patterns:
+                                       0x1111, 0x5555, 0x7777 (4, 8, 12 of 16 pairs exact);
+                                       noncausal only                                          */
 } fp4attn_operands;
 
 /*
@@ -175,7 +182,8 @@ typedef struct {
  * of a query row takes the integer exponent E_B = ceil(max_j y_j), each score maps straight to
  * the E2M1 code q_j = Q_E2M1(2^(y_j - E_B + log2 6)) (p_map = IDEAL; with p_map = AFFINE the paper's
  * classifier q_j = Q_E2M1(max(0, u_j)), u_j = fl32(S_j * fl32(A c) + fl32(A (log2 6 - E_B) + B)), a single
- * fused multiply-add per score, replaces the exponential), and the block's E8M0 byte is
+ * fused multiply-add per score, replaces the exponential; with p_map = HYBRID a fixed pattern of element
+ * pairs, exact_pairs, keeps the exponential and the rest takes the classifier), and the block's E8M0 byte is
  * E_B - mu + 127 for an integer row reference mu that never exceeds the running maximum by
  * construction (blocks whose byte would drop below 1 are zero blocks).  P V runs as a second
  * block-scaled FP4 product; the output is normalised by the sum of the same rounded values:

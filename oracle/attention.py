@@ -30,6 +30,10 @@ float32 so that a GPU reproduces the codes bit for bit:
     cA = fl32(A * c32),  bA = fl32(A * fl32(log2 6 - E_B) + B)  (one fma),  u = fl32(s32 * cA + bA)  (one fma).
 Block exponents, reference, denominator and output are unchanged.
 
+Mixed map (p_map="hybrid", the paper's EX2-density control, Appendix "SM103 launch and EX2 controls"):
+element pair k of a block (keys 2k, 2k+1) takes the ideal map where bit k of `exact_pairs` is set and the
+affine map elsewhere; which pairs pay for an exponential is a fixed pattern, so a GPU reproduces it.
+
 Second block-exponent rule (p_scale="thr16"): Eq. "mx-scale" allows either neighbouring power of two
 as the amplitude; besides the ceiling (default) the oracle offers the threshold rule
 E_B = floor(fl32(max y + fl32(log2 1.6))), i.e. alpha_B = 2^floor(log2(1.6 a_B)): the block maximum then
@@ -96,7 +100,8 @@ def _fma32(a, b, c):
 
 
 def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int = 128, tile_order=None,
-                  p_map: str = "ideal", affine=(1.5, 1.2), p_scale: str = "ceil", row_index=None):
+                  p_map: str = "ideal", affine=(1.5, 1.2), p_scale: str = "ceil", row_index=None,
+                  exact_pairs: int = 0xFFFF):
     """Direct-P online softmax + PV for a set of query rows of one (batch, head).
 
     s32  [R, N] float32 tensor-core-facing scores;  Vhat [N, d] float64 reconstructed V.
@@ -114,7 +119,10 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
     O = np.zeros((R, Vhat.shape[1]))
     codes_all = np.zeros((R, N), dtype=np.uint8)
     EB_all = np.zeros((R, N // P_BLOCK), dtype=np.int64)
-    assert p_map in ("ideal", "affine")
+    assert p_map in ("ideal", "affine", "hybrid")
+    # hybrid: element pair k (keys 2k, 2k+1 of a block) takes the ideal map where bit k of exact_pairs is set,
+    # the affine map elsewhere
+    pair_exact = ((int(exact_pairs) >> (np.arange(P_BLOCK) // 2)) & 1).astype(bool)
     A32, B32 = np.float32(affine[0]), np.float32(affine[1])
     cA = np.float32(A32 * np.float32(c32))
     order = range(N // tile) if tile_order is None else tile_order
@@ -134,13 +142,14 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
             e_B = np.where(seen, E_B - mu, -np.inf)
             live = (e_B + 127) >= 1
             b_B32 = np.float32(LOG2_6_32 - E_B.astype(np.float32))
-            if p_map == "ideal":
+            if p_map in ("ideal", "hybrid"):
                 x = yx[:, bj:bj + P_BLOCK] + b_B32.astype(np.float64)[:, None]
                 code = e2m1_encode_mag(np.exp2(x))
-            else:
+            if p_map in ("affine", "hybrid"):
                 bA = _fma32(A32, b_B32, B32)
                 u = _fma32(s32[:, bj:bj + P_BLOCK], cA, bA[:, None])
-                code = e2m1_encode_mag(np.maximum(u, np.float32(0)).astype(np.float64))
+                code_a = e2m1_encode_mag(np.maximum(u, np.float32(0)).astype(np.float64))
+                code = code_a if p_map == "affine" else np.where(pair_exact[None, :], code, code_a)
             code = np.where(live[:, None], code, 0).astype(np.uint8)
             q = E2M1_VALUES[code]
             alpha = np.where(live, np.exp2(np.where(live, e_B, 0.0)), 0.0)
@@ -156,7 +165,7 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
 
 def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int = 128,
                      rows=None, heads=None, tile_order=None, p_map: str = "ideal", affine=(1.5, 1.2),
-                     p_scale: str = "ceil", causal: bool = False, kv_group: int = 1):
+                     p_scale: str = "ceil", causal: bool = False, kv_group: int = 1, exact_pairs: int = 0xFFFF):
     """Whole-operator oracle.  qd/kd/vd come from oracle.quantize.quantize_qk / quantize_v.
 
     rows : optional 1-D index array of query rows evaluated for every (b, h) (rows are
@@ -174,7 +183,7 @@ def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int
         s32 = scores_fp32(qd, kd, b, h, rows, hk)
         Vhat = dequantize({**vd, "nib": vd["nib"][b, hk][None, None], "sf": vd["sf"][b, hk][None, None]})[0, 0].T
         O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order, p_map, affine, p_scale,
-                                        ridx if causal else None)
+                                        ridx if causal else None, exact_pairs)
         Os.append(O)
         Ls.append(lse)
     return np.stack(Os), np.stack(Ls)

@@ -193,9 +193,16 @@ __device__ __forceinline__ void exp2_poly6(float x0, float x1, float& p0, float&
 //   ideal map  (Eq. "ideal-code-path"):  q = Q_E2M1(2^x),            x = y - E_B + log2 6
 //   affine map (Eq. "affine-code-map"):  q = Q_E2M1(max(0, A x + B)), folded into one fused multiply-add
 //                                        per element: u = s * fl32(A c) + fma(A, log2 6 - E_B, B)
-template <bool AFFINE, bool MASKED, bool THR16>
+// PMAP: 0 ideal map for every element, 1 affine map for every element, 2..4 mixed (the EX2-density control
+// of Appendix "SM103 launch and EX2 controls"): element pair k of the block takes the ideal map where bit
+// k of the pattern is set, the affine map elsewhere.
+__host__ __device__ constexpr uint32_t exact_pairs_of(int pmap) {
+  return pmap == 0 ? 0xFFFFu : pmap == 1 ? 0x0000u : pmap == 2 ? 0x1111u : pmap == 3 ? 0x5555u : 0x7777u;
+}
+template <int PMAP, bool MASKED, bool THR16>
 __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float A, float B, int visible, int& E,
                                                uint32_t* words) {
+  constexpr uint32_t kExact = exact_pairs_of(PMAP);
   const float LOG2_6 = 2.5849625007211560f;
   if (MASKED) {                                                 // causal diagonal: keys beyond the query get -inf
 #pragma unroll
@@ -212,37 +219,32 @@ __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float 
   const float t = THR16 ? __fadd_rd(__fadd_rn(ymax, 0.6780719161033630f), M) : __fadd_ru(ymax, M);
   E = (int)(__float_as_uint(t) - 0x4B400000u);
   const float bB = __fsub_rn(LOG2_6, __fsub_rn(t, M));          // t - M = (float)E, exact
-  if (AFFINE) {
-    const float cA = __fmul_rn(A, c32), bA = __fmaf_rn(A, bB, B);
+  const float cA = __fmul_rn(A, c32), bA = __fmaf_rn(A, bB, B);  // affine pairs only
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      float pv[8];
+  for (int w = 0; w < 4; ++w) {
+    float pv[8];
 #pragma unroll
-      for (int i = 0; i < 8; i += 2)
-        fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), cA, bA, pv[i], pv[i + 1]);
-      words[w] = cvt_e2m1x8_relu(pv);                            // the conversion clamps negative inputs to +0
-    }
-  } else {
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      float pv[8];
-#pragma unroll
-      for (int i = 0; i < 8; i += 2) {
+    for (int i = 0; i < 8; i += 2) {
+      const int pair = 4 * w + i / 2;
+      if ((kExact >> pair) & 1u) {
         float x0, x1;
         fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), c32, bB, x0, x1);
-        if ((FP4ATTN_POLY_MASK >> (4 * w + i / 2)) & 1u) {
+        if ((FP4ATTN_POLY_MASK >> pair) & 1u) {
           exp2_poly6(x0, x1, pv[i], pv[i + 1]);
         } else {
           pv[i] = ex2_approx(x0);
           pv[i + 1] = ex2_approx(x1);
         }
+      } else {
+        fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), cA, bA, pv[i], pv[i + 1]);
       }
-      words[w] = cvt_e2m1x8(pv);
     }
+    // the conversion clamps negative inputs to +0 (affine pairs; exact pairs are positive anyway)
+    words[w] = kExact == 0xFFFFu ? cvt_e2m1x8(pv) : cvt_e2m1x8_relu(pv);
   }
 }
 
-template <int D, bool NV, bool AFFINE, bool CAUSAL, bool THR16>
+template <int D, bool NV, int PMAP, bool CAUSAL, bool THR16>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -589,23 +591,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tmem_ld_32x32b_x32(tS, sraw);
         tmem_wait_ld();
         if (!CAUSAL || g != gdiag) {
-          direct_p_block<AFFINE, false, THR16>(sraw, c32, p.aff_a, p.aff_b, 32, E0, w0);
+          direct_p_block<PMAP, false, THR16>(sraw, c32, p.aff_a, p.aff_b, 32, E0, w0);
           tmem_ld_32x32b_x32(tS + 32, sraw);
           tmem_wait_ld();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(sempty);                   // pair may take the stage after next
-          direct_p_block<AFFINE, false, THR16>(sraw, c32, p.aff_a, p.aff_b, 32, E1, w1);
+          direct_p_block<PMAP, false, THR16>(sraw, c32, p.aff_a, p.aff_b, 32, E1, w1);
         } else {
           // causal diagonal stage: this row sees keys 0..row of the stage; the team's tile starts at key 64*(team&1)
           const int v0 = row - 64 * (team & 1) + 1;
-          direct_p_block<AFFINE, true, THR16>(sraw, c32, p.aff_a, p.aff_b, v0, E0, w0);
+          direct_p_block<PMAP, true, THR16>(sraw, c32, p.aff_a, p.aff_b, v0, E0, w0);
           tmem_ld_32x32b_x32(tS + 32, sraw);
           tmem_wait_ld();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(sempty);
-          direct_p_block<AFFINE, true, THR16>(sraw, c32, p.aff_a, p.aff_b, v0 - 32, E1, w1);
+          direct_p_block<PMAP, true, THR16>(sraw, c32, p.aff_a, p.aff_b, v0 - 32, E1, w1);
         }
         if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
         if (!ok) break;
@@ -704,13 +706,13 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint6
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool NV, bool AFFINE, bool CAUSAL, bool THR16>
+template <int D, bool NV, int PMAP, bool CAUSAL, bool THR16>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
   const int Hkv = prm.Hkv;
   using C = Cfg<D, NV>;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV, AFFINE, CAUSAL, THR16>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
       return FP4ATTN_ERR_CUDA;
     attr_set = true;
   }
@@ -725,7 +727,7 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return FP4ATTN_ERR_CUDA;
   const unsigned grid = (unsigned)(prm.n_items < sms ? prm.n_items : sms);     // persistent: one CTA per SM
-  attn_fwd_kernel<D, NV, AFFINE, CAUSAL, THR16><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, tmO, prm);
+  attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, tmO, prm);
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
 
@@ -743,11 +745,17 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   if (!(d == 64 || d == 128) || N < 128 || N % 128 != 0) return FP4ATTN_ERR_UNSUPPORTED_SHAPE;
   if ((uint64_t)B * H * N >= (1ull << 31)) return FP4ATTN_ERR_UNSUPPORTED_SHAPE;
   if (!(ops->softmax_scale >= 0.f)) return FP4ATTN_ERR_INVALID_ARG;
-  if (ops->p_map != FP4ATTN_PMAP_IDEAL && ops->p_map != FP4ATTN_PMAP_AFFINE) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->p_map != FP4ATTN_PMAP_IDEAL && ops->p_map != FP4ATTN_PMAP_AFFINE && ops->p_map != FP4ATTN_PMAP_HYBRID)
+    return FP4ATTN_ERR_INVALID_ARG;
+  int pmap = ops->p_map;                                          // kernel instance: 0 ideal, 1 affine, 2..4 mixed patterns
+  if (ops->p_map == FP4ATTN_PMAP_HYBRID) {
+    pmap = ops->exact_pairs == 0x1111 ? 2 : ops->exact_pairs == 0x5555 ? 3 : ops->exact_pairs == 0x7777 ? 4 : -1;
+    if (pmap < 0 || ops->causal) return FP4ATTN_ERR_INVALID_ARG;    // three patterns, noncausal only
+  }
   if (ops->p_scale_rule != FP4ATTN_PSCALE_CEIL && ops->p_scale_rule != FP4ATTN_PSCALE_THR16) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->kv_heads < 0 || (ops->kv_heads > 0 && H % ops->kv_heads != 0) || (ops->causal != 0 && ops->causal != 1))
     return FP4ATTN_ERR_INVALID_ARG;
-  if (ops->p_map == FP4ATTN_PMAP_AFFINE && !(ops->affine_a >= 0.f && ops->affine_a < 16.f && fabsf(ops->affine_b) < 16.f))
+  if (ops->p_map != FP4ATTN_PMAP_IDEAL && !(ops->affine_a >= 0.f && ops->affine_a < 16.f && fabsf(ops->affine_b) < 16.f))
     return FP4ATTN_ERR_INVALID_ARG;
   const uintptr_t a128 = (uintptr_t)ops->q | (uintptr_t)ops->k | (uintptr_t)ops->v | (uintptr_t)ops->q_sf |
                          (uintptr_t)ops->k_sf | (uintptr_t)ops->v_sf;
@@ -766,29 +774,39 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.c_base = 1.4426950408889634f * scale;                        // fl32(log2e_32 * scale_32)
   cudaStream_t st = (cudaStream_t)stream;
   const bool nv = ops->qk_fmt == FP4ATTN_FMT_NVFP4;
-  const bool affine = ops->p_map == FP4ATTN_PMAP_AFFINE;
   prm.aff_a = ops->affine_a != 0.f ? ops->affine_a : 1.5f;         // the paper's generic `fast` fit
   prm.aff_b = ops->affine_a != 0.f ? ops->affine_b : 1.2f;
   prm.thr16 = ops->p_scale_rule == FP4ATTN_PSCALE_THR16;
   // one kernel instance per (d, Q/K format, P map, mask, P scale rule): nothing of these is decided at run time
-  const int variant = (prm.thr16 ? 16 : 0) | (prm.causal ? 8 : 0) | (d == 128 ? 4 : 0) | (nv ? 2 : 0) | (affine ? 1 : 0);
-#define FP4ATTN_CASE4(n, D_, NV_, AFF_)                                                         \
-  case n: return launch_attn<D_, NV_, AFF_, false, false>(ops, B, H, N, prm, st);                \
-  case n + 8: return launch_attn<D_, NV_, AFF_, true, false>(ops, B, H, N, prm, st);             \
-  case n + 16: return launch_attn<D_, NV_, AFF_, false, true>(ops, B, H, N, prm, st);            \
-  case n + 24: return launch_attn<D_, NV_, AFF_, true, true>(ops, B, H, N, prm, st);
-  switch (variant) {
-    FP4ATTN_CASE4(0, 64, false, false)
-    FP4ATTN_CASE4(1, 64, false, true)
-    FP4ATTN_CASE4(2, 64, true, false)
-    FP4ATTN_CASE4(3, 64, true, true)
-    FP4ATTN_CASE4(4, 128, false, false)
-    FP4ATTN_CASE4(5, 128, false, true)
-    FP4ATTN_CASE4(6, 128, true, false)
-    FP4ATTN_CASE4(7, 128, true, true)
-    default: return FP4ATTN_ERR_INVALID_ARG;
+  const int shape = (d == 128 ? 2 : 0) | (nv ? 1 : 0);
+#define FP4ATTN_SHAPES(PM_, CAU_, THR_)                                                  \
+  switch (shape) {                                                                       \
+    case 0: return launch_attn<64, false, PM_, CAU_, THR_>(ops, B, H, N, prm, st);       \
+    case 1: return launch_attn<64, true, PM_, CAU_, THR_>(ops, B, H, N, prm, st);        \
+    case 2: return launch_attn<128, false, PM_, CAU_, THR_>(ops, B, H, N, prm, st);      \
+    default: return launch_attn<128, true, PM_, CAU_, THR_>(ops, B, H, N, prm, st);      \
   }
-#undef FP4ATTN_CASE4
+#define FP4ATTN_MASKS(PM_)                                         \
+  if (prm.causal) {                                                \
+    if (prm.thr16) { FP4ATTN_SHAPES(PM_, true, true) }             \
+    else           { FP4ATTN_SHAPES(PM_, true, false) }            \
+  } else {                                                         \
+    if (prm.thr16) { FP4ATTN_SHAPES(PM_, false, true) }            \
+    else           { FP4ATTN_SHAPES(PM_, false, false) }           \
+  }
+#define FP4ATTN_NONCAUSAL(PM_)                                     \
+  if (prm.thr16) { FP4ATTN_SHAPES(PM_, false, true) }              \
+  else           { FP4ATTN_SHAPES(PM_, false, false) }
+  switch (pmap) {
+    case 0: FP4ATTN_MASKS(0)
+    case 1: FP4ATTN_MASKS(1)
+    case 2: FP4ATTN_NONCAUSAL(2)
+    case 3: FP4ATTN_NONCAUSAL(3)
+    default: FP4ATTN_NONCAUSAL(4)
+  }
+#undef FP4ATTN_SHAPES
+#undef FP4ATTN_MASKS
+#undef FP4ATTN_NONCAUSAL
 }
 
 extern "C" int fp4attn_mma_peak_probe(int iters, unsigned long long* cycles_out, fp4attn_stream_t stream) {

@@ -322,3 +322,54 @@ def test_causal_config2_full_size_sampled_rows():
     heads = [(0, 3), (2, 9), (3, 15)]
     Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows, causal=True)
     check_heads(Og, Lg, Oo, Lo, heads, rows)
+
+
+# ------------------------------------------------------------------ mixed map (p_map = HYBRID)
+HYBRID_CASES = [
+    ("cfg1", dict(), 0x1111, "ceil"),
+    ("cfg1", dict(N=384, H=3), 0x5555, "ceil"),
+    ("cfg1", dict(d=64, N=512), 0x7777, "ceil"),
+    ("cfg3", dict(B=2, H=2, N=512), 0x5555, "ceil"),
+    ("cfg3", dict(B=1, H=2, N=384, d=128), 0x1111, "thr16"),
+    ("cfg4", dict(H=2, N=1024), 0x7777, "ceil"),
+    ("cfg2", dict(B=2, H=3, N=2304), 0x5555, "thr16"),
+]
+
+
+@pytest.mark.parametrize("name,kw,mask,p_scale", HYBRID_CASES)
+def test_hybrid_map_matches_oracle_elementwise(name, kw, mask, p_scale):
+    """A fixed pattern of element pairs takes the exact map, the rest the affine classifier; both sides
+    fix the pattern and the fp32 arithmetic, so the codes agree and the usual tolerances hold."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    rule = Bd.PSCALE_THR16 if p_scale == "thr16" else Bd.PSCALE_CEIL
+    Og, Lg = run_gpu_general(w, q, k, v, p_map=Bd.PMAP_HYBRID, exact_pairs=mask, p_scale_rule=rule)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, p_map="hybrid", exact_pairs=mask, p_scale=p_scale)
+    check_heads(Og, Lg, Oo, Lo, heads)
+
+
+def test_hybrid_map_config2_full_size_sampled_rows():
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.WORKLOADS["cfg2"]
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu_general(w, q, k, v, p_map=Bd.PMAP_HYBRID, exact_pairs=0x5555)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    rng = np.random.default_rng(13)
+    rows = np.sort(rng.choice(w.N, size=128, replace=False))
+    heads = [(0, 3), (2, 9)]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows, p_map="hybrid", exact_pairs=0x5555)
+    check_heads(Og, Lg, Oo, Lo, heads, rows)
+
+
+def test_hybrid_map_rejects_other_patterns_and_the_causal_mask():
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg1"], N=128)
+    q, k, v = I.make_qkv(w)
+    ops = [Bd.fp4attn_quantize(_dev(a), w.qk_fmt if r != Bd.ROLE_V else Bd.FMT_MXFP4, r)
+           for a, r in ((q, Bd.ROLE_Q), (k, Bd.ROLE_K), (v, Bd.ROLE_V))]
+    for kw in (dict(exact_pairs=0x0101), dict(exact_pairs=0), dict(exact_pairs=0x5555, causal=True)):
+        with pytest.raises(Bd.Fp4AttnError):
+            Bd.fp4attn_fwd(*ops, p_map=Bd.PMAP_HYBRID, **kw)

@@ -354,3 +354,41 @@ def test_grouped_query_attention_equals_repeating_the_kv_heads():
     krep, vrep = np.repeat(k[:, :2], 2, axis=1), np.repeat(v[:, :2], 2, axis=1)
     O2, L2 = A.direct_p_forward(qd, Qz.quantize_qk(krep, "mx"), Qz.quantize_v(vrep), causal=True)
     assert np.array_equal(O, O2) and np.array_equal(L, L2)
+
+
+# ------------------------------------------------------------------ mixed map (EX2-density control)
+def test_hybrid_map_takes_each_pair_from_the_map_its_bit_names():
+    """Appendix "SM103 launch and EX2 controls": a fixed share of the elements pays for the exponential.
+    Element pair k of a block (keys 2k, 2k+1) must carry the ideal map's code where bit k of the pattern is
+    set and the affine map's code elsewhere - checked position by position against the two pinned maps,
+    for every supported pattern and for the two degenerate ones."""
+    w, _, qd, kd, vd = _cfg1(N=256)
+    c32 = A.score_constant(qd, kd, w.d)
+    s32 = A.scores_fp32(qd, kd, 0, 0)
+    Vhat = np.ascontiguousarray(Qz.dequantize(vd)[0, 0].T)
+    Oi, Li, ci, Ei, _ = A.direct_p_rows(s32, c32, Vhat)
+    Oa, La, ca, Ea, _ = A.direct_p_rows(s32, c32, Vhat, p_map="affine")
+    assert np.array_equal(Ei, Ea)                                   # block exponents do not depend on the map
+    assert np.mean(ci != ca) > 0.3                                  # the two maps really differ on this input
+    for mask in (0x1111, 0x5555, 0x7777, 0xFFFF, 0x0000):
+        Oh, Lh, ch, Eh, _ = A.direct_p_rows(s32, c32, Vhat, p_map="hybrid", exact_pairs=mask)
+        assert np.array_equal(Eh, Ei)
+        for key in range(256):
+            pair = (key % 32) // 2
+            want = ci if (mask >> pair) & 1 else ca
+            assert np.array_equal(ch[:, key], want[:, key]), (hex(mask), key)
+    assert np.array_equal(A.direct_p_rows(s32, c32, Vhat, p_map="hybrid", exact_pairs=0xFFFF)[0], Oi)
+    assert np.array_equal(A.direct_p_rows(s32, c32, Vhat, p_map="hybrid", exact_pairs=0x0000)[0], Oa)
+
+
+def test_hybrid_map_error_falls_with_the_share_of_exact_pairs():
+    """The control's purpose (Table "b300-tuning": cosine rises with EX2 density): against fp64 attention
+    the error of 0, 4, 8, 12, 16 exact pairs of 16 decreases monotonically."""
+    w, (q, k, v), qd, kd, vd = _cfg1(N=512)
+    x = [Qz.bf16_bits_to_f64(a) for a in (q, k, v)]
+    Oe = np.stack([A.exact_attention(x[0][0, h], x[1][0, h], x[2][0, h])[0] for h in range(w.H)])
+    errs = []
+    for mask in (0x0000, 0x1111, 0x5555, 0x7777, 0xFFFF):
+        O, _ = A.direct_p_forward(qd, kd, vd, p_map="hybrid", exact_pairs=mask)
+        errs.append(np.linalg.norm(O - Oe) / np.linalg.norm(Oe))
+    assert all(a > b for a, b in zip(errs, errs[1:])), errs
