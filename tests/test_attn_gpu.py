@@ -373,3 +373,31 @@ def test_hybrid_map_rejects_other_patterns_and_the_causal_mask():
     for kw in (dict(exact_pairs=0x0101), dict(exact_pairs=0), dict(exact_pairs=0x5555, causal=True)):
         with pytest.raises(Bd.Fp4AttnError):
             Bd.fp4attn_fwd(*ops, p_map=Bd.PMAP_HYBRID, **kw)
+
+
+# ------------------------------------------------------------------ size limits
+def test_longest_sequence_sampled_rows():
+    """N = 65536 keys in one head (512 stages per work item, 2^16-key rows, the ring wraps 85 times):
+    index arithmetic and the long-running row sum.  24 sampled rows of B1 H1 d128 against the oracle."""
+    w = I.shrink(I.WORKLOADS["cfg1"], H=1, N=65536)
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu(w, q, k, v)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    rng = np.random.default_rng(21)
+    rows = np.sort(rng.choice(w.N, size=24, replace=False))
+    rows[0], rows[-1] = 0, w.N - 1
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=[(0, 0)], rows=rows)
+    check_heads(Og, Lg, Oo, Lo, [(0, 0)], rows)
+
+
+def test_many_small_heads_more_items_than_one_wave():
+    """B*H = 1024 heads of N = 128: 1024 single-stage work items on 148 persistent CTAs (every item is an
+    item boundary: Q double buffer, epilogue overlap, reference reset).  All heads checked."""
+    w = I.shrink(I.WORKLOADS["cfg1"], B=8, H=128, N=128)
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu(w, q, k, v)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    rng = np.random.default_rng(22)
+    heads = [(int(b), int(h)) for b, h in zip(rng.integers(0, w.B, 48), rng.integers(0, w.H, 48))]
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads)
+    check_heads(Og, Lg, Oo, Lo, heads)
