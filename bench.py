@@ -341,7 +341,7 @@ def run_cuda(args, w):
     if world == 1 and not args.no_sweep:
         del dq, dk, dv, hq, hk, hv, ws, ho, hl
         torch.cuda.empty_cache()
-        for name in ("cfg5_N1024", "cfg5_N8192", "cfg5_N32768", "cfg3", "cfg4"):
+        for name in ("cfg5_N1024", "cfg5_N2048", "cfg5_N8192", "cfg5_N16384", "cfg5_N32768", "cfg3", "cfg4"):
             if name == w.name:
                 continue
             ww = I.WORKLOADS[name]
