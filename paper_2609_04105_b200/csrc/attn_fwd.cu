@@ -96,6 +96,8 @@ struct AttnParams {
   int thr16;               // block exponent rule: 0 = ceil(max y), 1 = floor(max y + log2 1.6)
   int causal;              // 1: query row i sees keys 0..i
   int H, Hkv;              // query heads, K/V heads (H % Hkv == 0: grouped-query attention)
+  int BH;                  // B * H
+  unsigned long long recip_qtiles, recip_bh;   // ceil(2^64 / (N / 128)), ceil(2^64 / BH); 0 for a divisor of 1
 };
 
 // One work item = one 128-row query tile of one (batch, query head).
@@ -106,22 +108,30 @@ struct WorkItem {
   int kvh;                 // b*Hkv + h / (H/Hkv): the K/V head this query head reads
   int T2;                  // 128-key stages to walk (causal: up to and including the diagonal)
 };
+// floor(n / d) for n < 2^31 through the precomputed reciprocal ceil(2^64 / d) (0 stands for d = 1): the
+// roles decode a work item on their critical path, and a 32-bit division costs some fifty instructions
+__device__ __forceinline__ int fast_div(int n, unsigned long long recip) {
+  return recip ? (int)__umul64hi((unsigned long long)n, recip) : n;
+}
 template <bool CAUSAL>
 __device__ __forceinline__ WorkItem decode_item(int item, const AttnParams& p, int qtiles) {
   WorkItem w;
   int bh;
   if (CAUSAL) {             // longest items first, so the persistent CTAs finish together
-    const int BH = p.n_items / qtiles;
-    w.qt = qtiles - 1 - item / BH;
-    bh = item % BH;
+    const int r = fast_div(item, p.recip_bh);
+    w.qt = qtiles - 1 - r;
+    bh = item - r * p.BH;
   } else {                  // consecutive items share K/V in L2
-    bh = item / qtiles;
+    bh = fast_div(item, p.recip_qtiles);
     w.qt = item - bh * qtiles;
   }
   w.qrow0 = bh * p.N + w.qt * BM;
   w.qtile_lin = bh * qtiles + w.qt;
-  const int b = bh / p.H, h = bh - b * p.H;
-  w.kvh = b * p.Hkv + h / (p.H / p.Hkv);
+  w.kvh = bh;
+  if (p.H != p.Hkv) {       // grouped-query attention
+    const int b = bh / p.H, h = bh - b * p.H;
+    w.kvh = b * p.Hkv + h / (p.H / p.Hkv);
+  }
   w.T2 = CAUSAL ? w.qt + 1 : p.stages;
   return w;
 }
@@ -767,6 +777,9 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.q_G = ops->q_G; prm.k_G = ops->k_G;
   prm.O = (__nv_bfloat16*)O; prm.LSE = LSE; prm.status = device_status;
   prm.N = N; prm.stages = N / BS; prm.n_items = B * H * (N / BM);
+  prm.BH = B * H;
+  prm.recip_qtiles = (N / BM) > 1 ? ~0ull / (unsigned long long)(N / BM) + 1 : 0;
+  prm.recip_bh = prm.BH > 1 ? ~0ull / (unsigned long long)prm.BH + 1 : 0;
   prm.causal = ops->causal ? 1 : 0;
   prm.H = H;
   prm.Hkv = ops->kv_heads > 0 ? ops->kv_heads : H;
