@@ -22,7 +22,8 @@
 // of the accumulator is sum_j 2^(u_B-127) q_j over exactly the codes and scale bytes PV consumed.
 //
 // Tensor memory (512 columns): S slots 0..255 | O 256..399 (d + 16 columns) | Q scales 400..415 (two
-// buffers) | K scales 416..431 (two slots) | V scales 432..447 (two slots of 8) | P scales 448..455.
+// buffers) | K scales 416..431 (two slots) | V scales 432..447 (two slots of 8) | P scales 448..455 |
+// P codes 456..487 (per stage parity and 64-key tile 8 columns: 64 keys x 4 bits per row).
 #include <cuda.h>
 
 #include "common.cuh"
@@ -43,7 +44,8 @@ constexpr int kRefHeadroom = 60; // ... and is then set this far ABOVE that expo
                                  // needs a jump of 124 octaves: E8M0 bytes stay within 1..191, blocks weaker
                                  // than 2^-66 of the row maximum become zero blocks
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256, kColSFQ = 400, kColSFK = 416, kColSFV = 432, kColSFP = 448;
+constexpr uint32_t kColS = 0, kColO = 256, kColSFQ = 400, kColSFK = 416, kColSFV = 432, kColSFP = 448,
+                   kColP = 456;      // P codes: [stage parity][tile] x 8 columns (64 keys x 4 bits per row)
 constexpr int kOnesRows = 16;    // rows of ones appended to V^T (the MMA's N must be a multiple of 16)
 
 template <int D, bool NV>
@@ -62,19 +64,17 @@ struct Cfg {
   static constexpr int OFF_KSF = K_BYTES + V_BYTES + ONES_BYTES;   // within a stage
   static constexpr int OFF_VSF = OFF_KSF + KSF_BYTES;
   static constexpr int STAGE_BYTES = OFF_VSF + VSF_BYTES;
-  static constexpr int NST = (D == 128) ? 6 : 8;                // ring depth (stages of 128 keys)
-  static constexpr int P_BYTES = BM * (BN / 2);                 // 4 KB per 64-key tile: [block][row][16 B]
+  static constexpr int NST = (D == 128) ? 7 : 8;                // ring depth (stages of 128 keys)
   static constexpr int PSF_BYTES = 512;                         // one atom per stage: bytes {0,1} tile 0, {2,3} tile 1
   static constexpr int META_BYTES = BM * 16;                    // per stage parity and row: {E_0, E_1} of tile 0, of tile 1
   // shared-memory map (offsets from a 1024-byte aligned base)
   static constexpr int OFF_Q = 0;                               // two buffers
   static constexpr int OFF_QSF = OFF_Q + 2 * Q_BYTES;           // two buffers of 1 KB
-  static constexpr int OFF_P = OFF_QSF + 2048;
-  static constexpr int OFF_PSF = OFF_P + kTeams * P_BYTES;
+  static constexpr int OFF_PSF = OFF_QSF + 2048;
   static constexpr int OFF_ONESF = OFF_PSF + 2 * PSF_BYTES;     // scale atom of 1.0 for the rows of ones
   static constexpr int OFF_META = OFF_ONESF + 512;
   static constexpr int OFF_STAGE = (OFF_META + 2 * META_BYTES + 1023) / 1024 * 1024;
-  static constexpr int OFF_OUT = OFF_STAGE + NST * STAGE_BYTES; // bf16 O tile staged for TMA stores: D/64 halves of [128 rows][128 B]
+  static constexpr int OFF_OUT = (OFF_STAGE + NST * STAGE_BYTES + 1023) / 1024 * 1024; // bf16 O tile staged for TMA stores: D/64 halves of [128 rows][128 B]
   static constexpr int OUT_BYTES = (D / 64) * BM * 128;
   static constexpr int OFF_BAR = OFF_OUT + OUT_BYTES;
   static constexpr int SMEM_BYTES = OFF_BAR + 1024 + 1024;      // barriers + alignment slack
@@ -272,7 +272,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   constexpr uint64_t kDescSF = (uint64_t)(16 >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
   constexpr uint64_t kDescQK = (uint64_t)(16 >> 4) << 16 | (uint64_t)((8 * C::ROW_BYTES) >> 4) << 32 | 1ull << 46 | C::SWZ_QK << 61;
   constexpr uint64_t kDescV = (uint64_t)(16 >> 4) << 16 | (uint64_t)(512 >> 4) << 32 | 1ull << 46 | kSwz64 << 61;
-  constexpr uint64_t kDescP = (uint64_t)((BM * 16) >> 4) << 16 | (uint64_t)(128 >> 4) << 32 | 1ull << 46;
   auto at = [](uint64_t tmpl, uint32_t addr) { return tmpl | (uint64_t)((addr & 0x3FFFFu) >> 4); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -437,13 +436,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           __syncwarp();
         }
         const uint64_t dV = at(kDescV, stp + C::K_BYTES);
-        const uint64_t dP = at(kDescP, sbase + C::OFF_P + C::P_BYTES * 2 * pr);
         if (elect_one()) {
           tc_cp_32x128b_warpx4(tSFP, at(kDescSF, sbase + C::OFF_PSF + 512 * pr));
           tc_cp_32x128b_warpx4(tSFV, at(kDescSF, stp + C::OFF_VSF));
-          // tile h of the stage: P slot 2*pr+h, keys 64h..64h+63 of V^T (32 bytes on), scale bytes {2h, 2h+1}
-          tc_mma_fp4_2x(tO, dP, dV, kIdPV0, tSFP, tSFV, s2 > 0);
-          tc_mma_fp4_2x(tO, dP + (C::P_BYTES >> 4), dV + 2, kIdPV1, tSFP, tSFV, 1);
+          // tile h of the stage: P codes from tensor memory (the A operand; written there by the teams, so
+          // no shared-memory round trip and no proxy fence), keys 64h..64h+63 of V^T (32 bytes on), scale
+          // bytes {2h, 2h+1}
+          tc_mma_fp4_2x_ta(tO, tmem + kColP + 16 * pr, dV, kIdPV0, tSFP, tSFV, s2 > 0);
+          tc_mma_fp4_2x_ta(tO, tmem + kColP + 16 * pr + 8, dV + 2, kIdPV1, tSFP, tSFV, 1);
           tc_commit(bar_empty(sp));                             // stage back to the producer
           tc_commit(bar(BAR_PFREE0 + pr));                      // P slots reusable; O holds this stage
           if (s2 == T2 - 1) tc_commit(bar(BAR_OFULL));
@@ -589,7 +589,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t tS = tmem + ((uint32_t)(quarter * 32) << 16) + kColS + BN * team;
     const uint32_t sfull = bar(BAR_SFULL0 + pr), sempty = bar(BAR_SEMPTY0 + pr);
     const uint32_t smdone = bar(BAR_SMDONE0 + pr), pfree = bar(BAR_PFREE0 + pr);
-    uint8_t* pbuf = sgen + C::OFF_P + C::P_BYTES * team + row * 16;
+    const uint32_t tP = tmem + ((uint32_t)(quarter * 32) << 16) + kColP + 8 * team;
     int2* meta = reinterpret_cast<int2*>(sgen + C::OFF_META + C::META_BYTES * pr + row * 16 + 8 * (team & 1));
     float c32;
     if (NV) c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G), __ldg(p.k_G)));
@@ -634,10 +634,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
         if (!ok) break;
-        *reinterpret_cast<uint4*>(pbuf) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
-        *reinterpret_cast<uint4*>(pbuf + BM * 16) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+        {
+          const uint32_t pw[8] = {w0[0], w0[1], w0[2], w0[3], w1[0], w1[1], w1[2], w1[3]};
+          tmem_st_32x32b_x8(tP, pw);
+        }
         *meta = make_int2(E0, E1);
-        fence_proxy_async_smem();
+        tmem_wait_st();
+        tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smdone);
       }
