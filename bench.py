@@ -29,7 +29,7 @@ from paper_2609_04105_b200 import inputs as I  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised in profiles/
 # (attention: profiles/attn_fwd_cfg2.md, quantizer: profiles/quantizers_cfg2.md); other workloads: not captured.
-NCU_TRAFFIC_BYTES = {"cfg2": {"attn": 53.52e6 + 23.36e6, "quant_rows": 67.12e6 + 3.08e6}}
+NCU_TRAFFIC_BYTES = {"cfg2": {"attn": 53.52e6 + 24.48e6, "quant_rows": 67.12e6 + 3.08e6}}
 
 METRIC = "fp4_attention_fwd_tflops"
 UNIT = "TFLOP/s"
