@@ -323,6 +323,25 @@ def run_cuda(args, w):
     h2d = 3 * B * H * N * d * 2
     d2h = B * H * N * d * 2 + B * H * N * 4
 
+    # ---- the same workload's attention launch under the other code maps (context beside the timed map)
+    other_maps = {}
+    if world == 1:
+        qd0, kd0, vd0 = state["ops"]
+        for name, kw in (("ideal", dict(p_map=Bd.PMAP_IDEAL)), ("hybrid8", dict(p_map=Bd.PMAP_HYBRID, exact_pairs=0x5555)),
+                         ("affine", dict(p_map=Bd.PMAP_AFFINE))):
+            if name == args.p_map:
+                continue
+            for _ in range(3):
+                Bd.fp4attn_fwd(qd0, kd0, vd0, out=O, status=status, p_scale_rule=pscale, **kw)
+            m0, m1 = E(), E()
+            flush.fill_(2)
+            m0.record()
+            for _ in range(10):
+                Bd.fp4attn_fwd(qd0, kd0, vd0, out=O, status=status, p_scale_rule=pscale, **kw)
+            m1.record()
+            torch.cuda.synchronize()
+            other_maps[name] = {"attn_tflops": w.flops / (m0.elapsed_time(m1) / 10 * 1e-3) / 1e12}
+
     # ---- measured dense FP4 issue rate of this device (context for the roofline)
     cyc = torch.zeros(1, dtype=torch.int64, device=dev)
     iters = 20000
@@ -411,7 +430,8 @@ def run_cuda(args, w):
                    "l2": "flushed between steps (256 MiB fill, outside the step's events)",
                    "flops": "4*B*H*N^2*d", "parallelism": f"replica x{world}, (batch, head) units, no collective"},
         "attn_only": {"value": attn_tflops, "unit": UNIT, "ms": attn_launch_ms,
-                      "note": "attention kernel alone (the paper's timing boundary excludes quantization)"},
+                      "note": "attention kernel alone (the paper's timing boundary excludes quantization)",
+                      "other_code_maps": other_maps},
         "roofline": {"kernel": "attn_fwd_kernel", "bound": "tensor", "achieved": w.flops / (attn_launch_ms * 1e-3) / 1e12,
                      "peak": fp4_peak, "unit": "TFLOP/s",
                      "frac": w.flops / (attn_launch_ms * 1e-3) / 1e12 / fp4_peak,
