@@ -207,10 +207,18 @@ size_t fp4attn_attention_host_workspace_bytes(int qk_fmt, int B, int H, int N, i
 /*
  * Whole path from HOST buffers: copies bf16 Q, K, V [B,H,N,d] from (preferably pinned) host
  * memory into the caller's device workspace, quantizes them (fp4attn_quantize x3), runs
- * fp4attn_fwd and copies O (bf16) and, if LSE_host is not NULL, LSE back to host memory, all on
- * `stream`; returns after enqueuing.  q_host/k_host/v_host/O_host/LSE_host are HOST pointers,
- * workspace is a DEVICE pointer of at least fp4attn_attention_host_workspace_bytes() bytes,
- * 256-byte aligned.  The caller synchronises the stream before reading O_host.
+ * fp4attn_fwd and copies O (bf16) and, if LSE_host is not NULL, LSE back to host memory; returns
+ * after enqueuing.  q_host/k_host/v_host/O_host/LSE_host are HOST pointers, workspace is a DEVICE
+ * pointer of at least fp4attn_attention_host_workspace_bytes() bytes, 256-byte aligned.  The caller
+ * synchronises `stream` before reading O_host: everything the call enqueues has completed by then.
+ *
+ * With MXFP4 Q, K and at least 8 (batch, head) units the call is pipelined over groups of units (they
+ * are independent and MXFP4 needs no tensor-wide pass): the copy in of one group, the kernels of the
+ * previous one and the copy out of the one before overlap, so the path costs about its largest leg
+ * instead of the sum.  The copies then run on two internal streams (created on the first such call per
+ * device and kept until the process exits; no device memory is allocated) that fork from `stream` and
+ * join back into it through events.  NVFP4 (tensor-wide amax first) and small problems run on `stream`
+ * alone.  Results are bit-identical either way.
  */
 int fp4attn_attention_host(const void* q_host, const void* k_host, const void* v_host,
                            int qk_fmt, float softmax_scale, int B, int H, int N, int d,
