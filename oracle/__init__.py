@@ -8,12 +8,18 @@ cpu-baseline leg may call it.
 Pinned by tests/test_oracle_*.py (run with -m "not gpu"):
   formats.py    E2M1 / E8M0 / E4M3 coders      -> printed codebook and boundaries, exhaustive
                                                   enumeration, closed forms, Table "p-range"
-  quantize.py   MXFP4 / NVFP4 operand quantizers -> closed forms, brute force, error bounds
+  quantize.py   MXFP4 / NVFP4 operand quantizers -> closed forms, brute force, error bounds; the three
+                                                  amplitude rules -> exact rational arithmetic on every
+                                                  bf16 significand, hand-computed blocks, saturation
   attention.py  tiled Direct-P forward          -> tile-size / tile-order invariance, V == 1,
                                                   equal keys, dominant key, brute-force exact
                                                   attention on losslessly representable inputs;
                                                   affine code map -> its printed decision boundaries
                                                   (t_j - B)/A, the same invariants, the paper's
                                                   all-MXFP4 accuracy band; threshold amplitude rule
-                                                  -> closed form, Table "p-range" MXFP4 row
+                                                  -> closed form, Table "p-range" MXFP4 row; causal mask
+                                                  and grouped-query attention -> first row, whole-tile
+                                                  prefixes, brute force, repeated K/V heads; mixed map
+                                                  -> position by position against the two pinned maps,
+                                                  error monotone in the share of exact pairs
 """
