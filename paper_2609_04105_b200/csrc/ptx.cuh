@@ -1,4 +1,4 @@
-// Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (no multicast anywhere), tcgen05
+// Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (loads of this CTA only), tcgen05
 // (tensor memory allocation, block-scaled FP4 MMA, scale-factor copy, TMEM loads/stores).
 // Every wait is bounded: a wait that runs out returns false and the caller unwinds.
 #pragma once
