@@ -547,19 +547,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // let TMA write it out, so O is released after four TMEM reads instead of after 16 global stores
       if (lane == 0) bulk_wait_read_all();                      // this warp's previous stores have read the buffer
       __syncwarp();
-#pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
-        uint32_t o[32];
-        tmem_ld_32x32b_x32(tO + c0, o);
-        tmem_wait_ld();
-        if (c0 + 32 == D) {                                     // last read of O: the next item's PV may overwrite it
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar(BAR_OFREE));
-        }
+      // 16-column chunks, the next one in flight from tensor memory while this one is normalised and stored
+      uint32_t oa[16], ob[16];
+      tmem_ld_32x32b_x16(tO, oa);
+      tmem_wait_ld();
+#pragma unroll
+      for (int c0 = 0; c0 < D; c0 += 16) {
+        uint32_t* o = ((c0 >> 4) & 1) ? ob : oa;
+        uint32_t* nx = ((c0 >> 4) & 1) ? oa : ob;
+        if (c0 + 16 < D) tmem_ld_32x32b_x16(tO + c0 + 16, nx);
         uint8_t* half = sgen + C::OFF_OUT + (c0 >> 6) * (BM * 128) + row * 128;
 #pragma unroll
-        for (int c = 0; c < 32; c += 8) {
+        for (int c = 0; c < 16; c += 8) {
           uint32_t pk[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -568,6 +567,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
           const int chunk = ((c0 & 63) + c) >> 3;               // 16-byte chunk of the 128-byte row
           *reinterpret_cast<uint4*>(half + ((chunk ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+        if (c0 + 16 < D) {
+          tmem_wait_ld();
+          if (c0 + 32 == D) {                                   // last read of O: the next item's PV may overwrite it
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_OFREE));
+          }
         }
       }
       fence_proxy_async_smem();
