@@ -406,3 +406,47 @@ def test_many_small_heads_more_items_than_one_wave():
     heads = [(int(b), int(h)) for b, h in zip(rng.integers(0, w.B, 48), rng.integers(0, w.H, 48))]
     Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads)
     check_heads(Og, Lg, Oo, Lo, heads)
+
+
+# ------------------------------------------------------------------ seeded random configurations
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_random_configurations_match_oracle(seed):
+    """Forty seeded draws of (d, Q/K format, N, B, heads, K/V head sharing, mask, code map, block-exponent rule,
+    softmax scale, outlier channels) per seed: every combination of options on small shapes, sampled rows of two
+    heads each against the oracle, usual tolerances."""
+    from paper_2609_04105_b200 import binding as Bd
+    rng = np.random.default_rng(seed)
+    for _ in range(40):
+        d = int(rng.choice([64, 128])); nv = bool(rng.integers(0, 2))
+        N = 128 * int(rng.integers(1, 9)); B = int(rng.integers(1, 4))
+        group = int(rng.choice([1, 1, 2, 4])); Hkv = int(rng.integers(1, 4)); H = Hkv * group
+        causal = bool(rng.integers(0, 2)); pm = int(rng.choice([0, 0, 1, 2])); thr = bool(rng.integers(0, 2))
+        mask = int(rng.choice([0x1111, 0x5555, 0x7777]))
+        if pm == 2:
+            causal = False
+        scale = float(rng.choice([0.0, 0.05, 0.3]))
+        x = [rng.standard_normal((B, h, N, d)).astype(np.float32) for h in (H, Hkv, Hkv)]
+        if rng.integers(0, 4) == 0:                              # outlier channels as in config 4
+            ch = rng.choice(d, size=3, replace=False)
+            x[0][..., ch] *= 20
+            x[1][..., ch] *= 20
+        bits = [I.f32_to_bf16_bits(a) for a in x]
+        fmt = Bd.FMT_NVFP4 if nv else Bd.FMT_MXFP4
+        ops = [Bd.fp4attn_quantize(_dev(bits[0]), fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(bits[1]), fmt, Bd.ROLE_K),
+               Bd.fp4attn_quantize(_dev(bits[2]), Bd.FMT_MXFP4, Bd.ROLE_V)]
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        O, L = Bd.fp4attn_fwd(*ops, softmax_scale=scale, status=status, p_map=pm, p_scale_rule=int(thr), causal=causal,
+                              exact_pairs=mask if pm == 2 else 0)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        f = "nv" if nv else "mx"
+        qd, kd, vd = Qz.quantize_qk(bits[0], f), Qz.quantize_qk(bits[1], f), Qz.quantize_v(bits[2])
+        heads = [(int(rng.integers(0, B)), int(rng.integers(0, H))) for _ in range(2)]
+        rows = np.sort(rng.choice(N, size=min(N, 48), replace=False))
+        rows[0], rows[-1] = 0, N - 1
+        okw = dict(p_map=["ideal", "affine", "hybrid"][pm], p_scale="thr16" if thr else "ceil", causal=causal, kv_group=group,
+                   softmax_scale=(scale if scale > 0 else None))
+        if pm == 2:
+            okw["exact_pairs"] = mask
+        Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows, **okw)
+        check_heads(O.float().cpu().numpy().astype(np.float64), L.cpu().numpy().astype(np.float64), Oo, Lo, heads, rows)
