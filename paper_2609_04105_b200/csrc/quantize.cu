@@ -40,7 +40,9 @@ __device__ __forceinline__ uint32_t mx_codes_x8(const uint4& raw, uint32_t u) {
   if (u >= 2u) {
     const float s6 = __uint_as_float(((256u - u) << 23) | 0x400000u);   // 1.5 * 2^(129-u) = 6 / alpha
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] *= s6;
+    for (int i = 0; i < 8; i += 2)                                        // two exact products per instruction
+      asm("{\n\t.reg .b64 a, b, c;\n\tmov.b64 a, {%2, %3};\n\tmov.b64 b, {%4, %4};\n\tmul.rn.f32x2 c, a, b;\n\tmov.b64 {%0, %1}, c;\n\t}"
+          : "=f"(v[i]), "=f"(v[i + 1]) : "f"(v[i]), "f"(v[i + 1]), "f"(s6));
   } else {                                                              // alpha = 2^-126: 6/alpha overflows fp32
     const float inv = mx_inv_amplitude(u);
 #pragma unroll
