@@ -445,7 +445,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_mma_fp4_2x_ta(tO, tmem + kColP + 16 * pr, dV, kIdPV0, tSFP, tSFV, s2 > 0);
           tc_mma_fp4_2x_ta(tO, tmem + kColP + 16 * pr + 8, dV + 2, kIdPV1, tSFP, tSFV, 1);
           tc_commit(bar_empty(sp));                             // stage back to the producer
-          tc_commit(bar(BAR_PFREE0 + pr));                      // P slots reusable; O holds this stage
+          tc_commit(bar(BAR_PFREE0 + pr));                      // the stage's P columns reusable; O holds this stage
           if (s2 == T2 - 1) tc_commit(bar(BAR_OFULL));
         }
         __syncwarp();
@@ -456,8 +456,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     __syncwarp();
   } else if (warp < kFirstSoftmaxWarp) {
     // ===================================================================== correction warps
-    // One thread per query row, tiles in key order.  Owns the integer row reference mu, the
-    // represented row sum and the O accumulator's scale; turns the teams' absolute block exponents
+    // One thread per query row, stages in key order.  Owns the integer row reference mu and the O
+    // accumulator's scale (numerator and row-sum columns alike); turns the teams' absolute block exponents
     // into the E8M0 bytes the PV instruction reads.
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
