@@ -1,12 +1,13 @@
-// Noncausal full-FP4 attention forward with Direct-P for sm_100a.
+// Full-FP4 attention forward with Direct-P for sm_100a (noncausal or causal, optional grouped K/V heads).
 //
 // Persistent kernel, one CTA per SM.  A CTA takes work items (one 128-row query tile of one
 // (batch, head)) round-robin and walks the keys of an item in stages of 128 (two 64-key tiles, four
 // N32 probability blocks).  Score tiles live in a ring of four 64-column TMEM slots (two per stage),
 // each served by its own team of four softmax warps, so four independent score->code streams share
 // every SM sub-partition; everything that is sequential in the key index (row reference, rescale of O,
-// scale bytes of P) is done by separate correction warps on four numbers per row and stage.  All roles keep running counters across items, so the next item's loads, QK products and
-// softmax overlap the previous item's epilogue.
+// scale bytes of P) is done by separate correction warps on four numbers per row and stage.  All roles
+// keep running counters across items, so the next item's loads, QK products and softmax overlap the
+// previous item's epilogue.
 //
 //   warp 0        TMA producer: Q tile per item (two buffers), ring of {K, V^T, K scales, V scales}
 //   warp 1        tensor-core issuer for S = Q K^T, one 128-key stage (two score slots) per issue
@@ -14,8 +15,9 @@
 //   warps 3-6     correction: integer row reference, E8M0 bytes of P, exact power-of-two rescale of
 //                 O, epilogue; one pass per stage
 //   warps 7-22    softmax teams 0..3, one thread per query row; team 2p+h serves the h-th 64 keys of
-//                 the stages with parity p: Algorithm "direct-p-pack" up to the codes and their
-//                 sums; codes do not depend on the row reference, so teams never wait for one another
+//                 the stages with parity p: Algorithm "direct-p-pack" up to the codes (written
+//                 straight into tensor memory, PV's A operand) and the block exponents; codes do not
+//                 depend on the row reference, so teams never wait for one another
 //
 // The represented row sum (the denominator of Eq. "represented-output") is produced by the same PV
 // instruction as the numerator: sixteen constant rows of ones follow V^T in every stage, so column d
