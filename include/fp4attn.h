@@ -99,7 +99,11 @@ int fp4attn_quantize(const void* x_bf16, int fmt, int role, int B, int H, int N,
  * maximum magnitude a (the paper fixes none; Section "Problem 2" names both neighbours). */
 enum { FP4ATTN_QSCALE_CEIL = 0,    /* alpha = 2^ceil(log2 a): the maximum lands in (3, 6], nothing saturates      */
        FP4ATTN_QSCALE_THR16 = 1,   /* alpha = 2^floor(log2(1.6 a)): maxima up to 1.25 alpha saturate at code 6    */
-       FP4ATTN_QSCALE_FLOOR = 2 }; /* alpha = 2^floor(log2 a): the maximum always saturates at code 6             */
+       FP4ATTN_QSCALE_FLOOR = 2,   /* alpha = 2^floor(log2 a): the maximum always saturates at code 6             */
+       FP4ATTN_QSCALE_MSE = 3 };   /* per block the better of floor and ceiling: squared error of the 32 codes,
+                                      fp32, d_i = 6 v_i/alpha - q_i exact, fl32(d_i^2) added left to right within
+                                      groups of eight, groups as (g0 + g1) + (g2 + g3); floor only if strictly
+                                      smaller than four times the ceiling's (its units are four times larger)   */
 
 /*
  * MXFP4 operand quantizer with a selectable amplitude rule (Eq. "mx-scale"): as fp4attn_quantize with

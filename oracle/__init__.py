@@ -10,7 +10,9 @@ Pinned by tests/test_oracle_*.py (run with -m "not gpu"):
                                                   enumeration, closed forms, Table "p-range"
   quantize.py   MXFP4 / NVFP4 operand quantizers -> closed forms, brute force, error bounds; the three
                                                   amplitude rules -> exact rational arithmetic on every
-                                                  bf16 significand, hand-computed blocks, saturation
+                                                  bf16 significand, hand-computed blocks, saturation;
+                                                  MSE rule -> block errors in exact rational arithmetic,
+                                                  its fp32 summation order operation by operation
   attention.py  tiled Direct-P forward          -> tile-size / tile-order invariance, V == 1,
                                                   equal keys, dominant key, brute-force exact
                                                   attention on losslessly representable inputs;

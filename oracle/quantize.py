@@ -39,7 +39,8 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
 def mx_amplitude_exponent(a: np.ndarray, rule: str) -> np.ndarray:
     """Exponent e of the amplitude alpha = 2**e for block maxima a > 0 (Eq. "mx-scale" allows either
     power of two next to a):  "ceil"  ceil(log2 a);  "floor"  floor(log2 a);
-    "thr16"  floor(log2(1.6 a)), i.e. round up exactly when a / 2**floor(log2 a) >= 1.25."""
+    "thr16"  floor(log2(1.6 a)), i.e. round up exactly when a / 2**floor(log2 a) >= 1.25.
+    (The fourth rule of mx_quantize_lastdim, "mse", picks between floor and ceil per block.)"""
     m, k = np.frexp(a)                      # a = m 2**k, m in [0.5, 1): exact
     fl = k.astype(np.int64) - 1             # floor(log2 a)
     if rule == "floor":
@@ -62,13 +63,43 @@ def mx_quantize_lastdim(x: np.ndarray, rule: str = "ceil"):
     xb = x.reshape(x.shape[:-1] + (L // MX_BLOCK, MX_BLOCK))
     a = np.abs(xb).max(axis=-1)
     nz = a > 0
-    e = ceil_log2(np.where(nz, a, 1.0)) if rule == "ceil" else mx_amplitude_exponent(np.where(nz, a, 1.0), rule)
-    u = np.clip(e + 127, 1, 254)
+    a1 = np.where(nz, a, 1.0)
+    if rule == "mse":
+        # per block the better of the two neighbouring powers of two (Eq. "mx-scale" names both); the squared
+        # error is taken in float32 in a fixed order (mx_block_error32) so that a GPU reproduces the choice;
+        # the floor wins only if its error is strictly smaller
+        uf = np.clip(mx_amplitude_exponent(a1, "floor") + 127, 1, 254).astype(np.uint8)
+        uc = np.clip(mx_amplitude_exponent(a1, "ceil") + 127, 1, 254).astype(np.uint8)
+        ef, cf = mx_block_error32(xb, uf)
+        ec, cc = mx_block_error32(xb, uc)
+        take_f = (uf != uc) & (ef < np.float32(4.0) * ec)       # ceil's error is in units four times larger
+        u = np.where(take_f, uf, uc)
+        codes = np.where(take_f[..., None], cf, cc)
+    else:
+        e = ceil_log2(a1) if rule == "ceil" else mx_amplitude_exponent(a1, rule)
+        u = np.clip(e + 127, 1, 254).astype(np.uint8)
+        codes = e2m1_encode(6.0 * xb / e8m0_decode(u)[..., None])
     u = np.where(nz, u, 0).astype(np.uint8)
-    alpha = e8m0_decode(u)
-    codes = e2m1_encode(6.0 * xb / alpha[..., None])
     codes = np.where(nz[..., None], codes, 0).astype(np.uint8)
     return codes.reshape(x.shape), u
+
+
+def mx_block_error32(xb: np.ndarray, u: np.ndarray):
+    """Squared error of MXFP4 blocks [..., 32] under scale bytes u, in units of (alpha/6)**2, as float32 in
+    a fixed order: d_i = 6 v_i/alpha - q_i (exact above the float32 subnormal range), s_i = fl32(d_i*d_i); the eight s_i of each group of eight
+    consecutive elements are added left to right, then the four group sums as (g0 + g1) + (g2 + g3).
+    Returns (error float32 [...], codes uint8 [..., 32])."""
+    t = 6.0 * xb / e8m0_decode(u)[..., None]                   # exact, and exactly representable in float32
+    codes = e2m1_encode(t)
+    d = (t - e2m1_decode(codes)).astype(np.float32)
+    inexact = d.astype(np.float64) != t - e2m1_decode(codes)    # only below the float32 normal range, where
+    assert np.all(np.abs(t[inexact]) < 2.0 ** -126)             # fl32(d*d) is 0 whichever way d was rounded
+    s = (d * d).astype(np.float32).reshape(d.shape[:-1] + (4, 8))
+    g = s[..., 0]
+    for i in range(1, 8):
+        g = (g + s[..., i]).astype(np.float32)
+    err = ((g[..., 0] + g[..., 1]).astype(np.float32) + (g[..., 2] + g[..., 3]).astype(np.float32)).astype(np.float32)
+    return err, codes
 
 
 def mx_dequantize_lastdim(nib: np.ndarray, u: np.ndarray, hw: bool = False) -> np.ndarray:

@@ -16,7 +16,7 @@ FMT_MXFP4, FMT_NVFP4 = 0, 1
 ROLE_Q, ROLE_K, ROLE_V = 0, 1, 2
 PMAP_IDEAL, PMAP_AFFINE, PMAP_HYBRID = 0, 1, 2
 PSCALE_CEIL, PSCALE_THR16 = 0, 1
-QSCALE_CEIL, QSCALE_THR16, QSCALE_FLOOR = 0, 1, 2
+QSCALE_CEIL, QSCALE_THR16, QSCALE_FLOOR, QSCALE_MSE = 0, 1, 2, 3
 ERR_TIMEOUT = 7
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

@@ -1,5 +1,7 @@
 // Operand quantizers: bf16 -> packed E2M1 + scale bytes in the 128x4 atom order.
 // HBM-bound: 128-bit loads, block amax by lane shuffles, 32-bit / 128-bit stores.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace fp4attn {
@@ -34,21 +36,65 @@ __device__ __forceinline__ uint32_t mx_scale_byte_bf16(uint32_t a16) {
   const uint32_t up = RULE == FP4ATTN_QSCALE_CEIL ? (m != 0) : RULE == FP4ATTN_QSCALE_THR16 ? (m >= 32u) : 0u;
   return min(max((a16 >> 7) + up, 1u), 254u);
 }
-__device__ __forceinline__ uint32_t mx_codes_x8(const uint4& raw, uint32_t u) {
-  float v[8];
-  bf16x8_to_f32(raw, v);
+// v[i] <- 6 v[i] / alpha for the amplitude of byte u: exact in fp32 (one multiply by 1.5 * 2^k)
+template <int N_>
+__device__ __forceinline__ void mx_scale_values(float* v, uint32_t u) {
   if (u >= 2u) {
     const float s6 = __uint_as_float(((256u - u) << 23) | 0x400000u);   // 1.5 * 2^(129-u) = 6 / alpha
 #pragma unroll
-    for (int i = 0; i < 8; i += 2)                                        // two exact products per instruction
+    for (int i = 0; i < N_; i += 2)                                       // two exact products per instruction
       asm("{\n\t.reg .b64 a, b, c;\n\tmov.b64 a, {%2, %3};\n\tmov.b64 b, {%4, %4};\n\tmul.rn.f32x2 c, a, b;\n\tmov.b64 {%0, %1}, c;\n\t}"
           : "=f"(v[i]), "=f"(v[i + 1]) : "f"(v[i]), "f"(v[i + 1]), "f"(s6));
   } else {                                                              // alpha = 2^-126: 6/alpha overflows fp32
     const float inv = mx_inv_amplitude(u);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = (v[i] * inv) * 6.0f;
+    for (int i = 0; i < N_; ++i) v[i] = (v[i] * inv) * 6.0f;
   }
+}
+__device__ __forceinline__ uint32_t mx_codes_x8(const uint4& raw, uint32_t u) {
+  float v[8];
+  bf16x8_to_f32(raw, v);
+  mx_scale_values<8>(v, u);
   return cvt_e2m1x8(v);
+}
+// Squared error of eight scaled values t against their codes (one word), in code units: d = t - q exact,
+// fl32(d * d) added left to right in fp32 - the order the MSE amplitude rule is defined with.
+__device__ __forceinline__ float mx_error_x8(const float* t, uint32_t codes) {
+  float acc = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint32_t h2;
+    asm("{\n\t.reg .b8 b;\n\t.reg .b32 s;\n\tshr.b32 s, %1, %2;\n\tcvt.u8.u32 b, s;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}"
+        : "=r"(h2) : "r"(codes), "r"(8 * i));
+    const float2 q = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+    const float d0 = __fsub_rn(t[2 * i], q.x), d1 = __fsub_rn(t[2 * i + 1], q.y);
+    const float s0 = __fmul_rn(d0, d0), s1 = __fmul_rn(d1, d1);
+    acc = (i == 0) ? s0 : __fadd_rn(acc, s0);
+    acc = __fadd_rn(acc, s1);
+  }
+  return acc;
+}
+// MSE rule, blocks along d: the four eight-element groups of a block sit in four adjacent lanes, so the
+// group sums meet as (g0 + g1) + (g2 + g3) in every lane.  The floor's error is in units four times
+// smaller than the ceiling's, hence the factor; the floor wins only if strictly better.  Returns the
+// chosen byte, `word` gets this lane's codes under it.
+__device__ __forceinline__ uint32_t mx_choose_mse_rows(const uint4& raw, uint32_t a16, uint32_t& word) {
+  const uint32_t uf = mx_scale_byte_bf16<FP4ATTN_QSCALE_FLOOR>(a16), uc = mx_scale_byte_bf16<FP4ATTN_QSCALE_CEIL>(a16);
+  float tf[8], tc[8];
+  bf16x8_to_f32(raw, tf);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tc[i] = tf[i];
+  mx_scale_values<8>(tf, uf);
+  mx_scale_values<8>(tc, uc);
+  const uint32_t wf = cvt_e2m1x8(tf), wc = cvt_e2m1x8(tc);
+  float ef = mx_error_x8(tf, wf), ec = mx_error_x8(tc, wc);
+  ef = __fadd_rn(ef, __shfl_xor_sync(0xffffffffu, ef, 1));
+  ec = __fadd_rn(ec, __shfl_xor_sync(0xffffffffu, ec, 1));
+  ef = __fadd_rn(ef, __shfl_xor_sync(0xffffffffu, ef, 2));
+  ec = __fadd_rn(ec, __shfl_xor_sync(0xffffffffu, ec, 2));
+  const bool take_f = (uf != uc) && (ef < __fmul_rn(4.0f, ec));
+  word = take_f ? wf : wc;
+  return take_f ? uf : uc;
 }
 
 // grid (N * D/8 / kGroupsPerCta, B*H)
@@ -70,8 +116,14 @@ quant_mx_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
     uint32_t a = absmax_bf16x8(raw[k]);
     a = max(a, __shfl_xor_sync(0xffffffffu, a, 1));
     a = max(a, __shfl_xor_sync(0xffffffffu, a, 2));
-    const uint32_t u = mx_scale_byte_bf16<RULE>(a);
-    packed[gbase + g] = mx_codes_x8(raw[k], u);
+    uint32_t u, word;
+    if (RULE == FP4ATTN_QSCALE_MSE) {
+      u = mx_choose_mse_rows(raw[k], a, word);
+    } else {
+      u = mx_scale_byte_bf16<RULE>(a);
+      word = mx_codes_x8(raw[k], u);
+    }
+    packed[gbase + g] = word;
     const uint32_t row = g / GPR, seg = g % GPR;
     uint8_t* p = sfb + (row >> 7) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4;
     if ((seg & 3) == 0) p[seg >> 2] = (uint8_t)u;                    // one lane per 32-block
@@ -111,24 +163,41 @@ quant_mx_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ packed, uint8
   }
 #pragma unroll
   for (int c = 0; c < 2; ++c) {                    // low half = column 2cp, high half = column 2cp+1
-    const uint32_t u = mx_scale_byte_bf16<RULE>(c ? (m >> 16) : (m & 0xFFFFu));
+    const uint32_t a16 = c ? (m >> 16) : (m & 0xFFFFu);
+    uint32_t u = mx_scale_byte_bf16<RULE == FP4ATTN_QSCALE_MSE ? FP4ATTN_QSCALE_CEIL : RULE>(a16);
     float v[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(c ? (w[i] & 0xFFFF0000u) : (w[i] << 16));
-    if (u >= 2u) {
-      const float s6 = __uint_as_float(((256u - u) << 23) | 0x400000u);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] *= s6;
-    } else {
-      const float inv = mx_inv_amplitude(u);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = (v[i] * inv) * 6.0f;
-    }
     uint4 out;
-    out.x = cvt_e2m1x8(v);
-    out.y = cvt_e2m1x8(v + 8);
-    out.z = cvt_e2m1x8(v + 16);
-    out.w = cvt_e2m1x8(v + 24);
+    if (RULE == FP4ATTN_QSCALE_MSE) {
+      // both amplitudes; group sums of eight consecutive keys combined as (g0 + g1) + (g2 + g3)
+      const uint32_t uf = mx_scale_byte_bf16<FP4ATTN_QSCALE_FLOOR>(a16);
+      float tf[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) tf[i] = v[i];
+      mx_scale_values<32>(tf, uf);
+      mx_scale_values<32>(v, u);
+      uint32_t wf[4], wc[4];
+      float gf[4], gc[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        wf[j] = cvt_e2m1x8(tf + 8 * j);
+        wc[j] = cvt_e2m1x8(v + 8 * j);
+        gf[j] = mx_error_x8(tf + 8 * j, wf[j]);
+        gc[j] = mx_error_x8(v + 8 * j, wc[j]);
+      }
+      const float ef = __fadd_rn(__fadd_rn(gf[0], gf[1]), __fadd_rn(gf[2], gf[3]));
+      const float ec = __fadd_rn(__fadd_rn(gc[0], gc[1]), __fadd_rn(gc[2], gc[3]));
+      const bool take_f = (uf != u) && (ef < __fmul_rn(4.0f, ec));
+      out = take_f ? make_uint4(wf[0], wf[1], wf[2], wf[3]) : make_uint4(wc[0], wc[1], wc[2], wc[3]);
+      u = take_f ? uf : u;
+    } else {
+      mx_scale_values<32>(v, u);
+      out.x = cvt_e2m1x8(v);
+      out.y = cvt_e2m1x8(v + 8);
+      out.z = cvt_e2m1x8(v + 16);
+      out.w = cvt_e2m1x8(v + 24);
+    }
     const int col = 2 * cp + c;
     packed[((bh * D + col) * (size_t)(N / 2) + (size_t)kt * 64 + kb * 16) / 16] = out;
     sfb[col * 4 + kb] = (uint8_t)u;
@@ -282,6 +351,7 @@ int launch_quantize(const void* x, int fmt, int role, int B, int H, int N, int d
   if (fmt == FP4ATTN_FMT_MXFP4) {
     if (mx_rule == FP4ATTN_QSCALE_THR16)      launch_mx<FP4ATTN_QSCALE_THR16>(xs, role, B, H, N, d, packed, scales, st);
     else if (mx_rule == FP4ATTN_QSCALE_FLOOR) launch_mx<FP4ATTN_QSCALE_FLOOR>(xs, role, B, H, N, d, packed, scales, st);
+    else if (mx_rule == FP4ATTN_QSCALE_MSE)   launch_mx<FP4ATTN_QSCALE_MSE>(xs, role, B, H, N, d, packed, scales, st);
     else                                      launch_mx<FP4ATTN_QSCALE_CEIL>(xs, role, B, H, N, d, packed, scales, st);
   } else {
     const int n_partials = (int)(grid < (unsigned)kMaxPartials ? grid : kMaxPartials);
@@ -322,7 +392,8 @@ extern "C" int fp4attn_quantize(const void* x, int fmt, int role, int B, int H, 
 
 extern "C" int fp4attn_quantize_mxfp4_rule(const void* x, int role, int scale_rule, int B, int H, int N, int d,
                                            void* packed, void* scales, fp4attn_stream_t stream) {
-  if (scale_rule != FP4ATTN_QSCALE_CEIL && scale_rule != FP4ATTN_QSCALE_THR16 && scale_rule != FP4ATTN_QSCALE_FLOOR)
+  if (scale_rule != FP4ATTN_QSCALE_CEIL && scale_rule != FP4ATTN_QSCALE_THR16 && scale_rule != FP4ATTN_QSCALE_FLOOR &&
+      scale_rule != FP4ATTN_QSCALE_MSE)
     return FP4ATTN_ERR_INVALID_ARG;
   int rc = validate_quantize(x, FP4ATTN_FMT_MXFP4, role, B, H, N, d, packed, scales, nullptr);
   if (rc != FP4ATTN_OK) return rc;

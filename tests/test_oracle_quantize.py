@@ -155,3 +155,75 @@ def test_mx_amplitude_rules_closed_forms_and_saturation():
             assert np.all(np.abs(xr).reshape(64, 8, 32).max(axis=-1) <= 2.0 ** np.ceil(np.log2(xb.max(axis=-1))))
     assert err["thr16"] < err["ceil"] < err["floor"]
     assert 0.10 < err["thr16"] < 0.12 and 0.17 < err["floor"] < 0.19
+
+
+def test_mx_mse_rule_against_exact_rational_errors():
+    """The MSE rule keeps, per block, whichever of the two amplitudes Eq. "mx-scale" allows reconstructs the
+    block better.  Pins: (1) the chosen (byte, codes) always equal the floor rule's or the ceiling rule's output
+    for that block; (2) the choice agrees with the two reconstruction errors computed in exact rational
+    arithmetic from the dequantized values, except where those are within 1e-5 relative of each other (the rule
+    sums in fp32); (3) hand-made blocks; (4) on Gaussian data its error is below the threshold rule's."""
+    from fractions import Fraction
+    rng = np.random.default_rng(11)
+    x = Qz.bf16_bits_to_f64(I.f32_to_bf16_bits((rng.standard_normal((40, 128)) * rng.choice([1e-3, 1.0, 37.0], (40, 1))).astype(np.float32)))
+    out = {r: Qz.mx_quantize_lastdim(x, r) for r in ("mse", "floor", "ceil")}
+    xr = {r: Qz.mx_dequantize_lastdim(*out[r]) for r in out}
+    picked_floor = 0
+    for r in range(40):
+        for b in range(4):
+            sl = slice(32 * b, 32 * b + 32)
+            is_f = out["mse"][1][r, b] == out["floor"][1][r, b] and np.array_equal(out["mse"][0][r, sl], out["floor"][0][r, sl])
+            is_c = out["mse"][1][r, b] == out["ceil"][1][r, b] and np.array_equal(out["mse"][0][r, sl], out["ceil"][0][r, sl])
+            assert is_f or is_c
+            ef = sum((Fraction(float(p)) - Fraction(float(q))) ** 2 for p, q in zip(xr["floor"][r, sl], x[r, sl]))
+            ec = sum((Fraction(float(p)) - Fraction(float(q))) ** 2 for p, q in zip(xr["ceil"][r, sl], x[r, sl]))
+            if abs(ef - ec) > Fraction(1, 100000) * max(ef, ec):
+                assert is_f == (ef < ec) or (is_f and is_c), (r, b, float(ef), float(ec))
+            picked_floor += bool(is_f and not is_c)
+    assert 20 < picked_floor < 140                                   # both amplitudes are in use
+    # maximum 1.0078125, eight values 0.25.  alpha 1: 6.046875 -> 6 (d^2 = 0.0022), 1.5 exact.  alpha 2:
+    # 0.75 is a tie -> 1.0 (even code), d = 0.25 eight times: the floor is far better
+    blk = np.zeros((1, 32)); blk[0, 0] = 1.0078125; blk[0, 1:9] = 0.25
+    nib, u = Qz.mx_quantize_lastdim(blk, "mse")
+    assert u[0, 0] == 127 and nib[0, 0] == 7 and nib[0, 1] == 3 and nib[0, 9] == 0
+    # maximum 1.5, three values 0.5 (exact on both grids).  alpha 1: 9 saturates at 6, d = 3 -> 9 units;
+    # alpha 2: 4.5 -> 4 (tie to the even code), d = 0.5 -> 4 * 0.25 = 1 in the same units: the ceiling is kept
+    blk = np.zeros((1, 32)); blk[0, 0] = 1.5; blk[0, 1:4] = 0.5
+    nib, u = Qz.mx_quantize_lastdim(blk, "mse")
+    assert u[0, 0] == 128 and nib[0, 0] == 6 and nib[0, 1] == 3
+    # equal errors keep the ceiling: maximum 1.25 alone -> alpha 1: 7.5 -> 6, 2.25; alpha 2: 3.75 -> 4, 4 * 0.0625
+    blk = np.zeros((1, 32)); blk[0, 0] = 1.25
+    assert Qz.mx_quantize_lastdim(blk, "mse")[1][0, 0] == 128
+    blk = np.zeros((1, 32)); blk[0, 0] = 2.0; blk[0, 5] = 0.3125         # power of two: only one candidate
+    assert Qz.mx_quantize_lastdim(blk, "mse")[1][0, 0] == Qz.mx_quantize_lastdim(blk, "floor")[1][0, 0] == 128
+    xg = Qz.bf16_bits_to_f64(I.f32_to_bf16_bits(np.random.default_rng(2).standard_normal((64, 256)).astype(np.float32)))
+    err = {}
+    for rule in ("mse", "thr16"):
+        nib, u = Qz.mx_quantize_lastdim(xg, rule)
+        err[rule] = np.linalg.norm(Qz.mx_dequantize_lastdim(nib, u) - xg) / np.linalg.norm(xg)
+    assert err["mse"] < err["thr16"] and 0.10 < err["mse"] < 0.12
+
+
+def test_mx_mse_rule_error_sum_is_order_pinned():
+    """mx_block_error32 against its definition written out with Python floats rounded through float32 one
+    operation at a time (left to right within groups of eight, groups as (g0 + g1) + (g2 + g3))."""
+    import struct
+    f32 = lambda v: struct.unpack("f", struct.pack("f", v))[0]
+    rng = np.random.default_rng(3)
+    xb = Qz.bf16_bits_to_f64(I.f32_to_bf16_bits(rng.standard_normal((6, 32)).astype(np.float32)))
+    u = np.full((6,), 128, dtype=np.uint8)
+    err, codes = Qz.mx_block_error32(xb, u)
+    grid = [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+    for r in range(6):
+        g = []
+        for j in range(4):
+            acc = None
+            for i in range(8):
+                t = 6.0 * float(xb[r, 8 * j + i]) / 2.0
+                q = min(grid, key=lambda c: (abs(abs(t) - c), grid.index(c) % 2))     # nearest, ties to the even code
+                assert grid[int(codes[r, 8 * j + i]) & 7] == q
+                d = abs(t) - q
+                s = f32(d * d)
+                acc = s if acc is None else f32(acc + s)
+            g.append(acc)
+        assert float(err[r]) == f32(f32(g[0] + g[1]) + f32(g[2] + g[3]))

@@ -80,7 +80,7 @@ def test_full_size_quantizer_sampled(tmp_path):
     _check_operand(got, Qz.quantize_v(v), Bd.ROLE_V)
 
 
-RULES = [("ceil", 0), ("thr16", 1), ("floor", 2)]
+RULES = [("ceil", 0), ("thr16", 1), ("floor", 2), ("mse", 3)]
 
 
 @pytest.mark.parametrize("rule,code", RULES)
