@@ -223,6 +223,11 @@ size_t fp4attn_attention_host_workspace_bytes(int qk_fmt, int B, int H, int N, i
  * device and kept until the process exits; no device memory is allocated) that fork from `stream` and
  * join back into it through events.  NVFP4 (tensor-wide amax first) and small problems run on `stream`
  * alone.  Results are bit-identical either way.
+ *
+ * Threads: every entry point may be called from several host threads (each on its own stream and
+ * buffers); the pipelined host path serialises its enqueue phase on an internal lock because the
+ * copy streams and events are shared per device.  On an error return the call still joins the
+ * internal streams into `stream`, so whatever was enqueued stays ordered before later work there.
  */
 int fp4attn_attention_host(const void* q_host, const void* k_host, const void* v_host,
                            int qk_fmt, float softmax_scale, int B, int H, int N, int d,

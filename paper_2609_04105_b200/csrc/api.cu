@@ -5,16 +5,17 @@ namespace fp4attn {
 
 int check_device_sm100() {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return FP4ATTN_ERR_CUDA;
-  static int cached_dev = -1, cached_rc = FP4ATTN_OK;
-  if (dev == cached_dev) return cached_rc;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FP4ATTN_ERR_CUDA;
+  static std::atomic<int> cached[kMaxDevices];                 // 0 unknown, else status + 1
+  const int c = cached[dev].load(std::memory_order_acquire);
+  if (c) return c - 1;
   int major = 0, minor = 0;
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess)
     return FP4ATTN_ERR_CUDA;
-  cached_rc = (major == 10 && minor == 0) ? FP4ATTN_OK : FP4ATTN_ERR_UNSUPPORTED_ARCH;
-  cached_dev = dev;
-  return cached_rc;
+  const int rc = (major == 10 && minor == 0) ? FP4ATTN_OK : FP4ATTN_ERR_UNSUPPORTED_ARCH;
+  cached[dev].store(rc + 1, std::memory_order_release);
+  return rc;
 }
 
 }  // namespace fp4attn
@@ -74,41 +75,46 @@ struct HostPipe {
   cudaEvent_t start = nullptr, end = nullptr, in[kMaxGroups] = {}, done[kMaxGroups] = {};
   bool ready = false;
 };
+void destroy(HostPipe& hp) {
+  if (hp.h2d) cudaStreamDestroy(hp.h2d);
+  if (hp.d2h) cudaStreamDestroy(hp.d2h);
+  if (hp.start) cudaEventDestroy(hp.start);
+  if (hp.end) cudaEventDestroy(hp.end);
+  for (int c = 0; c < kMaxGroups; ++c) {
+    if (hp.in[c]) cudaEventDestroy(hp.in[c]);
+    if (hp.done[c]) cudaEventDestroy(hp.done[c]);
+  }
+  hp = HostPipe();
+}
+std::mutex g_pipe_mutex;                                        // one pipelined enqueue at a time: the events are shared
+// caller holds g_pipe_mutex
 HostPipe* host_pipe() {
-  constexpr int kMaxDevices = 64;
+  constexpr int kMaxDevices = fp4attn::kMaxDevices;
   static HostPipe pipes[kMaxDevices];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
   HostPipe& hp = pipes[dev];
   if (!hp.ready) {
-    if (cudaStreamCreateWithFlags(&hp.h2d, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    if (cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&hp.end, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    for (int c = 0; c < kMaxGroups; ++c)
-      if (cudaEventCreateWithFlags(&hp.in[c], cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&hp.done[c], cudaEventDisableTiming) != cudaSuccess)
-        return nullptr;
+    bool ok = cudaStreamCreateWithFlags(&hp.h2d, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.end, cudaEventDisableTiming) == cudaSuccess;
+    for (int c = 0; ok && c < kMaxGroups; ++c)
+      ok = cudaEventCreateWithFlags(&hp.in[c], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.done[c], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { destroy(hp); return nullptr; }                   // nothing half-made is kept
     hp.ready = true;
   }
   return &hp;
 }
-int attention_host_pipelined(const void* q_host, const void* k_host, const void* v_host, float softmax_scale, int B, int H,
-                             int N, int d, void* O_host, float* LSE_host, char* ws, const HostPlan& p,
-                             size_t workspace_bytes, cudaStream_t st) {
-  const int BH = B * H;
-  const int groups = BH < 8 ? 1 : (BH < 2 * kMaxGroups ? 4 : 8);   // (16 groups measured slower than 8: more, smaller copies)
-  if (groups == 1) return kNoPipeline;
-  HostPipe* hp = host_pipe();
-  if (!hp) return kNoPipeline;
+int enqueue_groups(HostPipe* hp, int groups, const void* q_host, const void* k_host, const void* v_host, float softmax_scale,
+                   int BH, int N, int d, void* O_host, float* LSE_host, char* ws, const HostPlan& p, size_t workspace_bytes,
+                   cudaStream_t st) {
   const size_t head_elems = (size_t)N * d;
   const size_t sfq_head = fp4attn_scale_bytes(FP4ATTN_FMT_MXFP4, FP4ATTN_ROLE_Q, 1, 1, N, d);
   const size_t sfv_head = fp4attn_scale_bytes(FP4ATTN_FMT_MXFP4, FP4ATTN_ROLE_V, 1, 1, N, d);
   const char* src[3] = {(const char*)q_host, (const char*)k_host, (const char*)v_host};
 #define FP4ATTN_CUDA_OK(call) do { if ((call) != cudaSuccess) return FP4ATTN_ERR_CUDA; } while (0)
-  FP4ATTN_CUDA_OK(cudaEventRecord(hp->start, st));              // fork: the copies start after the stream's earlier work
-  FP4ATTN_CUDA_OK(cudaStreamWaitEvent(hp->h2d, hp->start, 0));
-  FP4ATTN_CUDA_OK(cudaStreamWaitEvent(hp->d2h, hp->start, 0));
   for (int c = 0; c < groups; ++c) {
     const int h0 = (int)((long long)BH * c / groups), nh = (int)((long long)BH * (c + 1) / groups) - h0;
     for (int i = 0; i < 3; ++i)
@@ -143,10 +149,28 @@ int attention_host_pipelined(const void* q_host, const void* k_host, const void*
       FP4ATTN_CUDA_OK(cudaMemcpyAsync(LSE_host + (size_t)h0 * N, (float*)(ws + p.LSE) + (size_t)h0 * N, (size_t)nh * N * 4,
                                       cudaMemcpyDeviceToHost, hp->d2h));
   }
-  FP4ATTN_CUDA_OK(cudaEventRecord(hp->end, hp->d2h));            // join
-  FP4ATTN_CUDA_OK(cudaStreamWaitEvent(st, hp->end, 0));
 #undef FP4ATTN_CUDA_OK
   return FP4ATTN_OK;
+}
+int attention_host_pipelined(const void* q_host, const void* k_host, const void* v_host, float softmax_scale, int B, int H,
+                             int N, int d, void* O_host, float* LSE_host, char* ws, const HostPlan& p,
+                             size_t workspace_bytes, cudaStream_t st) {
+  const int BH = B * H;
+  const int groups = BH < 8 ? 1 : (BH < 2 * kMaxGroups ? 4 : 8);   // (16 groups measured slower than 8: more, smaller copies)
+  if (groups == 1) return kNoPipeline;
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  HostPipe* hp = host_pipe();
+  if (!hp) return kNoPipeline;
+  if (cudaEventRecord(hp->start, st) != cudaSuccess ||         // fork: the copies start after the stream's earlier work
+      cudaStreamWaitEvent(hp->h2d, hp->start, 0) != cudaSuccess || cudaStreamWaitEvent(hp->d2h, hp->start, 0) != cudaSuccess)
+    return FP4ATTN_ERR_CUDA;
+  const int rc = enqueue_groups(hp, groups, q_host, k_host, v_host, softmax_scale, BH, N, d, O_host, LSE_host, ws, p,
+                                workspace_bytes, st);
+  // join on every exit, also a failed one: whatever reached the internal streams stays ordered before the
+  // caller's later work on its stream (which may reuse the workspace and the host buffers)
+  bool joined = cudaEventRecord(hp->end, hp->h2d) == cudaSuccess && cudaStreamWaitEvent(st, hp->end, 0) == cudaSuccess;
+  joined = joined && cudaEventRecord(hp->end, hp->d2h) == cudaSuccess && cudaStreamWaitEvent(st, hp->end, 0) == cudaSuccess;
+  return rc != FP4ATTN_OK ? rc : (joined ? FP4ATTN_OK : FP4ATTN_ERR_CUDA);
 }
 }  // namespace
 

@@ -715,13 +715,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
+  static std::atomic<EncodeTiledFn> cached{nullptr};
+  EncodeTiledFn fn = cached.load(std::memory_order_acquire);
   if (!fn) {
     void* ptr = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
       fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    cached.store(fn, std::memory_order_release);
   }
   return fn;
 }
@@ -745,11 +747,16 @@ template <int D, bool NV, int PMAP, bool CAUSAL, bool THR16>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
   const int Hkv = prm.Hkv;
   using C = Cfg<D, NV>;
-  static bool attr_set = false;
-  if (!attr_set) {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return FP4ATTN_ERR_CUDA;
+  // the shared-memory opt-in is a per-device property of the function: set it once on every device used
+  static std::atomic<bool> attr_set[kMaxDevices];
+  if (dev < 0 || dev >= kMaxDevices) return FP4ATTN_ERR_CUDA;
+  if (!attr_set[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
       return FP4ATTN_ERR_CUDA;
-    attr_set = true;
+    attr_set[dev].store(true, std::memory_order_release);
   }
   CUtensorMap tmQ, tmK, tmV, tmO;
   const uint64_t rows = (uint64_t)B * H * N, kv_rows = (uint64_t)B * Hkv * N;
@@ -757,9 +764,6 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
       !make_map(&tmK, ops->k, C::ROW_BYTES, kv_rows, C::ROW_BYTES, BS) ||
       !make_map(&tmV, ops->v, (uint64_t)N / 2, (uint64_t)B * Hkv * D, BS / 2, D) ||
       !make_map(&tmO, prm.O, (uint64_t)D * 2, rows, 128, 32))
-    return FP4ATTN_ERR_CUDA;
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return FP4ATTN_ERR_CUDA;
   const unsigned grid = (unsigned)(prm.n_items < sms ? prm.n_items : sms);     // persistent: one CTA per SM
   attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, tmO, prm);

@@ -4,6 +4,9 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "../../include/fp4attn.h"
 
 namespace fp4attn {
@@ -67,6 +70,8 @@ __device__ __forceinline__ uint32_t mx_scale_byte(float a) {
 __device__ __forceinline__ float mx_inv_amplitude(uint32_t u) {
   return __uint_as_float(u == 254u ? 0x00400000u : ((254u - u) << 23));
 }
+
+constexpr int kMaxDevices = 64;      // per-device host-side caches are arrays of this length
 
 int check_device_sm100();            // FP4ATTN_OK or FP4ATTN_ERR_UNSUPPORTED_ARCH / _CUDA
 

@@ -417,7 +417,6 @@ extern "C" int fp4attn_quantize_nvfp4_noalloc(const void* x, int role, int B, in
   if (rc != FP4ATTN_OK) return rc;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return FP4ATTN_ERR_CUDA;
-  constexpr int kMaxDevices = 64;
   static float* scratch_addr[kMaxDevices] = {};          // per-device address of g_noalloc_partials
   if (dev < 0 || dev >= kMaxDevices) return FP4ATTN_ERR_INVALID_ARG;
   if (!scratch_addr[dev]) {

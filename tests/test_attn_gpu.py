@@ -153,6 +153,46 @@ def test_host_buffer_entry_point_matches_device_path(kw):
         assert np.array_equal(lse.numpy().astype(np.float64), Lg)
 
 
+def test_host_buffer_entry_point_from_two_threads():
+    """Two host threads, each with its own stream, workspace and host buffers, enqueue the pipelined host
+    path at the same time (the library's internal copy streams and events are shared and guarded by a
+    lock): each must get exactly what the device path returns for its inputs."""
+    import threading
+    from paper_2609_04105_b200 import binding as Bd
+    jobs = []
+    for t in range(2):
+        w = I.shrink(I.WORKLOADS["cfg1"], H=5 + 4 * t, N=384)                 # 10 and 18 heads: 4 groups each
+        q, k, v = I.make_qkv(w)                                                # shapes differ, so do the tensors
+        Og, Lg = run_gpu(w, q, k, v)
+        host = [torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory() for a in (q, k, v)]
+        ws = torch.empty(Bd.fp4attn_attention_host_workspace_bytes(w.qk_fmt, w.B, w.H, w.N, w.d), dtype=torch.uint8, device="cuda")
+        out = torch.zeros((w.B, w.H, w.N, w.d), dtype=torch.bfloat16).pin_memory()
+        lse = torch.zeros((w.B, w.H, w.N), dtype=torch.float32).pin_memory()
+        jobs.append((w, host, ws, out, lse, Og, Lg, torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    errors = []
+
+    def work(job):
+        w, host, ws, out, lse, _, _, stream = job
+        try:
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    Bd.fp4attn_attention_host(host[0], host[1], host[2], w.qk_fmt, out, lse, ws)
+            stream.synchronize()
+        except Exception as e:                                                 # surfaces in the main thread below
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for w, host, ws, out, lse, Og, Lg, _ in jobs:
+        assert np.array_equal(out.float().numpy().astype(np.float64), Og)
+        assert np.array_equal(lse.numpy().astype(np.float64), Lg)
+
+
 def test_invalid_arguments_are_rejected_before_launch():
     from paper_2609_04105_b200 import binding as Bd
     x = torch.zeros((1, 1, 100, 128), dtype=torch.bfloat16, device="cuda")
