@@ -90,6 +90,11 @@ size_t fp4attn_quantize_workspace_bytes(int fmt, int role, int B, int H, int N, 
  * x_bf16 [B,H,N,d]; packed_out / scales_out sized by the queries above; tensor_scale_out is
  * required for NVFP4 and ignored (may be NULL) for MXFP4; workspace may be NULL when the size
  * query returns 0.  Outputs are fully overwritten (padding included).
+ *
+ * Inputs are expected to be finite.  A non-finite value never leads to an out-of-range access or
+ * an error return (no address depends on the data); under MXFP4 it only affects its own block
+ * (amplitude 2^127, its own code saturated at 6), under NVFP4 it reaches every block through G,
+ * and the attention result for such operands is unspecified.
  */
 int fp4attn_quantize(const void* x_bf16, int fmt, int role, int B, int H, int N, int d,
                      void* packed_out, void* scales_out, float* tensor_scale_out,

@@ -127,3 +127,28 @@ def test_mx_amplitude_rule_rejects_unknown_rule():
     x = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(Bd.Fp4AttnError):
         Bd.fp4attn_quantize_mxfp4_rule(x, Bd.ROLE_Q, 7)
+
+
+def test_mx_non_finite_values_stay_in_their_block():
+    """An infinity and a NaN, each in a block of its own: the call succeeds, every other block carries exactly
+    the oracle's bytes, and the two blocks get the largest amplitude byte with a saturated code."""
+    from paper_2609_04105_b200 import binding as Bd
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((1, 2, 128, 128)).astype(np.float32)
+    clean = I.f32_to_bf16_bits(x)
+    bits = clean.copy()
+    bits[0, 0, 5, 40] = 0x7F80                                  # +inf: row 5, block 1
+    bits[0, 1, 77, 100] = 0xFFC1                                # a NaN: row 77, block 3
+    got = Bd.fp4attn_quantize(_dev(bits), Bd.FMT_MXFP4, Bd.ROLE_Q)
+    torch.cuda.synchronize()
+    want = Qz.quantize_qk(clean, "mx")
+    pk_g = Qz.strip_negative_zero(got.packed.cpu().numpy()).reshape(1, 2, 128, 4, 16)     # 16 bytes per 32-block
+    pk_w = Qz.strip_negative_zero(Qz.pack_nibbles(want["nib"]).reshape(-1)).reshape(1, 2, 128, 4, 16)
+    touched = np.zeros((1, 2, 128, 4), dtype=bool)
+    touched[0, 0, 5, 1] = touched[0, 1, 77, 3] = True
+    assert ((pk_g == pk_w).all(axis=-1) | touched).all()
+    sf_clean = Bd.fp4attn_quantize(_dev(clean), Bd.FMT_MXFP4, Bd.ROLE_Q).scales.cpu().numpy()
+    sf_g = got.scales.cpu().numpy()
+    assert np.array_equal(sf_clean, Qz.swizzle_scales(want["sf"]).reshape(-1))
+    assert (sf_g != sf_clean).sum() == 2 and set(sf_g[sf_g != sf_clean]) == {254}
+    assert (pk_g[0, 0, 5, 1, (40 - 32) // 2] & 0xF) == 7        # +inf (even element: low nibble) saturates at +6
