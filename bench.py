@@ -340,14 +340,16 @@ def run_cuda(args, w):
     other_maps = {}
     if world == 1:
         qd0, kd0, vd0 = state["ops"]
+        O_alt = torch.empty_like(O)                                 # O keeps the timed map's result for the parity sample
         for name, kw in (("ideal", dict(p_map=Bd.PMAP_IDEAL)), ("hybrid8", dict(p_map=Bd.PMAP_HYBRID, exact_pairs=0x5555)),
                          ("affine", dict(p_map=Bd.PMAP_AFFINE))):
             if name == args.p_map:
                 continue
             for _ in range(3):
-                Bd.fp4attn_fwd(qd0, kd0, vd0, out=O, status=status, p_scale_rule=pscale, **kw)
-            ms_map = time_flushed(lambda: Bd.fp4attn_fwd(qd0, kd0, vd0, out=O, status=status, p_scale_rule=pscale, **kw), 10, flush, E)
+                Bd.fp4attn_fwd(qd0, kd0, vd0, out=O_alt, status=status, p_scale_rule=pscale, **kw)
+            ms_map = time_flushed(lambda: Bd.fp4attn_fwd(qd0, kd0, vd0, out=O_alt, status=status, p_scale_rule=pscale, **kw), 10, flush, E)
             other_maps[name] = {"attn_tflops": w.flops / (ms_map * 1e-3) / 1e12}
+        del O_alt
 
     # ---- measured dense FP4 issue rate of this device (context for the roofline)
     cyc = torch.zeros(1, dtype=torch.int64, device=dev)
@@ -455,7 +457,9 @@ def run_cuda(args, w):
         rel = max(float(np.linalg.norm(Og[i] - Oo[i]) / np.linalg.norm(Oo[i])) for i in range(len(heads)))
         sample = f"{len(heads)} (batch, head) pairs x {n_rows} seeded query rows of {w.name}, {dt:.1f} s"
         out["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "sample": sample}
-        out["parity_on_sample"] = {"rel_fro_max": rel, "max_abs": float(np.abs(Og - Oo).max())}
+        max_abs = float(np.abs(Og - Oo).max())
+        out["parity_on_sample"] = {"rel_fro_max": rel, "max_abs": max_abs, "tolerance": {"rel_fro": 5e-3, "max_abs": 2e-2},
+                                   "ok": bool(rel <= 5e-3 and max_abs <= 2e-2)}
         out["accuracy_vs_fp64"] = accuracy_vs_fp64(w, q, k, v, heads, rows, Og, Oo)
     print(json.dumps(out))
     if world > 1:
