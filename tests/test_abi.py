@@ -65,3 +65,38 @@ def test_host_detectable_errors_return_codes_without_a_gpu(lib):
     assert lib.fp4attn_quantize(*args(0x1004, 0, 0, 128, 128)) == 4       # misaligned
     assert lib.fp4attn_quantize(*args(0x1000, 1, 2, 128, 128, vp(0x3000))) == 1   # NVFP4 V
     assert lib.fp4attn_quantize(*args(0x1000, 1, 0, 128, 128, vp(0x3000))) == 5   # NVFP4 without workspace
+
+
+def test_header_is_plain_c_and_the_struct_layout_matches_the_binding(lib, tmp_path):
+    """The boundary is usable from C: the header compiles as strict C99, a C program links against the
+    library and calls it, and the operand struct it sees has the layout the Python binding marshals."""
+    import shutil
+    import subprocess
+    from paper_2609_04105_b200 import binding, build
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    fields = [n for n, _ in binding._Operands._fields_]
+    src = tmp_path / "abi.c"
+    lines = ['#include <stddef.h>', '#include <stdio.h>', '#include <string.h>', '#include "fp4attn.h"', 'int main(void) {',
+             '  fp4attn_operands ops;', '  memset(&ops, 0, sizeof ops);',
+             '  printf("sizeof %zu\\n", sizeof(fp4attn_operands));']
+    lines += [f'  printf("{n} %zu\\n", offsetof(fp4attn_operands, {n}));' for n in fields]
+    lines += ['  printf("version %d\\n", fp4attn_version());',
+              '  printf("packed %zu\\n", fp4attn_packed_bytes(4, 16, 4096, 128));',
+              '  printf("null_ops %d\\n", fp4attn_fwd(NULL, 1, 1, 128, 128, NULL, NULL, NULL, NULL));',
+              '  printf("status %s\\n", fp4attn_status_string(FP4ATTN_ERR_INVALID_ARG));',
+              '  return 0;', '}']
+    src.write_text("\n".join(lines) + "\n")
+    libpath = build.build()
+    exe = tmp_path / "abi"
+    subprocess.run([gcc, "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src),
+                    "-o", str(exe), libpath, f"-Wl,-rpath,{os.path.dirname(libpath)}"], check=True)
+    out = dict(l.split(" ", 1) for l in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines())
+    assert int(out["sizeof"]) == ctypes.sizeof(binding._Operands)
+    for n in fields:
+        assert int(out[n]) == getattr(binding._Operands, n).offset, n
+    assert int(out["version"]) == lib.fp4attn_version()
+    assert int(out["packed"]) == 4 * 16 * 4096 * 128 // 2
+    assert int(out["null_ops"]) == binding.ERR_INVALID_ARG if hasattr(binding, "ERR_INVALID_ARG") else int(out["null_ops"]) != 0
+    assert out["status"] == "invalid argument"
