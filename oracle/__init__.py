@@ -12,7 +12,9 @@ Pinned by tests/test_oracle_*.py (run with -m "not gpu"):
                                                   amplitude rules -> exact rational arithmetic on every
                                                   bf16 significand, hand-computed blocks, saturation;
                                                   MSE rule -> block errors in exact rational arithmetic,
-                                                  its fp32 summation order operation by operation
+                                                  its fp32 summation order operation by operation;
+                                                  per-(batch, head) NVFP4 factors -> power-of-two scaling
+                                                  of a head moves only its factor, error bound per head
   attention.py  tiled Direct-P forward          -> tile-size / tile-order invariance, V == 1,
                                                   equal keys, dominant key, brute-force exact
                                                   attention on losslessly representable inputs;
@@ -23,5 +25,7 @@ Pinned by tests/test_oracle_*.py (run with -m "not gpu"):
                                                   and grouped-query attention -> first row, whole-tile
                                                   prefixes, brute force, repeated K/V heads; mixed map
                                                   -> position by position against the two pinned maps,
-                                                  error monotone in the share of exact pairs
+                                                  error monotone in the share of exact pairs; per-head
+                                                  factors -> bit-identical output under 2^a / 2^-a scaling
+                                                  of a query head and its key head
 """

@@ -68,18 +68,24 @@ def block_exponent(ymax32: np.ndarray, p_scale: str = "ceil") -> np.ndarray:
     return np.floor((np.asarray(ymax32, np.float32) + LOG2_1P6_32).astype(np.float32).astype(np.float64))
 
 
-def score_constant(qd: dict, kd: dict, d: int, softmax_scale=None) -> np.float32:
+def score_constant(qd: dict, kd: dict, d: int, softmax_scale=None, unit=None) -> np.float32:
     """c32: multiplies the tensor-core-facing score S_hw to give y = z*log2(e).
 
     MXFP4 x MXFP4: S_hw carries 6*6 (amplitude convention) -> c = fl32(fl32(log2e*scale)/36).
     NVFP4 x NVFP4: S_hw carries G_q*G_k              -> c = fl32(fl32(log2e*scale)/fl32(G_q*G_k)).
+    With per-(batch, head) factors (G arrays [B, H]) `unit` = (b, h, hk) names the query unit and the
+    K/V head it reads, and the constant is that pair's.
     """
     scale = np.float32(1.0 / math.sqrt(d)) if softmax_scale is None else np.float32(softmax_scale)
     base = np.float32(LOG2E_32 * scale)
     if qd["fmt"] == "mx" and kd["fmt"] == "mx":
         return np.float32(base / np.float32(36.0))
     assert qd["fmt"] == "nv" and kd["fmt"] == "nv"
-    return np.float32(base / np.float32(np.float32(qd["G"]) * np.float32(kd["G"])))
+    Gq, Gk = qd["G"], kd["G"]
+    if np.ndim(Gq) or np.ndim(Gk):
+        b, h, hk = unit
+        Gq, Gk = np.asarray(Gq)[b, h], np.asarray(Gk)[b, hk]
+    return np.float32(base / np.float32(np.float32(Gq) * np.float32(Gk)))
 
 
 def scores_fp32(qd: dict, kd: dict, b: int, h: int, rows=None, hk=None) -> np.ndarray:
@@ -175,11 +181,11 @@ def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int
     B, H, N, d = qd["nib"].shape
     assert H % kv_group == 0 and kd["nib"].shape[1] == H // kv_group and vd["nib"].shape[1] == H // kv_group
     heads = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
-    c32 = score_constant(qd, kd, d, softmax_scale)
     ridx = np.arange(N) if rows is None else np.asarray(rows)
     Os, Ls = [], []
     for (b, h) in heads:
         hk = h // kv_group                                       # K/V head shared by the group
+        c32 = score_constant(qd, kd, d, softmax_scale, (b, h, hk))
         s32 = scores_fp32(qd, kd, b, h, rows, hk)
         Vhat = dequantize({**vd, "nib": vd["nib"][b, hk][None, None], "sf": vd["sf"][b, hk][None, None]})[0, 0].T
         O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order, p_map, affine, p_scale,

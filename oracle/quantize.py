@@ -151,17 +151,32 @@ def nv_dequantize_lastdim(nib: np.ndarray, sbyte: np.ndarray, G=None, hw: bool =
     q = e2m1_decode(nib).reshape(nib.shape[:-1] + (L // NV_BLOCK, NV_BLOCK))
     v = q * e4m3_decode(sbyte)[..., None]
     if not hw:
-        v = v / np.float64(G)
+        G = np.asarray(G, dtype=np.float64)                      # one factor, or one per (batch, head) [B, H]
+        v = v / G.reshape(G.shape + (1,) * (v.ndim - G.ndim))
     return v.reshape(nib.shape)
 
 
 # --------------------------------------------------------------------------- roles
-def quantize_qk(bits: np.ndarray, fmt: str, rule: str = "ceil"):
-    """Q or K, bf16 bit patterns [B,H,N,d] -> dict(nib [B,H,N,d], sf [B,H,N,d/blk], G)."""
+def quantize_qk(bits: np.ndarray, fmt: str, rule: str = "ceil", per_head: bool = False):
+    """Q or K, bf16 bit patterns [B,H,N,d] -> dict(nib [B,H,N,d], sf [B,H,N,d/blk], G).
+
+    NVFP4: G is one encode factor for the whole tensor, or with per_head one per (batch, head) unit,
+    float32 [B, H], each taken from that unit's own maximum (Section "Pass the forward quantization into
+    backward" saves per-head Q-K global factors): every unit is then quantized as if it were a tensor."""
     x = bf16_bits_to_f64(bits)
     if fmt == "mx":
         nib, sf = mx_quantize_lastdim(x, rule)
         return {"nib": nib, "sf": sf, "G": None, "fmt": "mx"}
+    if per_head:
+        B, H = x.shape[:2]
+        G = np.empty((B, H), dtype=np.float32)
+        nib = np.empty(x.shape, dtype=np.uint8)
+        sf = np.empty(x.shape[:-1] + (x.shape[-1] // NV_BLOCK,), dtype=np.uint8)
+        for b in range(B):
+            for h in range(H):
+                G[b, h] = nv_tensor_scale(x[b, h])
+                nib[b, h], sf[b, h] = nv_quantize_lastdim(x[b, h], G[b, h])
+        return {"nib": nib, "sf": sf, "G": G, "fmt": "nv"}
     G = nv_tensor_scale(x)
     nib, sf = nv_quantize_lastdim(x, G)
     return {"nib": nib, "sf": sf, "G": G, "fmt": "nv"}

@@ -392,3 +392,36 @@ def test_hybrid_map_error_falls_with_the_share_of_exact_pairs():
         O, _ = A.direct_p_forward(qd, kd, vd, p_map="hybrid", exact_pairs=mask)
         errs.append(np.linalg.norm(O - Oe) / np.linalg.norm(Oe))
     assert all(a > b for a, b in zip(errs, errs[1:])), errs
+
+
+def test_per_head_nvfp4_factors_make_attention_invariant_to_head_scaling():
+    """With one encode factor per (batch, head) unit, multiplying a query head by 2^a and the key head it
+    reads by 2^-a changes neither a code, nor a scale byte, nor the product G_q G_k: output and LSE are
+    identical bit for bit (with tensor-wide factors they are not).  And every head stays in the accuracy band
+    of the method against exact attention on the bf16 inputs when head magnitudes differ by 2^10."""
+    w = I.shrink(I.WORKLOADS["cfg3"], B=1, H=2, N=256)
+    q, k, v = I.make_qkv(w)
+    xq, xk = Qz.bf16_bits_to_f64(q), Qz.bf16_bits_to_f64(k)
+    vd = Qz.quantize_v(v)
+    qd, kd = Qz.quantize_qk(q, "nv", per_head=True), Qz.quantize_qk(k, "nv", per_head=True)
+    O, L = A.direct_p_forward(qd, kd, vd)
+    xq2, xk2 = xq.copy(), xk.copy()
+    xq2[0, 1] *= 2.0 ** 4
+    xk2[0, 1] *= 2.0 ** -4
+    q2, k2 = I.f32_to_bf16_bits(xq2.astype(np.float32)), I.f32_to_bf16_bits(xk2.astype(np.float32))
+    qd2, kd2 = Qz.quantize_qk(q2, "nv", per_head=True), Qz.quantize_qk(k2, "nv", per_head=True)
+    O2, L2 = A.direct_p_forward(qd2, kd2, vd)
+    assert np.array_equal(O2, O) and np.array_equal(L2, L)
+    Ot, _ = A.direct_p_forward(Qz.quantize_qk(q2, "nv"), Qz.quantize_qk(k2, "nv"), vd)
+    assert not np.array_equal(Ot, O)
+    # head 1 of Q and K 2^-10 times smaller, softmax_scale unchanged: its logits shrink, the method still tracks
+    xq3, xk3 = xq.copy(), xk.copy()
+    xq3[0, 1] *= 2.0 ** -5
+    xk3[0, 1] *= 2.0 ** -5
+    q3, k3 = I.f32_to_bf16_bits(xq3.astype(np.float32)), I.f32_to_bf16_bits(xk3.astype(np.float32))
+    O3, _ = A.direct_p_forward(Qz.quantize_qk(q3, "nv", per_head=True), Qz.quantize_qk(k3, "nv", per_head=True), vd)
+    V = Qz.bf16_bits_to_f64(v)
+    for h in range(2):
+        Oe, _ = A.exact_attention(Qz.bf16_bits_to_f64(q3)[0, h], Qz.bf16_bits_to_f64(k3)[0, h], V[0, h])
+        cos = float((O3[h] * Oe).sum() / np.linalg.norm(O3[h]) / np.linalg.norm(Oe))
+        assert cos > 0.95, (h, cos)

@@ -227,3 +227,38 @@ def test_mx_mse_rule_error_sum_is_order_pinned():
                 acc = s if acc is None else f32(acc + s)
             g.append(acc)
         assert float(err[r]) == f32(f32(g[0] + g[1]) + f32(g[2] + g[3]))
+
+
+def test_nv_per_head_factors_power_of_two_invariance_and_error():
+    """Per-(batch, head) encode factors (Section "Pass the forward quantization into backward": per-head
+    Q-K global factors).  (1) Scaling a head by 2^k leaves its codes and scale bytes untouched and moves only
+    its factor, by exactly 2^-k; the other heads do not change at all.  (2) The tensor maximum's block of every
+    head gets the largest scale byte.  (3) With head magnitudes 1 : 2^-20 one tensor-wide factor flushes
+    the small head's blocks to zero scale, per-head factors keep every head inside the NVFP4 error bound."""
+    w = I.shrink(I.WORKLOADS["cfg3"], B=2, H=3, N=128)
+    q, _, _ = I.make_qkv(w)
+    base = Qz.quantize_qk(q, "nv", per_head=True)
+    assert base["G"].shape == (2, 3) and base["G"].dtype == np.float32
+    x = Qz.bf16_bits_to_f64(q)
+    for b in range(2):
+        for h in range(3):
+            assert base["G"][b, h] == np.float32(2688.0) / np.float32(np.abs(x[b, h]).max())
+            assert base["sf"][b, h].max() == 0x7E
+    scaled = x.copy()
+    scaled[1, 2] *= 2.0 ** 5
+    sd = Qz.quantize_qk(I.f32_to_bf16_bits(scaled.astype(np.float32)), "nv", per_head=True)
+    assert np.array_equal(sd["nib"], base["nib"]) and np.array_equal(sd["sf"], base["sf"])
+    want_G = base["G"].copy()
+    want_G[1, 2] /= np.float32(32.0)
+    assert np.array_equal(sd["G"], want_G)
+    assert np.array_equal(Qz.dequantize(sd)[1, 2], Qz.dequantize(base)[1, 2] * 32.0)
+    small = x.copy()
+    small[0, 1] *= 2.0 ** -20
+    bits = I.f32_to_bf16_bits(small.astype(np.float32))
+    xs = Qz.bf16_bits_to_f64(bits)
+    one, per = Qz.quantize_qk(bits, "nv"), Qz.quantize_qk(bits, "nv", per_head=True)
+    rel = lambda qd, b, h: np.linalg.norm(Qz.dequantize(qd)[b, h] - xs[b, h]) / np.linalg.norm(xs[b, h])
+    assert rel(one, 0, 1) > 0.9 and not one["sf"][0, 1].any()          # a_B G / 6 < 2^-10: every scale byte is zero
+    for b in range(2):
+        for h in range(3):
+            assert rel(per, b, h) < 0.11
