@@ -153,6 +153,21 @@ int fp4attn_quantize_nvfp4_noalloc(const void* x_bf16, int role, int B, int H, i
                                    void* packed_out, void* scales_out, float* tensor_scale_out,
                                    fp4attn_stream_t stream);
 
+/*
+ * NVFP4 quantizer (Q, K) with one encode factor per (batch, head) unit instead of one per tensor (Section
+ * "Pass the forward quantization into backward": the forward saves per-head Q-K global factors): unit
+ * (b, h) is quantized exactly as fp4attn_quantize would quantize it alone, with
+ * G[b*H + h] = fl32(2688 / max|x[b, h]|) (1 for an all-zero unit).  tensor_scale_out receives B*H floats.
+ * Pass the operands to fp4attn_fwd with g_per_head = 1.  Units no longer share a scale, so a head with
+ * small magnitudes keeps its precision and (batch, head) units stay independent problems.
+ * workspace: device scratch of fp4attn_quantize_nvfp4_per_head_workspace_bytes() bytes, 16-byte aligned.
+ * Other arguments, layouts and status codes as for fp4attn_quantize.
+ */
+size_t fp4attn_quantize_nvfp4_per_head_workspace_bytes(int B, int H, int N, int d);
+int fp4attn_quantize_nvfp4_per_head(const void* x_bf16, int role, int B, int H, int N, int d,
+                                    void* packed_out, void* scales_out, float* tensor_scale_out,
+                                    void* workspace, size_t workspace_bytes, fp4attn_stream_t stream);
+
 /* how the integer exponent E_B of a 32-key probability block follows from its maximum y (Eq. "mx-scale"
  * allows either neighbouring power of two as the amplitude) */
 enum { FP4ATTN_PSCALE_CEIL = 0,    /* E_B = ceil(max y): nothing saturates                              */
@@ -178,6 +193,9 @@ typedef struct {
                                        is set, the affine map elsewhere.  Supported patterns:
                                        0x1111, 0x5555, 0x7777 (4, 8, 12 of 16 pairs exact);
                                        noncausal only                                          */
+  int g_per_head;                   /* NVFP4 only: 0 - q_G and k_G point to one factor each; 1 - q_G holds
+                                       B*H factors and k_G B*kv_heads, one per (batch, head) unit
+                                       (fp4attn_quantize_nvfp4_per_head)                        */
 } fp4attn_operands;
 
 /*

@@ -17,7 +17,8 @@ ROLE_Q, ROLE_K, ROLE_V = 0, 1, 2
 PMAP_IDEAL, PMAP_AFFINE, PMAP_HYBRID = 0, 1, 2
 PSCALE_CEIL, PSCALE_THR16 = 0, 1
 QSCALE_CEIL, QSCALE_THR16, QSCALE_FLOOR, QSCALE_MSE = 0, 1, 2, 3
-ERR_TIMEOUT = 7
+(OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_ARCH, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA,
+ ERR_TIMEOUT) = range(8)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libfp4attn.so")
@@ -27,6 +28,7 @@ EXPORTS = [
     "fp4attn_quantize_workspace_bytes", "fp4attn_quantize", "fp4attn_fwd",
     "fp4attn_attention_host_workspace_bytes", "fp4attn_attention_host", "fp4attn_mma_peak_probe",
     "fp4attn_quantize_nvfp4_noalloc", "fp4attn_selftest_bounded_wait", "fp4attn_quantize_mxfp4_rule",
+    "fp4attn_quantize_nvfp4_per_head_workspace_bytes", "fp4attn_quantize_nvfp4_per_head",
 ]
 
 
@@ -41,7 +43,7 @@ class _Operands(ctypes.Structure):
                 ("qk_fmt", ctypes.c_int), ("softmax_scale", ctypes.c_float),
                 ("p_map", ctypes.c_int), ("affine_a", ctypes.c_float), ("affine_b", ctypes.c_float),
                 ("p_scale_rule", ctypes.c_int), ("causal", ctypes.c_int), ("kv_heads", ctypes.c_int),
-                ("exact_pairs", ctypes.c_int)]
+                ("exact_pairs", ctypes.c_int), ("g_per_head", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:
@@ -71,6 +73,10 @@ def _load() -> ctypes.CDLL:
     lib.fp4attn_quantize_mxfp4_rule.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp]
     lib.fp4attn_quantize_nvfp4_noalloc.restype = i
     lib.fp4attn_quantize_nvfp4_noalloc.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp]
+    lib.fp4attn_quantize_nvfp4_per_head_workspace_bytes.restype = sz
+    lib.fp4attn_quantize_nvfp4_per_head_workspace_bytes.argtypes = [i, i, i, i]
+    lib.fp4attn_quantize_nvfp4_per_head.restype = i
+    lib.fp4attn_quantize_nvfp4_per_head.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, sz, vp]
     lib.fp4attn_selftest_bounded_wait.restype = i
     lib.fp4attn_selftest_bounded_wait.argtypes = [ctypes.c_longlong, vp, vp]
     lib.fp4attn_mma_peak_probe.restype = i
@@ -109,6 +115,7 @@ class QuantizedOperand:
     fmt: int
     role: int
     shape: Tuple[int, int, int, int]  # (B, H, N, d) of the source tensor
+    per_head: bool = False            # NVFP4: G holds one factor per (batch, head) unit
 
 
 def fp4attn_quantize(x: torch.Tensor, fmt: int, role: int, workspace: Optional[torch.Tensor] = None) -> QuantizedOperand:
@@ -151,6 +158,28 @@ def fp4attn_quantize_mxfp4_rule(x: torch.Tensor, role: int, scale_rule: int) -> 
     return QuantizedOperand(packed, scales, None, FMT_MXFP4, role, (B, H, N, d))
 
 
+def fp4attn_quantize_nvfp4_per_head(x: torch.Tensor, role: int) -> QuantizedOperand:
+    """NVFP4 quantizer with one encode factor per (batch, head) unit; G comes back as fp32 [B*H]."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 4
+    B, H, N, d = x.shape
+    L = lib()
+    nb = L.fp4attn_packed_bytes(B, H, N, d)
+    ns = L.fp4attn_scale_bytes(FMT_NVFP4, role, B, H, N, d)
+    nw = L.fp4attn_quantize_nvfp4_per_head_workspace_bytes(B, H, N, d)
+    if nb == 0 or ns == 0 or nw == 0:
+        _check(L.fp4attn_quantize_nvfp4_per_head(x.data_ptr(), role, B, H, N, d, 1, 1, 1, None, 0, _stream()),
+               "fp4attn_quantize_nvfp4_per_head")
+        raise Fp4AttnError("fp4attn_quantize_nvfp4_per_head: unsupported arguments")
+    packed = torch.empty(nb, dtype=torch.uint8, device=x.device)
+    scales = torch.empty(ns, dtype=torch.uint8, device=x.device)
+    G = torch.empty(B * H, dtype=torch.float32, device=x.device)
+    ws = torch.empty(nw, dtype=torch.uint8, device=x.device)
+    _check(L.fp4attn_quantize_nvfp4_per_head(x.data_ptr(), role, B, H, N, d, packed.data_ptr(), scales.data_ptr(),
+                                             G.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "fp4attn_quantize_nvfp4_per_head")
+    return QuantizedOperand(packed, scales, G, FMT_NVFP4, role, (B, H, N, d), True)
+
+
 def fp4attn_quantize_nvfp4_noalloc(x: torch.Tensor, role: int, packed: torch.Tensor, scales: torch.Tensor,
                                    G: torch.Tensor) -> QuantizedOperand:
     """NVFP4 quantizer that allocates nothing: the caller passes every output buffer and the library
@@ -172,6 +201,7 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
     B, H, N, d = q.shape
     Hkv = k.shape[1]                                   # grouped-query attention when Hkv < H
     assert k.shape == v.shape and k.shape == (B, Hkv, N, d) and H % Hkv == 0 and q.fmt == k.fmt and v.fmt == FMT_MXFP4
+    assert q.per_head == k.per_head, "Q and K must both carry per-head factors, or neither"
     dev = q.packed.device
     if out is None:
         out = torch.empty((B, H, N, d), dtype=torch.bfloat16, device=dev)
@@ -180,7 +210,7 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
     ops = _Operands(q.packed.data_ptr(), k.packed.data_ptr(), v.packed.data_ptr(),
                     q.scales.data_ptr(), k.scales.data_ptr(), v.scales.data_ptr(),
                     _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b), int(p_scale_rule), int(bool(causal)), int(Hkv),
-                    int(exact_pairs))
+                    int(exact_pairs), int(q.per_head))
     _check(lib().fp4attn_fwd(ctypes.byref(ops), B, H, N, d, out.data_ptr(), lse.data_ptr(), _ptr(status), _stream()),
            "fp4attn_fwd")
     return out, lse

@@ -99,6 +99,7 @@ struct AttnParams {
   int causal;              // 1: query row i sees keys 0..i
   int H, Hkv;              // query heads, K/V heads (H % Hkv == 0: grouped-query attention)
   int BH;                  // B * H
+  int g_per_head;          // NVFP4: q_G holds B*H factors and k_G B*Hkv, one per (batch, head) unit
   unsigned long long recip_qtiles, recip_bh;   // ceil(2^64 / (N / 128)), ceil(2^64 / BH); 0 for a divisor of 1
 };
 
@@ -108,6 +109,7 @@ struct WorkItem {
   int qrow0;               // first row of the tile in the [B*H*N] row space of Q, O, LSE
   int qtile_lin;           // (b*H + h) * qtiles + qt: index of the tile's Q scale atom(s)
   int kvh;                 // b*Hkv + h / (H/Hkv): the K/V head this query head reads
+  int bh;                  // b*H + h
   int T2;                  // 128-key stages to walk (causal: up to and including the diagonal)
 };
 // floor(n / d) for n < 2^31 through the precomputed reciprocal ceil(2^64 / d) (0 stands for d = 1): the
@@ -130,6 +132,7 @@ __device__ __forceinline__ WorkItem decode_item(int item, const AttnParams& p, i
   w.qrow0 = bh * p.N + w.qt * BM;
   w.qtile_lin = bh * qtiles + w.qt;
   w.kvh = bh;
+  w.bh = bh;
   if (p.H != p.Hkv) {       // grouped-query attention
     const int b = bh / p.H, h = bh - b * p.H;
     w.kvh = b * p.Hkv + h / (p.H / p.Hkv);
@@ -612,6 +615,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
         T2 = wi.T2;
         gdiag = CAUSAL ? g0 + (uint32_t)wi.qt : 0xFFFFFFFFu;
+        if (NV && p.g_per_head)                                 // this unit's own pair of encode factors
+          c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G + wi.bh), __ldg(p.k_G + wi.kvh)));
       }
       for (uint32_t g = g0 + ((g0 & 1) != (uint32_t)pr); g < g0 + T2; g += 2) {   // this team's stages of the item
         const uint32_t m = g >> 1;
@@ -792,6 +797,7 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
     if (pmap < 0 || ops->causal) return FP4ATTN_ERR_INVALID_ARG;    // three patterns, noncausal only
   }
   if (ops->p_scale_rule != FP4ATTN_PSCALE_CEIL && ops->p_scale_rule != FP4ATTN_PSCALE_THR16) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->g_per_head != 0 && ops->g_per_head != 1) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->kv_heads < 0 || (ops->kv_heads > 0 && H % ops->kv_heads != 0) || (ops->causal != 0 && ops->causal != 1))
     return FP4ATTN_ERR_INVALID_ARG;
   if (ops->p_map != FP4ATTN_PMAP_IDEAL && !(ops->affine_a >= 0.f && ops->affine_a < 16.f && fabsf(ops->affine_b) < 16.f))
@@ -807,6 +813,7 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.O = (__nv_bfloat16*)O; prm.LSE = LSE; prm.status = device_status;
   prm.N = N; prm.stages = N / BS; prm.n_items = B * H * (N / BM);
   prm.BH = B * H;
+  prm.g_per_head = (ops->qk_fmt == FP4ATTN_FMT_NVFP4 && ops->g_per_head) ? 1 : 0;
   prm.recip_qtiles = (N / BM) > 1 ? ~0ull / (unsigned long long)(N / BM) + 1 : 0;
   prm.recip_bh = prm.BH > 1 ? ~0ull / (unsigned long long)prm.BH + 1 : 0;
   prm.causal = ops->causal ? 1 : 0;

@@ -10,6 +10,7 @@ constexpr int kThreads = 256;
 constexpr int kGroupsPerThread = 4;          // 16-byte loads in flight per thread
 constexpr int kGroupsPerCta = kThreads * kGroupsPerThread;
 constexpr int kMaxPartials = 1024;           // NVFP4 amax pass: one partial maximum per block
+constexpr int kPartialsPerHead = 32;         // the same, per (batch, head) unit, for per-head factors
 
 __device__ __forceinline__ float amax8(const float* v) {
   float a = 0.f;
@@ -210,9 +211,13 @@ quant_mx_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ packed, uint8
   }
 }
 
-// ---------------------------------------------------------------- NVFP4 pass 1: tensor-wide amax partials
+// ---------------------------------------------------------------- NVFP4 pass 1: amax partials
+// grid (P, U): U = 1 for the tensor-wide maximum, U = B*H for one maximum per (batch, head) unit; row y of
+// the grid covers groups [y * n_groups, (y + 1) * n_groups) and writes partials[y * P .. y * P + P)
 __global__ void __launch_bounds__(kThreads)
 amax_partials_kernel(const uint4* __restrict__ x, size_t n_groups, float* __restrict__ partials) {
+  x += (size_t)blockIdx.y * n_groups;
+  partials += (size_t)blockIdx.y * gridDim.x;
   float a = 0.f;
   for (size_t g = (size_t)blockIdx.x * kThreads + threadIdx.x; g < n_groups; g += (size_t)gridDim.x * kThreads) {
     float v[8];
@@ -246,11 +251,13 @@ __device__ __forceinline__ float e4m3_byte_to_f32(uint32_t b) {
 template <int D>
 __global__ void __launch_bounds__(kThreads)
 quant_nv_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed, uint8_t* __restrict__ sf,
-                     const float* __restrict__ partials, int n_partials, float* __restrict__ G_out, int N) {
+                     const float* __restrict__ partials, int n_partials, float* __restrict__ G_out, int N, int per_head) {
   constexpr int GPR = D / 8;
   constexpr int CT = (D / 16 + 3) / 4;
   __shared__ float s_G;
   {
+    // per_head: this block's (batch, head) unit has its own n_partials maxima and its own factor
+    if (per_head) { partials += (size_t)blockIdx.y * n_partials; G_out += blockIdx.y; }
     float a = 0.f;
     for (int i = threadIdx.x; i < n_partials; i += kThreads) a = fmaxf(a, partials[i]);
 #pragma unroll
@@ -262,7 +269,7 @@ quant_nv_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
       for (int i = 1; i < kThreads / 32; ++i) a = fmaxf(a, wmax[i]);
       const float G = (a == 0.f) ? 1.0f : __fdiv_rn(2688.0f, a);
       s_G = G;
-      if (blockIdx.x == 0 && blockIdx.y == 0) *G_out = G;
+      if (blockIdx.x == 0 && (per_head || blockIdx.y == 0)) *G_out = G;
     }
     __syncthreads();
   }
@@ -343,7 +350,7 @@ static void launch_mx(const uint4* xs, int role, int B, int H, int N, int d, voi
 }
 
 int launch_quantize(const void* x, int fmt, int role, int B, int H, int N, int d, void* packed, void* scales,
-                    float* G_out, float* partials, cudaStream_t st, int mx_rule) {
+                    float* G_out, float* partials, cudaStream_t st, int mx_rule, bool per_head = false) {
   const size_t n_groups = (size_t)B * H * N * d / 8;
   const unsigned grid = (unsigned)(n_groups / kGroupsPerCta);
   const dim3 grid2((unsigned)((size_t)N * d / 8 / kGroupsPerCta), (unsigned)(B * H));   // N % 128 == 0 makes this exact
@@ -354,10 +361,16 @@ int launch_quantize(const void* x, int fmt, int role, int B, int H, int N, int d
     else if (mx_rule == FP4ATTN_QSCALE_MSE)   launch_mx<FP4ATTN_QSCALE_MSE>(xs, role, B, H, N, d, packed, scales, st);
     else                                      launch_mx<FP4ATTN_QSCALE_CEIL>(xs, role, B, H, N, d, packed, scales, st);
   } else {
-    const int n_partials = (int)(grid < (unsigned)kMaxPartials ? grid : kMaxPartials);
-    amax_partials_kernel<<<n_partials, kThreads, 0, st>>>(xs, n_groups, partials);
-    if (d == 128) quant_nv_rows_kernel<128><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N);
-    else          quant_nv_rows_kernel<64><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N);
+    int n_partials;
+    if (per_head) {
+      n_partials = (int)(grid2.x < (unsigned)kPartialsPerHead ? grid2.x : kPartialsPerHead);
+      amax_partials_kernel<<<dim3(n_partials, B * H), kThreads, 0, st>>>(xs, n_groups / ((size_t)B * H), partials);
+    } else {
+      n_partials = (int)(grid < (unsigned)kMaxPartials ? grid : kMaxPartials);
+      amax_partials_kernel<<<n_partials, kThreads, 0, st>>>(xs, n_groups, partials);
+    }
+    if (d == 128) quant_nv_rows_kernel<128><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N, per_head);
+    else          quant_nv_rows_kernel<64><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N, per_head);
   }
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
@@ -401,6 +414,25 @@ extern "C" int fp4attn_quantize_mxfp4_rule(const void* x, int role, int scale_ru
   if (rc != FP4ATTN_OK) return rc;
   return launch_quantize(x, FP4ATTN_FMT_MXFP4, role, B, H, N, d, packed, scales, nullptr, nullptr, (cudaStream_t)stream,
                          scale_rule);
+}
+
+extern "C" size_t fp4attn_quantize_nvfp4_per_head_workspace_bytes(int B, int H, int N, int d) {
+  if (!shape_ok(B, H, N, d)) return 0;
+  return (size_t)B * H * kPartialsPerHead * sizeof(float);
+}
+
+extern "C" int fp4attn_quantize_nvfp4_per_head(const void* x, int role, int B, int H, int N, int d, void* packed,
+                                               void* scales, float* G_out, void* workspace, size_t workspace_bytes,
+                                               fp4attn_stream_t stream) {
+  int rc = validate_quantize(x, FP4ATTN_FMT_NVFP4, role, B, H, N, d, packed, scales, G_out);
+  if (rc != FP4ATTN_OK) return rc;
+  const size_t need = fp4attn_quantize_nvfp4_per_head_workspace_bytes(B, H, N, d);
+  if (!workspace || workspace_bytes < need) return FP4ATTN_ERR_WORKSPACE;
+  if ((uintptr_t)workspace & 15) return FP4ATTN_ERR_ALIGNMENT;
+  rc = check_device_sm100();
+  if (rc != FP4ATTN_OK) return rc;
+  return launch_quantize(x, FP4ATTN_FMT_NVFP4, role, B, H, N, d, packed, scales, G_out, (float*)workspace,
+                         (cudaStream_t)stream, FP4ATTN_QSCALE_CEIL, true);
 }
 
 // ---------------------------------------------------------------- allocation-free NVFP4 variant

@@ -98,5 +98,5 @@ def test_header_is_plain_c_and_the_struct_layout_matches_the_binding(lib, tmp_pa
         assert int(out[n]) == getattr(binding._Operands, n).offset, n
     assert int(out["version"]) == lib.fp4attn_version()
     assert int(out["packed"]) == 4 * 16 * 4096 * 128 // 2
-    assert int(out["null_ops"]) == binding.ERR_INVALID_ARG if hasattr(binding, "ERR_INVALID_ARG") else int(out["null_ops"]) != 0
+    assert int(out["null_ops"]) == binding.ERR_INVALID_ARG
     assert out["status"] == "invalid argument"

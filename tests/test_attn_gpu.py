@@ -490,3 +490,32 @@ def test_random_configurations_match_oracle(seed):
             okw["exact_pairs"] = mask
         Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows, **okw)
         check_heads(O.float().cpu().numpy().astype(np.float64), L.cpu().numpy().astype(np.float64), Oo, Lo, heads, rows)
+
+
+@pytest.mark.parametrize("kw,group,causal", [(dict(B=2, H=4, N=512), 1, False), (dict(B=1, H=4, N=384, d=128), 2, True),
+                                             (dict(B=2, H=6, N=256), 3, False)])
+def test_nvfp4_per_head_factors_attention_matches_oracle(kw, group, causal):
+    """NVFP4 Q, K with one encode factor per (batch, head) unit (heads scaled by 2^-6..2^6 so that the factors
+    differ), also with grouped K/V heads (the key factor is the K/V head's) and the causal mask."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg3"], **kw)
+    q, k, v = I.make_qkv(w)
+    rng = np.random.default_rng(11)
+    Hkv = w.H // group
+    xq = Qz.bf16_bits_to_f64(q) * 2.0 ** rng.integers(-6, 7, size=(w.B, w.H, 1, 1))
+    xk = Qz.bf16_bits_to_f64(k)[:, :Hkv] * 2.0 ** rng.integers(-6, 7, size=(w.B, Hkv, 1, 1))
+    q2, k2 = I.f32_to_bf16_bits(xq.astype(np.float32)), I.f32_to_bf16_bits(xk.astype(np.float32))
+    v2 = np.ascontiguousarray(v[:, :Hkv])
+    # logits stay in a sane range: the softmax scale undoes the average head scaling
+    qd = Bd.fp4attn_quantize_nvfp4_per_head(_dev(q2), Bd.ROLE_Q)
+    kd = Bd.fp4attn_quantize_nvfp4_per_head(_dev(k2), Bd.ROLE_K)
+    vd = Bd.fp4attn_quantize(_dev(v2), Bd.FMT_MXFP4, Bd.ROLE_V)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    O, lse = Bd.fp4attn_fwd(qd, kd, vd, status=status, causal=causal)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    Og, Lg = O.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+    oq, ok_ = Qz.quantize_qk(q2, "nv", per_head=True), Qz.quantize_qk(k2, "nv", per_head=True)
+    heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    Oo, Lo = A.direct_p_forward(oq, ok_, Qz.quantize_v(v2), heads=heads, causal=causal, kv_group=group)
+    check_heads(Og, Lg, Oo, Lo, heads)

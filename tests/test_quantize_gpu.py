@@ -152,3 +152,37 @@ def test_mx_non_finite_values_stay_in_their_block():
     assert np.array_equal(sf_clean, Qz.swizzle_scales(want["sf"]).reshape(-1))
     assert (sf_g != sf_clean).sum() == 2 and set(sf_g[sf_g != sf_clean]) == {254}
     assert (pk_g[0, 0, 5, 1, (40 - 32) // 2] & 0xF) == 7        # +inf (even element: low nibble) saturates at +6
+
+
+@pytest.mark.parametrize("kw", [dict(B=2, H=3, N=256), dict(B=1, H=5, N=1152, d=128), dict(B=3, H=1, N=128)])
+def test_nvfp4_per_head_factors_match_oracle(kw):
+    """One encode factor per (batch, head) unit: bytes and the B*H factors equal the oracle's; heads are given
+    magnitudes from 2^-20 to 2^9 (and one unit is all zero) so that a tensor-wide factor would not do."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg3"], **kw)
+    q, k, _ = I.make_qkv(w)
+    rng = np.random.default_rng(3)
+    for bits, role in ((q, Bd.ROLE_Q), (k, Bd.ROLE_K)):
+        x = Qz.bf16_bits_to_f64(bits)
+        x *= 2.0 ** rng.integers(-20, 10, size=(w.B, w.H, 1, 1))
+        if role == Bd.ROLE_K:
+            x[w.B - 1, w.H - 1] = 0.0
+        bits2 = I.f32_to_bf16_bits(x.astype(np.float32))
+        got = Bd.fp4attn_quantize_nvfp4_per_head(_dev(bits2), role)
+        want = Qz.quantize_qk(bits2, "nv", per_head=True)
+        G = want.pop("G")
+        _check_operand(got, {**want, "G": None}, role)
+        assert np.array_equal(got.G.cpu().numpy(), G.reshape(-1))
+        assert got.per_head
+
+
+def test_nvfp4_per_head_rejects_v_and_missing_workspace():
+    from paper_2609_04105_b200 import binding as Bd
+    x = torch.zeros((1, 2, 128, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_quantize_nvfp4_per_head(x, Bd.ROLE_V)
+    L = Bd.lib()
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    rc = L.fp4attn_quantize_nvfp4_per_head(x.data_ptr(), Bd.ROLE_Q, 1, 2, 128, 64, buf.data_ptr(), buf.data_ptr(),
+                                           buf.data_ptr(), None, 0, None)
+    assert rc == Bd.ERR_WORKSPACE
