@@ -452,7 +452,7 @@ def test_many_small_heads_more_items_than_one_wave():
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_random_configurations_match_oracle(seed):
     """Forty seeded draws of (d, Q/K format, N, B, heads, K/V head sharing, mask, code map, block-exponent rule,
-    softmax scale, outlier channels) per seed: every combination of options on small shapes, sampled rows of two
+    softmax scale, outlier channels, NVFP4 factors per tensor or per head, MXFP4 amplitude rule) per seed: every combination of options on small shapes, sampled rows of two
     heads each against the oracle, usual tolerances."""
     from paper_2609_04105_b200 import binding as Bd
     rng = np.random.default_rng(seed)
@@ -471,16 +471,23 @@ def test_random_configurations_match_oracle(seed):
             x[0][..., ch] *= 20
             x[1][..., ch] *= 20
         bits = [I.f32_to_bf16_bits(a) for a in x]
-        fmt = Bd.FMT_NVFP4 if nv else Bd.FMT_MXFP4
-        ops = [Bd.fp4attn_quantize(_dev(bits[0]), fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(bits[1]), fmt, Bd.ROLE_K),
-               Bd.fp4attn_quantize(_dev(bits[2]), Bd.FMT_MXFP4, Bd.ROLE_V)]
+        per_head = bool(rng.integers(0, 2))                       # NVFP4: one factor per (batch, head) unit
+        rule = int(rng.integers(0, 4))                            # MXFP4 amplitude rule of Q, K and V
+        rname = ["ceil", "thr16", "floor", "mse"][rule]
+        if nv:
+            quant = Bd.fp4attn_quantize_nvfp4_per_head if per_head else (lambda t, role: Bd.fp4attn_quantize(t, Bd.FMT_NVFP4, role))
+            ops = [quant(_dev(bits[0]), Bd.ROLE_Q), quant(_dev(bits[1]), Bd.ROLE_K), Bd.fp4attn_quantize(_dev(bits[2]), Bd.FMT_MXFP4, Bd.ROLE_V)]
+        else:
+            ops = [Bd.fp4attn_quantize_mxfp4_rule(_dev(bits[i]), role, rule) for i, role in enumerate((Bd.ROLE_Q, Bd.ROLE_K, Bd.ROLE_V))]
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         O, L = Bd.fp4attn_fwd(*ops, softmax_scale=scale, status=status, p_map=pm, p_scale_rule=int(thr), causal=causal,
                               exact_pairs=mask if pm == 2 else 0)
         torch.cuda.synchronize()
         assert int(status.item()) == 0
-        f = "nv" if nv else "mx"
-        qd, kd, vd = Qz.quantize_qk(bits[0], f), Qz.quantize_qk(bits[1], f), Qz.quantize_v(bits[2])
+        if nv:
+            qd, kd, vd = Qz.quantize_qk(bits[0], "nv", per_head=per_head), Qz.quantize_qk(bits[1], "nv", per_head=per_head), Qz.quantize_v(bits[2])
+        else:
+            qd, kd, vd = Qz.quantize_qk(bits[0], "mx", rname), Qz.quantize_qk(bits[1], "mx", rname), Qz.quantize_v(bits[2], rname)
         heads = [(int(rng.integers(0, B)), int(rng.integers(0, H))) for _ in range(2)]
         rows = np.sort(rng.choice(N, size=min(N, 48), replace=False))
         rows[0], rows[-1] = 0, N - 1
@@ -506,7 +513,7 @@ def test_nvfp4_per_head_factors_attention_matches_oracle(kw, group, causal):
     xk = Qz.bf16_bits_to_f64(k)[:, :Hkv] * 2.0 ** rng.integers(-6, 7, size=(w.B, Hkv, 1, 1))
     q2, k2 = I.f32_to_bf16_bits(xq.astype(np.float32)), I.f32_to_bf16_bits(xk.astype(np.float32))
     v2 = np.ascontiguousarray(v[:, :Hkv])
-    # logits stay in a sane range: the softmax scale undoes the average head scaling
+    # logits range from 2^-12 to 2^12 times the usual: flat rows as well as one-hot ones
     qd = Bd.fp4attn_quantize_nvfp4_per_head(_dev(q2), Bd.ROLE_Q)
     kd = Bd.fp4attn_quantize_nvfp4_per_head(_dev(k2), Bd.ROLE_K)
     vd = Bd.fp4attn_quantize(_dev(v2), Bd.FMT_MXFP4, Bd.ROLE_V)
