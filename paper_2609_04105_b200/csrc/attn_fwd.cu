@@ -471,22 +471,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     bool ok = true;
     int i = 0;
     int T2 = 0;
-    int mu_next = -(1 << 28);                                   // reference of the item whose first stage was served early
+    int mu_next = -(1 << 28);                                   // reference of the item whose first stage was served ahead
     bool first_served = false;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i, g0 += T2) {
       const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
       T2 = wi.T2;
-      // (measured: +1..2 % with any exponentials in the map, -1 % with none, so the pure affine map skips it)
-      const uint32_t g_end = g0 + (uint32_t)T2 + ((PMAP != 1 && item + (int)gridDim.x < p.n_items) ? 1u : 0u);
+      const bool has_next = item + (int)gridDim.x < p.n_items;
       int mu = first_served ? mu_next : -(1 << 28);
-      int mu_item = mu;
-      // One pass per 128-key stage (both of its tiles).  After the item's last stage the loop also serves the
-      // NEXT item's first stage (the teams run ahead and have it encoded, or will shortly - nothing they need
-      // depends on this item's epilogue): its PV then waits for O only, not for the epilogue as well.
-      for (uint32_t g = g0 + (first_served ? 1u : 0u); g < g_end; ++g) {
-        const bool first_of_item = (g == g0) || (g == g0 + (uint32_t)T2);
+      // One pass per 128-key stage (both of its tiles).  The item's first stage may already have been served
+      // from inside the previous item's epilogue.
+      for (uint32_t g = g0 + (first_served ? 1u : 0u); g < g0 + (uint32_t)T2; ++g) {
+        const bool first_of_item = g == g0;
         const int pr = g & 1;
-        if (g == g0 + (uint32_t)T2) { mu_item = mu; mu = -(1 << 28); }
         ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + pr), (g >> 1) & 1, abortf));
         if (!ok) break;
         const int4 me = *reinterpret_cast<const int4*>(sgen + C::OFF_META + C::META_BYTES * pr + row * 16);
@@ -533,8 +529,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + pr));
       }
       if (!ok) break;
-      first_served = g_end > g0 + (uint32_t)T2;
-      if (first_served) { mu_next = mu; mu = mu_item; } else { mu_item = mu; }
+      first_served = false;
       // ---- epilogue: with L_hw = column d of the accumulator, O = O_hw / (6 L_hw), LSE = ln2 (mu + log2(L_hw / 6))
       ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFULL), i & 1, abortf));
       if (!ok) break;
@@ -581,6 +576,26 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (lane == 0) mbar_arrive(bar(BAR_OFREE));
           }
         }
+      }
+      if (has_next) {
+        // O is released; before the stores go out, serve the next item's first stage (the teams run ahead and
+        // have it encoded, or will shortly - nothing they need depends on this epilogue), so that its PV waits
+        // for neither the rest of this epilogue nor a pass after it.  A first stage starts a fresh reference,
+        // kRefHeadroom above its largest block exponent, and never touches O.  (Measured against serving it
+        // before the epilogue: +1 % with exponentials in the map, +-1 % without.)
+        const uint32_t g = g0 + (uint32_t)T2;
+        const int pr = g & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + pr), (g >> 1) & 1, abortf));
+        if (!ok) break;
+        const int4 me = *reinterpret_cast<const int4*>(sgen + C::OFF_META + C::META_BYTES * pr + row * 16);
+        mu_next = max(max(me.x, me.y), max(me.z, me.w)) + kRefHeadroom;
+        const uint32_t u0 = (uint32_t)max(me.x - mu_next + 127, 0), u1 = (uint32_t)max(me.y - mu_next + 127, 0);
+        const uint32_t u2 = (uint32_t)max(me.z - mu_next + 127, 0), u3 = (uint32_t)max(me.w - mu_next + 127, 0);
+        *reinterpret_cast<uint32_t*>(sgen + C::OFF_PSF + 512 * pr + lane * 16 + quarter * 4) = u0 | (u1 << 8) | (u2 << 16) | (u3 << 24);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + pr));
+        first_served = true;
       }
       fence_proxy_async_smem();
       __syncwarp();
