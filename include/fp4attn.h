@@ -195,7 +195,8 @@ typedef struct {
                                        noncausal only                                          */
   int g_per_head;                   /* NVFP4 only: 0 - q_G and k_G point to one factor each; 1 - q_G holds
                                        B*H factors and k_G B*kv_heads, one per (batch, head) unit
-                                       (fp4attn_quantize_nvfp4_per_head)                        */
+                                       (fp4attn_quantize_nvfp4_per_head); with the ideal and the
+                                       affine map, not with FP4ATTN_PMAP_HYBRID                 */
 } fp4attn_operands;
 
 /*

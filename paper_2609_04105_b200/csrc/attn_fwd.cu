@@ -99,7 +99,6 @@ struct AttnParams {
   int causal;              // 1: query row i sees keys 0..i
   int H, Hkv;              // query heads, K/V heads (H % Hkv == 0: grouped-query attention)
   int BH;                  // B * H
-  int g_per_head;          // NVFP4: q_G holds B*H factors and k_G B*Hkv, one per (batch, head) unit
   unsigned long long recip_qtiles, recip_bh;   // ceil(2^64 / (N / 128)), ceil(2^64 / BH); 0 for a divisor of 1
 };
 
@@ -259,12 +258,15 @@ __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float 
   }
 }
 
-template <int D, bool NV, int PMAP, bool CAUSAL, bool THR16>
+// NV: 0 - MXFP4 Q, K; 1 - NVFP4 with one encode factor per tensor; 2 - NVFP4 with one factor per (batch, head)
+// unit (an instance of its own: a score constant that changes per work item costs the tensor-wide variant
+// 2-8 % when it is only a run-time branch)
+template <int D, int NV, int PMAP, bool CAUSAL, bool THR16>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
                 const AttnParams p) {
-  using C = Cfg<D, NV>;
+  using C = Cfg<D, (NV != 0)>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
@@ -577,12 +579,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
       }
-      if (has_next) {
+      if (PMAP != 1 && has_next) {
         // O is released; before the stores go out, serve the next item's first stage (the teams run ahead and
         // have it encoded, or will shortly - nothing they need depends on this epilogue), so that its PV waits
         // for neither the rest of this epilogue nor a pass after it.  A first stage starts a fresh reference,
         // kRefHeadroom above its largest block exponent, and never touches O.  (Measured against serving it
-        // before the epilogue: +1 % with exponentials in the map, +-1 % without.)
+        // before the epilogue: +1 % with exponentials in the map; the pure affine map loses 1 % at long
+        // sequences either way and serves the stage in its own loop, after the epilogue.)
         const uint32_t g = g0 + (uint32_t)T2;
         const int pr = g & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + pr), (g >> 1) & 1, abortf));
@@ -630,7 +633,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
         T2 = wi.T2;
         gdiag = CAUSAL ? g0 + (uint32_t)wi.qt : 0xFFFFFFFFu;
-        if (NV && p.g_per_head)                                 // this unit's own pair of encode factors
+        if (NV == 2)                                            // this unit's own pair of encode factors
           c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G + wi.bh), __ldg(p.k_G + wi.kvh)));
       }
       for (uint32_t g = g0 + ((g0 & 1) != (uint32_t)pr); g < g0 + T2; g += 2) {   // this team's stages of the item
@@ -763,10 +766,10 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint6
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool NV, int PMAP, bool CAUSAL, bool THR16>
+template <int D, int NV, int PMAP, bool CAUSAL, bool THR16>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
   const int Hkv = prm.Hkv;
-  using C = Cfg<D, NV>;
+  using C = Cfg<D, (NV != 0)>;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return FP4ATTN_ERR_CUDA;
@@ -813,6 +816,7 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   }
   if (ops->p_scale_rule != FP4ATTN_PSCALE_CEIL && ops->p_scale_rule != FP4ATTN_PSCALE_THR16) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->g_per_head != 0 && ops->g_per_head != 1) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->g_per_head && ops->p_map == FP4ATTN_PMAP_HYBRID) return FP4ATTN_ERR_INVALID_ARG;   // ideal and affine maps only
   if (ops->kv_heads < 0 || (ops->kv_heads > 0 && H % ops->kv_heads != 0) || (ops->causal != 0 && ops->causal != 1))
     return FP4ATTN_ERR_INVALID_ARG;
   if (ops->p_map != FP4ATTN_PMAP_IDEAL && !(ops->affine_a >= 0.f && ops->affine_a < 16.f && fabsf(ops->affine_b) < 16.f))
@@ -828,7 +832,6 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.O = (__nv_bfloat16*)O; prm.LSE = LSE; prm.status = device_status;
   prm.N = N; prm.stages = N / BS; prm.n_items = B * H * (N / BM);
   prm.BH = B * H;
-  prm.g_per_head = (ops->qk_fmt == FP4ATTN_FMT_NVFP4 && ops->g_per_head) ? 1 : 0;
   prm.recip_qtiles = (N / BM) > 1 ? ~0ull / (unsigned long long)(N / BM) + 1 : 0;
   prm.recip_bh = prm.BH > 1 ? ~0ull / (unsigned long long)prm.BH + 1 : 0;
   prm.causal = ops->causal ? 1 : 0;
@@ -842,13 +845,18 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.aff_b = ops->affine_a != 0.f ? ops->affine_b : 1.2f;
   prm.thr16 = ops->p_scale_rule == FP4ATTN_PSCALE_THR16;
   // one kernel instance per (d, Q/K format, P map, mask, P scale rule): nothing of these is decided at run time
+  const bool per_head = nv && ops->g_per_head;
   const int shape = (d == 128 ? 2 : 0) | (nv ? 1 : 0);
 #define FP4ATTN_SHAPES(PM_, CAU_, THR_)                                                  \
+  if (per_head && PM_ <= 1) {                                                            \
+    if (d == 64) return launch_attn<64, 2, (PM_ <= 1 ? PM_ : 0), CAU_, THR_>(ops, B, H, N, prm, st);   \
+    return launch_attn<128, 2, (PM_ <= 1 ? PM_ : 0), CAU_, THR_>(ops, B, H, N, prm, st); \
+  }                                                                                      \
   switch (shape) {                                                                       \
-    case 0: return launch_attn<64, false, PM_, CAU_, THR_>(ops, B, H, N, prm, st);       \
-    case 1: return launch_attn<64, true, PM_, CAU_, THR_>(ops, B, H, N, prm, st);        \
-    case 2: return launch_attn<128, false, PM_, CAU_, THR_>(ops, B, H, N, prm, st);      \
-    default: return launch_attn<128, true, PM_, CAU_, THR_>(ops, B, H, N, prm, st);      \
+    case 0: return launch_attn<64, 0, PM_, CAU_, THR_>(ops, B, H, N, prm, st);           \
+    case 1: return launch_attn<64, 1, PM_, CAU_, THR_>(ops, B, H, N, prm, st);           \
+    case 2: return launch_attn<128, 0, PM_, CAU_, THR_>(ops, B, H, N, prm, st);          \
+    default: return launch_attn<128, 1, PM_, CAU_, THR_>(ops, B, H, N, prm, st);         \
   }
 #define FP4ATTN_MASKS(PM_)                                         \
   if (prm.causal) {                                                \

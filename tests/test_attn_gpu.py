@@ -409,6 +409,15 @@ def test_hybrid_map_config2_full_size_sampled_rows():
     check_heads(Og, Lg, Oo, Lo, heads, rows)
 
 
+def test_hybrid_map_rejects_per_head_factors():
+    from paper_2609_04105_b200 import binding as Bd
+    x = torch.randn((1, 2, 128, 64), device="cuda").bfloat16()
+    q, k = Bd.fp4attn_quantize_nvfp4_per_head(x, Bd.ROLE_Q), Bd.fp4attn_quantize_nvfp4_per_head(x, Bd.ROLE_K)
+    v = Bd.fp4attn_quantize(x, Bd.FMT_MXFP4, Bd.ROLE_V)
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_fwd(q, k, v, p_map=Bd.PMAP_HYBRID, exact_pairs=0x5555)
+
+
 def test_hybrid_map_rejects_other_patterns_and_the_causal_mask():
     from paper_2609_04105_b200 import binding as Bd
     w = I.shrink(I.WORKLOADS["cfg1"], N=128)
@@ -471,7 +480,7 @@ def test_random_configurations_match_oracle(seed):
             x[0][..., ch] *= 20
             x[1][..., ch] *= 20
         bits = [I.f32_to_bf16_bits(a) for a in x]
-        per_head = bool(rng.integers(0, 2))                       # NVFP4: one factor per (batch, head) unit
+        per_head = bool(rng.integers(0, 2)) and pm != 2           # NVFP4: one factor per (batch, head) unit (not with the mixed map)
         rule = int(rng.integers(0, 4))                            # MXFP4 amplitude rule of Q, K and V
         rname = ["ceil", "thr16", "floor", "mse"][rule]
         if nv:
