@@ -250,7 +250,7 @@ def run_cuda(args, w):
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     qws = torch.empty(max(16, Bd.lib().fp4attn_quantize_workspace_bytes(w.qk_fmt, 0, B, H, N, d)), dtype=torch.uint8, device=dev)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)      # > 126 MB L2
-    launches_per_step = 4 if w.qk_fmt == I.FMT_MXFP4 else 6
+    launches_per_step = 4 if w.qk_fmt == I.FMT_MXFP4 else 8          # NVFP4: amax pass + encode factor + codes, for Q and for K
     pmap = Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_HYBRID if args.p_map in HYBRID_PATTERNS else Bd.PMAP_IDEAL
     pairs = HYBRID_PATTERNS.get(args.p_map, 0)
     pscale = Bd.PSCALE_THR16 if args.p_scale == "thr16" else Bd.PSCALE_CEIL

@@ -12,13 +12,6 @@ constexpr int kGroupsPerCta = kThreads * kGroupsPerThread;
 constexpr int kMaxPartials = 1024;           // NVFP4 amax pass: one partial maximum per block
 constexpr int kPartialsPerHead = 32;         // the same, per (batch, head) unit, for per-head factors
 
-__device__ __forceinline__ float amax8(const float* v) {
-  float a = 0.f;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(v[i]));
-  return a;
-}
-
 // ---------------------------------------------------------------- MXFP4, blocks along d (Q, K)
 // |bf16| bit patterns order like the magnitudes, so the block maximum is taken on packed 16-bit
 // integers; 6 v / alpha = v * (1.5 * 2^(129-u)) is one exact fp32 multiply.
@@ -218,12 +211,33 @@ __global__ void __launch_bounds__(kThreads)
 amax_partials_kernel(const uint4* __restrict__ x, size_t n_groups, float* __restrict__ partials) {
   x += (size_t)blockIdx.y * n_groups;
   partials += (size_t)blockIdx.y * gridDim.x;
-  float a = 0.f;
-  for (size_t g = (size_t)blockIdx.x * kThreads + threadIdx.x; g < n_groups; g += (size_t)gridDim.x * kThreads) {
-    float v[8];
-    bf16x8_to_f32(__ldg(x + g), v);
-    a = fmaxf(a, amax8(v));
+  // |bf16| bit patterns order like the magnitudes: packed 16-bit maxima, four independent loads per trip
+  uint32_t m = 0;
+  const size_t stride = (size_t)gridDim.x * kThreads;
+  size_t g = (size_t)blockIdx.x * kThreads + threadIdx.x;
+  for (; g + 3 * stride < n_groups; g += 4 * stride) {
+    const uint4 r0 = __ldg(x + g), r1 = __ldg(x + g + stride), r2 = __ldg(x + g + 2 * stride), r3 = __ldg(x + g + 3 * stride);
+    m = max(max(m, absmax_bf16x8(r0)), max(absmax_bf16x8(r1), max(absmax_bf16x8(r2), absmax_bf16x8(r3))));
   }
+  for (; g < n_groups; g += stride) m = max(m, absmax_bf16x8(__ldg(x + g)));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+  __shared__ uint32_t wmax[kThreads / 32];
+  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < kThreads / 32; ++i) m = max(m, wmax[i]);
+    partials[blockIdx.x] = __uint_as_float(m << 16);
+  }
+}
+
+// One block per encode factor: G = fl32(2688 / max of its partial maxima) (1 for an all-zero tensor or unit).
+// grid (U): block y reads partials[y * n_partials ..) and writes G_out[y]
+__global__ void __launch_bounds__(kThreads)
+nv_encode_factor_kernel(const float* __restrict__ partials, int n_partials, float* __restrict__ G_out) {
+  partials += (size_t)blockIdx.x * n_partials;
+  float a = 0.f;
+  for (int i = threadIdx.x; i < n_partials; i += kThreads) a = fmaxf(a, partials[i]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
   __shared__ float wmax[kThreads / 32];
@@ -231,7 +245,7 @@ amax_partials_kernel(const uint4* __restrict__ x, size_t n_groups, float* __rest
   __syncthreads();
   if (threadIdx.x == 0) {
     for (int i = 1; i < kThreads / 32; ++i) a = fmaxf(a, wmax[i]);
-    partials[blockIdx.x] = a;
+    G_out[blockIdx.x] = (a == 0.f) ? 1.0f : __fdiv_rn(2688.0f, a);
   }
 }
 
@@ -246,34 +260,15 @@ __device__ __forceinline__ float e4m3_byte_to_f32(uint32_t b) {
   return __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
 }
 
-// ---------------------------------------------------------------- NVFP4 pass 2, blocks of 16 along d (Q, K)
+// ---------------------------------------------------------------- NVFP4 pass 3, blocks of 16 along d (Q, K)
 // grid (N * D/8 / kGroupsPerCta, B*H)
 template <int D>
 __global__ void __launch_bounds__(kThreads)
 quant_nv_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed, uint8_t* __restrict__ sf,
-                     const float* __restrict__ partials, int n_partials, float* __restrict__ G_out, int N, int per_head) {
+                     const float* __restrict__ G_in, int N, int per_head) {
   constexpr int GPR = D / 8;
   constexpr int CT = (D / 16 + 3) / 4;
-  __shared__ float s_G;
-  {
-    // per_head: this block's (batch, head) unit has its own n_partials maxima and its own factor
-    if (per_head) { partials += (size_t)blockIdx.y * n_partials; G_out += blockIdx.y; }
-    float a = 0.f;
-    for (int i = threadIdx.x; i < n_partials; i += kThreads) a = fmaxf(a, partials[i]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-    __shared__ float wmax[kThreads / 32];
-    if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = a;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      for (int i = 1; i < kThreads / 32; ++i) a = fmaxf(a, wmax[i]);
-      const float G = (a == 0.f) ? 1.0f : __fdiv_rn(2688.0f, a);
-      s_G = G;
-      if (blockIdx.x == 0 && (per_head || blockIdx.y == 0)) *G_out = G;
-    }
-    __syncthreads();
-  }
-  const float G = s_G;
+  const float G = __ldg(G_in + (per_head ? blockIdx.y : 0));    // this block's (batch, head) unit, or the tensor's
   const uint32_t bh = blockIdx.y;
   const uint32_t gl = blockIdx.x * kGroupsPerCta + threadIdx.x;
   const size_t gbase = (size_t)bh * N * GPR;
@@ -369,8 +364,9 @@ int launch_quantize(const void* x, int fmt, int role, int B, int H, int N, int d
       n_partials = (int)(grid < (unsigned)kMaxPartials ? grid : kMaxPartials);
       amax_partials_kernel<<<n_partials, kThreads, 0, st>>>(xs, n_groups, partials);
     }
-    if (d == 128) quant_nv_rows_kernel<128><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N, per_head);
-    else          quant_nv_rows_kernel<64><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, partials, n_partials, G_out, N, per_head);
+    nv_encode_factor_kernel<<<per_head ? B * H : 1, kThreads, 0, st>>>(partials, n_partials, G_out);
+    if (d == 128) quant_nv_rows_kernel<128><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, G_out, N, per_head);
+    else          quant_nv_rows_kernel<64><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, G_out, N, per_head);
   }
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
