@@ -300,11 +300,11 @@ def run_cuda(args, w):
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
-        Bd.fp4attn_quantize(dq, Bd.FMT_MXFP4, Bd.ROLE_Q)
+        Bd.fp4attn_quantize(dq, w.qk_fmt, Bd.ROLE_Q, qws)
     torch.cuda.current_stream().wait_stream(side)
-    with torch.cuda.graph(qgraph):
+    with torch.cuda.graph(qgraph):                                   # the Q/K quantizer of the workload's own format
         for r in range(12):
-            state["q_only"] = Bd.fp4attn_quantize((dq, dk, dv)[r % 3], Bd.FMT_MXFP4, Bd.ROLE_Q)
+            state["q_only"] = Bd.fp4attn_quantize((dq, dk, dv)[r % 3], w.qk_fmt, Bd.ROLE_Q, qws)
     qb = [E(), E()]
     qgraph.replay()
     flush.fill_(1)
@@ -313,7 +313,10 @@ def run_cuda(args, w):
     qb[1].record()
     torch.cuda.synchronize()
     q_ms = qb[0].elapsed_time(qb[1]) / 12
-    q_bytes = B * H * N * d * (2 + 0.5 + 1.0 / 32)
+    # algorithmic bytes per element: bf16 in, 4-bit codes and scale bytes out; NVFP4 reads the tensor twice
+    q_bpe = (2 + 0.5 + 1.0 / 32) if w.qk_fmt == I.FMT_MXFP4 else (2 + 2 + 0.5 + 1.0 / 16)
+    q_kernel = "quant_mx_rows_kernel" if w.qk_fmt == I.FMT_MXFP4 else "amax_partials_kernel + nv_encode_factor_kernel + quant_nv_rows_kernel"
+    q_bytes = B * H * N * d * q_bpe
 
     # ---- end to end through the host-buffer entry point (pinned host in, host out)
     ho = torch.empty((B, H, N, d), dtype=torch.bfloat16).pin_memory()
@@ -432,11 +435,11 @@ def run_cuda(args, w):
                      "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get("attn"),
                      "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x nominal fp4:bf16 ratio 4",
                      "fp4_issue_probe_tflops": probe_tflops, "fp4_issue_probe_flop_per_clk_per_sm": probe_flop_per_clk_sm},
-        "roofline_quantize": {"kernel": "quant_mx_rows_kernel", "bound": "hbm", "achieved": q_bytes / (q_ms * 1e-3) / 1e9,
+        "roofline_quantize": {"kernel": q_kernel, "bound": "hbm", "achieved": q_bytes / (q_ms * 1e-3) / 1e9,
                               "peak": peaks["hbm_gbs"], "unit": "GB/s",
                               "frac": q_bytes / (q_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                               "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get("quant_rows"),
-                              "bytes_per_element": 2 + 0.5 + 1.0 / 32},
+                              "bytes_per_element": q_bpe},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "api": "fp4attn_attention_host (pinned host buffers)"},
         "attn_other_workloads": sweep,
