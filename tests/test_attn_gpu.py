@@ -535,3 +535,26 @@ def test_nvfp4_per_head_factors_attention_matches_oracle(kw, group, causal):
     heads = [(b, h) for b in range(w.B) for h in range(w.H)]
     Oo, Lo = A.direct_p_forward(oq, ok_, Qz.quantize_v(v2), heads=heads, causal=causal, kv_group=group)
     check_heads(Og, Lg, Oo, Lo, heads)
+
+
+@pytest.mark.parametrize("growth,scale", [(1.0, 2.0), (3.0, 2.0), (-0.11, 2.0), (1.0, 0.02)])
+def test_row_reference_raises_of_every_size(growth, scale):
+    """Scores that climb (or fall) by whole binades from one 128-key stage to the next: the keys of stage s are
+    scaled by 1 + growth * s, and the softmax scale puts a row's stage maximum near 90 log2 units at s = 0.
+    growth 1: the row reference rises by ~90 octaves per stage (raise capped at 126 octaves, old terms kept);
+    growth 3: by ~270 (old terms drop out entirely); negative growth: later blocks fall far below the reference
+    (zero blocks); small scale: the ordinary lazy regime.  The oracle keeps an exact running integer reference."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg1"], N=1024)
+    q, k, v = I.make_qkv(w)
+    xk = Qz.bf16_bits_to_f64(k)
+    s = (np.arange(w.N) // 128).astype(np.float64)
+    xk = xk * (1.0 + growth * s)[None, None, :, None]
+    k2 = I.f32_to_bf16_bits(xk.astype(np.float32))
+    Og, Lg = run_gpu(w, q, k2, v, softmax_scale=scale)
+    qd, kd, vd = oracle_operands(w, q, k2, v)
+    heads = [(0, 0), (0, 1)]
+    rows = np.arange(0, w.N, 7)
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows, softmax_scale=scale)
+    assert np.isfinite(Og).all() and np.isfinite(Lg).all()
+    check_heads(Og, Lg, Oo, Lo, heads, rows)
