@@ -480,6 +480,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       T2 = wi.T2;
       const bool has_next = item + (int)gridDim.x < p.n_items;
       int mu = first_served ? mu_next : -(1 << 28);
+      int runmax = first_served ? mu_next - kRefHeadroom : -(1 << 28);   // largest block exponent of the row so far
       // One pass per 128-key stage (both of its tiles).  The item's first stage may already have been served
       // from inside the previous item's epilogue.
       for (uint32_t g = g0 + (first_served ? 1u : 0u); g < g0 + (uint32_t)T2; ++g) {
@@ -489,18 +490,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         const int4 me = *reinterpret_cast<const int4*>(sgen + C::OFF_META + C::META_BYTES * pr + row * 16);
         const int Emax = max(max(me.x, me.y), max(me.z, me.w));
+        runmax = max(runmax, Emax);
         const bool need = Emax > mu + kLazyShift;
         if (__any_sync(0xffffffffu, need)) {
-          float f = 1.0f;
-          if (need) {
-            // new reference: kRefHeadroom above the offending exponent, but never more than 126 octaves
-            // above the old one while the old contributions can still matter (they reach up to
-            // mu + kLazyShift); only when even that is out of reach are they dropped (f = 0)
-            int delta = Emax + kRefHeadroom - mu;
-            if (delta > 126 && Emax <= mu + 126 + kLazyShift) delta = 126;
-            f = (delta > 126) ? 0.f : __uint_as_float((uint32_t)(127 - delta) << 23);
-            mu = (delta > 126) ? Emax + kRefHeadroom : mu + delta;
-          }
+          // New reference: kRefHeadroom above the row's largest block exponent so far, but never more than 126
+          // octaves above the old one while the old contributions can still matter (they reach up to
+          // mu + kLazyShift); only when even that is out of reach are they dropped (f = 0).  The pass over O is
+          // paid for by the whole warp, so the rows that did not ask for it re-centre as well (for them
+          // 0 <= delta <= kLazyShift + kRefHeadroom): every row has its full span again afterwards, which keeps
+          // passes rare for the warp as a whole (with outlier channels one raise per row would otherwise mean
+          // a pass in every few stages).
+          int delta = runmax + kRefHeadroom - mu;
+          if (delta > 126 && runmax <= mu + 126 + kLazyShift) delta = 126;
+          const float f = (delta > 126) ? 0.f : __uint_as_float((uint32_t)(127 - delta) << 23);
+          mu = (delta > 126) ? runmax + kRefHeadroom : mu + delta;
           if (!first_of_item) {
             // O holds the item's earlier stages once their PV has landed (an item's first stage never
             // touches O: it may still belong to the previous item)
