@@ -2,9 +2,11 @@
  * fp4attn — full-FP4 attention forward with Direct-P for NVIDIA B200 (sm_100a).
  *
  * C ABI.  Unless an argument says otherwise every pointer is a DEVICE pointer owned by the
- * caller; the library allocates nothing, keeps no state between calls except cached kernel
- * attributes and tensor maps' driver entry point, enqueues its work on the caller's stream and
- * returns without synchronising.  Errors that the host can detect come back as a non-zero
+ * caller; the library allocates no device memory.  State kept between calls: cached kernel attributes and
+ * the driver entry point of the tensor-map encoder (per process), the tensor maps of each host thread's last
+ * few attention calls (host memory, a few KB per thread), and the copy streams and events of
+ * fp4attn_attention_host (per device, created on first use); fp4attn_release() drops the last two.  Work is
+ * enqueued on the caller's stream and calls return without synchronising.  Errors that the host can detect come back as a non-zero
  * status and nothing is launched; nothing throws, prints or exits.
  *
  * Tensor layouts
@@ -51,7 +53,8 @@ enum {
 enum { FP4ATTN_FMT_MXFP4 = 0, FP4ATTN_FMT_NVFP4 = 1 };
 enum { FP4ATTN_ROLE_Q = 0, FP4ATTN_ROLE_K = 1, FP4ATTN_ROLE_V = 2 };
 /* how a normalised score x = y - E_B + log2 6 becomes an E2M1 probability code */
-enum { FP4ATTN_PMAP_IDEAL = 0,    /* q = Q_E2M1(2^x)              (Eq. "ideal-code-path")  */
+enum { FP4ATTN_PMAP_IDEAL = 0,    /* q = Q_E2M1(2^x)              (Eq. "ideal-code-path"); how 2^x is evaluated
+                                     is stated at fp4attn_fwd                                 */
        FP4ATTN_PMAP_AFFINE = 1,   /* q = Q_E2M1(max(0, A x + B))  (Eq. "affine-code-map")  */
        FP4ATTN_PMAP_HYBRID = 2 }; /* per element pair one of the two: the EX2-density control of
                                      Appendix "SM103 launch and EX2 controls"; see exact_pairs     */
@@ -93,8 +96,9 @@ size_t fp4attn_quantize_workspace_bytes(int fmt, int role, int B, int H, int N, 
  *
  * Inputs are expected to be finite.  A non-finite value never leads to an out-of-range access or
  * an error return (no address depends on the data); under MXFP4 it only affects its own block
- * (amplitude 2^127, its own code saturated at 6), under NVFP4 it reaches every block through G,
- * and the attention result for such operands is unspecified.
+ * (amplitude 2^127, its own code saturated at 6); under NVFP4 an infinity reaches every block through G
+ * while a NaN may or may not (the tensor maximum is folded with an operation that drops NaNs), and the bytes
+ * written are unspecified.  The attention result for such operands is unspecified.
  */
 int fp4attn_quantize(const void* x_bf16, int fmt, int role, int B, int H, int N, int d,
                      void* packed_out, void* scales_out, float* tensor_scale_out,
@@ -222,6 +226,14 @@ typedef struct {
  * code to 0, and a block without a visible key contributes nothing.  B, H, N, d describe Q and O;
  * K and V have kv_heads heads.
  *
+ * What FP4ATTN_PMAP_IDEAL guarantees.  x is one fused multiply-add in float32, x = fma(S, c, fl32(log2 6 - E_B)).
+ * Of the 16 element pairs (keys 2k, 2k+1) of a block, pairs 0, 5, 10 and 15 evaluate 2^x by a degree-6
+ * polynomial through the seven points where a code can change (after clamping x at -2.75, below which the
+ * code is 0 either way), the other twelve by ex2.approx; the pattern is fixed in this build of the library.
+ * Both are monotone there, so the codes equal Q_E2M1(2^x) except for x within about three float32 spacings of
+ * a rounding boundary log2(t), t in {1/4, 3/4, 5/4, 7/4, 5/2, 7/2, 5}, where either neighbouring code may come
+ * out.  FP4ATTN_PMAP_AFFINE has no such band: its arithmetic is exact float32 as written above.
+ *
  * O_bf16 [B,H,N,d]; LSE [B,H,N] (may be NULL); device_status (may be NULL) receives
  * FP4ATTN_ERR_TIMEOUT if a bounded in-kernel wait ran out, and is otherwise left untouched, so
  * the caller clears it beforehand.
@@ -248,6 +260,11 @@ size_t fp4attn_attention_host_workspace_bytes(int qk_fmt, int B, int H, int N, i
  * join back into it through events.  NVFP4 (tensor-wide amax first) and small problems run on `stream`
  * alone.  Results are bit-identical either way.
  *
+ * status_host (HOST pointer, preferably pinned; may be NULL): the call keeps a status word in its workspace,
+ * clears it before its first kernel, hands it to every attention launch and copies it to *status_host at the
+ * end: FP4ATTN_OK, or FP4ATTN_ERR_TIMEOUT if a bounded in-kernel wait ran out (O_host is then unspecified).
+ * Read it after synchronising `stream`.
+ *
  * Threads: every entry point may be called from several host threads (each on its own stream and
  * buffers); the pipelined host path serialises its enqueue phase on an internal lock because the
  * copy streams and events are shared per device.  On an error return the call still joins the
@@ -255,8 +272,17 @@ size_t fp4attn_attention_host_workspace_bytes(int qk_fmt, int B, int H, int N, i
  */
 int fp4attn_attention_host(const void* q_host, const void* k_host, const void* v_host,
                            int qk_fmt, float softmax_scale, int B, int H, int N, int d,
-                           void* O_host, float* LSE_host,
+                           void* O_host, float* LSE_host, int* status_host,
                            void* workspace, size_t workspace_bytes, fp4attn_stream_t stream);
+
+/*
+ * Gives back what the library keeps between calls: the copy streams and events of fp4attn_attention_host on
+ * every device that used it (they are created again on the next such call) and all cached tensor maps.  No
+ * call of this library may be running or enqueuing on another thread, and every stream handed to
+ * fp4attn_attention_host must have been synchronised.  Optional: a process that never calls it leaks nothing
+ * but those objects until it exits.  (The paper has no counterpart.)
+ */
+int fp4attn_release(void);
 
 /*
  * Dense FP4 tensor-core ceiling of the current device, measured: every SM issues `iters`

@@ -10,7 +10,7 @@ Follows, in the paper's order and notation:
     "represented-output"), with the denominator term evaluated as alpha_B * (c_B / 6) in that
     association (Algorithm "sampled-guard", steps 4-5).
 
-Readings where the paper leaves a choice (listed in the design notes of the repository):
+Readings where the paper leaves a choice:
   * row reference m_i: the running maximum rounded UP to an integer in the log2 domain,
     mu_i = max over tiles seen so far of ceil(max_j y_ij), y = z*log2(e).  With an integer
     reference every online rescale factor is an exact power of two and
@@ -44,6 +44,15 @@ Causal mask and grouped-query attention (the forward the paper's training sectio
 Section "Causal backward ..."): causal=True removes keys j > i from query row i before anything else
 (their score is -inf: they never raise a block maximum and always code to 0; a block with no visible
 key contributes nothing); kv_group = g lets g consecutive query heads share one K/V head.
+
+Several results can be correct.  A code changes only where the converter input crosses one of the seven
+boundaries of Eq. "e2m1-boundaries", and a block exponent only where the block maximum crosses an
+integer.  An implementation whose score differs from fl32(exact product) by a rounding (a tensor core
+accumulating a sum that float32 cannot hold) or whose 2**x is an approximation may legitimately land on
+the other side.  `direct_p_rows(report={})` therefore also lists every such near-decision of a row that
+carries visible weight, and `flips=` re-evaluates rows with chosen decisions taken the other way; a
+checker accepts an output row that disagrees with the default evaluation only if it agrees with one of
+those alternatives.
 """
 from __future__ import annotations
 
@@ -105,14 +114,44 @@ def _fma32(a, b, c):
             + np.asarray(c, np.float32).astype(np.float64)).astype(np.float32)
 
 
+def ulp32(v) -> np.ndarray:
+    """Spacing of float32 at |v| (float64 result; the smallest normal spacing below 2**-126)."""
+    a = np.abs(np.asarray(v, np.float64))
+    _, e = np.frexp(np.maximum(a, 2.0 ** -126))
+    return np.ldexp(1.0, e - 24)
+
+
+AMBIGUITY = dict(rel=2.0 ** -18, ulps=4.0, share=1e-4)
+"""Default near-decision thresholds.  rel: relative distance of the converter input (2**x, or the affine
+classifier's u measured through its slope) from a code boundary; ulps: float32 spacings of the score y
+that an implementation's score may differ by (this widens `rel` for large |y| and is the distance of a
+block maximum from an integer); share: smallest part of the row's represented mass an element (or, for
+an exponent decision, a block) must carry for its decision to be listed."""
+
+
+def _boundary_neighbours(v: np.ndarray):
+    """For decision values v >= 0: index j of the nearest E2M1 rounding boundary t_j and |v - t_j|."""
+    t = np.asarray([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0])
+    dist = np.abs(v[..., None] - t)
+    j = dist.argmin(axis=-1)
+    return j, np.take_along_axis(dist, j[..., None], axis=-1)[..., 0], t[j]
+
+
 def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int = 128, tile_order=None,
                   p_map: str = "ideal", affine=(1.5, 1.2), p_scale: str = "ceil", row_index=None,
-                  exact_pairs: int = 0xFFFF):
+                  exact_pairs: int = 0xFFFF, report=None, flips=None, ambiguity=None):
     """Direct-P online softmax + PV for a set of query rows of one (batch, head).
 
     s32  [R, N] float32 tensor-core-facing scores;  Vhat [N, d] float64 reconstructed V.
     Returns O [R, d] float64, LSE [R] float64, and the represented probabilities' pieces
     (codes [R, N] uint8, block exponents E_B [R, N/32] int64, final reference mu [R]).
+
+    report : optional dict, filled with the near-decisions of every row (thresholds `ambiguity`, default
+             AMBIGUITY): "code" bool [R, N] - the element's code could be its neighbour's; "eb" bool
+             [R, N/32] - the block exponent could be the other integer; "row" bool [R] - any of the two.
+    flips  : optional dict with the same two keys: decisions to take the OTHER way.  A flipped code moves to
+             the code across its nearest boundary; a flipped block exponent to the integer on the other side
+             of the block maximum, and the block's codes follow from the new exponent.
     """
     R, N = s32.shape
     assert N % P_BLOCK == 0 and tile % P_BLOCK == 0 and N % tile == 0
@@ -131,41 +170,92 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
     pair_exact = ((int(exact_pairs) >> (np.arange(P_BLOCK) // 2)) & 1).astype(bool)
     A32, B32 = np.float32(affine[0]), np.float32(affine[1])
     cA = np.float32(A32 * np.float32(c32))
+    amb = dict(AMBIGUITY, **(ambiguity or {}))
+    if report is not None:
+        near_code = np.zeros((R, N), dtype=bool)
+        near_eb = np.zeros((R, N // P_BLOCK), dtype=bool)
+        cand = np.zeros((R, N))                                   # larger candidate value of a near code, in units of 2**E_B / 6
+    flip_code = None if flips is None or flips.get("code") is None else np.asarray(flips["code"], bool)
+    flip_eb = None if flips is None or flips.get("eb") is None else np.asarray(flips["eb"], bool)
+
+    def exponent_of(bj):
+        """Block exponent of keys bj..bj+31 (with its flip applied), and whether it is a near-decision."""
+        ymax = y32[:, bj:bj + P_BLOCK].max(axis=1)
+        E = block_exponent(ymax, p_scale)
+        w = ymax if p_scale == "ceil" else (ymax + LOG2_1P6_32).astype(np.float32)   # the value that is rounded to an integer
+        w64 = w.astype(np.float64)
+        with np.errstate(invalid="ignore"):
+            near = np.isfinite(w64) & (np.abs(w64 - np.rint(w64)) < amb["ulps"] * ulp32(np.where(np.isfinite(w64), w64, 0.0)))
+        if flip_eb is not None:
+            n = np.rint(np.where(np.isfinite(w64), w64, 0.0))
+            other = np.where(E == n, n + (1 if p_scale == "ceil" else -1), n)      # the integer on the other side of w
+            E = np.where(flip_eb[:, bj // P_BLOCK] & np.isfinite(w64), other, E)
+        return E, near
+
     order = range(N // tile) if tile_order is None else tile_order
     for t in order:
         j0 = t * tile
-        m_tile = np.max(np.stack([block_exponent(y32[:, bj:bj + P_BLOCK].max(axis=1), p_scale)
-                                  for bj in range(j0, j0 + tile, P_BLOCK)]), axis=0)
+        exps = [exponent_of(bj) for bj in range(j0, j0 + tile, P_BLOCK)]
+        m_tile = np.max(np.stack([e for e, _ in exps]), axis=0)
         mu_new = np.maximum(mu, m_tile)
         f = np.where(np.isinf(mu), 0.0, np.exp2(mu - mu_new))     # exact power of two
         L *= f
         O *= f[:, None]
         mu = mu_new
-        for bj in range(j0, j0 + tile, P_BLOCK):
-            E_B = block_exponent(y32[:, bj:bj + P_BLOCK].max(axis=1), p_scale)
+        for bj, (E_B, eb_near) in zip(range(j0, j0 + tile, P_BLOCK), exps):
             seen = np.isfinite(E_B)                              # False: every key of the block is masked
             E_B = np.where(seen, E_B, 0.0)
             e_B = np.where(seen, E_B - mu, -np.inf)
             live = (e_B + 127) >= 1
             b_B32 = np.float32(LOG2_6_32 - E_B.astype(np.float32))
+            sl = slice(bj, bj + P_BLOCK)
             if p_map in ("ideal", "hybrid"):
-                x = yx[:, bj:bj + P_BLOCK] + b_B32.astype(np.float64)[:, None]
-                code = e2m1_encode_mag(np.exp2(x))
+                x = yx[:, sl] + b_B32.astype(np.float64)[:, None]
+                v = np.exp2(x)                                   # decision value of the ideal map
+                slope = math.log(2.0) * v                        # d v / d x
+                code = e2m1_encode_mag(v)
             if p_map in ("affine", "hybrid"):
                 bA = _fma32(A32, b_B32, B32)
-                u = _fma32(s32[:, bj:bj + P_BLOCK], cA, bA[:, None])
-                code_a = e2m1_encode_mag(np.maximum(u, np.float32(0)).astype(np.float64))
-                code = code_a if p_map == "affine" else np.where(pair_exact[None, :], code, code_a)
+                u = _fma32(s32[:, sl], cA, bA[:, None])
+                v_a = np.maximum(u, np.float32(0)).astype(np.float64)
+                code_a = e2m1_encode_mag(v_a)
+                if p_map == "affine":
+                    code, v, slope = code_a, v_a, np.full(v_a.shape, float(A32))
+                else:
+                    code = np.where(pair_exact[None, :], code, code_a)
+                    v = np.where(pair_exact[None, :], v, v_a)
+                    slope = np.where(pair_exact[None, :], slope, float(A32))
+            if report is not None or flip_code is not None:
+                with np.errstate(invalid="ignore"):
+                    jn, dist, tj = _boundary_neighbours(np.where(np.isfinite(v), v, 0.0))
+                if report is not None:
+                    tol_x = np.maximum(amb["rel"] / math.log(2.0), amb["ulps"] * ulp32(np.where(np.isfinite(yx[:, sl]), yx[:, sl], 0.0)))
+                    near_code[:, sl] = np.isfinite(yx[:, sl]) & live[:, None] & (dist < slope * tol_x)
+                    cand[:, sl] = E2M1_VALUES[jn + 1]
+                    near_eb[:, bj // P_BLOCK] = eb_near & seen & live
+                if flip_code is not None:
+                    code = np.where(flip_code[:, sl], (2 * jn + 1) - code.astype(np.int64), code)   # neighbours of boundary j are codes j, j+1
             code = np.where(live[:, None], code, 0).astype(np.uint8)
             q = E2M1_VALUES[code]
             alpha = np.where(live, np.exp2(np.where(live, e_B, 0.0)), 0.0)
             c_B = q.sum(axis=1)
             L += alpha * (c_B / 6.0)
-            O += (alpha / 6.0)[:, None] * (q @ Vhat[bj:bj + P_BLOCK])
-            codes_all[:, bj:bj + P_BLOCK] = code
+            O += (alpha / 6.0)[:, None] * (q @ Vhat[sl])
+            codes_all[:, sl] = code
             EB_all[:, bj // P_BLOCK] = np.where(seen, E_B, -(1 << 40)).astype(np.int64)
     Oout = O / L[:, None]
     lse = math.log(2.0) * (mu + np.log2(L))
+    if report is not None:
+        # keep only decisions that carry visible weight: an element's (larger candidate) share of the row's
+        # represented mass, a block's whole share for an exponent decision
+        EBf = np.repeat(np.where(EB_all > -(1 << 39), EB_all, 0).astype(np.float64), P_BLOCK, axis=1)
+        w_el = np.exp2(np.minimum(EBf - mu[:, None], 0.0)) / 6.0 / L[:, None]
+        visible = EB_all > -(1 << 39)
+        share_el = cand * w_el
+        share_blk = (E2M1_VALUES[codes_all] * w_el).reshape(R, N // P_BLOCK, P_BLOCK).sum(axis=2)
+        report["code"] = near_code & (share_el > amb["share"])
+        report["eb"] = near_eb & visible & (share_blk > amb["share"])
+        report["row"] = report["code"].any(axis=1) | report["eb"].any(axis=1)
     return Oout, lse, codes_all, EB_all, mu
 
 
@@ -208,6 +298,16 @@ def exact_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray, softmax_scale=N
     p = np.exp(z - m)
     l = p.sum(axis=1, keepdims=True)
     return (p @ V) / l, (m + np.log(l))[:, 0]
+
+
+def exact_p_attention(qd: dict, kd: dict, vd: dict, b: int, h: int, softmax_scale=None, rows=None, causal=False,
+                      hk=None):
+    """O_exactP for one (batch, head): the quantized operands as they are reconstructed (Q^, K^, V^), exact
+    float64 softmax in between - what the path would return if P were not quantized."""
+    hk = h if hk is None else hk
+    one = lambda dd, i: dequantize({**dd, "nib": dd["nib"][b, i][None, None], "sf": dd["sf"][b, i][None, None],
+                                    "G": (None if dd["G"] is None else (np.asarray(dd["G"])[b, i] if np.ndim(dd["G"]) else dd["G"]))})[0, 0]
+    return exact_attention(one(qd, h), one(kd, hk), one(vd, hk).T, softmax_scale, rows, causal)
 
 
 def bf16_round(x: np.ndarray) -> np.ndarray:

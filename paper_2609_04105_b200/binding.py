@@ -28,7 +28,7 @@ EXPORTS = [
     "fp4attn_quantize_workspace_bytes", "fp4attn_quantize", "fp4attn_fwd",
     "fp4attn_attention_host_workspace_bytes", "fp4attn_attention_host", "fp4attn_mma_peak_probe",
     "fp4attn_quantize_nvfp4_noalloc", "fp4attn_selftest_bounded_wait", "fp4attn_quantize_mxfp4_rule",
-    "fp4attn_quantize_nvfp4_per_head_workspace_bytes", "fp4attn_quantize_nvfp4_per_head",
+    "fp4attn_quantize_nvfp4_per_head_workspace_bytes", "fp4attn_quantize_nvfp4_per_head", "fp4attn_release",
 ]
 
 
@@ -68,7 +68,9 @@ def _load() -> ctypes.CDLL:
     lib.fp4attn_attention_host_workspace_bytes.restype = sz
     lib.fp4attn_attention_host_workspace_bytes.argtypes = [i, i, i, i, i]
     lib.fp4attn_attention_host.restype = i
-    lib.fp4attn_attention_host.argtypes = [vp, vp, vp, i, ctypes.c_float, i, i, i, i, vp, vp, vp, sz, vp]
+    lib.fp4attn_attention_host.argtypes = [vp, vp, vp, i, ctypes.c_float, i, i, i, i, vp, vp, vp, vp, sz, vp]
+    lib.fp4attn_release.restype = i
+    lib.fp4attn_release.argtypes = []
     lib.fp4attn_quantize_mxfp4_rule.restype = i
     lib.fp4attn_quantize_mxfp4_rule.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp]
     lib.fp4attn_quantize_nvfp4_noalloc.restype = i
@@ -221,14 +223,21 @@ def fp4attn_attention_host_workspace_bytes(qk_fmt: int, B: int, H: int, N: int, 
 
 
 def fp4attn_attention_host(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, qk_fmt: int, out: torch.Tensor,
-                           lse: Optional[torch.Tensor], workspace: torch.Tensor, softmax_scale: float = 0.0) -> None:
+                           lse: Optional[torch.Tensor], workspace: torch.Tensor, softmax_scale: float = 0.0,
+                           status: Optional[torch.Tensor] = None) -> None:
     """Host (pinned) bf16 Q, K, V -> host O (and LSE); copies, quantizers and attention are enqueued
-    on the current stream.  `workspace` is a CUDA uint8 tensor of the queried size."""
-    assert not q.is_cuda and not out.is_cuda and workspace.is_cuda
+    on the current stream.  `workspace` is a CUDA uint8 tensor of the queried size; `status` an optional
+    HOST int32 tensor that receives the call's status word (0, or ERR_TIMEOUT) once the stream is synchronised."""
+    assert not q.is_cuda and not out.is_cuda and workspace.is_cuda and (status is None or not status.is_cuda)
     B, H, N, d = q.shape
     _check(lib().fp4attn_attention_host(q.data_ptr(), k.data_ptr(), v.data_ptr(), qk_fmt, float(softmax_scale),
-                                        B, H, N, d, out.data_ptr(), _ptr(lse), workspace.data_ptr(),
+                                        B, H, N, d, out.data_ptr(), _ptr(lse), _ptr(status), workspace.data_ptr(),
                                         workspace.numel(), _stream()), "fp4attn_attention_host")
+
+
+def fp4attn_release() -> None:
+    """Destroys the host path's internal streams and events and forgets cached tensor maps."""
+    _check(lib().fp4attn_release(), "fp4attn_release")
 
 
 def fp4attn_mma_peak_probe(iters: int, cycles_out: torch.Tensor) -> None:

@@ -34,7 +34,7 @@ extern "C" const char* fp4attn_status_string(int status) {
   }
 }
 
-extern "C" int fp4attn_version(void) { return 100; }
+extern "C" int fp4attn_version(void) { return 200; }
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -87,13 +87,12 @@ void destroy(HostPipe& hp) {
   hp = HostPipe();
 }
 std::mutex g_pipe_mutex;                                        // one pipelined enqueue at a time: the events are shared
+HostPipe g_pipes[fp4attn::kMaxDevices];                         // guarded by g_pipe_mutex
 // caller holds g_pipe_mutex
 HostPipe* host_pipe() {
-  constexpr int kMaxDevices = fp4attn::kMaxDevices;
-  static HostPipe pipes[kMaxDevices];
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-  HostPipe& hp = pipes[dev];
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= fp4attn::kMaxDevices) return nullptr;
+  HostPipe& hp = g_pipes[dev];
   if (!hp.ready) {
     bool ok = cudaStreamCreateWithFlags(&hp.h2d, cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking) == cudaSuccess &&
@@ -109,7 +108,7 @@ HostPipe* host_pipe() {
 }
 int enqueue_groups(HostPipe* hp, int groups, const void* q_host, const void* k_host, const void* v_host, float softmax_scale,
                    int BH, int N, int d, void* O_host, float* LSE_host, char* ws, const HostPlan& p, size_t workspace_bytes,
-                   cudaStream_t st) {
+                   int* dev_status, cudaStream_t st) {
   const size_t head_elems = (size_t)N * d;
   const size_t sfq_head = fp4attn_scale_bytes(FP4ATTN_FMT_MXFP4, FP4ATTN_ROLE_Q, 1, 1, N, d);
   const size_t sfv_head = fp4attn_scale_bytes(FP4ATTN_FMT_MXFP4, FP4ATTN_ROLE_V, 1, 1, N, d);
@@ -138,7 +137,7 @@ int enqueue_groups(HostPipe* hp, int groups, const void* q_host, const void* k_h
     ops.q_sf = ws + p.sf[0] + h0 * sfq_head; ops.k_sf = ws + p.sf[1] + h0 * sfq_head; ops.v_sf = ws + p.sf[2] + h0 * sfv_head;
     ops.qk_fmt = FP4ATTN_FMT_MXFP4;
     ops.softmax_scale = softmax_scale;
-    const int rc = fp4attn_fwd(&ops, 1, nh, N, d, ws + p.O + h0 * head_elems * 2, (float*)(ws + p.LSE) + (size_t)h0 * N, nullptr,
+    const int rc = fp4attn_fwd(&ops, 1, nh, N, d, ws + p.O + h0 * head_elems * 2, (float*)(ws + p.LSE) + (size_t)h0 * N, dev_status,
                                (fp4attn_stream_t)st);
     if (rc != FP4ATTN_OK) return rc;
     FP4ATTN_CUDA_OK(cudaEventRecord(hp->done[c], st));
@@ -154,7 +153,7 @@ int enqueue_groups(HostPipe* hp, int groups, const void* q_host, const void* k_h
 }
 int attention_host_pipelined(const void* q_host, const void* k_host, const void* v_host, float softmax_scale, int B, int H,
                              int N, int d, void* O_host, float* LSE_host, char* ws, const HostPlan& p,
-                             size_t workspace_bytes, cudaStream_t st) {
+                             size_t workspace_bytes, int* dev_status, cudaStream_t st) {
   const int BH = B * H;
   const int groups = BH < 8 ? 1 : (BH < 2 * kMaxGroups ? 4 : 8);   // (16 groups measured slower than 8: more, smaller copies)
   if (groups == 1) return kNoPipeline;
@@ -165,7 +164,7 @@ int attention_host_pipelined(const void* q_host, const void* k_host, const void*
       cudaStreamWaitEvent(hp->h2d, hp->start, 0) != cudaSuccess || cudaStreamWaitEvent(hp->d2h, hp->start, 0) != cudaSuccess)
     return FP4ATTN_ERR_CUDA;
   const int rc = enqueue_groups(hp, groups, q_host, k_host, v_host, softmax_scale, BH, N, d, O_host, LSE_host, ws, p,
-                                workspace_bytes, st);
+                                workspace_bytes, dev_status, st);
   // join on every exit, also a failed one: whatever reached the internal streams stays ordered before the
   // caller's later work on its stream (which may reuse the workspace and the host buffers)
   bool joined = cudaEventRecord(hp->end, hp->h2d) == cudaSuccess && cudaStreamWaitEvent(st, hp->end, 0) == cudaSuccess;
@@ -179,9 +178,21 @@ extern "C" size_t fp4attn_attention_host_workspace_bytes(int qk_fmt, int B, int 
   return plan(qk_fmt, B, H, N, d, &p) ? p.total : 0;
 }
 
+// The status word of the host path lives in the 256-byte slot of the workspace that also holds the two
+// NVFP4 encode factors (floats 0 and 1); it is cleared on the caller's stream before the first kernel of the
+// call and handed to every attention launch of the call.
+static int* host_status_word(char* ws, const HostPlan& p) { return reinterpret_cast<int*>(ws + p.G + 64); }
+
+static int finish_host_call(int rc, int* dev_status, int* status_host, cudaStream_t st) {
+  if (rc == FP4ATTN_OK && status_host &&
+      cudaMemcpyAsync(status_host, dev_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return FP4ATTN_ERR_CUDA;
+  return rc;
+}
+
 extern "C" int fp4attn_attention_host(const void* q_host, const void* k_host, const void* v_host, int qk_fmt,
                                       float softmax_scale, int B, int H, int N, int d, void* O_host,
-                                      float* LSE_host, void* workspace, size_t workspace_bytes,
+                                      float* LSE_host, int* status_host, void* workspace, size_t workspace_bytes,
                                       fp4attn_stream_t stream) {
   if (!q_host || !k_host || !v_host || !O_host) return FP4ATTN_ERR_INVALID_ARG;
   if (qk_fmt != FP4ATTN_FMT_MXFP4 && qk_fmt != FP4ATTN_FMT_NVFP4) return FP4ATTN_ERR_INVALID_ARG;
@@ -193,10 +204,12 @@ extern "C" int fp4attn_attention_host(const void* q_host, const void* k_host, co
   char* ws = (char*)workspace;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t elems = (size_t)B * H * N * d;
+  int* dev_status = host_status_word(ws, p);
+  if (cudaMemsetAsync(dev_status, 0, sizeof(int), st) != cudaSuccess) return FP4ATTN_ERR_CUDA;
   if (qk_fmt == FP4ATTN_FMT_MXFP4) {
     const int rc = attention_host_pipelined(q_host, k_host, v_host, softmax_scale, B, H, N, d, O_host, LSE_host, ws, p,
-                                            workspace_bytes, st);
-    if (rc != kNoPipeline) return rc;
+                                            workspace_bytes, dev_status, st);
+    if (rc != kNoPipeline) return finish_host_call(rc, dev_status, status_host, st);
   }
   const void* src[3] = {q_host, k_host, v_host};
   for (int i = 0; i < 3; ++i)
@@ -216,11 +229,28 @@ extern "C" int fp4attn_attention_host(const void* q_host, const void* k_host, co
   ops.k_G = qk_fmt == FP4ATTN_FMT_NVFP4 ? G + 1 : nullptr;
   ops.qk_fmt = qk_fmt;
   ops.softmax_scale = softmax_scale;
-  int rc = fp4attn_fwd(&ops, B, H, N, d, ws + p.O, (float*)(ws + p.LSE), nullptr, stream);
+  int rc = fp4attn_fwd(&ops, B, H, N, d, ws + p.O, (float*)(ws + p.LSE), dev_status, stream);
   if (rc != FP4ATTN_OK) return rc;
   if (cudaMemcpyAsync(O_host, ws + p.O, elems * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FP4ATTN_ERR_CUDA;
   if (LSE_host &&
       cudaMemcpyAsync(LSE_host, ws + p.LSE, (size_t)B * H * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return FP4ATTN_ERR_CUDA;
-  return FP4ATTN_OK;
+  return finish_host_call(FP4ATTN_OK, dev_status, status_host, st);
+}
+
+namespace fp4attn { void drop_tensor_map_cache(); }
+
+extern "C" int fp4attn_release(void) {
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  int prev = 0;
+  const bool have_dev = cudaGetDevice(&prev) == cudaSuccess;
+  bool ok = true;
+  for (int dev = 0; dev < fp4attn::kMaxDevices; ++dev) {
+    if (!g_pipes[dev].ready) continue;
+    ok = cudaSetDevice(dev) == cudaSuccess && ok;
+    destroy(g_pipes[dev]);
+  }
+  if (have_dev) cudaSetDevice(prev);
+  fp4attn::drop_tensor_map_cache();
+  return ok ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }

@@ -142,7 +142,7 @@ __device__ __forceinline__ WorkItem decode_item(int item, const AttnParams& p, i
 
 // barrier slots (8 bytes each)
 enum { BAR_QFULL0 = 0, BAR_QFREE0 = 2, BAR_OFULL = 4, BAR_OFREE = 5, BAR_SFULL0 = 6, BAR_SEMPTY0 = 8,
-       BAR_PFULL0 = 10, BAR_PFREE0 = 12, BAR_SMDONE0 = 14, BAR_RING = 16 };
+       BAR_PFULL0 = 10, BAR_PFREE0 = 12, BAR_SMDONE0 = 14, BAR_DRAIN0 = 16, BAR_RING = 18 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -184,6 +184,9 @@ __device__ __forceinline__ void fma2(float s0, float s1, float c, float b, float
 #ifndef FP4ATTN_POLY_MASK
 #define FP4ATTN_POLY_MASK 0x8421u      // which of a block's 16 element pairs take the polynomial path
 #endif
+// The header states which pairs take which evaluation (fp4attn.h, FP4ATTN_PMAP_IDEAL); a build with another
+// pattern would change codes within rounding distance of a boundary, so it has to change that text as well.
+static_assert(FP4ATTN_POLY_MASK == 0x8421u, "the pattern of polynomial pairs is part of the documented behaviour");
 __device__ __forceinline__ uint64_t pack2(float a, float b) {
   uint64_t r;
   asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
@@ -296,6 +299,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     mbar_init(bar(BAR_OFULL), 1);
     mbar_init(bar(BAR_OFREE), 4);
+    mbar_init(bar(BAR_DRAIN0), 1);             // time-out path only: one per tensor-core issuer
+    mbar_init(bar(BAR_DRAIN0 + 1), 1);
     for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
     *abortf = 0;
     fence_barrier_init();
@@ -408,6 +413,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (++sq == C::NST) { sq = 0; phq ^= 1; stq = sbase + C::OFF_STAGE; }
       }
     }
+    if (*abortf && elect_one()) tc_commit(bar(BAR_DRAIN0));      // completes when this warp's products and copies have
     __syncwarp();
   } else if (warp == 2) {
     // ===================================================================== PV issuer: O += P V, one stage per issue
@@ -460,6 +466,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (++sp == C::NST) { sp = 0; stp = sbase + C::OFF_STAGE; }
       }
     }
+    if (*abortf && elect_one()) tc_commit(bar(BAR_DRAIN0 + 1));
     __syncwarp();
   } else if (warp < kFirstSoftmaxWarp) {
     // ===================================================================== correction warps
@@ -685,6 +692,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __syncthreads();
   if (*abortf && threadIdx.x == 0 && p.status) *p.status = FP4ATTN_ERR_TIMEOUT;
   if (warp == 1) {
+    if (*abortf && lane == 0) {
+      // time-out path: the issuers may have left with products or scale copies in flight; give them a bounded
+      // time to finish before tensor memory and shared memory are given up
+      for (int r = 0; r < 2; ++r)
+        for (int spin = 0; spin < (1 << 14) && !mbar_try_wait(bar(BAR_DRAIN0 + r), 0); ++spin) {}
+    }
+    __syncwarp();
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
@@ -769,6 +783,49 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint6
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The four tensor maps of a launch depend only on the operand and output addresses and the shape, and encoding
+// them costs more host time than launching a short kernel, so each host thread remembers the maps of its last
+// few distinct calls (a map holds addresses and extents, no reference to the memory: a stale entry is harmless
+// and is simply never matched again).
+struct MapKey {
+  const void *q, *k, *v, *o;
+  int B, H, Hkv, N, D;
+  bool operator==(const MapKey& r) const {
+    return q == r.q && k == r.k && v == r.v && o == r.o && B == r.B && H == r.H && Hkv == r.Hkv && N == r.N && D == r.D;
+  }
+};
+struct MapEntry {
+  MapKey key;
+  unsigned long long epoch;             // value of g_map_epoch when the entry was made; 0 = empty
+  alignas(64) CUtensorMap tm[4];
+};
+constexpr int kMapCacheEntries = 8;
+static std::atomic<unsigned long long> g_map_epoch{1};          // bumped by fp4attn_release: older entries are dead
+static thread_local MapEntry t_maps[kMapCacheEntries];
+static thread_local unsigned t_map_next = 0;
+void drop_tensor_map_cache() { g_map_epoch.fetch_add(1, std::memory_order_acq_rel); }
+
+template <int D>
+static const CUtensorMap* tensor_maps(const fp4attn_operands* ops, void* O, int B, int H, int Hkv, int N) {
+  constexpr int ROW_BYTES = D / 2;
+  const MapKey key{ops->q, ops->k, ops->v, O, B, H, Hkv, N, D};
+  const unsigned long long epoch = g_map_epoch.load(std::memory_order_acquire);
+  for (int i = 0; i < kMapCacheEntries; ++i)
+    if (t_maps[i].epoch == epoch && t_maps[i].key == key) return t_maps[i].tm;
+  MapEntry& e = t_maps[t_map_next];
+  e.epoch = 0;
+  const uint64_t rows = (uint64_t)B * H * N, kv_rows = (uint64_t)B * Hkv * N;
+  if (!make_map(&e.tm[0], ops->q, ROW_BYTES, rows, ROW_BYTES, BM) ||
+      !make_map(&e.tm[1], ops->k, ROW_BYTES, kv_rows, ROW_BYTES, BS) ||
+      !make_map(&e.tm[2], ops->v, (uint64_t)N / 2, (uint64_t)B * Hkv * D, BS / 2, D) ||
+      !make_map(&e.tm[3], O, (uint64_t)D * 2, rows, 128, 32))
+    return nullptr;
+  e.key = key;
+  e.epoch = epoch;
+  t_map_next = (t_map_next + 1) % kMapCacheEntries;
+  return e.tm;
+}
+
 template <int D, int NV, int PMAP, bool CAUSAL, bool THR16>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
   const int Hkv = prm.Hkv;
@@ -784,15 +841,10 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
       return FP4ATTN_ERR_CUDA;
     attr_set[dev].store(true, std::memory_order_release);
   }
-  CUtensorMap tmQ, tmK, tmV, tmO;
-  const uint64_t rows = (uint64_t)B * H * N, kv_rows = (uint64_t)B * Hkv * N;
-  if (!make_map(&tmQ, ops->q, C::ROW_BYTES, rows, C::ROW_BYTES, BM) ||
-      !make_map(&tmK, ops->k, C::ROW_BYTES, kv_rows, C::ROW_BYTES, BS) ||
-      !make_map(&tmV, ops->v, (uint64_t)N / 2, (uint64_t)B * Hkv * D, BS / 2, D) ||
-      !make_map(&tmO, prm.O, (uint64_t)D * 2, rows, 128, 32))
-    return FP4ATTN_ERR_CUDA;
+  const CUtensorMap* tm = tensor_maps<D>(ops, prm.O, B, H, Hkv, N);
+  if (!tm) return FP4ATTN_ERR_CUDA;
   const unsigned grid = (unsigned)(prm.n_items < sms ? prm.n_items : sms);     // persistent: one CTA per SM
-  attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tmQ, tmK, tmV, tmO, prm);
+  attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tm[0], tm[1], tm[2], tm[3], prm);
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
 

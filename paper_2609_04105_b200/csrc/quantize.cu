@@ -445,13 +445,15 @@ extern "C" int fp4attn_quantize_nvfp4_noalloc(const void* x, int role, int B, in
   if (rc != FP4ATTN_OK) return rc;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return FP4ATTN_ERR_CUDA;
-  static float* scratch_addr[kMaxDevices] = {};          // per-device address of g_noalloc_partials
+  // per-device address of g_noalloc_partials; several host threads may make the first call on a device at
+  // once (they all store the same address)
+  static std::atomic<float*> scratch_addr[kMaxDevices];
   if (dev < 0 || dev >= kMaxDevices) return FP4ATTN_ERR_INVALID_ARG;
-  if (!scratch_addr[dev]) {
-    float* ptr = nullptr;
-    if (cudaGetSymbolAddress((void**)&ptr, g_noalloc_partials) != cudaSuccess || !ptr) return FP4ATTN_ERR_CUDA;
-    scratch_addr[dev] = ptr;
+  float* scratch = scratch_addr[dev].load(std::memory_order_acquire);
+  if (!scratch) {
+    if (cudaGetSymbolAddress((void**)&scratch, g_noalloc_partials) != cudaSuccess || !scratch) return FP4ATTN_ERR_CUDA;
+    scratch_addr[dev].store(scratch, std::memory_order_release);
   }
-  return launch_quantize(x, FP4ATTN_FMT_NVFP4, role, B, H, N, d, packed, scales, G_out, scratch_addr[dev],
+  return launch_quantize(x, FP4ATTN_FMT_NVFP4, role, B, H, N, d, packed, scales, G_out, scratch,
                          (cudaStream_t)stream, FP4ATTN_QSCALE_CEIL);
 }

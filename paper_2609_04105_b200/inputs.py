@@ -86,20 +86,22 @@ def outlier_channels(w: Workload) -> np.ndarray:
     return np.stack([np.sort(rng.choice(w.d, size=k, replace=False)) for _ in range(w.H)])
 
 
-def make_qkv(w: Workload, heads=None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
-    """bf16 bit patterns of Q, K, V, each [B, H, N, d] (uint16).
+def make_operand_f32(w: Workload, t: int) -> np.ndarray:
+    """The float32 draw of operand t (0 = Q, 1 = K, 2 = V) before rounding to bfloat16, [B, H, N, d].
 
     Streams: Q seed = BASE_SEED + 10*cfg, K = +1, V = +2, outlier channels = +3.
     """
-    shape = (w.B, w.H, w.N, w.d)
-    out = []
-    for t in range(3):
-        x = _normal_bf16(BASE_SEED + 10 * w.cfg + t, shape)
-        if w.outliers and t < 2:
-            ch = outlier_channels(w)
-            for h in range(w.H):
-                x[:, h, :, ch[h]] *= np.float32(20.0)
-        out.append(f32_to_bf16_bits(x))
+    x = _normal_bf16(BASE_SEED + 10 * w.cfg + t, (w.B, w.H, w.N, w.d))
+    if w.outliers and t < 2:
+        ch = outlier_channels(w)
+        for h in range(w.H):
+            x[:, h, :, ch[h]] *= np.float32(20.0)
+    return x
+
+
+def make_qkv(w: Workload, heads=None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """bf16 bit patterns of Q, K, V, each [B, H, N, d] (uint16): make_operand_f32 rounded to nearest even."""
+    out = [f32_to_bf16_bits(make_operand_f32(w, t)) for t in range(3)]
     return out[0], out[1], out[2]
 
 

@@ -96,41 +96,58 @@ def test_run_to_run_determinism():
     assert np.array_equal(O1, O2) and np.array_equal(L1, L2)
 
 
-def _sampled_case(name, n_rows, n_heads, seed):
+def _full_size_case(name, n_rows, n_heads, seed, whole_heads=0):
+    """One launch of a whole configuration as bench.py launches it.  `n_heads` (batch, head) units are compared on
+    `n_rows` sampled query rows each, and `whole_heads` further units on ALL their rows under the protocol for
+    outputs with more than one correct value (tests/parity.py); the statistics of those are printed."""
+    import parity
     w = I.WORKLOADS[name]
     q, k, v = I.make_qkv(w)
     Og, Lg = run_gpu(w, q, k, v)
     qd, kd, vd = oracle_operands(w, q, k, v)
     rng = np.random.default_rng(seed)
-    rows = np.sort(rng.choice(w.N, size=n_rows, replace=False))
-    rows[0], rows[-1] = 0, w.N - 1
     all_heads = [(b, h) for b in range(w.B) for h in range(w.H)]
-    pick = rng.choice(len(all_heads), size=min(n_heads, len(all_heads)), replace=False)
-    heads = [all_heads[i] for i in sorted(pick)]
-    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows)
-    return check_heads(Og, Lg, Oo, Lo, heads, rows)
+    pick = [all_heads[i] for i in rng.choice(len(all_heads), size=min(n_heads + whole_heads, len(all_heads)), replace=False)]
+    if n_heads:
+        rows = np.sort(rng.choice(w.N, size=n_rows, replace=False))
+        rows[0], rows[-1] = 0, w.N - 1
+        heads = sorted(pick[:n_heads])
+        Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows)
+        check_heads(Og, Lg, Oo, Lo, heads, rows)
+    for (b, h) in pick[n_heads:]:
+        st = parity.compare_head(Og[b, h], Lg[b, h], qd, kd, vd, b, h)
+        print(f"{name} whole head: {st}")
+        assert st["lse_err"] <= 1e-3 or st["rows_failing_strict"] > 0, st
 
 
-def test_config2_full_size_sampled_rows():
-    """B4 H16 N4096 d128 as bench.py launches it; 8 heads x 256 sampled query rows vs the oracle."""
-    _sampled_case("cfg2", 256, 8, 2)
+def test_config2_full_size_sampled_rows_and_whole_heads():
+    """B4 H16 N4096 d128 as bench.py launches it; 8 heads x 256 sampled query rows and 2 whole heads."""
+    _full_size_case("cfg2", 256, 8, 2, whole_heads=2)
 
 
-def test_config3_full_size_sampled_rows():
-    """B8 H16 N8192 d64, NVFP4 Q/K; 4 heads x 128 sampled rows."""
-    _sampled_case("cfg3", 128, 4, 3)
+def test_config3_full_size_sampled_rows_and_whole_heads():
+    """B8 H16 N8192 d64, NVFP4 Q/K (scores are sums float32 cannot always hold); 4 heads x 128 sampled rows and
+    2 whole heads (all 8192 rows)."""
+    _full_size_case("cfg3", 128, 4, 3, whole_heads=2)
 
 
-def test_config4_full_size_sampled_rows():
-    """B1 H32 N16384 d128 with x20 outlier channels (|y| ~ 300: moving reference, zero blocks);
-    3 heads x 96 sampled rows."""
-    _sampled_case("cfg4", 96, 3, 4)
+def test_config4_full_size_sampled_rows_and_whole_heads():
+    """B1 H32 N16384 d128 with x20 outlier channels (|y| ~ 300: moving reference, zero blocks, near one-hot
+    rows where one code decision can move an output row); 3 heads x 96 sampled rows and 2 whole heads (all
+    16384 rows)."""
+    _full_size_case("cfg4", 96, 3, 4, whole_heads=2)
 
 
-@pytest.mark.parametrize("N", [1024, 8192, 32768])
+@pytest.mark.parametrize("N", [1024, 2048, 4096, 8192, 16384])
 def test_config5_sweep_full_size_sampled_rows(N):
-    """Sequence sweep at B*N = 32768 tokens, H=16, d=128: shortest, middle and longest point."""
-    _sampled_case(f"cfg5_N{N}", 128 if N < 32768 else 64, 8 if N < 32768 else 2, 5)
+    """Sequence sweep at B*N = 32768 tokens, H=16, d=128: every point below the longest on sampled rows."""
+    _full_size_case(f"cfg5_N{N}", 128 if N < 16384 else 96, 8 if N < 8192 else 4, 5)
+
+
+def test_config5_longest_sequence_whole_head():
+    """N = 32768 (B=1, H=16, d=128), the workload bench.py times: one whole head (all 32768 rows) and sampled rows
+    of two more."""
+    _full_size_case("cfg5_N32768", 64, 2, 5, whole_heads=1)
 
 
 @pytest.mark.parametrize("kw", [dict(N=512), dict(B=3, H=8, N=256), dict(B=2, H=17, N=128)])
@@ -144,13 +161,17 @@ def test_host_buffer_entry_point_matches_device_path(kw):
     Og, Lg = run_gpu(w, q, k, v)
     host = [torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory() for a in (q, k, v)]
     ws = torch.empty(Bd.fp4attn_attention_host_workspace_bytes(w.qk_fmt, w.B, w.H, w.N, w.d), dtype=torch.uint8, device="cuda")
-    for _ in range(2):
+    for rep in range(3):
         out = torch.zeros((w.B, w.H, w.N, w.d), dtype=torch.bfloat16).pin_memory()
         lse = torch.zeros((w.B, w.H, w.N), dtype=torch.float32).pin_memory()
-        Bd.fp4attn_attention_host(host[0], host[1], host[2], w.qk_fmt, out, lse, ws)
+        st = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+        Bd.fp4attn_attention_host(host[0], host[1], host[2], w.qk_fmt, out, lse, ws, status=st)
         torch.cuda.synchronize()
+        assert int(st[0]) == 0                                  # the call's status word: no bounded wait ran out
         assert np.array_equal(out.float().numpy().astype(np.float64), Og)
         assert np.array_equal(lse.numpy().astype(np.float64), Lg)
+        if rep == 1:
+            Bd.fp4attn_release()                                # internal streams, events, tensor maps: made again on the next call
 
 
 def test_host_buffer_entry_point_from_two_threads():
@@ -191,6 +212,29 @@ def test_host_buffer_entry_point_from_two_threads():
     for w, host, ws, out, lse, Og, Lg, _ in jobs:
         assert np.array_equal(out.float().numpy().astype(np.float64), Og)
         assert np.array_equal(lse.numpy().astype(np.float64), Lg)
+
+
+def test_cached_tensor_maps_follow_the_buffers():
+    """The library remembers the tensor maps of a thread's last few calls by operand address and shape.  Calls
+    that alternate between two operand sets and two output buffers, more distinct calls than the cache holds,
+    and a call after fp4attn_release() must each read and write the buffers they were given."""
+    from paper_2609_04105_b200 import binding as Bd
+    sets = []
+    for i, kw in enumerate((dict(N=256), dict(N=384), dict(N=256, H=3))):
+        w = I.shrink(I.WORKLOADS["cfg1"], **kw)
+        q, k, v = I.make_qkv(I.shrink(w, cfg=w.cfg + i))
+        ops = [Bd.fp4attn_quantize(_dev(a), Bd.FMT_MXFP4, r) for a, r in ((q, Bd.ROLE_Q), (k, Bd.ROLE_K), (v, Bd.ROLE_V))]
+        ref, _ = Bd.fp4attn_fwd(*ops)
+        sets.append((ops, ref.clone()))
+    outs = [torch.zeros_like(sets[j % 3][1]) for j in range(12)]          # twelve distinct output buffers > cache entries
+    for rnd in range(2):
+        for j, o in enumerate(outs):
+            o.zero_()
+            Bd.fp4attn_fwd(*sets[j % 3][0], out=o)
+        torch.cuda.synchronize()
+        for j, o in enumerate(outs):
+            assert torch.equal(o, sets[j % 3][1]), (rnd, j)
+        Bd.fp4attn_release()
 
 
 def test_invalid_arguments_are_rejected_before_launch():

@@ -425,3 +425,129 @@ def test_per_head_nvfp4_factors_make_attention_invariant_to_head_scaling():
         Oe, _ = A.exact_attention(Qz.bf16_bits_to_f64(q3)[0, h], Qz.bf16_bits_to_f64(k3)[0, h], V[0, h])
         cos = float((O3[h] * Oe).sum() / np.linalg.norm(O3[h]) / np.linalg.norm(Oe))
         assert cos > 0.95, (h, cos)
+
+
+# ------------------------------------------------------------------ several results can be correct
+def _plain_definition(y, E_B, codes, V):
+    """Eq. "represented-output" written out for one row, Python floats: p~_j = 2**E_B(j) * value(code_j) / 6."""
+    vals = [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+    top = max(E_B)
+    num = [0.0] * V.shape[1]
+    den = 0.0
+    for j in range(len(y)):
+        p = 2.0 ** (E_B[j // 32] - top) * vals[codes[j]] / 6.0
+        den += p
+        for c in range(V.shape[1]):
+            num[c] += p * float(V[j, c])
+    return np.array(num) / den, math.log(2.0) * (top + math.log2(den))
+
+
+@pytest.mark.parametrize("k", range(7))
+def test_score_on_a_code_boundary_is_reported_and_can_be_taken_either_way(k):
+    """One key of a row sits (to float32 precision) on boundary t_k of Eq. "e2m1-boundaries": the report lists
+    exactly that element, and flipping it moves exactly that code to its neighbour; both outputs equal the
+    plain definition evaluated with the respective code."""
+    t = float(F.E2M1_BOUNDARIES[k])
+    rng = np.random.default_rng(40 + k)
+    N, d = 64, 5
+    y = (-rng.uniform(0.05, 2.2, size=(1, N))).astype(np.float32)
+    y[0, 0] = y[0, 32] = 0.0                                       # both blocks: maximum 0 -> E_B = 0 (an integer: see the next test)
+    j = 7
+    y[0, j] = np.float32(math.log2(t / 6.0))                       # 2**(y - 0 + log2 6) = t up to float32 rounding
+    # keep every other element away from a boundary, so that the one planted is the only near-decision
+    for jj in range(N):
+        if jj not in (0, 32, j):
+            while np.min(np.abs(6.0 * 2.0 ** float(y[0, jj]) / F.E2M1_BOUNDARIES - 1.0)) < 1e-3:
+                y[0, jj] -= np.float32(0.01)
+    V = rng.standard_normal((N, d))
+    rep = {}
+    O, lse, codes, EB, _ = A.direct_p_rows(y, np.float32(1.0), V, tile=32, report=rep, ambiguity=dict(ulps=0.0))
+    assert rep["code"].sum() == 1 and rep["code"][0, j] and rep["row"][0]
+    assert codes[0, j] in (k, k + 1)
+    flip = np.zeros((1, N), dtype=bool)
+    flip[0, j] = True
+    O2, lse2, codes2, EB2, _ = A.direct_p_rows(y, np.float32(1.0), V, tile=32, flips={"code": flip})
+    assert codes2[0, j] == 2 * k + 1 - codes[0, j]
+    assert np.array_equal(np.delete(codes2[0], j), np.delete(codes[0], j)) and np.array_equal(EB, EB2)
+    for o, l, c in ((O, lse, codes), (O2, lse2, codes2)):
+        od, ld = _plain_definition(y[0], [0, 0], c[0], V)
+        assert np.abs(o[0] - od).max() < 1e-14 and abs(l[0] - ld) < 1e-13
+    assert np.abs(O2 - O).max() > 1e-4                             # the decision is visible in the output
+
+
+@pytest.mark.parametrize("p_scale,w0", [("ceil", 3.0), ("thr16", 5.0)])
+def test_integer_block_maximum_is_reported_and_can_be_taken_either_way(p_scale, w0):
+    """A block whose rounded quantity (max y, or fl32(max y + log2 1.6) under the threshold rule) is an integer
+    up to a float32 spacing: reported as an exponent near-decision; flipped, the block takes the integer on the
+    other side and all its codes follow from it (plain definition with that exponent)."""
+    rng = np.random.default_rng(50)
+    N, d = 96, 4
+    y = rng.uniform(-3.0, 1.5, size=(1, N)).astype(np.float32)
+    ymax = np.float32(w0) if p_scale == "ceil" else np.float32(np.float32(w0) - A.LOG2_1P6_32)
+    y[0, 40] = ymax                                                # block 1
+    V = rng.standard_normal((N, d))
+    rep = {}
+    O, lse, codes, EB, _ = A.direct_p_rows(y, np.float32(1.0), V, tile=32, p_scale=p_scale, report=rep)
+    assert rep["eb"].tolist() == [[False, True, False]] and rep["row"][0]
+    fl = np.zeros((1, 3), dtype=bool)
+    fl[0, 1] = True
+    O2, lse2, codes2, EB2, _ = A.direct_p_rows(y, np.float32(1.0), V, tile=32, p_scale=p_scale, flips={"eb": fl})
+    assert abs(int(EB2[0, 1]) - int(EB[0, 1])) == 1 and EB2[0, 0] == EB[0, 0] and EB2[0, 2] == EB[0, 2]
+    assert {int(EB[0, 1]), int(EB2[0, 1])} == ({3, 4} if p_scale == "ceil" else {4, 5})
+    for o, l, c, e in ((O, lse, codes, EB), (O2, lse2, codes2, EB2)):
+        want = F.e2m1_encode_mag(6.0 * 2.0 ** (y[0].astype(np.float64) - np.repeat(e[0], 32)))
+        assert np.array_equal(c[0], want)
+        od, ld = _plain_definition(y[0], list(e[0]), c[0], V)
+        assert np.abs(o[0] - od).max() < 1e-14 and abs(l[0] - ld) < 1e-13
+
+
+def test_near_decisions_without_visible_weight_are_not_reported_and_no_flip_changes_nothing():
+    """A boundary score in a block 2**-40 below the row maximum carries no visible weight: not reported.
+    Empty flip masks reproduce the default evaluation bit for bit; on Gaussian operands reports are rare."""
+    N, d = 64, 3
+    y = np.full((1, N), -1.3, dtype=np.float32)
+    y[0, 0] = 0.0
+    y[0, 32:] -= 40.0
+    y[0, 32] = -40.0
+    y[0, 50] = np.float32(-40.0 + math.log2(2.5 / 6.0))            # on a boundary, but 2**-40 of the row
+    V = np.random.default_rng(1).standard_normal((N, d))
+    rep = {}
+    A.direct_p_rows(y, np.float32(1.0), V, tile=32, report=rep, ambiguity=dict(ulps=0.0))
+    assert not rep["code"].any()
+    rep2 = {}
+    A.direct_p_rows(y, np.float32(1.0), V, tile=32, report=rep2, ambiguity=dict(ulps=0.0, share=0.0))
+    assert rep2["code"][0, 50] and rep2["code"].sum() == 1
+
+    w, _, qd, kd, vd = _cfg1(N=512)
+    c32 = A.score_constant(qd, kd, w.d)
+    s32 = A.scores_fp32(qd, kd, 0, 0)
+    Vhat = np.ascontiguousarray(Qz.dequantize({**vd, "nib": vd["nib"][0, 0][None, None], "sf": vd["sf"][0, 0][None, None]})[0, 0].T)
+    rep3 = {}
+    base = A.direct_p_rows(s32, c32, Vhat, report=rep3)
+    none = A.direct_p_rows(s32, c32, Vhat, flips={"code": np.zeros(s32.shape, bool), "eb": np.zeros((512, 16), bool)})
+    for a, b in zip(base, none):
+        assert np.array_equal(a, b)
+    # FP4 operands make scores discrete (a score of exactly 0 under E_B = 3 gives 2**x = 0.75, a boundary), so
+    # near-decisions are not rare per row, but they are per element, and every one reported is within the
+    # stated distance of a boundary when recomputed from the returned block exponents
+    assert rep3["code"].mean() < 2e-3 and not rep3["eb"].any()
+    i, j = np.nonzero(rep3["code"])
+    v = 6.0 * 2.0 ** (s32[i, j].astype(np.float64) * float(c32) - base[3][i, j // 32])
+    assert np.all(np.min(np.abs(v[:, None] / F.E2M1_BOUNDARIES[None, :] - 1.0), axis=1) < 2.0 ** -17)
+    assert np.any(s32[i, j] == 0)
+
+
+def test_exact_p_output_sits_between_direct_p_and_unquantized_attention():
+    """O_exactP (quantized Q, K, V, exact softmax) is what is left when P is not quantized: it equals exact
+    attention on the reconstructed operands, and is closer to unquantized attention than Direct-P is."""
+    w, (q, k, v), qd, kd, vd = _cfg1(N=512)
+    Oe, _ = A.exact_p_attention(qd, kd, vd, 0, 1)
+    Qh, Kh, Vh = (Qz.dequantize(qd)[0, 1], Qz.dequantize(kd)[0, 1], Qz.dequantize(vd)[0, 1].T)
+    z = Qh @ Kh.T / math.sqrt(w.d)
+    p = np.exp(z - z.max(axis=1, keepdims=True))
+    assert np.abs(Oe - (p / p.sum(axis=1, keepdims=True)) @ Vh).max() < 1e-13
+    x = [Qz.bf16_bits_to_f64(a[0, 1]) for a in (q, k, v)]
+    O64, _ = A.exact_attention(*x)
+    Od, _ = A.direct_p_forward(qd, kd, vd, heads=[(0, 1)])
+    rel = lambda a: np.linalg.norm(a - O64) / np.linalg.norm(O64)
+    assert rel(Oe) < rel(Od[0]) and 0.15 < rel(Oe) < 0.26 and 0.22 < rel(Od[0]) < 0.32

@@ -80,6 +80,24 @@ def test_full_size_quantizer_sampled(tmp_path):
     _check_operand(got, Qz.quantize_v(v), Bd.ROLE_V)
 
 
+def test_full_size_nvfp4_quantizer_all_bytes():
+    """Config 3's full Q tensor (B8 H16 N8192 d64: 2^26 elements, 2^23 sixteen-byte groups, so every block of
+    the tensor-wide amax pass walks its strided loop several times): encode factor, every scale byte and
+    every code against the oracle; then the per-(batch, head) variant on the same tensor."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.WORKLOADS["cfg3"]
+    q, _, _ = I.make_qkv(w)
+    x = _dev(q)
+    got = Bd.fp4attn_quantize(x, Bd.FMT_NVFP4, Bd.ROLE_Q)
+    _check_operand(got, Qz.quantize_qk(q, "nv"), Bd.ROLE_Q)
+    got = Bd.fp4attn_quantize_nvfp4_per_head(x, Bd.ROLE_Q)
+    want = Qz.quantize_qk(q, "nv", per_head=True)
+    assert np.array_equal(got.G.cpu().numpy().reshape(w.B, w.H), want["G"])
+    assert np.array_equal(Qz.strip_negative_zero(got.packed.cpu().numpy()),
+                          Qz.strip_negative_zero(Qz.pack_nibbles(want["nib"]).reshape(-1)))
+    assert np.array_equal(got.scales.cpu().numpy(), Qz.swizzle_scales(want["sf"]).reshape(-1))
+
+
 RULES = [("ceil", 0), ("thr16", 1), ("floor", 2), ("mse", 3)]
 
 
@@ -186,3 +204,14 @@ def test_nvfp4_per_head_rejects_v_and_missing_workspace():
     rc = L.fp4attn_quantize_nvfp4_per_head(x.data_ptr(), Bd.ROLE_Q, 1, 2, 128, 64, buf.data_ptr(), buf.data_ptr(),
                                            buf.data_ptr(), None, 0, None)
     assert rc == Bd.ERR_WORKSPACE
+
+
+def test_device_rounding_of_the_seeded_draws_equals_the_host_recipe():
+    """bench.py rounds the seeded float32 draws to bfloat16 on the device; the bits must be those of the host
+    rounding that the tests and the oracle use (round to nearest even), including the scaled outlier channels."""
+    w = I.shrink(I.WORKLOADS["cfg4"], H=2, N=1024)
+    want = I.make_qkv(w)
+    for t in range(3):
+        x = I.make_operand_f32(w, t)
+        got = torch.from_numpy(x).cuda().to(torch.bfloat16).view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(got, want[t])
