@@ -178,6 +178,15 @@ enum { FP4ATTN_PSCALE_CEIL = 0,    /* E_B = ceil(max y): nothing saturates      
        FP4ATTN_PSCALE_THR16 = 1 }; /* E_B = floor(fl32(max y + fl32(log2 1.6))): the block maximum lands in
                                       [3.75, 7.5) code units, values above 6 saturate; lower P error    */
 
+/* how query tiles are assigned to thread blocks (Section "Two-query execution model") */
+enum { FP4ATTN_SCHEDULE_ONE_QUERY = 0,   /* one 128-row query tile per thread block: every shape                 */
+       FP4ATTN_SCHEDULE_TWO_QUERY = 1 }; /* two query tiles of a head share every K / V stage and run as two
+                                            independent chains with an accumulator each.  Exists where tensor
+                                            memory holds two accumulators beside the score slots without overlays:
+                                            d = 64, N a multiple of 256, noncausal, one NVFP4 factor per tensor;
+                                            anything else returns FP4ATTN_ERR_UNSUPPORTED_SHAPE.  Same results, bit
+                                            for bit, as FP4ATTN_SCHEDULE_ONE_QUERY                                */
+
 typedef struct {
   const void *q, *k, *v;            /* packed E2M1 (V transposed)                           */
   const void *q_sf, *k_sf, *v_sf;   /* scale atoms                                           */
@@ -201,6 +210,7 @@ typedef struct {
                                        B*H factors and k_G B*kv_heads, one per (batch, head) unit
                                        (fp4attn_quantize_nvfp4_per_head); with the ideal and the
                                        affine map, not with FP4ATTN_PMAP_HYBRID                 */
+  int schedule;                     /* FP4ATTN_SCHEDULE_ONE_QUERY (0, default) or _TWO_QUERY */
 } fp4attn_operands;
 
 /*

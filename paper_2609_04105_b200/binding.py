@@ -16,6 +16,7 @@ FMT_MXFP4, FMT_NVFP4 = 0, 1
 ROLE_Q, ROLE_K, ROLE_V = 0, 1, 2
 PMAP_IDEAL, PMAP_AFFINE, PMAP_HYBRID = 0, 1, 2
 PSCALE_CEIL, PSCALE_THR16 = 0, 1
+SCHEDULE_ONE_QUERY, SCHEDULE_TWO_QUERY = 0, 1
 QSCALE_CEIL, QSCALE_THR16, QSCALE_FLOOR, QSCALE_MSE = 0, 1, 2, 3
 (OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_ARCH, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA,
  ERR_TIMEOUT) = range(8)
@@ -43,7 +44,7 @@ class _Operands(ctypes.Structure):
                 ("qk_fmt", ctypes.c_int), ("softmax_scale", ctypes.c_float),
                 ("p_map", ctypes.c_int), ("affine_a", ctypes.c_float), ("affine_b", ctypes.c_float),
                 ("p_scale_rule", ctypes.c_int), ("causal", ctypes.c_int), ("kv_heads", ctypes.c_int),
-                ("exact_pairs", ctypes.c_int), ("g_per_head", ctypes.c_int)]
+                ("exact_pairs", ctypes.c_int), ("g_per_head", ctypes.c_int), ("schedule", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:
@@ -197,7 +198,7 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
                 out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
                 status: Optional[torch.Tensor] = None, p_map: int = PMAP_IDEAL, affine_a: float = 0.0,
                 affine_b: float = 0.0, p_scale_rule: int = PSCALE_CEIL, causal: bool = False,
-                exact_pairs: int = 0) -> Tuple[torch.Tensor, torch.Tensor]:
+                exact_pairs: int = 0, schedule: int = SCHEDULE_ONE_QUERY) -> Tuple[torch.Tensor, torch.Tensor]:
     """Direct-P attention forward on quantized operands -> (O bf16 [B,H,N,d], LSE fp32 [B,H,N]).
     p_map selects the exact code map or the affine classifier (affine_a = 0: A = 1.5, B = 1.2)."""
     B, H, N, d = q.shape
@@ -212,7 +213,7 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
     ops = _Operands(q.packed.data_ptr(), k.packed.data_ptr(), v.packed.data_ptr(),
                     q.scales.data_ptr(), k.scales.data_ptr(), v.scales.data_ptr(),
                     _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b), int(p_scale_rule), int(bool(causal)), int(Hkv),
-                    int(exact_pairs), int(q.per_head))
+                    int(exact_pairs), int(q.per_head), int(schedule))
     _check(lib().fp4attn_fwd(ctypes.byref(ops), B, H, N, d, out.data_ptr(), lse.data_ptr(), _ptr(status), _stream()),
            "fp4attn_fwd")
     return out, lse

@@ -602,3 +602,67 @@ def test_row_reference_raises_of_every_size(growth, scale):
     Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows, softmax_scale=scale)
     assert np.isfinite(Og).all() and np.isfinite(Lg).all()
     check_heads(Og, Lg, Oo, Lo, heads, rows)
+
+
+# ------------------------------------------------------------------ two-query schedule (d = 64)
+TWO_QUERY_CASES = [
+    ("cfg3", dict(B=2, H=2, N=512), dict()),                                   # NVFP4 Q/K, exact map
+    ("cfg3", dict(B=1, H=3, N=256), dict(p_map=1)),                            # one tile pair per head, affine map
+    ("cfg3", dict(B=2, H=2, N=1024), dict(p_map=2, exact_pairs=0x5555)),       # mixed map
+    ("cfg1", dict(d=64, N=768, H=5), dict(p_map=1)),                           # MXFP4 Q/K at d = 64, odd number of pairs
+    ("cfg1", dict(d=64, N=512, H=4), dict(p_scale_rule=1)),                    # threshold rule
+    ("cfg4", dict(d=64, H=2, N=1024), dict()),                                 # outlier channels: the row reference moves
+    ("cfg3", dict(B=3, H=40, N=2304), dict(p_map=1)),                          # more tile pairs than one wave of thread blocks
+]
+
+
+@pytest.mark.parametrize("name,kw,okw", TWO_QUERY_CASES)
+def test_two_query_schedule_matches_oracle_and_the_one_query_schedule(name, kw, okw):
+    """Two query tiles per thread block sharing every K/V stage (d = 64): same codes, same accumulation order per
+    row, so the output must equal the one-query schedule's bit for bit, and the oracle within the tolerances."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    O1, L1 = run_gpu_general(w, q, k, v, **okw)
+    O2, L2 = run_gpu_general(w, q, k, v, schedule=Bd.SCHEDULE_TWO_QUERY, **okw)
+    assert np.array_equal(O1, O2) and np.array_equal(L1, L2)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    rng = np.random.default_rng(8)
+    all_heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    heads = [all_heads[i] for i in sorted(rng.choice(len(all_heads), size=min(4, len(all_heads)), replace=False))]
+    rows = np.sort(rng.choice(w.N, size=min(w.N, 256), replace=False))
+    rows[0], rows[-1] = 0, w.N - 1
+    omap = {0: "ideal", 1: "affine", 2: "hybrid"}[okw.get("p_map", 0)]
+    extra = dict(exact_pairs=okw["exact_pairs"]) if "exact_pairs" in okw else {}
+    Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, rows=rows, p_map=omap,
+                                p_scale="thr16" if okw.get("p_scale_rule") else "ceil", **extra)
+    check_heads(O2, L2, Oo, Lo, heads, rows)
+
+
+def test_two_query_schedule_grouped_kv_heads_and_config3_full_size():
+    """Grouped K/V heads under the two-query schedule, and config 3 (B8 H16 N8192 d64) at full size: bit-identical to
+    the one-query launch."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg3"], B=1, H=6, N=512)
+    q, k, v = I.make_qkv(w)
+    k, v = k[:, :2], v[:, :2]
+    O1, L1 = run_gpu_general(w, q, k, v)
+    O2, L2 = run_gpu_general(w, q, k, v, schedule=Bd.SCHEDULE_TWO_QUERY)
+    assert np.array_equal(O1, O2) and np.array_equal(L1, L2)
+    w = I.WORKLOADS["cfg3"]
+    q, k, v = I.make_qkv(w)
+    for okw in (dict(), dict(p_map=Bd.PMAP_AFFINE)):
+        O1, L1 = run_gpu_general(w, q, k, v, **okw)
+        O2, L2 = run_gpu_general(w, q, k, v, schedule=Bd.SCHEDULE_TWO_QUERY, **okw)
+        assert np.array_equal(O1, O2) and np.array_equal(L1, L2)
+
+
+def test_two_query_schedule_rejects_what_it_does_not_cover():
+    from paper_2609_04105_b200 import binding as Bd
+    for kw, okw in ((dict(N=256), dict()),                          # d = 128
+                    (dict(d=64, N=384), dict()),                    # N not a multiple of 256
+                    (dict(d=64, N=512), dict(causal=True))):
+        w = I.shrink(I.WORKLOADS["cfg1"], **kw)
+        q, k, v = I.make_qkv(w)
+        with pytest.raises(Bd.Fp4AttnError):
+            run_gpu_general(w, q, k, v, schedule=Bd.SCHEDULE_TWO_QUERY, **okw)
