@@ -1,0 +1,113 @@
+#!/usr/bin/env python
+"""Every row of every (batch, head) unit of a configuration, CUDA path against the oracle.
+
+The pytest suite compares whole heads of each configuration (a few units each) so that it stays within minutes;
+this script is the same comparison (tests/parity.py: strict figures, and the protocol for rows with more than one
+correct value) over ALL units, for the record.  One launch of the configuration as bench.py launches it, then the
+oracle on a pool of host processes, one unit per task.
+
+  python tests/run_full_parity.py cfg4 [--p-map affine] [--workers 12] [--units 0:32]
+
+Prints one JSON line per unit and a summary line.  Needs a B200; imports the oracle (test infrastructure).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import multiprocessing as mp
+import os
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+from paper_2609_04105_b200 import inputs as I  # noqa: E402
+
+_G = {}
+
+
+def _unit(task):
+    """Oracle operands of one unit from its bf16 bits, then the whole-head comparison."""
+    import parity
+    from oracle import quantize as Qz
+    try:                                                         # one BLAS thread per worker process
+        from threadpoolctl import threadpool_limits
+        threadpool_limits(1)
+    except Exception:
+        pass
+    b, h = task
+    w, q, k, v, Og, Lg, Gq, Gk, okw = (_G[x] for x in ("w", "q", "k", "v", "O", "L", "Gq", "Gk", "okw"))
+    one = lambda a: np.ascontiguousarray(a[b, h][None, None])
+    if w.qk_fmt == I.FMT_NVFP4:
+        nq, sq = Qz.nv_quantize_lastdim(Qz.bf16_bits_to_f64(one(q)), Gq)
+        nk, sk = Qz.nv_quantize_lastdim(Qz.bf16_bits_to_f64(one(k)), Gk)
+        qd = {"nib": nq, "sf": sq, "G": Gq, "fmt": "nv"}
+        kd = {"nib": nk, "sf": sk, "G": Gk, "fmt": "nv"}
+    else:
+        qd, kd = Qz.quantize_qk(one(q), "mx"), Qz.quantize_qk(one(k), "mx")
+    vd = Qz.quantize_v(one(v))
+    t0 = time.perf_counter()
+    try:
+        st = parity.compare_head(Og[b, h].astype(np.float64), Lg[b, h].astype(np.float64), qd, kd, vd, 0, 0, **okw)
+        st["ok"] = True
+    except AssertionError as e:
+        st = {"ok": False, "error": str(e)[:400]}
+    st["head"] = (b, h)
+    st["oracle_s"] = round(time.perf_counter() - t0, 1)
+    return st
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("workload", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine"])
+    ap.add_argument("--workers", type=int, default=max(1, len(os.sched_getaffinity(0)) - 2))
+    ap.add_argument("--units", default=None, help="begin:end slice of the (batch, head) units, default all")
+    args = ap.parse_args()
+    import torch
+    from oracle import quantize as Qz
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.WORKLOADS[args.workload]
+    q, k, v = I.make_qkv(w)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    qg = Bd.fp4attn_quantize(dev(q), w.qk_fmt, Bd.ROLE_Q)
+    kg = Bd.fp4attn_quantize(dev(k), w.qk_fmt, Bd.ROLE_K)
+    vg = Bd.fp4attn_quantize(dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    O, L = Bd.fp4attn_fwd(qg, kg, vg, status=status, p_map=Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_IDEAL)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    _G.update(w=w, q=q, k=k, v=v, O=O.float().cpu().numpy(), L=L.cpu().numpy(), Gq=None, Gk=None,
+              okw=dict(p_map=args.p_map))
+    if w.qk_fmt == I.FMT_NVFP4:
+        _G["Gq"] = Qz.nv_tensor_scale(Qz.bf16_bits_to_f64(q))
+        _G["Gk"] = Qz.nv_tensor_scale(Qz.bf16_bits_to_f64(k))
+    del qg, kg, vg, O, L
+    torch.cuda.empty_cache()
+    units = [(b, h) for b in range(w.B) for h in range(w.H)]
+    if args.units:
+        lo, hi = (int(x) for x in args.units.split(":"))
+        units = units[lo:hi]
+    t0 = time.perf_counter()
+    with mp.get_context("fork").Pool(args.workers) as pool:        # workers inherit the arrays; they never touch CUDA
+        res = []
+        for st in pool.imap_unordered(_unit, units):
+            print(json.dumps(st), flush=True)
+            res.append(st)
+    good = [r for r in res if r["ok"]]
+    summary = {"workload": w.name, "p_map": args.p_map, "units": len(res), "units_ok": len(good),
+               "rows": int(sum(r["rows"] for r in good)), "wall_s": round(time.perf_counter() - t0, 1)}
+    if good:
+        summary.update(rel_fro_strict_max=max(r["rel_fro_strict"] for r in good), max_abs_strict=max(r["max_abs_strict"] for r in good),
+                       lse_err_max=max(r["lse_err"] for r in good), rows_failing_strict=int(sum(r["rows_failing_strict"] for r in good)),
+                       accepted_with_flips=int(sum(r["accepted_with_flips"] for r in good)))
+    print("SUMMARY " + json.dumps(summary), flush=True)
+    sys.exit(0 if len(good) == len(res) else 1)
+
+
+if __name__ == "__main__":
+    main()
