@@ -51,7 +51,7 @@ METRIC = "fp4_attention_fwd_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_FP4_OVER_BF16 = 4.0          # dense 9 PFLOP/s fp4 : 2.25 PFLOP/s bf16
 DEFAULT_WORKLOAD = "cfg5_N32768"
-SUB_RECORDS = ("cfg5_N8192", "cfg5_N16384", "cfg4", "cfg3", "cfg2", "cfg5_N4096", "cfg5_N2048", "cfg5_N1024")
+SUB_RECORDS = ("cfg5_N8192", "cfg5_N16384", "cfg4", "cfg3", "cfg3_N32768", "cfg2", "cfg5_N4096", "cfg5_N2048", "cfg5_N1024")
 
 
 def _peaks():
@@ -281,9 +281,9 @@ def timed_launches(fn, n, flush, E, sync):
     return [a.elapsed_time(b) for a, b in pairs]
 
 
-def roofline_record(w, ms, fp4_peak, peaks):
+def roofline_record(w, ms, fp4_peak, peaks, kernel="attn_fwd_kernel"):
     tf = w.flops / (ms * 1e-3) / 1e12
-    return {"kernel": "attn_fwd_kernel", "bound": "tensor", "achieved": tf, "peak": fp4_peak, "unit": "TFLOP/s",
+    return {"kernel": kernel, "bound": "tensor", "achieved": tf, "peak": fp4_peak, "unit": "TFLOP/s",
             "frac": tf / fp4_peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name, {}).get("attn"),
             "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x nominal fp4:bf16 ratio 4"}
 
@@ -325,6 +325,7 @@ def run_cuda(args, w):
     pmap = Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_HYBRID if args.p_map in HYBRID_PATTERNS else Bd.PMAP_IDEAL
     pairs = HYBRID_PATTERNS.get(args.p_map, 0)
     pscale = Bd.PSCALE_THR16 if args.p_scale == "thr16" else Bd.PSCALE_CEIL
+    sched = Bd.SCHEDULE_TWO_QUERY if args.schedule == "two-query" else Bd.SCHEDULE_ONE_QUERY
     state = {}
     E = lambda: torch.cuda.Event(enable_timing=True)
 
@@ -334,7 +335,8 @@ def run_cuda(args, w):
         vd = Bd.fp4attn_quantize(dv, Bd.FMT_MXFP4, Bd.ROLE_V)
         if ev is not None:
             ev[0].record()
-        Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status, p_map=pmap, p_scale_rule=pscale, exact_pairs=pairs)
+        Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status, p_map=pmap, p_scale_rule=pscale, exact_pairs=pairs,
+                       schedule=sched)
         if ev is not None:
             ev[1].record()
         state["ops"] = (qd, kd, vd)
@@ -510,7 +512,11 @@ def run_cuda(args, w):
             del xq, xk, xv
             so = torch.empty((ww.B, ww.H, ww.N, ww.d), dtype=torch.bfloat16, device=dev)
             rec = {"workload": _workload_text(ww), "launches": n_it, "inputs": "seeded recipe of the configuration"}
-            for key, kw, share in (("", {}, 1.0), ("affine_", dict(p_map=Bd.PMAP_AFFINE), 1.0), ("causal_", dict(causal=True), 0.5)):
+            variants = [("", {}, 1.0), ("affine_", dict(p_map=Bd.PMAP_AFFINE), 1.0), ("causal_", dict(causal=True), 0.5)]
+            if ww.d == 64 and ww.N % 256 == 0:                       # the two-query schedule beside the one-query one
+                variants += [("two_query_", dict(schedule=Bd.SCHEDULE_TWO_QUERY), 1.0),
+                             ("two_query_affine_", dict(schedule=Bd.SCHEDULE_TWO_QUERY, p_map=Bd.PMAP_AFFINE), 1.0)]
+            for key, kw, share in variants:
                 fn = lambda: Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status, **kw)
                 for _ in range(3):
                     fn()
@@ -533,7 +539,7 @@ def run_cuda(args, w):
             dist.destroy_process_group()
         return
 
-    roof = roofline_record(w, attn_launch_ms, fp4_peak, peaks)
+    roof = roofline_record(w, attn_launch_ms, fp4_peak, peaks, "attn_fwd_2q_kernel" if args.schedule == "two-query" else "attn_fwd_kernel")
     roof.update({"fp4_issue_probe_tflops": probe_tflops, "fp4_issue_probe_flop_per_clk_per_sm": probe_flop_per_clk_sm,
                  "launch_ms_mean": attn_launch_ms, "launch_ms_median": statistics.median(attn_ms)})
     out = {
@@ -541,7 +547,7 @@ def run_cuda(args, w):
         "warmup": n_warm, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate)", "data": "synthetic",
         "config": {"workload": _workload_text(w), "step": "quantize Q,K,V + attention forward", "p_map": args.p_map, "p_scale": args.p_scale,
-                   "l2": "flushed between steps (256 MiB fill, outside the step's events)",
+                   "schedule": args.schedule, "l2": "flushed between steps (256 MiB fill, outside the step's events)",
                    "warmup": f"{n_warm} steps (at least --warmup and 300 ms)",
                    "flops": "4*B*H*N^2*d", "parallelism": f"replica x{world}, (batch, head) units, no collective"},
         "attn_only": {"value": attn_tflops, "unit": UNIT, "ms": attn_launch_ms,
@@ -596,6 +602,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the attention-only timings of the other configurations")
     ap.add_argument("--p-scale", default="ceil", choices=["ceil", "thr16"],
                     help="block-exponent rule of P: ceiling (default) or floor(max y + log2 1.6)")
+    ap.add_argument("--schedule", default="one-query", choices=["one-query", "two-query"],
+                    help="query tiles per thread block in the timed step (two-query: d = 64 workloads only)")
     ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine", "hybrid4", "hybrid8", "hybrid12"],
                     help="score->code map of the timed path: exact codes (default), the paper's affine classifier, or "
                          "4 / 8 / 12 of every 16 element pairs exact and the rest affine (EX2-density control)")

@@ -55,6 +55,9 @@ WORKLOADS: Dict[str, Workload] = {
 }
 for _n in (1024, 2048, 4096, 8192, 16384, 32768):
     WORKLOADS[f"cfg5_N{_n}"] = sweep_workload(_n)
+# configuration 3's formats and head dimension at the longest sequence (same token count per head as the sweep's
+# longest point): the second shape on which the two schedules of d = 64 are timed side by side
+WORKLOADS["cfg3_N32768"] = Workload("cfg3_N32768", 6, 2, 16, 32768, 64, FMT_NVFP4)
 
 
 def shrink(w: Workload, **kw) -> Workload:
