@@ -43,8 +43,9 @@ from paper_2609_04105_b200 import inputs as I  # noqa: E402
 # algorithmic bytes.  Workloads without a capture report null.
 NCU_TRAFFIC_BYTES = {
     "cfg2": {"attn": 53.5e6 + 24.2e6, "quant_rows": 67.12e6 + 3.08e6},
-    "cfg3": {"attn": 113.3e6 + 97.4e6},
+    "cfg3": {"attn": 114.6e6 + 97.6e6},
     "cfg4": {"attn": 107.3e6 + 95.9e6},
+    "cfg5_N32768": {"attn": 107.4e6 + 96.0e6},
 }
 
 METRIC = "fp4_attention_fwd_tflops"
