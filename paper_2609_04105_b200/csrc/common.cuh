@@ -11,15 +11,6 @@
 
 namespace fp4attn {
 
-// Two floats -> one byte of two E2M1 codes, round to nearest even, saturating:
-// `lo` lands in bits 0-3, `hi` in bits 4-7.
-__device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi) {
-  uint16_t r;
-  asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %2, %1; mov.b16 %0, {t, 0}; }"
-      : "=h"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-
 // Eight floats -> one 32-bit word of eight E2M1 codes (element k in nibble k).
 __device__ __forceinline__ uint32_t cvt_e2m1x8(const float* v) {
   uint32_t w;
@@ -55,15 +46,6 @@ __device__ __forceinline__ void bf16x8_to_f32(const uint4& raw, float* v) {
     v[2 * i] = __uint_as_float(w[i] << 16);
     v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
   }
-}
-
-// E8M0 byte of the MXFP4 amplitude convention: u = clamp(127 + ceil(log2 a), 1, 254), 0 for a == 0.
-// `a` is a non-negative finite float; ceil(log2 a) is read from exponent and mantissa bits.
-__device__ __forceinline__ uint32_t mx_scale_byte(float a) {
-  const uint32_t bits = __float_as_uint(a);
-  if (bits == 0) return 0;
-  uint32_t u = (bits >> 23) + ((bits & 0x7FFFFFu) != 0 ? 1u : 0u);
-  return min(max(u, 1u), 254u);
 }
 
 // 2^(127-u) for u in [0, 254] (u = 254 needs the subnormal 2^-127).
