@@ -126,81 +126,104 @@ quant_mx_rows_kernel(const uint4* __restrict__ x, uint32_t* __restrict__ packed,
 }
 
 // ---------------------------------------------------------------- MXFP4, blocks along keys (V), transposed out
-// A [128 keys x D] tile goes through shared memory; a thread owns two adjacent head-dim columns and
-// one 32-key block, reads them as bf16x2 words (conflict-free) and writes two 16-byte code groups.
-// grid (N / 128, B*H), 2*D threads
+// A [128 keys x D] tile (contiguous in memory) goes through shared memory; a thread owns two adjacent head-dim
+// columns and one 32-key block, reads them as bf16x2 words (conflict-free) and writes two 16-byte code groups.
+// Persistent CTAs walk the tiles with two tile buffers: the asynchronous copies (cp.async, 16 bytes per thread
+// and copy, no registers in between) of the next tile are in flight while the current one is converted, so the
+// memory system always has work although each tile passes through a load -> barrier -> convert sequence.
+// grid min(tiles, CTAs that fit) , 2*D threads, dynamic shared memory kVSmem<D>
+template <int D> constexpr int kVTileBytes = 128 * D * 2;
+template <int D> constexpr int kVSmem = 2 * kVTileBytes<D> + 512;
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
 template <int D, int RULE>
-__global__ void __launch_bounds__(2 * D)
-quant_mx_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ packed, uint8_t* __restrict__ sf, int N) {
+__global__ void __launch_bounds__(2 * D, RULE == FP4ATTN_QSCALE_MSE ? 1 : (D == 128 ? 3 : 6))
+quant_mx_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ packed, uint8_t* __restrict__ sf, int N, int n_tiles) {
   constexpr int T = 2 * D;                         // threads: D/2 column pairs x 4 key blocks
-  __shared__ __align__(16) uint32_t tile[128 * D / 2];
-  __shared__ uint8_t sfb[128 * 4];
-  const int kt = blockIdx.x;                       // 128-key tile
-  const size_t bh = blockIdx.y;
-  const uint4* src = x + (bh * N + (size_t)kt * 128) * (D / 8);
-  constexpr int LOADS = 128 * D / 8 / T;           // 8
-  uint4 raw[LOADS];
-#pragma unroll
-  for (int k = 0; k < LOADS; ++k) raw[k] = __ldg(src + threadIdx.x + k * T);
-#pragma unroll
-  for (int k = 0; k < LOADS; ++k) reinterpret_cast<uint4*>(tile)[threadIdx.x + k * T] = raw[k];
-  if (threadIdx.x < 128) reinterpret_cast<uint32_t*>(sfb)[threadIdx.x] = 0;
-  __syncthreads();
+  constexpr int LOADS = 128 * D / 8 / T;           // 16-byte copies per thread and tile: 8
+  extern __shared__ __align__(16) uint8_t vsm[];
+  uint8_t* sfb = vsm + 2 * kVTileBytes<D>;
+  const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(vsm);
+  const int tiles_per_head = N / 128;
   const int cp = threadIdx.x % (D / 2);            // column pair: columns 2cp, 2cp+1
   const int kb = threadIdx.x / (D / 2);            // key block 0..3
-  uint32_t w[32];
-  uint32_t m = 0;
+  auto issue = [&](int t, int buf) {               // tile t is contiguous: 128 keys x D bf16 starting at key 128 t of the flat [B*H*N] key space
+    const uint4* src = x + (size_t)t * (128 * D / 8);
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    w[i] = tile[(kb * 32 + i) * (D / 2) + cp];
-    m = __vmaxu2(m, w[i] & 0x7FFF7FFFu);
-  }
+    for (int k = 0; k < LOADS; ++k)
+      cp_async_16(sbase + buf * kVTileBytes<D> + (threadIdx.x + k * T) * 16, src + threadIdx.x + k * T);
+    cp_async_commit();
+  };
+  int t = blockIdx.x, i = 0;
+  if (t < n_tiles) issue(t, 0);
+  for (; t < n_tiles; t += gridDim.x, ++i) {
+    const int tn = t + gridDim.x;
+    if (tn < n_tiles) { issue(tn, (i + 1) & 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+    if (threadIdx.x < 128) reinterpret_cast<uint32_t*>(sfb)[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t* tile = reinterpret_cast<const uint32_t*>(vsm + (i & 1) * kVTileBytes<D>);
+    const size_t bh = t / tiles_per_head;
+    const int kt = t - (int)bh * tiles_per_head;     // 128-key tile within the head
+    uint32_t w[32];
+    uint32_t m = 0;
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {                    // low half = column 2cp, high half = column 2cp+1
-    const uint32_t a16 = c ? (m >> 16) : (m & 0xFFFFu);
-    uint32_t u = mx_scale_byte_bf16<RULE == FP4ATTN_QSCALE_MSE ? FP4ATTN_QSCALE_CEIL : RULE>(a16);
-    float v[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(c ? (w[i] & 0xFFFF0000u) : (w[i] << 16));
-    uint4 out;
-    if (RULE == FP4ATTN_QSCALE_MSE) {
-      // both amplitudes; group sums of eight consecutive keys combined as (g0 + g1) + (g2 + g3)
-      const uint32_t uf = mx_scale_byte_bf16<FP4ATTN_QSCALE_FLOOR>(a16);
-      float tf[32];
-#pragma unroll
-      for (int i = 0; i < 32; ++i) tf[i] = v[i];
-      mx_scale_values<32>(tf, uf);
-      mx_scale_values<32>(v, u);
-      uint32_t wf[4], wc[4];
-      float gf[4], gc[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        wf[j] = cvt_e2m1x8(tf + 8 * j);
-        wc[j] = cvt_e2m1x8(v + 8 * j);
-        gf[j] = mx_error_x8(tf + 8 * j, wf[j]);
-        gc[j] = mx_error_x8(v + 8 * j, wc[j]);
-      }
-      const float ef = __fadd_rn(__fadd_rn(gf[0], gf[1]), __fadd_rn(gf[2], gf[3]));
-      const float ec = __fadd_rn(__fadd_rn(gc[0], gc[1]), __fadd_rn(gc[2], gc[3]));
-      const bool take_f = (uf != u) && (ef < __fmul_rn(4.0f, ec));
-      out = take_f ? make_uint4(wf[0], wf[1], wf[2], wf[3]) : make_uint4(wc[0], wc[1], wc[2], wc[3]);
-      u = take_f ? uf : u;
-    } else {
-      mx_scale_values<32>(v, u);
-      out.x = cvt_e2m1x8(v);
-      out.y = cvt_e2m1x8(v + 8);
-      out.z = cvt_e2m1x8(v + 16);
-      out.w = cvt_e2m1x8(v + 24);
+    for (int r = 0; r < 32; ++r) {
+      w[r] = tile[(kb * 32 + r) * (D / 2) + cp];
+      m = __vmaxu2(m, w[r] & 0x7FFF7FFFu);
     }
-    const int col = 2 * cp + c;
-    packed[((bh * D + col) * (size_t)(N / 2) + (size_t)kt * 64 + kb * 16) / 16] = out;
-    sfb[col * 4 + kb] = (uint8_t)u;
-  }
-  __syncthreads();
-  if (threadIdx.x < 128) {
-    const int r = threadIdx.x;                     // head-dim row; rows >= D are zero padding
-    uint8_t* p = sf + (bh * (size_t)(N / 128) + kt) * 512 + (r & 31) * 16 + (r >> 5) * 4;
-    *reinterpret_cast<uint32_t*>(p) = reinterpret_cast<const uint32_t*>(sfb)[r];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {                    // low half = column 2cp, high half = column 2cp+1
+      const uint32_t a16 = c ? (m >> 16) : (m & 0xFFFFu);
+      uint32_t u = mx_scale_byte_bf16<RULE == FP4ATTN_QSCALE_MSE ? FP4ATTN_QSCALE_CEIL : RULE>(a16);
+      float v[32];
+#pragma unroll
+      for (int r = 0; r < 32; ++r) v[r] = __uint_as_float(c ? (w[r] & 0xFFFF0000u) : (w[r] << 16));
+      uint4 out;
+      if (RULE == FP4ATTN_QSCALE_MSE) {
+        // both amplitudes; group sums of eight consecutive keys combined as (g0 + g1) + (g2 + g3)
+        const uint32_t uf = mx_scale_byte_bf16<FP4ATTN_QSCALE_FLOOR>(a16);
+        float tf[32];
+#pragma unroll
+        for (int r = 0; r < 32; ++r) tf[r] = v[r];
+        mx_scale_values<32>(tf, uf);
+        mx_scale_values<32>(v, u);
+        uint32_t wf[4], wc[4];
+        float gf[4], gc[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          wf[j] = cvt_e2m1x8(tf + 8 * j);
+          wc[j] = cvt_e2m1x8(v + 8 * j);
+          gf[j] = mx_error_x8(tf + 8 * j, wf[j]);
+          gc[j] = mx_error_x8(v + 8 * j, wc[j]);
+        }
+        const float ef = __fadd_rn(__fadd_rn(gf[0], gf[1]), __fadd_rn(gf[2], gf[3]));
+        const float ec = __fadd_rn(__fadd_rn(gc[0], gc[1]), __fadd_rn(gc[2], gc[3]));
+        const bool take_f = (uf != u) && (ef < __fmul_rn(4.0f, ec));
+        out = take_f ? make_uint4(wf[0], wf[1], wf[2], wf[3]) : make_uint4(wc[0], wc[1], wc[2], wc[3]);
+        u = take_f ? uf : u;
+      } else {
+        mx_scale_values<32>(v, u);
+        out.x = cvt_e2m1x8(v);
+        out.y = cvt_e2m1x8(v + 8);
+        out.z = cvt_e2m1x8(v + 16);
+        out.w = cvt_e2m1x8(v + 24);
+      }
+      const int col = 2 * cp + c;
+      packed[((bh * D + col) * (size_t)(N / 2) + (size_t)kt * 64 + kb * 16) / 16] = out;
+      sfb[col * 4 + kb] = (uint8_t)u;
+    }
+    __syncthreads();
+    if (threadIdx.x < 128) {
+      const int r = threadIdx.x;                     // head-dim row; rows >= D are zero padding
+      uint8_t* p = sf + (bh * (size_t)tiles_per_head + kt) * 512 + (r & 31) * 16 + (r >> 5) * 4;
+      *reinterpret_cast<uint32_t*>(p) = reinterpret_cast<const uint32_t*>(sfb)[r];
+    }
+    __syncthreads();                                 // the tile buffer and the scale staging are free again
   }
 }
 
@@ -330,6 +353,26 @@ extern "C" size_t fp4attn_quantize_workspace_bytes(int fmt, int role, int B, int
 }
 
 namespace fp4attn {
+// V kernel: persistent CTAs, as many as fit per SM with two tile buffers each (the opt-in to more than 48 KB of
+// dynamic shared memory is set once per device and instance)
+template <int D, int RULE>
+static void launch_mx_v(const uint4* xs, int n_tiles, int N, void* packed, void* scales, cudaStream_t st) {
+  static std::atomic<int> ctas[kMaxDevices];        // 0 unknown, else CTAs of the persistent grid
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return;   // the launch check below reports it
+  int grid = ctas[dev].load(std::memory_order_acquire);
+  if (!grid) {
+    int sms = 0, per_sm = 0;
+    if (cudaFuncSetAttribute(quant_mx_v_kernel<D, RULE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kVSmem<D>) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quant_mx_v_kernel<D, RULE>, 2 * D, kVSmem<D>) != cudaSuccess || per_sm < 1)
+      return;
+    grid = sms * per_sm;
+    ctas[dev].store(grid, std::memory_order_release);
+  }
+  quant_mx_v_kernel<D, RULE><<<n_tiles < grid ? n_tiles : grid, 2 * D, kVSmem<D>, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N, n_tiles);
+}
+
 // Shared by fp4attn_quantize and the variants that bring their own scratch.
 template <int RULE>
 static void launch_mx(const uint4* xs, int role, int B, int H, int N, int d, void* packed, void* scales, cudaStream_t st) {
@@ -337,10 +380,10 @@ static void launch_mx(const uint4* xs, int role, int B, int H, int N, int d, voi
     const dim3 grid2((unsigned)((size_t)N * d / 8 / kGroupsPerCta), (unsigned)(B * H));   // N % 128 == 0 makes this exact
     if (d == 128) quant_mx_rows_kernel<128, RULE><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
     else          quant_mx_rows_kernel<64, RULE><<<grid2, kThreads, 0, st>>>(xs, (uint32_t*)packed, (uint8_t*)scales, N);
+  } else if (d == 128) {
+    launch_mx_v<128, RULE>(xs, B * H * (N / 128), N, packed, scales, st);
   } else {
-    dim3 g2(N / 128, B * H);
-    if (d == 128) quant_mx_v_kernel<128, RULE><<<g2, 256, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
-    else          quant_mx_v_kernel<64, RULE><<<g2, 128, 0, st>>>(xs, (uint4*)packed, (uint8_t*)scales, N);
+    launch_mx_v<64, RULE>(xs, B * H * (N / 128), N, packed, scales, st);
   }
 }
 
