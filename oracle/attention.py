@@ -285,6 +285,56 @@ def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int
     return np.stack(Os), np.stack(Ls)
 
 
+# ----------------------------------------------------------------------------------------------- FP8 P/V route
+P8_SHIFT = 8      # probabilities are carried as 2**8 * p, so the largest (p = 1) is 256 <= 448, the E4M3 maximum
+
+
+def fp8_pv_rows(s32: np.ndarray, c32: np.float32, V8hat: np.ndarray, row_index=None):
+    """FP8 probabilities and values for a set of query rows of one (batch, head) (the route the paper retains for
+    training, Section "Training stability selects FP8 P/V"; it prints no algorithm, reading taken here).
+
+    s32 [R, N] float32 scores facing the tensor core, V8hat [N, d] float64 reconstructed E4M3 V.
+      mu_i  = ceil(max_j y_ij), y = fl32(s32 * c32): an integer row reference, the row maximum rounded up, known
+              before any probability is formed, so that nothing depends on a tile order;
+      p8_ij = Q_E4M3(2**(y_ij - mu_i + 8)), round to nearest even on the E4M3 grid (three mantissa bits, subnormals
+              of 2**-9; below 2**-10 the value is 0): one 8-bit float per probability, NO block scales;
+      O_i   = sum_j p8_ij V^_j / sum_j p8_ij (the same rounded values in numerator and denominator, Eq.
+              "represented-output" carried over), LSE_i = ln2 (mu_i - 8 + log2 sum_j p8_ij).
+    Returns O [R, d], LSE [R], the E4M3 bytes [R, N] and mu [R]."""
+    from .formats import e4m3_decode, e4m3_encode_unsigned
+    R, N = s32.shape
+    if row_index is not None:
+        s32 = np.where(np.arange(N)[None, :] > np.asarray(row_index)[:, None], np.float32(-np.inf), s32).astype(np.float32)
+    y32 = (s32 * np.float32(c32)).astype(np.float32)
+    mu = np.ceil(y32.max(axis=1).astype(np.float64))
+    b32 = np.float32(np.float32(P8_SHIFT) - mu.astype(np.float32))
+    x = s32.astype(np.float64) * np.float64(c32) + b32.astype(np.float64)[:, None]
+    byte = e4m3_encode_unsigned(np.exp2(x))
+    p8 = e4m3_decode(byte)
+    L = p8.sum(axis=1)
+    O = (p8 @ V8hat) / L[:, None]
+    lse = math.log(2.0) * (mu - P8_SHIFT + np.log2(L))
+    return O, lse, byte, mu
+
+
+def fp8_pv_forward(qd: dict, kd: dict, v8: dict, softmax_scale=None, rows=None, heads=None, causal: bool = False,
+                   kv_group: int = 1):
+    """Whole-operator oracle of the FP8-P/V route: FP4 Q, K as in direct_p_forward, v8 from quantize_v_e4m3."""
+    from .quantize import dequantize_v_e4m3
+    B, H, N, d = qd["nib"].shape
+    heads = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
+    ridx = np.arange(N) if rows is None else np.asarray(rows)
+    Os, Ls = [], []
+    for (b, h) in heads:
+        hk = h // kv_group
+        c32 = score_constant(qd, kd, d, softmax_scale, (b, h, hk))
+        s32 = scores_fp32(qd, kd, b, h, rows, hk)
+        O, lse, _, _ = fp8_pv_rows(s32, c32, np.ascontiguousarray(dequantize_v_e4m3(v8, b, hk).T), ridx if causal else None)
+        Os.append(O)
+        Ls.append(lse)
+    return np.stack(Os), np.stack(Ls)
+
+
 def exact_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray, softmax_scale=None, rows=None, causal=False):
     """Eq. "exact-attention" in float64 for one head: Q [N,d], K [N,d], V [N,d] -> O, LSE."""
     d = Q.shape[1]

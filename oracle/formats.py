@@ -81,3 +81,12 @@ def e4m3_encode_unsigned(t) -> np.ndarray:
     out = (ebits.astype(np.int64) << 3 | mant.astype(np.int64)).astype(np.uint8)
     out = np.where(t > 0, out, 0).astype(np.uint8)
     return out
+
+
+def e4m3_encode(t) -> np.ndarray:
+    """Signed E4M3 byte of the value nearest to t (ties to even mantissa, saturating at +-448); a result that rounds
+    to zero keeps sign bit 0."""
+    t = np.asarray(t, dtype=np.float64)
+    mag = e4m3_encode_unsigned(np.abs(t))
+    sign = ((t < 0) & (mag > 0)).astype(np.uint8)
+    return (mag | (sign << 7)).astype(np.uint8)

@@ -23,7 +23,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from .formats import (ceil_log2, e2m1_decode, e2m1_encode, e4m3_decode,
+from .formats import (ceil_log2, e2m1_decode, e2m1_encode, e4m3_decode, e4m3_encode,
                       e4m3_encode_unsigned, e8m0_decode)
 
 MX_BLOCK = 32
@@ -187,6 +187,28 @@ def quantize_v(bits: np.ndarray, rule: str = "ceil"):
     xt = np.ascontiguousarray(np.swapaxes(bf16_bits_to_f64(bits), -1, -2))
     nib, sf = mx_quantize_lastdim(xt, rule)
     return {"nib": nib, "sf": sf, "G": None, "fmt": "mx"}
+
+
+def quantize_v_e4m3(bits: np.ndarray):
+    """V bf16 [B,H,N,d] -> E4M3 bytes of V^T, dict(byte [B,H,d,N] uint8, G float32 [B,H], fmt "e4m3").
+
+    The FP8 value operand of the FP8-P/V route (Section "Training stability selects FP8 P/V": "E4M3 V views"); the
+    paper gives no scale rule, reading taken here: one encode factor per (batch, head) unit, like the per-head
+    NVFP4 factors, G = fl32(448 / max|V[b,h]|) (1 for an all-zero unit), byte = Q_E4M3(fl32(v * G)) round to nearest
+    even; a value is reconstructed as decode(byte) / G."""
+    x = bf16_bits_to_f64(bits)
+    B, H = x.shape[:2]
+    a = np.abs(x).reshape(B, H, -1).max(axis=2).astype(np.float32)
+    with np.errstate(divide="ignore"):
+        G = np.where(a > 0, np.float32(448.0) / np.where(a > 0, a, np.float32(1)), np.float32(1)).astype(np.float32)
+    t = (x.astype(np.float32) * G[:, :, None, None]).astype(np.float32)
+    byte = e4m3_encode(t.astype(np.float64))
+    return {"byte": np.ascontiguousarray(np.swapaxes(byte, -1, -2)), "G": G, "fmt": "e4m3"}
+
+
+def dequantize_v_e4m3(vd: dict, b: int, h: int) -> np.ndarray:
+    """Reconstructed V^T of one unit, [d, N] float64."""
+    return e4m3_decode(vd["byte"][b, h]) / np.float64(vd["G"][b, h])
 
 
 def dequantize(qd: dict, hw: bool = False) -> np.ndarray:
