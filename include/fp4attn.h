@@ -187,6 +187,11 @@ enum { FP4ATTN_SCHEDULE_ONE_QUERY = 0,   /* one 128-row query tile per thread bl
                                             anything else returns FP4ATTN_ERR_UNSUPPORTED_SHAPE.  Same results, bit
                                             for bit, as FP4ATTN_SCHEDULE_ONE_QUERY                                */
 
+/* format of the probabilities and of V in the second product */
+enum { FP4ATTN_PV_MXFP4 = 0,   /* Direct-P: E2M1 codes with E8M0 block scales for P and V (the path of this library)   */
+       FP4ATTN_PV_E4M3 = 1 };  /* FP8 P/V (Section "Training stability selects FP8 P/V"): one E4M3 byte per probability
+                                  and per value, no block scales; see fp4attn_fwd and fp4attn_quantize_v_e4m3           */
+
 typedef struct {
   const void *q, *k, *v;            /* packed E2M1 (V transposed)                           */
   const void *q_sf, *k_sf, *v_sf;   /* scale atoms                                           */
@@ -211,6 +216,10 @@ typedef struct {
                                        (fp4attn_quantize_nvfp4_per_head); with the ideal and the
                                        affine map, not with FP4ATTN_PMAP_HYBRID                 */
   int schedule;                     /* FP4ATTN_SCHEDULE_ONE_QUERY (0, default) or _TWO_QUERY */
+  int pv_fmt;                       /* FP4ATTN_PV_MXFP4 (0, default) or FP4ATTN_PV_E4M3: then v holds E4M3 bytes of V^T
+                                       [B, kv_heads, d, N] from fp4attn_quantize_v_e4m3, v_sf is ignored, v_G is required;
+                                       with the ideal map, the ceiling rule and the one-query schedule only          */
+  const float* v_G;                 /* FP4ATTN_PV_E4M3: device fp32 encode factors of V, one per (batch, K/V head)    */
 } fp4attn_operands;
 
 /*
@@ -250,6 +259,27 @@ typedef struct {
  */
 int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int d,
                 void* O_bf16, float* LSE, int* device_status, fp4attn_stream_t stream);
+
+/*
+ * E4M3 quantizer of V for the FP8 P/V route (Section "Training stability selects FP8 P/V": the retained training
+ * route keeps "E4M3 V views"; the paper states no scale rule).  Every (batch, head) unit gets one encode factor
+ * G[b*H + h] = fl32(448 / max|V[b, h]|) (1 for an all-zero unit), written to unit_scale_out (B*H floats), and
+ * every value the byte Q_E4M3(fl32(v * G)), round to nearest even; a value is reconstructed as decode(byte) / G.
+ * bytes_out receives V^T, [B, H, d, N] bytes (key index contiguous: the contraction-major layout of the second
+ * product).  workspace: device scratch of fp4attn_quantize_v_e4m3_workspace_bytes() bytes, 16-byte aligned.
+ * Shapes, alignment and status codes as for fp4attn_quantize.
+ *
+ * With pv_fmt = FP4ATTN_PV_E4M3 fp4attn_fwd computes, for FP4 Q and K exactly as described above,
+ *   mu_i = ceil(max_j y_ij),  p8_ij = Q_E4M3(2^(y_ij - mu_i + 8)),  O_i = sum_j p8_ij V^_j / sum_j p8_ij,
+ *   LSE_i = ln2 (mu_i - 8 + log2 sum_j p8_ij):
+ * the row reference is the row's own maximum rounded up to an integer, taken by a first sweep over the keys
+ * before any probability is formed (without block scales a rounded probability cannot be re-scaled later), so the
+ * result does not depend on any tile order.  2^x is ex2.approx: a byte can differ from the exact rounding within
+ * a few float32 spacings of x at a rounding boundary of the E4M3 grid.
+ */
+size_t fp4attn_quantize_v_e4m3_workspace_bytes(int B, int H, int N, int d);
+int fp4attn_quantize_v_e4m3(const void* x_bf16, int B, int H, int N, int d, void* bytes_out, float* unit_scale_out,
+                            void* workspace, size_t workspace_bytes, fp4attn_stream_t stream);
 
 /* Bytes of device scratch fp4attn_attention_host needs for a problem of this size. */
 size_t fp4attn_attention_host_workspace_bytes(int qk_fmt, int B, int H, int N, int d);

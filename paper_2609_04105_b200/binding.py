@@ -17,6 +17,7 @@ ROLE_Q, ROLE_K, ROLE_V = 0, 1, 2
 PMAP_IDEAL, PMAP_AFFINE, PMAP_HYBRID = 0, 1, 2
 PSCALE_CEIL, PSCALE_THR16 = 0, 1
 SCHEDULE_ONE_QUERY, SCHEDULE_TWO_QUERY = 0, 1
+PV_MXFP4, PV_E4M3 = 0, 1
 QSCALE_CEIL, QSCALE_THR16, QSCALE_FLOOR, QSCALE_MSE = 0, 1, 2, 3
 (OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_ARCH, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA,
  ERR_TIMEOUT) = range(8)
@@ -30,6 +31,7 @@ EXPORTS = [
     "fp4attn_attention_host_workspace_bytes", "fp4attn_attention_host", "fp4attn_mma_peak_probe",
     "fp4attn_quantize_nvfp4_noalloc", "fp4attn_selftest_bounded_wait", "fp4attn_quantize_mxfp4_rule",
     "fp4attn_quantize_nvfp4_per_head_workspace_bytes", "fp4attn_quantize_nvfp4_per_head", "fp4attn_release",
+    "fp4attn_quantize_v_e4m3_workspace_bytes", "fp4attn_quantize_v_e4m3",
 ]
 
 
@@ -44,7 +46,8 @@ class _Operands(ctypes.Structure):
                 ("qk_fmt", ctypes.c_int), ("softmax_scale", ctypes.c_float),
                 ("p_map", ctypes.c_int), ("affine_a", ctypes.c_float), ("affine_b", ctypes.c_float),
                 ("p_scale_rule", ctypes.c_int), ("causal", ctypes.c_int), ("kv_heads", ctypes.c_int),
-                ("exact_pairs", ctypes.c_int), ("g_per_head", ctypes.c_int), ("schedule", ctypes.c_int)]
+                ("exact_pairs", ctypes.c_int), ("g_per_head", ctypes.c_int), ("schedule", ctypes.c_int),
+                ("pv_fmt", ctypes.c_int), ("v_G", ctypes.c_void_p)]
 
 
 def _load() -> ctypes.CDLL:
@@ -72,6 +75,10 @@ def _load() -> ctypes.CDLL:
     lib.fp4attn_attention_host.argtypes = [vp, vp, vp, i, ctypes.c_float, i, i, i, i, vp, vp, vp, vp, sz, vp]
     lib.fp4attn_release.restype = i
     lib.fp4attn_release.argtypes = []
+    lib.fp4attn_quantize_v_e4m3_workspace_bytes.restype = sz
+    lib.fp4attn_quantize_v_e4m3_workspace_bytes.argtypes = [i, i, i, i]
+    lib.fp4attn_quantize_v_e4m3.restype = i
+    lib.fp4attn_quantize_v_e4m3.argtypes = [vp, i, i, i, i, vp, vp, vp, sz, vp]
     lib.fp4attn_quantize_mxfp4_rule.restype = i
     lib.fp4attn_quantize_mxfp4_rule.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp]
     lib.fp4attn_quantize_nvfp4_noalloc.restype = i
@@ -194,6 +201,26 @@ def fp4attn_quantize_nvfp4_noalloc(x: torch.Tensor, role: int, packed: torch.Ten
     return QuantizedOperand(packed, scales, G, FMT_NVFP4, role, (B, H, N, d))
 
 
+FMT_E4M3 = 2          # QuantizedOperand.fmt of an E4M3 V (fp4attn_quantize_v_e4m3); not a format of the C quantize calls
+
+
+def fp4attn_quantize_v_e4m3(x: torch.Tensor) -> QuantizedOperand:
+    """E4M3 bytes of V^T [B,H,d,N] with one encode factor per (batch, head) unit (G fp32 [B*H]); `scales` is empty."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 4
+    B, H, N, d = x.shape
+    L = lib()
+    nw = L.fp4attn_quantize_v_e4m3_workspace_bytes(B, H, N, d)
+    if nw == 0:
+        _check(L.fp4attn_quantize_v_e4m3(x.data_ptr(), B, H, N, d, 1, 1, None, 0, _stream()), "fp4attn_quantize_v_e4m3")
+        raise Fp4AttnError("fp4attn_quantize_v_e4m3: unsupported arguments")
+    out = torch.empty(B * H * d * N, dtype=torch.uint8, device=x.device)
+    G = torch.empty(B * H, dtype=torch.float32, device=x.device)
+    ws = torch.empty(nw, dtype=torch.uint8, device=x.device)
+    _check(L.fp4attn_quantize_v_e4m3(x.data_ptr(), B, H, N, d, out.data_ptr(), G.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "fp4attn_quantize_v_e4m3")
+    return QuantizedOperand(out, torch.empty(0, dtype=torch.uint8, device=x.device), G, FMT_E4M3, ROLE_V, (B, H, N, d), True)
+
+
 def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, softmax_scale: float = 0.0,
                 out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
                 status: Optional[torch.Tensor] = None, p_map: int = PMAP_IDEAL, affine_a: float = 0.0,
@@ -203,7 +230,8 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
     p_map selects the exact code map or the affine classifier (affine_a = 0: A = 1.5, B = 1.2)."""
     B, H, N, d = q.shape
     Hkv = k.shape[1]                                   # grouped-query attention when Hkv < H
-    assert k.shape == v.shape and k.shape == (B, Hkv, N, d) and H % Hkv == 0 and q.fmt == k.fmt and v.fmt == FMT_MXFP4
+    assert k.shape == v.shape and k.shape == (B, Hkv, N, d) and H % Hkv == 0 and q.fmt == k.fmt and v.fmt in (FMT_MXFP4, FMT_E4M3)
+    fp8 = v.fmt == FMT_E4M3
     assert q.per_head == k.per_head, "Q and K must both carry per-head factors, or neither"
     dev = q.packed.device
     if out is None:
@@ -211,9 +239,9 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
     if lse is None:
         lse = torch.empty((B, H, N), dtype=torch.float32, device=dev)
     ops = _Operands(q.packed.data_ptr(), k.packed.data_ptr(), v.packed.data_ptr(),
-                    q.scales.data_ptr(), k.scales.data_ptr(), v.scales.data_ptr(),
+                    q.scales.data_ptr(), k.scales.data_ptr(), None if fp8 else v.scales.data_ptr(),
                     _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b), int(p_scale_rule), int(bool(causal)), int(Hkv),
-                    int(exact_pairs), int(q.per_head), int(schedule))
+                    int(exact_pairs), int(q.per_head), int(schedule), PV_E4M3 if fp8 else PV_MXFP4, _ptr(v.G) if fp8 else None)
     _check(lib().fp4attn_fwd(ctypes.byref(ops), B, H, N, d, out.data_ptr(), lse.data_ptr(), _ptr(status), _stream()),
            "fp4attn_fwd")
     return out, lse

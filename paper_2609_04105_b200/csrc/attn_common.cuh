@@ -240,5 +240,7 @@ __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float 
 // Tensor maps of a launch (Q, K, V^T, O in that order) from the calling thread's cache; nullptr if the driver
 // refuses to encode one.  Defined beside the one-query kernel.
 const CUtensorMap* attention_tensor_maps(int D, const fp4attn_operands* ops, void* O, int B, int H, int Hkv, int N);
+// The same with V^T held as E4M3 bytes [B, Hkv, d, N] (box: 128 keys x d rows, 128-byte swizzle).
+const CUtensorMap* attention_tensor_maps_fp8v(int D, const fp4attn_operands* ops, void* O, int B, int H, int Hkv, int N);
 
 }  // namespace fp4attn

@@ -559,9 +559,9 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint6
 // and is simply never matched again).
 struct MapKey {
   const void *q, *k, *v, *o;
-  int B, H, Hkv, N, D;
+  int B, H, Hkv, N, D, v8;              // v8: V^T is E4M3 bytes (FP8 P/V route), not packed E2M1
   bool operator==(const MapKey& r) const {
-    return q == r.q && k == r.k && v == r.v && o == r.o && B == r.B && H == r.H && Hkv == r.Hkv && N == r.N && D == r.D;
+    return q == r.q && k == r.k && v == r.v && o == r.o && B == r.B && H == r.H && Hkv == r.Hkv && N == r.N && D == r.D && v8 == r.v8;
   }
 };
 struct MapEntry {
@@ -576,9 +576,9 @@ static thread_local unsigned t_map_next = 0;
 void drop_tensor_map_cache() { g_map_epoch.fetch_add(1, std::memory_order_acq_rel); }
 
 template <int D>
-static const CUtensorMap* tensor_maps(const fp4attn_operands* ops, void* O, int B, int H, int Hkv, int N) {
+static const CUtensorMap* tensor_maps(const fp4attn_operands* ops, void* O, int B, int H, int Hkv, int N, bool v8 = false) {
   constexpr int ROW_BYTES = D / 2;
-  const MapKey key{ops->q, ops->k, ops->v, O, B, H, Hkv, N, D};
+  const MapKey key{ops->q, ops->k, ops->v, O, B, H, Hkv, N, D, v8 ? 1 : 0};
   const unsigned long long epoch = g_map_epoch.load(std::memory_order_acquire);
   for (int i = 0; i < kMapCacheEntries; ++i)
     if (t_maps[i].epoch == epoch && t_maps[i].key == key) return t_maps[i].tm;
@@ -587,7 +587,8 @@ static const CUtensorMap* tensor_maps(const fp4attn_operands* ops, void* O, int 
   const uint64_t rows = (uint64_t)B * H * N, kv_rows = (uint64_t)B * Hkv * N;
   if (!make_map(&e.tm[0], ops->q, ROW_BYTES, rows, ROW_BYTES, BM) ||
       !make_map(&e.tm[1], ops->k, ROW_BYTES, kv_rows, ROW_BYTES, BS) ||
-      !make_map(&e.tm[2], ops->v, (uint64_t)N / 2, (uint64_t)B * Hkv * D, BS / 2, D) ||
+      !(v8 ? make_map(&e.tm[2], ops->v, (uint64_t)N, (uint64_t)B * Hkv * D, BS, D)
+           : make_map(&e.tm[2], ops->v, (uint64_t)N / 2, (uint64_t)B * Hkv * D, BS / 2, D)) ||
       !make_map(&e.tm[3], O, (uint64_t)D * 2, rows, 128, 32))
     return nullptr;
   e.key = key;
@@ -598,6 +599,10 @@ static const CUtensorMap* tensor_maps(const fp4attn_operands* ops, void* O, int 
 
 const CUtensorMap* attention_tensor_maps(int D, const fp4attn_operands* ops, void* O, int B, int H, int Hkv, int N) {
   return D == 128 ? tensor_maps<128>(ops, O, B, H, Hkv, N) : tensor_maps<64>(ops, O, B, H, Hkv, N);
+}
+
+const CUtensorMap* attention_tensor_maps_fp8v(int D, const fp4attn_operands* ops, void* O, int B, int H, int Hkv, int N) {
+  return D == 128 ? tensor_maps<128>(ops, O, B, H, Hkv, N, true) : tensor_maps<64>(ops, O, B, H, Hkv, N, true);
 }
 
 template <int D, int NV, int PMAP, bool CAUSAL, bool THR16>
@@ -623,6 +628,7 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
 }
 
 int launch_attn_two_query(const fp4attn_operands* ops, int B, int H, int N, int d, int pmap, AttnParams prm, cudaStream_t st);
+int launch_attn_fp8pv(const fp4attn_operands* ops, int B, int H, int N, int d, AttnParams prm, cudaStream_t st);
 
 }  // namespace fp4attn
 
@@ -630,8 +636,8 @@ using namespace fp4attn;
 
 extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int d, void* O, float* LSE,
                            int* device_status, fp4attn_stream_t stream) {
-  if (!ops || !O || !ops->q || !ops->k || !ops->v || !ops->q_sf || !ops->k_sf || !ops->v_sf)
-    return FP4ATTN_ERR_INVALID_ARG;
+  if (!ops || !O || !ops->q || !ops->k || !ops->v || !ops->q_sf || !ops->k_sf) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->pv_fmt != FP4ATTN_PV_E4M3 && !ops->v_sf) return FP4ATTN_ERR_INVALID_ARG;   // E4M3 V carries no block scales
   if (ops->qk_fmt != FP4ATTN_FMT_MXFP4 && ops->qk_fmt != FP4ATTN_FMT_NVFP4) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->qk_fmt == FP4ATTN_FMT_NVFP4 && (!ops->q_G || !ops->k_G)) return FP4ATTN_ERR_INVALID_ARG;
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return FP4ATTN_ERR_INVALID_ARG;
@@ -676,6 +682,8 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.aff_b = ops->affine_a != 0.f ? ops->affine_b : 1.2f;
   prm.thr16 = ops->p_scale_rule == FP4ATTN_PSCALE_THR16;
   if (ops->schedule != FP4ATTN_SCHEDULE_ONE_QUERY && ops->schedule != FP4ATTN_SCHEDULE_TWO_QUERY) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->pv_fmt != FP4ATTN_PV_MXFP4 && ops->pv_fmt != FP4ATTN_PV_E4M3) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->pv_fmt == FP4ATTN_PV_E4M3) return launch_attn_fp8pv(ops, B, H, N, d, prm, st);
   if (ops->schedule == FP4ATTN_SCHEDULE_TWO_QUERY) return launch_attn_two_query(ops, B, H, N, d, pmap, prm, st);
   // one kernel instance per (d, Q/K format, P map, mask, P scale rule): nothing of these is decided at run time
   const bool per_head = nv && ops->g_per_head;

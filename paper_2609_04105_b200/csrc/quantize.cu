@@ -227,6 +227,85 @@ quant_mx_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ packed, uint8
   }
 }
 
+// ---------------------------------------------------------------- E4M3 V (FP8 P/V route), transposed out
+// Same tile pipeline as the MXFP4 V kernel; a thread owns two adjacent head-dim columns and one 32-key block and
+// writes 32 bytes per column: byte = Q_E4M3(fl32(v * G)), G the unit's encode factor (one per (batch, head)).
+__device__ __forceinline__ uint32_t cvt_e4m3x4(float a, float b, float c, float d) {   // a in bits 0-7 ... d in bits 24-31
+  uint32_t w;
+  asm("{\n\t.reg .b16 lo, hi;\n\t"
+      "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+      "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+      "mov.b32 %0, {lo, hi};\n\t}"
+      : "=r"(w) : "f"(a), "f"(b), "f"(c), "f"(d));
+  return w;
+}
+template <int D>
+__global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 6)
+quant_e4m3_v_kernel(const uint4* __restrict__ x, uint4* __restrict__ bytes_out, const float* __restrict__ G_in, int N, int n_tiles) {
+  constexpr int T = 2 * D;
+  constexpr int LOADS = 128 * D / 8 / T;
+  extern __shared__ __align__(16) uint8_t vsm[];
+  const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(vsm);
+  const int tiles_per_head = N / 128;
+  const int cp = threadIdx.x % (D / 2);
+  const int kb = threadIdx.x / (D / 2);
+  auto issue = [&](int t, int buf) {
+    const uint4* src = x + (size_t)t * (128 * D / 8);
+#pragma unroll
+    for (int k = 0; k < LOADS; ++k)
+      cp_async_16(sbase + buf * kVTileBytes<D> + (threadIdx.x + k * T) * 16, src + threadIdx.x + k * T);
+    cp_async_commit();
+  };
+  int t = blockIdx.x, i = 0;
+  if (t < n_tiles) issue(t, 0);
+  for (; t < n_tiles; t += gridDim.x, ++i) {
+    const int tn = t + gridDim.x;
+    if (tn < n_tiles) { issue(tn, (i + 1) & 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+    __syncthreads();
+    const uint32_t* tile = reinterpret_cast<const uint32_t*>(vsm + (i & 1) * kVTileBytes<D>);
+    const size_t bh = t / tiles_per_head;
+    const int kt = t - (int)bh * tiles_per_head;
+    const float G = __ldg(G_in + bh);
+    uint32_t w[32];
+#pragma unroll
+    for (int r = 0; r < 32; ++r) w[r] = tile[(kb * 32 + r) * (D / 2) + cp];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t o[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float v[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          v[e] = __fmul_rn(__uint_as_float(c ? (w[4 * j + e] & 0xFFFF0000u) : (w[4 * j + e] << 16)), G);
+        o[j] = cvt_e4m3x4(v[0], v[1], v[2], v[3]);
+      }
+      const int col = 2 * cp + c;
+      uint4* dst = bytes_out + ((bh * D + col) * (size_t)N + (size_t)kt * 128 + kb * 32) / 16;
+      dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+      dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+    __syncthreads();
+  }
+}
+
+// One block per unit: G = fl32(448 / max of the unit's partial maxima) (1 for an all-zero unit)
+__global__ void __launch_bounds__(kThreads)
+e4m3_encode_factor_kernel(const float* __restrict__ partials, int n_partials, float* __restrict__ G_out) {
+  partials += (size_t)blockIdx.x * n_partials;
+  float a = 0.f;
+  for (int i = threadIdx.x; i < n_partials; i += kThreads) a = fmaxf(a, partials[i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+  __shared__ float wmax[kThreads / 32];
+  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = a;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < kThreads / 32; ++i) a = fmaxf(a, wmax[i]);
+    G_out[blockIdx.x] = (a == 0.f) ? 1.0f : __fdiv_rn(448.0f, a);
+  }
+}
+
 // ---------------------------------------------------------------- NVFP4 pass 1: amax partials
 // grid (P, U): U = 1 for the tensor-wide maximum, U = B*H for one maximum per (batch, head) unit; row y of
 // the grid covers groups [y * n_groups, (y + 1) * n_groups) and writes partials[y * P .. y * P + P)
@@ -499,4 +578,53 @@ extern "C" int fp4attn_quantize_nvfp4_noalloc(const void* x, int role, int B, in
   }
   return launch_quantize(x, FP4ATTN_FMT_NVFP4, role, B, H, N, d, packed, scales, G_out, scratch,
                          (cudaStream_t)stream, FP4ATTN_QSCALE_CEIL);
+}
+
+// ---------------------------------------------------------------- E4M3 V of the FP8 P/V route
+extern "C" size_t fp4attn_quantize_v_e4m3_workspace_bytes(int B, int H, int N, int d) {
+  if (!shape_ok(B, H, N, d)) return 0;
+  return (size_t)B * H * kPartialsPerHead * sizeof(float);
+}
+
+template <int D>
+static int launch_e4m3_v(const uint4* xs, int BH, int N, void* bytes_out, const float* G, cudaStream_t st) {
+  static std::atomic<int> ctas[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FP4ATTN_ERR_CUDA;
+  int grid = ctas[dev].load(std::memory_order_acquire);
+  if (!grid) {
+    int sms = 0, per_sm = 0;
+    if (cudaFuncSetAttribute(quant_e4m3_v_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kVTileBytes<D>) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quant_e4m3_v_kernel<D>, 2 * D, 2 * kVTileBytes<D>) != cudaSuccess || per_sm < 1)
+      return FP4ATTN_ERR_CUDA;
+    grid = sms * per_sm;
+    ctas[dev].store(grid, std::memory_order_release);
+  }
+  const int n_tiles = BH * (N / 128);
+  quant_e4m3_v_kernel<D><<<n_tiles < grid ? n_tiles : grid, 2 * D, 2 * kVTileBytes<D>, st>>>(xs, (uint4*)bytes_out, G, N, n_tiles);
+  return FP4ATTN_OK;
+}
+
+extern "C" int fp4attn_quantize_v_e4m3(const void* x, int B, int H, int N, int d, void* bytes_out, float* G_out,
+                                       void* workspace, size_t workspace_bytes, fp4attn_stream_t stream) {
+  if (!x || !bytes_out || !G_out) return FP4ATTN_ERR_INVALID_ARG;
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return FP4ATTN_ERR_INVALID_ARG;
+  if (!shape_ok(B, H, N, d)) return FP4ATTN_ERR_UNSUPPORTED_SHAPE;
+  if (((uintptr_t)x | (uintptr_t)bytes_out) & 15) return FP4ATTN_ERR_ALIGNMENT;
+  const size_t need = fp4attn_quantize_v_e4m3_workspace_bytes(B, H, N, d);
+  if (!workspace || workspace_bytes < need) return FP4ATTN_ERR_WORKSPACE;
+  if ((uintptr_t)workspace & 15) return FP4ATTN_ERR_ALIGNMENT;
+  int rc = check_device_sm100();
+  if (rc != FP4ATTN_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const uint4* xs = reinterpret_cast<const uint4*>(x);
+  const size_t groups_per_unit = (size_t)N * d / 8;
+  const unsigned gx = (unsigned)(groups_per_unit / kGroupsPerCta);
+  const int n_partials = (int)(gx < (unsigned)kPartialsPerHead ? gx : kPartialsPerHead);
+  amax_partials_kernel<<<dim3(n_partials, B * H), kThreads, 0, st>>>(xs, groups_per_unit, (float*)workspace);
+  e4m3_encode_factor_kernel<<<B * H, kThreads, 0, st>>>((const float*)workspace, n_partials, G_out);
+  rc = d == 128 ? launch_e4m3_v<128>(xs, B * H, N, bytes_out, G_out, st) : launch_e4m3_v<64>(xs, B * H, N, bytes_out, G_out, st);
+  if (rc != FP4ATTN_OK) return rc;
+  return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
