@@ -188,18 +188,23 @@ def oracle_sample(w, q, k, v, n_heads, rows, p_map="ideal", p_scale="ceil", amax
     return dt, flops / dt / 1e12, O, lse, (qd, kd, vd)
 
 
-def accuracy_vs_fp64(q, k, v, ops, rows, O_gpu, O_oracle):
+def accuracy_vs_fp64(q, k, v, ops, rows, O_gpu, O_oracle, O_gpu_fp8=None):
     """cos / rel-L2 against unquantised fp64 attention of: the CUDA path, the oracle, and O_exactP (quantised
     Q, K, V with an exact softmax - what is left when P is not quantised)."""
     from oracle import attention as A
     from oracle import quantize as Qz
-    keys = ("gpu", "oracle", "exact_p")
+    keys = ("gpu", "oracle", "exact_p") + (("gpu_fp8_pv", "oracle_fp8_pv") if O_gpu_fp8 is not None else ())
     num = {key: [0.0, 0.0, 0.0, 0.0] for key in keys}
+    v8 = Qz.quantize_v_e4m3(v) if O_gpu_fp8 is not None else None
     for n in range(q.shape[1]):
         x = [Qz.bf16_bits_to_f64(a[0, n]) for a in (q, k, v)]
         Oe, _ = A.exact_attention(x[0], x[1], x[2], rows=rows)
         Op, _ = A.exact_p_attention(ops[0], ops[1], ops[2], 0, n, rows=rows)
-        for key, O in (("gpu", O_gpu[n]), ("oracle", O_oracle[n]), ("exact_p", Op)):
+        outs = [("gpu", O_gpu[n]), ("oracle", O_oracle[n]), ("exact_p", Op)]
+        if O_gpu_fp8 is not None:
+            O8, _ = A.fp8_pv_forward(ops[0], ops[1], v8, rows=rows, heads=[(0, n)])
+            outs += [("gpu_fp8_pv", O_gpu_fp8[n]), ("oracle_fp8_pv", O8[0])]
+        for key, O in outs:
             acc = num[key]
             acc[0] += (O * Oe).sum(); acc[1] += (O * O).sum(); acc[2] += (Oe * Oe).sum(); acc[3] += ((O - Oe) ** 2).sum()
     out = {}
@@ -465,7 +470,17 @@ def run_cuda(args, w):
             ms_map = statistics.median(timed_launches(fn, 10, flush, E, torch.cuda.synchronize))
             other_maps[name] = {"attn_ms": ms_map, "attn_tflops": w.flops / (ms_map * 1e-3) / 1e12,
                                 "roofline_frac": w.flops / (ms_map * 1e-3) / 1e12 / fp4_peak}
-        del O_alt
+        # the FP8 P/V route on the same Q, K (E4M3 V with per-unit factors, E4M3 probabilities)
+        v8 = Bd.fp4attn_quantize_v_e4m3(dv)
+        fn = lambda: Bd.fp4attn_fwd(qd0, kd0, v8, out=O_alt, status=status)
+        for _ in range(3):
+            fn()
+        ms_map = statistics.median(timed_launches(fn, 10, flush, E, torch.cuda.synchronize))
+        other_maps["fp8_pv"] = {"attn_ms": ms_map, "attn_tflops": w.flops / (ms_map * 1e-3) / 1e12,
+                                "roofline_frac": w.flops / (ms_map * 1e-3) / 1e12 / fp4_peak,
+                                "note": "kind::f8f6f4 second product; its own denominator would be the FP8 roof, half the FP4 one"}
+        state["O_fp8"] = O_alt
+        del v8
 
     # ---- measured dense FP4 issue rate of this device (context for the roofline)
     cyc = torch.zeros(1, dtype=torch.int64, device=dev)
@@ -494,6 +509,9 @@ def run_cuda(args, w):
         amax = (float(dq.abs().max()), float(dk.abs().max())) if w.qk_fmt == I.FMT_NVFP4 else None
         sample = dict(rows=rows, heads=heads, q=pick(dq), k=pick(dk), v=pick(dv), amax=amax,
                       Og=np.stack([O[b, h].float().cpu().numpy().astype(np.float64)[rows] for b, h in heads]))
+        if "O_fp8" in state:
+            sample["Og8"] = np.stack([state["O_fp8"][b, h].float().cpu().numpy().astype(np.float64)[rows] for b, h in heads])
+    state.pop("O_fp8", None)
 
     # ---- attention kernel alone on the other configurations, each with a roofline fraction of its own (seeded
     # inputs of that configuration; every timed launch follows an L2 flush; median of the launches)
@@ -510,6 +528,7 @@ def run_cuda(args, w):
             sq = Bd.fp4attn_quantize(xq, ww.qk_fmt, Bd.ROLE_Q)
             sk = Bd.fp4attn_quantize(xk, ww.qk_fmt, Bd.ROLE_K)
             sv = Bd.fp4attn_quantize(xv, Bd.FMT_MXFP4, Bd.ROLE_V)
+            sv8 = Bd.fp4attn_quantize_v_e4m3(xv)
             del xq, xk, xv
             so = torch.empty((ww.B, ww.H, ww.N, ww.d), dtype=torch.bfloat16, device=dev)
             rec = {"workload": _workload_text(ww), "launches": n_it, "inputs": "seeded recipe of the configuration"}
@@ -517,8 +536,10 @@ def run_cuda(args, w):
             if ww.d == 64 and ww.N % 256 == 0:                       # the two-query schedule beside the one-query one
                 variants += [("two_query_", dict(schedule=Bd.SCHEDULE_TWO_QUERY), 1.0),
                              ("two_query_affine_", dict(schedule=Bd.SCHEDULE_TWO_QUERY, p_map=Bd.PMAP_AFFINE), 1.0)]
+            variants.append(("fp8_pv_", None, 1.0))
             for key, kw, share in variants:
-                fn = lambda: Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status, **kw)
+                fn = (lambda: Bd.fp4attn_fwd(sq, sk, sv8, out=so, status=status)) if kw is None else \
+                     (lambda: Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status, **kw))
                 for _ in range(3):
                     fn()
                 torch.cuda.synchronize()
@@ -531,7 +552,7 @@ def run_cuda(args, w):
                 else:
                     rec[key + "roofline_frac"] = share * ww.flops / (ms * 1e-3) / 1e12 / fp4_peak
             sweep[name] = rec
-            del sq, sk, sv, so
+            del sq, sk, sv, sv8, so
             torch.cuda.empty_cache()
         assert int(status.item()) == 0, "attention kernel reported a bounded-wait timeout"
 
@@ -584,7 +605,7 @@ def run_cuda(args, w):
                                    "rows_above_max_abs": int((row_abs > 2e-2).sum()),
                                    "tolerance": {"rel_fro": 5e-3, "max_abs": 2e-2},
                                    "ok": bool(rel <= 5e-3 and row_abs.max() <= 2e-2)}
-        out["accuracy_vs_fp64"] = accuracy_vs_fp64(sample["q"], sample["k"], sample["v"], ops, rows, Og, Oo)
+        out["accuracy_vs_fp64"] = accuracy_vs_fp64(sample["q"], sample["k"], sample["v"], ops, rows, Og, Oo, sample.get("Og8"))
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

@@ -6,7 +6,7 @@ this script is the same comparison (tests/parity.py: strict figures, and the pro
 correct value) over ALL units, for the record.  One launch of the configuration as bench.py launches it, then the
 oracle on a pool of host processes, one unit per task.
 
-  python tests/run_full_parity.py cfg4 [--p-map affine] [--workers 12] [--units 0:32]
+  python tests/run_full_parity.py cfg4 [--p-map affine] [--route fp8] [--workers 12] [--units 0:32]
 
 Prints one JSON line per unit and a summary line.  Needs a B200; imports the oracle (test infrastructure).
 """
@@ -49,10 +49,12 @@ def _unit(task):
         kd = {"nib": nk, "sf": sk, "G": Gk, "fmt": "nv"}
     else:
         qd, kd = Qz.quantize_qk(one(q), "mx"), Qz.quantize_qk(one(k), "mx")
-    vd = Qz.quantize_v(one(v))
     t0 = time.perf_counter()
     try:
-        st = parity.compare_head(Og[b, h].astype(np.float64), Lg[b, h].astype(np.float64), qd, kd, vd, 0, 0, **okw)
+        if _G["route"] == "fp8":
+            st = _fp8_head(Og[b, h].astype(np.float64), Lg[b, h].astype(np.float64), qd, kd, Qz.quantize_v_e4m3(one(v)))
+        else:
+            st = parity.compare_head(Og[b, h].astype(np.float64), Lg[b, h].astype(np.float64), qd, kd, Qz.quantize_v(one(v)), 0, 0, **okw)
         st["ok"] = True
     except AssertionError as e:
         st = {"ok": False, "error": str(e)[:400]}
@@ -61,10 +63,31 @@ def _unit(task):
     return st
 
 
+def _fp8_head(Og, Lg, qd, kd, v8, chunk=1024):
+    """FP8 P/V route: strict comparison of one unit, all rows (no alternative evaluations are defined for it)."""
+    import parity
+    from oracle import attention as A
+    N = Og.shape[0]
+    num = den = 0.0
+    worst = lse_err = 0.0
+    for r0 in range(0, N, chunk):
+        rows = np.arange(r0, min(N, r0 + chunk))
+        Oo, Lo = A.fp8_pv_forward(qd, kd, v8, rows=rows, heads=[(0, 0)])
+        num += ((Og[rows] - Oo[0]) ** 2).sum()
+        den += (Oo[0] ** 2).sum()
+        worst = max(worst, float(np.abs(Og[rows] - Oo[0]).max()))
+        lse_err = max(lse_err, float((np.abs(Lg[rows] - Lo[0]) - parity.LSE_REL * np.abs(Lo[0])).max()))
+    st = {"rows": int(N), "rel_fro_strict": float(np.sqrt(num / den)), "max_abs_strict": worst, "lse_err": lse_err,
+          "rows_failing_strict": 0, "accepted_with_flips": 0}
+    assert st["rel_fro_strict"] <= parity.REL_FRO and worst <= parity.MAX_ABS and lse_err <= parity.LSE_ABS, st
+    return st
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("workload", choices=sorted(I.WORKLOADS))
     ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine"])
+    ap.add_argument("--route", default="fp4", choices=["fp4", "fp8"], help="probability / value format: Direct-P FP4 or FP8 P/V")
     ap.add_argument("--workers", type=int, default=max(1, len(os.sched_getaffinity(0)) - 2))
     ap.add_argument("--units", default=None, help="begin:end slice of the (batch, head) units, default all")
     args = ap.parse_args()
@@ -76,12 +99,12 @@ def main():
     dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
     qg = Bd.fp4attn_quantize(dev(q), w.qk_fmt, Bd.ROLE_Q)
     kg = Bd.fp4attn_quantize(dev(k), w.qk_fmt, Bd.ROLE_K)
-    vg = Bd.fp4attn_quantize(dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    vg = Bd.fp4attn_quantize_v_e4m3(dev(v)) if args.route == "fp8" else Bd.fp4attn_quantize(dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     O, L = Bd.fp4attn_fwd(qg, kg, vg, status=status, p_map=Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_IDEAL)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    _G.update(w=w, q=q, k=k, v=v, O=O.float().cpu().numpy(), L=L.cpu().numpy(), Gq=None, Gk=None,
+    _G.update(route=args.route, w=w, q=q, k=k, v=v, O=O.float().cpu().numpy(), L=L.cpu().numpy(), Gq=None, Gk=None,
               okw=dict(p_map=args.p_map))
     if w.qk_fmt == I.FMT_NVFP4:
         _G["Gq"] = Qz.nv_tensor_scale(Qz.bf16_bits_to_f64(q))
@@ -99,7 +122,7 @@ def main():
             print(json.dumps(st), flush=True)
             res.append(st)
     good = [r for r in res if r["ok"]]
-    summary = {"workload": w.name, "p_map": args.p_map, "units": len(res), "units_ok": len(good),
+    summary = {"workload": w.name, "route": args.route, "p_map": args.p_map, "units": len(res), "units_ok": len(good),
                "rows": int(sum(r["rows"] for r in good)), "wall_s": round(time.perf_counter() - t0, 1)}
     if good:
         summary.update(rel_fro_strict_max=max(r["rel_fro_strict"] for r in good), max_abs_strict=max(r["max_abs_strict"] for r in good),
