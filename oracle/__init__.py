@@ -27,5 +27,10 @@ Pinned by tests/test_oracle_*.py (run with -m "not gpu"):
                                                   -> position by position against the two pinned maps,
                                                   error monotone in the share of exact pairs; per-head
                                                   factors -> bit-identical output under 2^a / 2^-a scaling
-                                                  of a query head and its key head
+                                                  of a query head and its key head;
+                                                  FP8 P/V route (E4M3 V per unit, E4M3 probabilities against the
+                                                  integer row maximum) -> the E4M3 grid written out independently,
+                                                  ties, saturation; closed forms of the V factor; representable
+                                                  probabilities against brute force; constant V, flushing, key
+                                                  permutation, causal prefix; the accuracy level the paper reports
 """
