@@ -123,3 +123,29 @@ def test_fp8_pv_rejects_the_fp4_only_options():
     for kw in (dict(p_map=Bd.PMAP_AFFINE), dict(p_scale_rule=Bd.PSCALE_THR16), dict(schedule=Bd.SCHEDULE_TWO_QUERY)):
         with pytest.raises(Bd.Fp4AttnError):
             Bd.fp4attn_fwd(qg, kg, vg, **kw)
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_fp8_pv_random_configurations_match_oracle(seed):
+    """Thirty seeded draws of (d, Q/K format, N, B, heads, K/V head sharing, mask, softmax scale, outlier channels)
+    per seed: sampled rows of two heads each against the oracle."""
+    from paper_2609_04105_b200 import binding as Bd
+    rng = np.random.default_rng(100 + seed)
+    for _ in range(30):
+        d = int(rng.choice([64, 128])); nv = bool(rng.integers(0, 2))
+        N = 128 * int(rng.integers(1, 9)); B = int(rng.integers(1, 4))
+        group = int(rng.choice([1, 1, 2, 4])); Hkv = int(rng.integers(1, 4)); H = Hkv * group
+        causal = bool(rng.integers(0, 2)); scale = float(rng.choice([0.0, 0.05, 0.3]))
+        x = [rng.standard_normal((B, h, N, d)).astype(np.float32) for h in (H, Hkv, Hkv)]
+        if rng.integers(0, 4) == 0:
+            ch = rng.choice(d, size=3, replace=False)
+            x[0][..., ch] *= 20
+            x[1][..., ch] *= 20
+        bits = [I.f32_to_bf16_bits(a) for a in x]
+        w = I.Workload("rand", 0, B, H, N, d, I.FMT_NVFP4 if nv else I.FMT_MXFP4)
+        Og, Lg = _run(w, bits[0], bits[1], bits[2], causal=causal, group=group, softmax_scale=scale)
+        heads = [(int(rng.integers(0, B)), int(rng.integers(0, H))) for _ in range(2)]
+        rows = np.sort(rng.choice(N, size=min(N, 48), replace=False))
+        rows[0], rows[-1] = 0, N - 1
+        _check(w, bits[0], bits[1], bits[2], Og, Lg, heads, rows, causal=causal, group=group,
+               softmax_scale=(scale if scale > 0 else None))
