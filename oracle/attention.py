@@ -34,6 +34,10 @@ Mixed map (p_map="hybrid", the paper's EX2-density control, Appendix "SM103 laun
 element pair k of a block (keys 2k, 2k+1) takes the ideal map where bit k of `exact_pairs` is set and the
 affine map elsewhere; which pairs pay for an exponential is a fixed pattern, so a GPU reproduces it.
 
+Third block-exponent rule (p_scale="mse"): per block the better of the two neighbouring powers by squared error of
+the represented values (see mse_exponent_of inside direct_p_rows); it reproduces the MXFP4 rows of Table "p-range" and
+is a near-decision wherever the two error sums almost tie.
+
 Second block-exponent rule (p_scale="thr16"): Eq. "mx-scale" allows either neighbouring power of two
 as the amplitude; besides the ceiling (default) the oracle offers the threshold rule
 E_B = floor(fl32(max y + fl32(log2 1.6))), i.e. alpha_B = 2^floor(log2(1.6 a_B)): the block maximum then
@@ -181,6 +185,8 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
     def exponent_of(bj):
         """Block exponent of keys bj..bj+31 (with its flip applied), and whether it is a near-decision."""
         ymax = y32[:, bj:bj + P_BLOCK].max(axis=1)
+        if p_scale == "mse":
+            return mse_exponent_of(bj, ymax)
         E = block_exponent(ymax, p_scale)
         w = ymax if p_scale == "ceil" else (ymax + LOG2_1P6_32).astype(np.float32)   # the value that is rounded to an integer
         w64 = w.astype(np.float64)
@@ -191,6 +197,27 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
             other = np.where(E == n, n + (1 if p_scale == "ceil" else -1), n)      # the integer on the other side of w
             E = np.where(flip_eb[:, bj // P_BLOCK] & np.isfinite(w64), other, E)
         return E, near
+
+    def mse_exponent_of(bj, ymax):
+        """Eq. "mx-scale" names both powers of two next to the block maximum; this rule takes, per block, the one
+        with the smaller squared error of the 32 represented values: with v = 6 * 2**(y - E_c) under the ceiling
+        E_c = ceil(max y), the floor E_c - 1 doubles every v (values above 6 saturate), and its error sum is in
+        units four times smaller, so the floor wins iff sum (2v - q(2v))**2 < 4 sum (v - q(v))**2 (strictly; a
+        block whose maximum is an integer has one candidate only).  Near-decision: the two sides within 1e-3 of
+        each other relative to their sum (an implementation evaluates 2**x approximately and sums in float32)."""
+        Ec = np.ceil(ymax.astype(np.float64))
+        fin = np.isfinite(Ec)
+        Ec0 = np.where(fin, Ec, 0.0)
+        b32 = np.float32(LOG2_6_32 - Ec0.astype(np.float32))
+        v = np.exp2(yx[:, bj:bj + P_BLOCK] + b32.astype(np.float64)[:, None])
+        ec = ((v - E2M1_VALUES[e2m1_encode_mag(v)]) ** 2).sum(axis=1)
+        ef = ((2 * v - E2M1_VALUES[e2m1_encode_mag(2 * v)]) ** 2).sum(axis=1)
+        two = fin & (ymax.astype(np.float64) != Ec)                # two candidates
+        take_f = two & (ef < 4.0 * ec)
+        near = two & (np.abs(ef - 4.0 * ec) <= 1e-3 * (ef + 4.0 * ec))
+        if flip_eb is not None:
+            take_f = np.where(flip_eb[:, bj // P_BLOCK] & two, ~take_f, take_f)
+        return np.where(fin, Ec0 - take_f, Ec), near
 
     order = range(N // tile) if tile_order is None else tile_order
     for t in order:

@@ -551,3 +551,69 @@ def test_exact_p_output_sits_between_direct_p_and_unquantized_attention():
     Od, _ = A.direct_p_forward(qd, kd, vd, heads=[(0, 1)])
     rel = lambda a: np.linalg.norm(a - O64) / np.linalg.norm(O64)
     assert rel(Oe) < rel(Od[0]) and 0.15 < rel(Oe) < 0.26 and 0.22 < rel(Od[0]) < 0.32
+
+
+# ------------------------------------------------------------------ MSE-selected block exponent for P
+def test_mse_rule_picks_the_exponent_with_the_smaller_block_error_brute_force():
+    """For every block the chosen exponent is one of ceil(max y), ceil(max y) - 1 and has the smaller squared error of
+    the represented probabilities in absolute units (brute force in Python floats); blocks whose maximum is an integer
+    keep the ceiling; codes under the chosen exponent are Q_E2M1(6 * 2**(y - E)) saturating at 6."""
+    rng = np.random.default_rng(9)
+    R, N = 6, 256
+    y = (rng.standard_normal((R, N)) * 2.0).astype(np.float32)
+    y[0, :32] = np.minimum(y[0, :32], 3.5)
+    y[0, 3] = 4.0                                               # an integer block maximum: no alternative
+    vals = [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+    _, _, codes, EB, _ = A.direct_p_rows(y, np.float32(1.0), np.ones((N, 1)), p_scale="mse")
+    n_floor = 0
+    for i in range(R):
+        for b in range(N // 32):
+            yb = [float(t) for t in y[i, 32 * b:32 * b + 32]]
+            Ec = math.ceil(max(yb))
+            errs = {}
+            for E in (Ec, Ec - 1):
+                err = 0.0
+                for t in yb:
+                    v = 6.0 * 2.0 ** (t - E)
+                    qv = min(vals, key=lambda c: (abs(c - min(v, 6.0)), c % 1.0 != 0 or (c / 0.5) % 2))   # nearest; exact ties do not occur here
+                    err += (2.0 ** E / 6.0) ** 2 * (v - qv) ** 2
+                errs[E] = err
+            want = Ec - 1 if (max(yb) != Ec and errs[Ec - 1] < errs[Ec]) else Ec
+            assert EB[i, b] == want, (i, b, errs)
+            n_floor += want != Ec
+            assert np.array_equal(codes[i, 32 * b:32 * b + 32], F.e2m1_encode_mag(6.0 * np.exp2(np.array(yb) - want)))
+    assert EB[0, 0] == 4 and 0.2 < n_floor / (R * N // 32) < 0.6     # the floor wins in roughly a third of Gaussian blocks
+
+
+def test_mse_rule_reproduces_table_p_range_mxfp4_row_and_reports_near_ties():
+    """Table "p-range", MXFP4 row at S = 1024: 0.188683 / 0.040178 / 0.146380 / 0.989846 (zero payload, lost mass,
+    P rel-L2, PV cosine).  The per-block least-squares choice reproduces it, closer than the threshold rule; a block
+    whose two error sums almost tie is reported and can be taken the other way."""
+    rng = np.random.default_rng(4)
+    S, d, R = 1024, 128, 192
+    q, k, V = rng.standard_normal((R, d)), rng.standard_normal((S, d)), rng.standard_normal((S, d))
+    z = q @ k.T / math.sqrt(d)
+    p = np.exp(z - z.max(axis=1, keepdims=True))
+    p /= p.sum(axis=1, keepdims=True)
+    y = np.log2(p).astype(np.float32)
+    rep = {}
+    _, _, codes, EB, _ = A.direct_p_rows(y, np.float32(1.0), V, tile=128, p_scale="mse", report=rep, ambiguity=dict(share=0.0))
+    phat = np.repeat(np.ldexp(1.0, EB), 32, axis=1) * F.E2M1_VALUES[codes] / 6.0
+    pn = phat / phat.sum(axis=1, keepdims=True)
+    rel = np.linalg.norm(pn - p) / np.linalg.norm(p)
+    o, oh = p @ V, pn @ V
+    assert np.mean(phat == 0) == pytest.approx(0.188683, rel=0.03)
+    assert np.mean((p * (phat == 0)).sum(axis=1)) == pytest.approx(0.040178, rel=0.04)
+    assert rel == pytest.approx(0.146380, rel=0.02)
+    assert (o * oh).sum() / np.linalg.norm(o) / np.linalg.norm(oh) == pytest.approx(0.989846, abs=1.5e-3)
+    _, _, c2, E2, _ = A.direct_p_rows(y, np.float32(1.0), V, tile=128, p_scale="thr16")
+    ph2 = np.repeat(np.ldexp(1.0, E2), 32, axis=1) * F.E2M1_VALUES[c2] / 6.0
+    pn2 = ph2 / ph2.sum(axis=1, keepdims=True)
+    assert rel <= np.linalg.norm(pn2 - p) / np.linalg.norm(p) * 1.002      # least squares per block is at least as good
+    near = rep["eb"]
+    assert 0 < near.mean() < 0.01                                   # near-ties exist and are rare
+    i, b = (int(t[0]) for t in np.nonzero(near))
+    fl = np.zeros((1, S // 32), bool)
+    fl[0, b] = True
+    _, _, _, E3, _ = A.direct_p_rows(y[i:i + 1], np.float32(1.0), V, tile=128, p_scale="mse", flips={"eb": fl})
+    assert abs(int(E3[0, b]) - int(EB[i, b])) == 1 and np.array_equal(np.delete(E3[0], b), np.delete(EB[i], b))
