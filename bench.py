@@ -330,7 +330,7 @@ def run_cuda(args, w):
     launches_per_step = 4 if w.qk_fmt == I.FMT_MXFP4 else 8          # NVFP4: amax pass + encode factor + codes, for Q and for K
     pmap = Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_HYBRID if args.p_map in HYBRID_PATTERNS else Bd.PMAP_IDEAL
     pairs = HYBRID_PATTERNS.get(args.p_map, 0)
-    pscale = Bd.PSCALE_THR16 if args.p_scale == "thr16" else Bd.PSCALE_CEIL
+    pscale = {"thr16": Bd.PSCALE_THR16, "mse": Bd.PSCALE_MSE}.get(args.p_scale, Bd.PSCALE_CEIL)
     sched = Bd.SCHEDULE_TWO_QUERY if args.schedule == "two-query" else Bd.SCHEDULE_ONE_QUERY
     state = {}
     E = lambda: torch.cuda.Event(enable_timing=True)
@@ -622,8 +622,9 @@ def main():
                     help="length of the median window that follows the K timed steps (0 skips it)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the attention-only timings of the other configurations")
-    ap.add_argument("--p-scale", default="ceil", choices=["ceil", "thr16"],
-                    help="block-exponent rule of P: ceiling (default) or floor(max y + log2 1.6)")
+    ap.add_argument("--p-scale", default="ceil", choices=["ceil", "thr16", "mse"],
+                    help="block-exponent rule of P: ceiling (default), floor(max y + log2 1.6), or per block the better of "
+                         "the two neighbouring exponents by squared error (ideal map only)")
     ap.add_argument("--schedule", default="one-query", choices=["one-query", "two-query"],
                     help="query tiles per thread block in the timed step (two-query: d = 64 workloads only)")
     ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine", "hybrid4", "hybrid8", "hybrid12"],

@@ -175,8 +175,14 @@ int fp4attn_quantize_nvfp4_per_head(const void* x_bf16, int role, int B, int H, 
 /* how the integer exponent E_B of a 32-key probability block follows from its maximum y (Eq. "mx-scale"
  * allows either neighbouring power of two as the amplitude) */
 enum { FP4ATTN_PSCALE_CEIL = 0,    /* E_B = ceil(max y): nothing saturates                              */
-       FP4ATTN_PSCALE_THR16 = 1 }; /* E_B = floor(fl32(max y + fl32(log2 1.6))): the block maximum lands in
+       FP4ATTN_PSCALE_THR16 = 1,   /* E_B = floor(fl32(max y + fl32(log2 1.6))): the block maximum lands in
                                       [3.75, 7.5) code units, values above 6 saturate; lower P error    */
+       FP4ATTN_PSCALE_MSE = 2 };   /* per block the better of ceil(max y) and ceil(max y) - 1 by squared error of the
+                                      32 represented probabilities: with v = 6 * 2^(y - ceil) the lower exponent wins
+                                      iff sum (2v - q(2v))^2 < 4 sum (v - q(v))^2 (fp32 sums over groups of eight keys,
+                                      groups as (g0 + g1) + (g2 + g3)); 2^x by ex2.approx, so a block whose two sums
+                                      almost tie may take either exponent.  With the ideal map, one NVFP4 factor per
+                                      tensor and the one-query schedule only; about twice the conversions per block */
 
 /* how query tiles are assigned to thread blocks (Section "Two-query execution model") */
 enum { FP4ATTN_SCHEDULE_ONE_QUERY = 0,   /* one 128-row query tile per thread block: every shape                 */
@@ -201,7 +207,7 @@ typedef struct {
   int p_map;                        /* FP4ATTN_PMAP_IDEAL, _AFFINE or _HYBRID                */
   float affine_a, affine_b;         /* classifier constants; affine_a == 0 selects the
                                        paper's generic fit A = 1.50, B = 1.20                */
-  int p_scale_rule;                 /* FP4ATTN_PSCALE_CEIL or FP4ATTN_PSCALE_THR16           */
+  int p_scale_rule;                 /* FP4ATTN_PSCALE_CEIL, _THR16 or _MSE                   */
   int causal;                       /* 1: query row i attends keys 0..i only; 0: all keys     */
   int kv_heads;                     /* K and V hold this many heads ([B, kv_heads, N, d]);
                                        H query heads share them in groups of H / kv_heads

@@ -15,7 +15,7 @@ import torch
 FMT_MXFP4, FMT_NVFP4 = 0, 1
 ROLE_Q, ROLE_K, ROLE_V = 0, 1, 2
 PMAP_IDEAL, PMAP_AFFINE, PMAP_HYBRID = 0, 1, 2
-PSCALE_CEIL, PSCALE_THR16 = 0, 1
+PSCALE_CEIL, PSCALE_THR16, PSCALE_MSE = 0, 1, 2
 SCHEDULE_ONE_QUERY, SCHEDULE_TWO_QUERY = 0, 1
 PV_MXFP4, PV_E4M3 = 0, 1
 QSCALE_CEIL, QSCALE_THR16, QSCALE_FLOOR, QSCALE_MSE = 0, 1, 2, 3

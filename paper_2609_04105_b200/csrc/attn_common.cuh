@@ -192,9 +192,16 @@ __device__ __forceinline__ void exp2_poly6(float x0, float x1, float& p0, float&
 __host__ __device__ constexpr uint32_t exact_pairs_of(int pmap) {
   return pmap == 0 ? 0xFFFFu : pmap == 1 ? 0x0000u : pmap == 2 ? 0x1111u : pmap == 3 ? 0x5555u : 0x7777u;
 }
-template <int PMAP, bool MASKED, bool THR16>
+// RULE: block exponent from the block maximum - 0 ceiling, 1 threshold rule, 2 the better of ceiling and ceiling - 1 by
+// squared error of the 32 represented values (ideal map only; see direct_p_block_mse)
+template <bool MASKED>
+__device__ __forceinline__ void direct_p_block_mse(uint32_t* sraw, float c32, int visible, int& E, uint32_t* words);
+
+template <int PMAP, bool MASKED, int RULE>
 __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float A, float B, int visible, int& E,
                                                uint32_t* words) {
+  if (RULE == 2) { direct_p_block_mse<MASKED>(sraw, c32, visible, E, words); return; }
+  constexpr bool THR16 = RULE == 1;
   constexpr uint32_t kExact = exact_pairs_of(PMAP);
   const float LOG2_6 = 2.5849625007211560f;
   if (MASKED) {                                                 // causal diagonal: keys beyond the query get -inf
@@ -235,6 +242,51 @@ __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float 
     // the conversion clamps negative inputs to +0 (affine pairs; exact pairs are positive anyway)
     words[w] = kExact == 0xFFFFu ? cvt_e2m1x8(pv) : cvt_e2m1x8_relu(pv);
   }
+}
+
+// Eq. "mx-scale" names both powers of two next to a block maximum.  Here every block takes, of E_c = ceil(max y) and
+// E_c - 1, the one with the smaller squared error of its 32 represented probabilities.  Under E_c the code units are
+// v = 6 * 2^(y - E_c) (every v through ex2.approx: the boundary polynomial is exact only where codes change); under
+// E_c - 1 they are 2v, saturating at 6, in units half as large: the floor wins iff
+//   sum (2v - q(2v))^2 < 4 sum (v - q(v))^2      (strictly; a block whose maximum is an integer has one candidate).
+// Error sums in fp32: eight consecutive keys left to right, the four group sums as (g0 + g1) + (g2 + g3).
+template <bool MASKED>
+__device__ __forceinline__ void direct_p_block_mse(uint32_t* sraw, float c32, int visible, int& E, uint32_t* words) {
+  const float LOG2_6 = 2.5849625007211560f;
+  if (MASKED) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) sraw[i] = (i < visible) ? sraw[i] : 0xFF800000u;
+  }
+  const float ymax = fminf(fmaxf(__fmul_rn(max32(sraw), c32), -2097152.0f), 2097152.0f);
+  const float M = 12582912.0f;
+  const float t = __fadd_ru(ymax, M);
+  const float Ec = __fsub_rn(t, M);                              // ceil(ymax), exact
+  const float bB = __fsub_rn(LOG2_6, Ec);
+  float gc[4], gf[4];
+  uint32_t wc[4], wf[4];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    float v[8], v2[8];
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+      float x0, x1;
+      fma2(__uint_as_float(sraw[8 * w + i]), __uint_as_float(sraw[8 * w + i + 1]), c32, bB, x0, x1);
+      v[i] = ex2_approx(x0);
+      v[i + 1] = ex2_approx(x1);
+      v2[i] = __fmul_rn(2.0f, v[i]);
+      v2[i + 1] = __fmul_rn(2.0f, v[i + 1]);
+    }
+    wc[w] = cvt_e2m1x8(v);
+    wf[w] = cvt_e2m1x8(v2);                                      // saturates at 6
+    gc[w] = mx_error_x8(v, wc[w]);
+    gf[w] = mx_error_x8(v2, wf[w]);
+  }
+  const float ec = __fadd_rn(__fadd_rn(gc[0], gc[1]), __fadd_rn(gc[2], gc[3]));
+  const float ef = __fadd_rn(__fadd_rn(gf[0], gf[1]), __fadd_rn(gf[2], gf[3]));
+  const bool take_f = (ymax != Ec) && (ef < __fmul_rn(4.0f, ec));
+  E = (int)(__float_as_uint(t) - 0x4B400000u) - (take_f ? 1 : 0);
+#pragma unroll
+  for (int w = 0; w < 4; ++w) words[w] = take_f ? wf[w] : wc[w];
 }
 
 // Tensor maps of a launch (Q, K, V^T, O in that order) from the calling thread's cache; nullptr if the driver

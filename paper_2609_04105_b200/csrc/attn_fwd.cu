@@ -34,7 +34,7 @@ using namespace ptx;
 // NV: 0 - MXFP4 Q, K; 1 - NVFP4 with one encode factor per tensor; 2 - NVFP4 with one factor per (batch, head)
 // unit (an instance of its own: a score constant that changes per work item costs the tensor-wide variant
 // 2-8 % when it is only a run-time branch)
-template <int D, int NV, int PMAP, bool CAUSAL, bool THR16>
+template <int D, int NV, int PMAP, bool CAUSAL, int THR16>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -605,7 +605,7 @@ const CUtensorMap* attention_tensor_maps_fp8v(int D, const fp4attn_operands* ops
   return D == 128 ? tensor_maps<128>(ops, O, B, H, Hkv, N, true) : tensor_maps<64>(ops, O, B, H, Hkv, N, true);
 }
 
-template <int D, int NV, int PMAP, bool CAUSAL, bool THR16>
+template <int D, int NV, int PMAP, bool CAUSAL, int THR16>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
   const int Hkv = prm.Hkv;
   using C = Cfg<D, (NV != 0)>;
@@ -651,7 +651,11 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
     pmap = ops->exact_pairs == 0x1111 ? 2 : ops->exact_pairs == 0x5555 ? 3 : ops->exact_pairs == 0x7777 ? 4 : -1;
     if (pmap < 0 || ops->causal) return FP4ATTN_ERR_INVALID_ARG;    // three patterns, noncausal only
   }
-  if (ops->p_scale_rule != FP4ATTN_PSCALE_CEIL && ops->p_scale_rule != FP4ATTN_PSCALE_THR16) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->p_scale_rule != FP4ATTN_PSCALE_CEIL && ops->p_scale_rule != FP4ATTN_PSCALE_THR16 && ops->p_scale_rule != FP4ATTN_PSCALE_MSE)
+    return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->p_scale_rule == FP4ATTN_PSCALE_MSE &&
+      (ops->p_map != FP4ATTN_PMAP_IDEAL || ops->g_per_head || ops->schedule != FP4ATTN_SCHEDULE_ONE_QUERY || ops->pv_fmt != FP4ATTN_PV_MXFP4))
+    return FP4ATTN_ERR_INVALID_ARG;                                 // ideal map, one factor per tensor, one-query schedule
   if (ops->g_per_head != 0 && ops->g_per_head != 1) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->g_per_head && ops->p_map == FP4ATTN_PMAP_HYBRID) return FP4ATTN_ERR_INVALID_ARG;   // ideal and affine maps only
   if (ops->kv_heads < 0 || (ops->kv_heads > 0 && H % ops->kv_heads != 0) || (ops->causal != 0 && ops->causal != 1))
@@ -685,6 +689,19 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   if (ops->pv_fmt != FP4ATTN_PV_MXFP4 && ops->pv_fmt != FP4ATTN_PV_E4M3) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->pv_fmt == FP4ATTN_PV_E4M3) return launch_attn_fp8pv(ops, B, H, N, d, prm, st);
   if (ops->schedule == FP4ATTN_SCHEDULE_TWO_QUERY) return launch_attn_two_query(ops, B, H, N, d, pmap, prm, st);
+  if (ops->p_scale_rule == FP4ATTN_PSCALE_MSE) {
+    const int sel = (d == 128 ? 4 : 0) | (nv ? 2 : 0) | (prm.causal ? 1 : 0);
+    switch (sel) {
+      case 0: return launch_attn<64, 0, 0, false, 2>(ops, B, H, N, prm, st);
+      case 1: return launch_attn<64, 0, 0, true, 2>(ops, B, H, N, prm, st);
+      case 2: return launch_attn<64, 1, 0, false, 2>(ops, B, H, N, prm, st);
+      case 3: return launch_attn<64, 1, 0, true, 2>(ops, B, H, N, prm, st);
+      case 4: return launch_attn<128, 0, 0, false, 2>(ops, B, H, N, prm, st);
+      case 5: return launch_attn<128, 0, 0, true, 2>(ops, B, H, N, prm, st);
+      case 6: return launch_attn<128, 1, 0, false, 2>(ops, B, H, N, prm, st);
+      default: return launch_attn<128, 1, 0, true, 2>(ops, B, H, N, prm, st);
+    }
+  }
   // one kernel instance per (d, Q/K format, P map, mask, P scale rule): nothing of these is decided at run time
   const bool per_head = nv && ops->g_per_head;
   const int shape = (d == 128 ? 2 : 0) | (nv ? 1 : 0);

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 
 #include <atomic>
@@ -39,6 +40,23 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8_relu(const float* v) {
   return w;
 }
 
+// Squared error of eight scaled values t against their codes (one word), in code units: d = t - q exact,
+// fl32(d * d) added left to right in fp32 - the order the MSE amplitude rule is defined with.
+__device__ __forceinline__ float mx_error_x8(const float* t, uint32_t codes) {
+  float acc = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint32_t h2;
+    asm("{\n\t.reg .b8 b;\n\t.reg .b32 s;\n\tshr.b32 s, %1, %2;\n\tcvt.u8.u32 b, s;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}"
+        : "=r"(h2) : "r"(codes), "r"(8 * i));
+    const float2 q = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+    const float d0 = __fsub_rn(t[2 * i], q.x), d1 = __fsub_rn(t[2 * i + 1], q.y);
+    const float s0 = __fmul_rn(d0, d0), s1 = __fmul_rn(d1, d1);
+    acc = (i == 0) ? s0 : __fadd_rn(acc, s0);
+    acc = __fadd_rn(acc, s1);
+  }
+  return acc;
+}
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& raw, float* v) {
   const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll

@@ -1,7 +1,5 @@
 // Operand quantizers: bf16 -> packed E2M1 + scale bytes in the 128x4 atom order.
 // HBM-bound: 128-bit loads, block amax by lane shuffles, 32-bit / 128-bit stores.
-#include <cuda_fp16.h>
-
 #include "common.cuh"
 
 namespace fp4attn {
@@ -50,23 +48,6 @@ __device__ __forceinline__ uint32_t mx_codes_x8(const uint4& raw, uint32_t u) {
   bf16x8_to_f32(raw, v);
   mx_scale_values<8>(v, u);
   return cvt_e2m1x8(v);
-}
-// Squared error of eight scaled values t against their codes (one word), in code units: d = t - q exact,
-// fl32(d * d) added left to right in fp32 - the order the MSE amplitude rule is defined with.
-__device__ __forceinline__ float mx_error_x8(const float* t, uint32_t codes) {
-  float acc = 0.f;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint32_t h2;
-    asm("{\n\t.reg .b8 b;\n\t.reg .b32 s;\n\tshr.b32 s, %1, %2;\n\tcvt.u8.u32 b, s;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}"
-        : "=r"(h2) : "r"(codes), "r"(8 * i));
-    const float2 q = __half22float2(*reinterpret_cast<const __half2*>(&h2));
-    const float d0 = __fsub_rn(t[2 * i], q.x), d1 = __fsub_rn(t[2 * i + 1], q.y);
-    const float s0 = __fmul_rn(d0, d0), s1 = __fmul_rn(d1, d1);
-    acc = (i == 0) ? s0 : __fadd_rn(acc, s0);
-    acc = __fadd_rn(acc, s1);
-  }
-  return acc;
 }
 // MSE rule, blocks along d: the four eight-element groups of a block sit in four adjacent lanes, so the
 // group sums meet as (g0 + g1) + (g2 + g3) in every lane.  The floor's error is in units four times

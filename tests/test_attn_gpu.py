@@ -666,3 +666,37 @@ def test_two_query_schedule_rejects_what_it_does_not_cover():
         q, k, v = I.make_qkv(w)
         with pytest.raises(Bd.Fp4AttnError):
             run_gpu_general(w, q, k, v, schedule=Bd.SCHEDULE_TWO_QUERY, **okw)
+
+
+# ------------------------------------------------------------------ MSE-selected block exponent for P
+@pytest.mark.parametrize("name,kw,causal", [("cfg1", dict(), False), ("cfg1", dict(d=64, N=512, H=3), False),
+                                            ("cfg3", dict(B=2, H=2, N=512), False), ("cfg4", dict(H=2, N=1024), False),
+                                            ("cfg2", dict(B=1, H=2, N=2304), True)])
+def test_mse_block_exponent_matches_oracle_with_near_ties_taken_either_way(name, kw, causal):
+    """Per block the better of the two neighbouring exponents by squared error.  The GPU forms 2^x with ex2.approx and
+    sums in fp32, so a block whose two error sums almost tie may take the other exponent: whole heads are compared
+    under the protocol that accepts a row only if it matches the oracle with some of its reported near-ties flipped."""
+    import parity
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    Og, Lg = run_gpu_general(w, q, k, v, p_scale_rule=Bd.PSCALE_MSE, causal=causal)
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    failing = 0
+    for b in range(w.B):
+        for h in range(w.H):
+            st = parity.compare_head(Og[b, h], Lg[b, h], qd, kd, vd, b, h, chunk=512, p_scale="mse", causal=causal)
+            failing += st["rows_failing_strict"]
+    print(f"{name}: rows that needed a flipped near-tie: {failing}")
+    # the rule is a different operator from the ceiling: on the same inputs the outputs differ visibly
+    Oc, _ = run_gpu_general(w, q, k, v, causal=causal)
+    assert np.abs(Oc - Og).max() > 1e-2
+
+
+def test_mse_block_exponent_rejects_other_maps_and_schedules():
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg1"], d=64, N=256)
+    q, k, v = I.make_qkv(w)
+    for kw in (dict(p_map=Bd.PMAP_AFFINE), dict(schedule=Bd.SCHEDULE_TWO_QUERY), dict(p_map=Bd.PMAP_HYBRID, exact_pairs=0x5555)):
+        with pytest.raises(Bd.Fp4AttnError):
+            run_gpu_general(w, q, k, v, p_scale_rule=Bd.PSCALE_MSE, **kw)
