@@ -464,7 +464,8 @@ def run_cuda(args, w):
                          ("affine", dict(p_map=Bd.PMAP_AFFINE))):
             if name == args.p_map:
                 continue
-            fn = lambda: Bd.fp4attn_fwd(qd0, kd0, vd0, out=O_alt, status=status, p_scale_rule=pscale, **kw)
+            rule = pscale if (pscale != Bd.PSCALE_MSE or name == "ideal") else Bd.PSCALE_CEIL     # the MSE rule exists for the ideal map
+            fn = lambda: Bd.fp4attn_fwd(qd0, kd0, vd0, out=O_alt, status=status, p_scale_rule=rule, **kw)
             for _ in range(3):
                 fn()
             ms_map = statistics.median(timed_launches(fn, 10, flush, E, torch.cuda.synchronize))
