@@ -700,3 +700,48 @@ def test_mse_block_exponent_rejects_other_maps_and_schedules():
     for kw in (dict(p_map=Bd.PMAP_AFFINE), dict(schedule=Bd.SCHEDULE_TWO_QUERY), dict(p_map=Bd.PMAP_HYBRID, exact_pairs=0x5555)):
         with pytest.raises(Bd.Fp4AttnError):
             run_gpu_general(w, q, k, v, p_scale_rule=Bd.PSCALE_MSE, **kw)
+
+
+# ------------------------------------------------------------------ repeated launches of every kernel family
+def test_every_kernel_family_is_deterministic_over_repeated_launches():
+    """Races between the roles of a kernel (a slot reused too early, a missing fence) show up as run-to-run differences
+    long before they show up as wrong averages: thirty launches of each family on a shape with many work items per CTA
+    and an odd number of stages must return bit-identical O and LSE, with other kernels interleaved on the stream."""
+    from paper_2609_04105_b200 import binding as Bd
+    cases = [
+        ("cfg2", dict(B=2, H=5, N=1152), dict()),                                    # one-query, exact map, d = 128
+        ("cfg2", dict(B=2, H=5, N=1152), dict(p_map=Bd.PMAP_AFFINE)),
+        ("cfg2", dict(B=2, H=5, N=1152), dict(causal=True)),
+        ("cfg2", dict(B=2, H=5, N=1152), dict(p_scale_rule=Bd.PSCALE_MSE)),
+        ("cfg4", dict(H=6, N=1152), dict()),                                         # the row reference moves
+        ("cfg3", dict(B=2, H=5, N=1280), dict()),                                    # d = 64, NVFP4
+        ("cfg3", dict(B=2, H=5, N=1280), dict(schedule=Bd.SCHEDULE_TWO_QUERY)),
+        ("cfg3", dict(B=2, H=5, N=1280), dict(schedule=Bd.SCHEDULE_TWO_QUERY, p_map=Bd.PMAP_AFFINE)),
+    ]
+    noise = torch.empty(64 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    for name, kw, okw in cases:
+        w = I.shrink(I.WORKLOADS[name], **kw)
+        q, k, v = I.make_qkv(w)
+        ops = [Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K),
+               Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)]
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        O0, L0 = Bd.fp4attn_fwd(*ops, status=status, **okw)
+        O0, L0 = O0.clone(), L0.clone()
+        for r in range(30):
+            if r % 3 == 0:
+                noise.fill_(r)                                    # evict L2, shift the timing of the loads
+            O, L = Bd.fp4attn_fwd(*ops, status=status, **okw)
+            assert torch.equal(O, O0) and torch.equal(L, L0), (name, okw, r)
+        assert int(status.item()) == 0
+    # the FP8 P/V route
+    w = I.shrink(I.WORKLOADS["cfg2"], B=2, H=5, N=1152)
+    q, k, v = I.make_qkv(w)
+    ops = [Bd.fp4attn_quantize(_dev(q), 0, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(k), 0, Bd.ROLE_K), Bd.fp4attn_quantize_v_e4m3(_dev(v))]
+    for okw in (dict(), dict(causal=True)):
+        O0, L0 = Bd.fp4attn_fwd(*ops, **okw)
+        O0, L0 = O0.clone(), L0.clone()
+        for r in range(30):
+            if r % 3 == 0:
+                noise.fill_(r)
+            O, L = Bd.fp4attn_fwd(*ops, **okw)
+            assert torch.equal(O, O0) and torch.equal(L, L0), ("fp8", okw, r)
