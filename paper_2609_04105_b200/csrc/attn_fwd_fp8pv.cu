@@ -12,11 +12,13 @@
 // stage.  The tensor pipe is three quarters idle in this kernel family, so the reference is taken by a first sweep
 // instead: every work item walks its keys TWICE - sweep A computes S and reduces the row maxima only, sweep B
 // computes S again, forms the bytes against the now final mu and feeds PV.  Nothing is ever rescaled, there is no
-// correction pass, and the result equals the plain (not online) definition above.
+// correction pass, and the result equals the plain (not online) definition above.  The second sweep of one item
+// and the first sweep of the CTA's next item run interleaved stage by stage (see the schedule comment in the
+// kernel), so that SFU-heavy and SFU-free visits alternate on every team.
 //
-//   warp 0        TMA producer: Q tile per item; ring of {K, K scales} in sweep A and {K, V8^T, K scales} in sweep B
-//   warp 1        QK issuer (both sweeps; in sweep A it also hands the ring slot back)
-//   warp 2        PV issuer (sweep B): four K32 products per 128-key stage, A operand from tensor memory
+//   warp 0        TMA producer: Q tile per item; ring of {K, K scales} for A-steps and {K, V8^T, K scales} for B-steps
+//   warp 1        QK issuer (both kinds of step; after an A-step it also hands the ring slot back)
+//   warp 2        PV issuer (B-steps): four K32 products per 128-key stage, A operand from tensor memory
 //   warps 3-6     epilogue: O = O_hw / (L_hw G_V), LSE
 //   warps 7-22    softmax teams as in attn_fwd.cu (team 2p + h: h-th 64 keys of the steps with parity p)
 //
@@ -41,7 +43,7 @@ struct Cfg8 {
   static constexpr int NST = (D == 128) ? 5 : 8;
   static constexpr int OFF_Q = 0;                                     // two buffers
   static constexpr int OFF_QSF = OFF_Q + 2 * C1::Q_BYTES;             // two buffers of 1 KB
-  static constexpr int OFF_RMAX = OFF_QSF + 2048;                     // [item parity][team][row] float
+  static constexpr int OFF_RMAX = OFF_QSF + 2048;                     // [item parity][first-sweep team][row] float
   static constexpr int OFF_MU = OFF_RMAX + 2 * 4 * BM * 4;            // [item parity][row] int
   static constexpr int OFF_STAGE = (OFF_MU + 2 * BM * 4 + 1023) / 1024 * 1024;
   static constexpr int OFF_OUT = OFF_STAGE + NST * STAGE_BYTES;
@@ -51,7 +53,7 @@ struct Cfg8 {
 };
 
 enum { B8_QFULL0 = 0, B8_QFREE0 = 2, B8_OFULL = 4, B8_OFREE = 5, B8_SFULL0 = 6, B8_SEMPTY0 = 8, B8_PFREE0 = 10,
-       B8_SMDONE0 = 12, B8_DRAIN0 = 14, B8_RMAX = 16, B8_RING = 17 };
+       B8_SMDONE0 = 12, B8_DRAIN0 = 14, B8_MURDY0 = 16, B8_RING = 18 };
 
 struct Fp8Params {
   AttnParams a;
@@ -124,20 +126,23 @@ attn_fwd_fp8pv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qtiles = p.N / BM;
+  // this CTA's work items are item(k) = blockIdx.x + k * gridDim.x, k = 0 .. n_my - 1
+  const int n_my = p.n_items > (int)blockIdx.x ? (p.n_items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  auto item_of = [&](int k) { return (int)blockIdx.x + k * (int)gridDim.x; };
 
   if (threadIdx.x == 0) {
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar(B8_QFULL0 + b), 1);
       mbar_init(bar(B8_QFREE0 + b), 1);
       mbar_init(bar(B8_SFULL0 + b), 1);
-      mbar_init(bar(B8_SEMPTY0 + b), 8);
+      mbar_init(bar(B8_SEMPTY0 + b), 8);       // the two teams of the pair, four warps each
       mbar_init(bar(B8_SMDONE0 + b), 8);
       mbar_init(bar(B8_PFREE0 + b), 1);
+      mbar_init(bar(B8_MURDY0 + b), 4 * kTeams);   // every softmax warp, once per item (slot by item parity)
       mbar_init(bar(B8_DRAIN0 + b), 1);
     }
     mbar_init(bar(B8_OFULL), 1);
     mbar_init(bar(B8_OFREE), 4);
-    mbar_init(bar(B8_RMAX), 4 * kTeams);       // every softmax warp, once per item
     for (int s = 0; s < C8::NST; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
     *abortf = 0;
     fence_barrier_init();
@@ -156,40 +161,53 @@ attn_fwd_fp8pv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   tc_fence_after();
   const uint32_t tmem = *tslot;
 
+  // Every role walks the same schedule.  Phase ph (0 .. n_my) carries the first sweep ("A": scores -> row maxima) of
+  // item ph and the second sweep ("B": scores -> bytes -> PV) of item ph - 1, stage by stage, in the order
+  // A B | B A | A B | ... ; the first phase has no B part, the last no A part.  Steps are numbered g = 0, 1, 2 ... in
+  // that order; step g uses score slot g & 1 and is served by the team pair g & 1 (teams 2p, 2p + 1), so each pair
+  // alternates between the SFU-heavy second sweep of one item and the SFU-free first sweep of the next, and the four
+  // warps of a scheduler are never all in the same kind of work.
   if (warp == 0) {
     // ===================================================================== TMA producer
     int s = 0, ph = 0;
     uint32_t gs = 0;
     uint32_t st = sbase + C8::OFF_STAGE;
     bool ok = true;
-    int i = 0;
-    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
-      const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
-      const int T2 = wi.T2;
-      const int qb = i & 1;
-      if (i >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_QFREE0 + qb), ((i >> 1) - 1) & 1, abortf));
-      if (!ok) break;
-      if (elect_one()) {
-        mbar_arrive_expect_tx(bar(B8_QFULL0 + qb), C::Q_BYTES + C::QSF_BYTES);
-        tma_load_2d(sbase + C8::OFF_Q + qb * C::Q_BYTES, &tmQ, 0, wi.qrow0, bar(B8_QFULL0 + qb));
-        bulk_load_1d(sbase + C8::OFF_QSF + qb * 1024, p.q_sf + (size_t)wi.qtile_lin * C::QSF_BYTES, C::QSF_BYTES, bar(B8_QFULL0 + qb));
-      }
-      const uint8_t* ksf = p.k_sf + (size_t)wi.kvh * qtiles * C::KSF_BYTES;
-      const int krow0 = wi.kvh * p.N, vrow0 = wi.kvh * D;
-      for (int s2 = 0; s2 < 2 * T2; ++s2, ++gs) {                 // sweep A: stages 0..T2-1 (K only), sweep B: again, with V8
-        const bool sweepB = s2 >= T2;
-        const int kt = sweepB ? s2 - T2 : s2;
-        if (gs >= (uint32_t)C8::NST) ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(s), ph ^ 1, abortf));
+    for (int phs = 0; ok && phs <= n_my; ++phs) {
+      WorkItem wa = {}, wb = {};
+      int TA = 0, TB = 0;
+      if (phs < n_my) { wa = decode_item<CAUSAL>(item_of(phs), p, qtiles); TA = wa.T2; }
+      if (phs >= 1) { wb = decode_item<CAUSAL>(item_of(phs - 1), p, qtiles); TB = wb.T2; }
+      if (phs < n_my) {
+        const int qb = phs & 1;
+        if (phs >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_QFREE0 + qb), ((phs >> 1) - 1) & 1, abortf));
         if (!ok) break;
-        const uint32_t fb = bar_full(s);
         if (elect_one()) {
-          mbar_arrive_expect_tx(fb, C::K_BYTES + C::KSF_BYTES + (sweepB ? C8::V_BYTES : 0));
-          tma_load_2d(st, &tmK, 0, krow0 + kt * BS, fb);
-          if (sweepB) tma_load_2d(st + C::K_BYTES, &tmV, kt * BS, vrow0, fb);
-          bulk_load_1d(st + C8::OFF_KSF, ksf + (size_t)kt * C::KSF_BYTES, C::KSF_BYTES, fb);
+          mbar_arrive_expect_tx(bar(B8_QFULL0 + qb), C::Q_BYTES + C::QSF_BYTES);
+          tma_load_2d(sbase + C8::OFF_Q + qb * C::Q_BYTES, &tmQ, 0, wa.qrow0, bar(B8_QFULL0 + qb));
+          bulk_load_1d(sbase + C8::OFF_QSF + qb * 1024, p.q_sf + (size_t)wa.qtile_lin * C::QSF_BYTES, C::QSF_BYTES, bar(B8_QFULL0 + qb));
         }
-        st += C8::STAGE_BYTES;
-        if (++s == C8::NST) { s = 0; ph ^= 1; st = sbase + C8::OFF_STAGE; }
+      }
+      const int TM = TA > TB ? TA : TB;
+      for (int s2 = 0; ok && s2 < TM; ++s2) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int kind = j ^ (s2 & 1);                            // 0: A-step of item phs, 1: B-step of item phs - 1
+          if (s2 >= (kind ? TB : TA)) continue;
+          const WorkItem& wi = kind ? wb : wa;
+          if (gs >= (uint32_t)C8::NST) ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(s), ph ^ 1, abortf));
+          if (!ok) break;
+          const uint32_t fb = bar_full(s);
+          if (elect_one()) {
+            mbar_arrive_expect_tx(fb, C::K_BYTES + C::KSF_BYTES + (kind ? C8::V_BYTES : 0));
+            tma_load_2d(st, &tmK, 0, wi.kvh * p.N + s2 * BS, fb);
+            if (kind) tma_load_2d(st + C::K_BYTES, &tmV, s2 * BS, wi.kvh * D, fb);
+            bulk_load_1d(st + C8::OFF_KSF, p.k_sf + ((size_t)wi.kvh * qtiles + s2) * C::KSF_BYTES, C::KSF_BYTES, fb);
+          }
+          ++gs;
+          st += C8::STAGE_BYTES;
+          if (++s == C8::NST) { s = 0; ph ^= 1; st = sbase + C8::OFF_STAGE; }
+        }
       }
     }
     if (*abortf && lane == 0) {
@@ -203,84 +221,103 @@ attn_fwd_fp8pv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     constexpr uint32_t kIdQK1 = NV ? make_idesc_fp4(BM, BS, false, 0, 0) : make_idesc_fp4(BM, BS, true, 2, 2);
     int sq = 0, phq = 0;
     uint32_t stq = sbase + C8::OFF_STAGE;
-    uint32_t g = 0;
+    uint32_t g = 0;                                             // steps issued so far (both kinds, all items)
     bool ok = true;
-    int i = 0;
-    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
-      const int T2 = decode_item<CAUSAL>(item, p, qtiles).T2;
-      const int qb = i & 1;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_QFULL0 + qb), (i >> 1) & 1, abortf));
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t tSFQ = tmem + kColSFQ + 8 * qb;
-      if (elect_one()) {
-#pragma unroll
-        for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFQ + 4 * a, at(kDescSF, sbase + C8::OFF_QSF + qb * 1024 + 512 * a));
-      }
-      const uint64_t dQ0 = at(kDescQK, sbase + C8::OFF_Q + qb * C::Q_BYTES);
-      for (int s2 = 0; s2 < 2 * T2; ++s2, ++g) {
-        const int pr = g & 1;
-        const uint32_t m = g >> 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_full(sq), phq, abortf));
-        if (ok && m > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_SEMPTY0 + pr), (m - 1) & 1, abortf));
+    for (int phs = 0; ok && phs <= n_my; ++phs) {
+      int TA = 0, TB = 0;
+      if (phs < n_my) TA = decode_item<CAUSAL>(item_of(phs), p, qtiles).T2;
+      if (phs >= 1) TB = decode_item<CAUSAL>(item_of(phs - 1), p, qtiles).T2;
+      if (phs < n_my) {
+        const int qb = phs & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_QFULL0 + qb), (phs >> 1) & 1, abortf));
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tSFK = tmem + kColSFK + 8 * pr;
-        const uint32_t tS = tmem + kColS + BS * pr;
-        const uint64_t dK0 = at(kDescQK, stq);
         if (elect_one()) {
 #pragma unroll
-          for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFK + 4 * a, at(kDescSF, stq + C8::OFF_KSF + 512 * a));
-          if (NV) {
-            tc_mma_fp4_4x(tS, dQ0, dK0, kIdQK0, tSFQ, tSFK, 0);
-            if (C::KBLK == 2) tc_mma_fp4_4x(tS, dQ0 + 2, dK0 + 2, kIdQK1, tSFQ + 4, tSFK + 4, 1);
-          } else {
-            tc_mma_fp4_2x(tS, dQ0, dK0, kIdQK0, tSFQ, tSFK, 0);
-            if (C::KBLK == 2) tc_mma_fp4_2x(tS, dQ0 + 2, dK0 + 2, kIdQK1, tSFQ, tSFK, 1);
-          }
-          tc_commit(bar(B8_SFULL0 + pr));
-          if (s2 < T2) tc_commit(bar_empty(sq));                 // sweep A: nothing else reads the stage
-          if (s2 == 2 * T2 - 1) tc_commit(bar(B8_QFREE0 + qb));
+          for (int a = 0; a < C::CTQ; ++a)
+            tc_cp_32x128b_warpx4(tmem + kColSFQ + 8 * qb + 4 * a, at(kDescSF, sbase + C8::OFF_QSF + qb * 1024 + 512 * a));
         }
         __syncwarp();
-        stq += C8::STAGE_BYTES;
-        if (++sq == C8::NST) { sq = 0; phq ^= 1; stq = sbase + C8::OFF_STAGE; }
+      }
+      const int TM = TA > TB ? TA : TB;
+      for (int s2 = 0; ok && s2 < TM; ++s2) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int kind = j ^ (s2 & 1);
+          if (s2 >= (kind ? TB : TA)) continue;
+          const int qb = (kind ? phs - 1 : phs) & 1;              // the Q buffer of the step's item
+          const int pr = g & 1;
+          const uint32_t m = g >> 1;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_full(sq), phq, abortf));
+          if (ok && m > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_SEMPTY0 + pr), (m - 1) & 1, abortf));   // both teams have read the slot
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t tSFQ = tmem + kColSFQ + 8 * qb;
+          const uint32_t tSFK = tmem + kColSFK + 8 * pr;
+          const uint32_t tS = tmem + kColS + BS * pr;
+          const uint64_t dQ0 = at(kDescQK, sbase + C8::OFF_Q + qb * C::Q_BYTES);
+          const uint64_t dK0 = at(kDescQK, stq);
+          if (elect_one()) {
+#pragma unroll
+            for (int a = 0; a < C::CTQ; ++a) tc_cp_32x128b_warpx4(tSFK + 4 * a, at(kDescSF, stq + C8::OFF_KSF + 512 * a));
+            if (NV) {
+              tc_mma_fp4_4x(tS, dQ0, dK0, kIdQK0, tSFQ, tSFK, 0);
+              if (C::KBLK == 2) tc_mma_fp4_4x(tS, dQ0 + 2, dK0 + 2, kIdQK1, tSFQ + 4, tSFK + 4, 1);
+            } else {
+              tc_mma_fp4_2x(tS, dQ0, dK0, kIdQK0, tSFQ, tSFK, 0);
+              if (C::KBLK == 2) tc_mma_fp4_2x(tS, dQ0 + 2, dK0 + 2, kIdQK1, tSFQ, tSFK, 1);
+            }
+            tc_commit(bar(B8_SFULL0 + pr));
+            if (kind == 0) tc_commit(bar_empty(sq));              // first sweep: nothing else reads the stage
+            if (kind == 1 && s2 == TB - 1) tc_commit(bar(B8_QFREE0 + qb));   // the item's Q buffer may take the item after next
+          }
+          __syncwarp();
+          ++g;
+          stq += C8::STAGE_BYTES;
+          if (++sq == C8::NST) { sq = 0; phq ^= 1; stq = sbase + C8::OFF_STAGE; }
+        }
       }
     }
     if (*abortf && elect_one()) tc_commit(bar(B8_DRAIN0));
     __syncwarp();
   } else if (warp == 2) {
-    // ===================================================================== PV issuer (sweep B)
+    // ===================================================================== PV issuer (B-steps)
     constexpr uint32_t kIdPV = make_idesc_f8(BM, C::DN);
     const uint32_t tO = tmem + kColO;
-    uint32_t gsl = 0;                                           // ring slots consumed so far by anyone (both sweeps)
-    uint32_t g = 0;
-    uint32_t nb[2] = {0, 0};                                    // sweep-B steps served so far, per step parity
+    uint32_t g = 0;                                             // steps so far (both kinds): ring slot and team pair of a step
+    uint32_t nb[2] = {0, 0};                                    // B-steps served so far, per team pair
     bool ok = true;
-    int i = 0;
-    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
-      const int T2 = decode_item<CAUSAL>(item, p, qtiles).T2;
-      gsl += T2;                                                // sweep A's slots
-      g += T2;
-      if (i >= 1) ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_OFREE), (i - 1) & 1, abortf));
-      for (int s2 = 0; ok && s2 < T2; ++s2, ++g, ++gsl) {
-        const int pr = g & 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_SMDONE0 + pr), (pr ? nb[1] : nb[0]) & 1, abortf));   // bytes of both tiles are in tensor memory
-        if (!ok) break;
-        if (pr) ++nb[1]; else ++nb[0];
-        tc_fence_after();
-        const uint32_t sp = gsl % C8::NST;
-        const uint32_t stp = sbase + C8::OFF_STAGE + sp * C8::STAGE_BYTES;
-        const uint64_t dV = at(kDescV, stp + C::K_BYTES);
-        if (elect_one()) {
+    for (int phs = 0; ok && phs <= n_my; ++phs) {
+      int TA = 0, TB = 0;
+      if (phs < n_my) TA = decode_item<CAUSAL>(item_of(phs), p, qtiles).T2;
+      if (phs >= 1) TB = decode_item<CAUSAL>(item_of(phs - 1), p, qtiles).T2;
+      if (phs >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_OFREE), (phs - 2) & 1, abortf));   // epilogue of item phs - 2 has read O
+      const int TM = TA > TB ? TA : TB;
+      for (int s2 = 0; ok && s2 < TM; ++s2) {
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk)                         // 32 keys per product: 8 columns of P, 32 bytes along V8^T's rows
-            tc_mma_f8_ta(tO, tmem + k8ColP + 32 * pr + 8 * kk, dV + 2 * kk, kIdPV, (s2 > 0 || kk > 0) ? 1u : 0u);
-          tc_commit(bar_empty(sp));
-          tc_commit(bar(B8_PFREE0 + pr));
-          if (s2 == T2 - 1) tc_commit(bar(B8_OFULL));
+        for (int j = 0; j < 2; ++j) {
+          const int kind = j ^ (s2 & 1);
+          if (s2 >= (kind ? TB : TA)) continue;
+          if (kind == 0) { ++g; continue; }                       // an A-step: only its slot is counted
+          const int pr = g & 1;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_SMDONE0 + pr), (pr ? nb[1] : nb[0]) & 1, abortf));   // bytes of both tiles are in tensor memory
+          if (!ok) break;
+          if (pr) ++nb[1]; else ++nb[0];
+          tc_fence_after();
+          const uint32_t sp = g % C8::NST;
+          const uint32_t stp = sbase + C8::OFF_STAGE + sp * C8::STAGE_BYTES;
+          const uint64_t dV = at(kDescV, stp + C::K_BYTES);
+          if (elect_one()) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)                         // 32 keys per product: 8 columns of P, 32 bytes along V8^T's rows
+              tc_mma_f8_ta(tO, tmem + k8ColP + 32 * pr + 8 * kk, dV + 2 * kk, kIdPV, (s2 > 0 || kk > 0) ? 1u : 0u);
+            tc_commit(bar_empty(sp));
+            tc_commit(bar(B8_PFREE0 + pr));
+            if (s2 == TB - 1) tc_commit(bar(B8_OFULL));
+          }
+          __syncwarp();
+          ++g;
         }
-        __syncwarp();
       }
     }
     if (*abortf && elect_one()) tc_commit(bar(B8_DRAIN0 + 1));
@@ -291,13 +328,12 @@ attn_fwd_fp8pv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const int row = quarter * 32 + lane;
     const uint32_t tO = tmem + ((uint32_t)(quarter * 32) << 16) + kColO;
     bool ok = true;
-    int i = 0;
-    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++i) {
-      const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_OFULL), i & 1, abortf));
+    for (int k = 0; ok && k < n_my; ++k) {
+      const WorkItem wi = decode_item<CAUSAL>(item_of(k), p, qtiles);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_OFULL), k & 1, abortf));
       if (!ok) break;
       tc_fence_after();
-      const int mu = reinterpret_cast<const int*>(sgen + C8::OFF_MU)[(i & 1) * BM + row];   // written before any PV of the item
+      const int mu = reinterpret_cast<const int*>(sgen + C8::OFF_MU)[(k & 1) * BM + row];   // written before any PV of the item
       float Lhw;
       {
         uint32_t r16[16];
@@ -344,92 +380,101 @@ attn_fwd_fp8pv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   } else {
     // ===================================================================== softmax teams
     const int team = (warp - kFirstSoftmaxWarp) >> 2;
-    const int pr = team >> 1;
+    const int pr = team >> 1;                                   // the steps with g & 1 == pr are this pair's
+    const int h = team & 1;                                     // which 64 keys of a stage
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const uint32_t tS = tmem + ((uint32_t)(quarter * 32) << 16) + kColS + BN * team;
     const uint32_t sfull = bar(B8_SFULL0 + pr), sempty = bar(B8_SEMPTY0 + pr);
     const uint32_t smdone = bar(B8_SMDONE0 + pr), pfree = bar(B8_PFREE0 + pr);
-    const uint32_t tP = tmem + ((uint32_t)(quarter * 32) << 16) + k8ColP + 32 * pr + 16 * (team & 1);
+    const uint32_t tP = tmem + ((uint32_t)(quarter * 32) << 16) + k8ColP + 32 * pr + 16 * h;
     float c32;
     if (NV) c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G), __ldg(p.k_G)));
     else    c32 = __fdiv_rn(p.c_base, 36.0f);
-    uint32_t g0 = 0;
-    uint32_t nbt = 0;                                           // sweep-B visits of this team so far (all items)
     bool ok = true;
-    int T2 = 0, i = 0;
-    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, g0 += 2 * T2, ++i) {
-      const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
-      T2 = wi.T2;
-      float* rmax = reinterpret_cast<float*>(sgen + C8::OFF_RMAX) + (i & 1) * 4 * BM;
-      // ---- sweep A: the maximum of this team's scores of the row (its half of the stages of its parity)
-      float smax = -INFINITY;
-      uint32_t g = g0 + ((g0 & 1) != (uint32_t)pr);
-      for (; g < g0 + T2; g += 2) {
-        ok = __all_sync(0xffffffffu, mbar_wait(sfull, (g >> 1) & 1, abortf));
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t sraw[32];
-        const bool diag = CAUSAL && (int)(g - g0) == wi.qt;
-        const int v0 = row - 64 * (team & 1) + 1;               // visible keys of the team's tile on the diagonal stage
-        tmem_ld_32x32b_x32(tS, sraw);
-        tmem_wait_ld();
-        if (diag) {
+    uint32_t g = 0;                                             // steps so far (both kinds, all pairs)
+    uint32_t nbt = 0;                                           // B-visits of this team so far
+    const int v0 = row - 64 * h + 1;                            // visible keys of the team's tile on a causal diagonal stage
+    float b = 0.f;                                              // 8 - mu of the item in its second sweep
+    for (int phs = 0; ok && phs <= n_my; ++phs) {
+      WorkItem wa = {}, wb = {};
+      int TA = 0, TB = 0;
+      if (phs < n_my) { wa = decode_item<CAUSAL>(item_of(phs), p, qtiles); TA = wa.T2; }
+      if (phs >= 1) { wb = decode_item<CAUSAL>(item_of(phs - 1), p, qtiles); TB = wb.T2; }
+      float smax = -INFINITY;                                   // this team's share of the maxima of item phs
+      const int TM = TA > TB ? TA : TB;
+      for (int s2 = 0; ok && s2 < TM; ++s2) {
 #pragma unroll
-          for (int k = 0; k < 32; ++k) sraw[k] = (k < v0) ? sraw[k] : 0xFF800000u;
-        }
-        smax = fmaxf(smax, max32(sraw));
-        tmem_ld_32x32b_x32(tS + 32, sraw);
-        tmem_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(sempty);
-        if (diag) {
+        for (int j = 0; j < 2; ++j) {
+          const int kind = j ^ (s2 & 1);
+          if (s2 >= (kind ? TB : TA)) continue;
+          if ((int)(g & 1) != pr) { ++g; continue; }              // the other pair's step
+          ok = __all_sync(0xffffffffu, mbar_wait(sfull, (g >> 1) & 1, abortf));
+          if (!ok) break;
+          tc_fence_after();
+          uint32_t sraw[32];
+          if (kind == 0) {
+            // ---- first sweep of item phs: maxima only
+            const bool diag = CAUSAL && s2 == wa.qt;
+            tmem_ld_32x32b_x32(tS, sraw);
+            tmem_wait_ld();
+            if (diag) {
 #pragma unroll
-          for (int k = 0; k < 32; ++k) sraw[k] = (k < v0 - 32) ? sraw[k] : 0xFF800000u;
+              for (int e = 0; e < 32; ++e) sraw[e] = (e < v0) ? sraw[e] : 0xFF800000u;
+            }
+            smax = fmaxf(smax, max32(sraw));
+            tmem_ld_32x32b_x32(tS + 32, sraw);
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sempty);
+            if (diag) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) sraw[e] = (e < v0 - 32) ? sraw[e] : 0xFF800000u;
+            }
+            smax = fmaxf(smax, max32(sraw));
+          } else {
+            // ---- second sweep of item phs - 1: bytes against its final reference
+            uint32_t w[16];
+            const bool diag = CAUSAL && s2 == wb.qt;
+            tmem_ld_32x32b_x32(tS, sraw);
+            tmem_wait_ld();
+            if (diag) fp8_p_block<true>(sraw, c32, b, v0, w);
+            else      fp8_p_block<false>(sraw, c32, b, 32, w);
+            tmem_ld_32x32b_x32(tS + 32, sraw);
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sempty);
+            if (diag) fp8_p_block<true>(sraw, c32, b, v0 - 32, w + 8);
+            else      fp8_p_block<false>(sraw, c32, b, 32, w + 8);
+            // the pair's probability slot was last read by the PV product of this team's previous B-visit
+            if (nbt > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (nbt - 1) & 1, abortf));
+            if (!ok) break;
+            tmem_st_32x32b_x16(tP, w);
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smdone);
+            ++nbt;
+          }
+          ++g;
         }
-        smax = fmaxf(smax, max32(sraw));
       }
       if (!ok) break;
-      // ---- the four teams meet: mu = ceil(c * max over all keys), as an integer on the FMA pipe
-      rmax[team * BM + row] = smax;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B8_RMAX));
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_RMAX), i & 1, abortf));     // a bounded wait, like every other hand-off
-      if (!ok) break;
-      const float mall = fmaxf(fmaxf(rmax[row], rmax[BM + row]), fmaxf(rmax[2 * BM + row], rmax[3 * BM + row]));
-      const float ymax = fminf(fmaxf(__fmul_rn(mall, c32), -2097152.0f), 2097152.0f);
-      const float tt = __fadd_ru(ymax, 12582912.0f);
-      const int mu = (int)(__float_as_uint(tt) - 0x4B400000u);
-      const float b = __fsub_rn(kP8Shift, __fsub_rn(tt, 12582912.0f));
-      if (team == 0) reinterpret_cast<int*>(sgen + C8::OFF_MU)[(i & 1) * BM + row] = mu;
-      // ---- sweep B: bytes against the final reference
-      for (; g < g0 + 2 * T2; g += 2, ++nbt) {
-        ok = __all_sync(0xffffffffu, mbar_wait(sfull, (g >> 1) & 1, abortf));
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t sraw[32], w[16];
-        const bool diag = CAUSAL && (int)(g - g0 - T2) == wi.qt;
-        const int v0 = row - 64 * (team & 1) + 1;
-        tmem_ld_32x32b_x32(tS, sraw);
-        tmem_wait_ld();
-        if (diag) fp8_p_block<true>(sraw, c32, b, v0, w);
-        else      fp8_p_block<false>(sraw, c32, b, 32, w);
-        tmem_ld_32x32b_x32(tS + 32, sraw);
-        tmem_wait_ld();
-        tc_fence_before();
+      if (phs < n_my) {
+        // ---- the sixteen softmax warps meet: mu of item phs = ceil(c * max over all its keys), on the FMA pipe
+        float* rmax = reinterpret_cast<float*>(sgen + C8::OFF_RMAX) + (phs & 1) * 4 * BM;
+        rmax[team * BM + row] = smax;                           // (-inf from a team that served none of the item's A-steps)
         __syncwarp();
-        if (lane == 0) mbar_arrive(sempty);
-        if (diag) fp8_p_block<true>(sraw, c32, b, v0 - 32, w + 8);
-        else      fp8_p_block<false>(sraw, c32, b, 32, w + 8);
-        // the P slot of this parity was last read by the PV product of this team's previous sweep-B visit
-        if (nbt > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (nbt - 1) & 1, abortf));
+        if (lane == 0) mbar_arrive(bar(B8_MURDY0 + (phs & 1)));
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(B8_MURDY0 + (phs & 1)), (phs >> 1) & 1, abortf));
         if (!ok) break;
-        tmem_st_32x32b_x16(tP, w);
-        tmem_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smdone);
+        const float mall = fmaxf(fmaxf(rmax[row], rmax[BM + row]), fmaxf(rmax[2 * BM + row], rmax[3 * BM + row]));
+        const float ymax = fminf(fmaxf(__fmul_rn(mall, c32), -2097152.0f), 2097152.0f);
+        const float tt = __fadd_ru(ymax, 12582912.0f);          // ceil, exact for |y| < 2^22
+        b = __fsub_rn(kP8Shift, __fsub_rn(tt, 12582912.0f));
+        if (team == 0) reinterpret_cast<int*>(sgen + C8::OFF_MU)[(phs & 1) * BM + row] = (int)(__float_as_uint(tt) - 0x4B400000u);
       }
     }
   }
