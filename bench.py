@@ -16,6 +16,11 @@ after an L2 flush (`value`, `ms_per_step`, `roofline.achieved` come from these);
 `window` (the paper's protocol is 300 ms warm-up and a median over a seconds-long window), with a
 clock-normalised figure beside the raw one.
 
+Rooflines: `roofline` holds the attention kernel against the tensor roof (measured bf16 burst x 4);
+`roofline_softmax_arith` holds the same kernel against what its softmax arithmetic alone allows on this device
+(the kernel's score -> code instruction stream run by itself, four warps per scheduler: with exact codes the
+special-function unit binds it); `roofline_quantize` the quantizers against the measured copy bandwidth.
+
 N > 1 is launched with torch.distributed.run (one rank per GPU); every rank runs the same
 workload on its own batch (independent (batch, head) units, no data-path collective), so the
 job is weak-scaled and `value` is the sum over ranks divided by the slowest rank's time.
@@ -469,8 +474,12 @@ def run_cuda(args, w):
             for _ in range(3):
                 fn()
             ms_map = statistics.median(timed_launches(fn, 10, flush, E, torch.cuda.synchronize))
+            cyc_m = torch.zeros(2, dtype=torch.int64, device=dev)
+            Bd.fp4attn_softmax_arith_probe(kw["p_map"], kw.get("exact_pairs", 0), 8192, cyc_m)
+            torch.cuda.synchronize()
             other_maps[name] = {"attn_ms": ms_map, "attn_tflops": w.flops / (ms_map * 1e-3) / 1e12,
-                                "roofline_frac": w.flops / (ms_map * 1e-3) / 1e12 / fp4_peak}
+                                "roofline_frac": w.flops / (ms_map * 1e-3) / 1e12 / fp4_peak,
+                                "softmax_arith_clk_per_block": int(cyc_m[0].item()) / (4.0 * 8192)}
         # the FP8 P/V route on the same Q, K (E4M3 V with per-unit factors, E4M3 probabilities)
         v8 = Bd.fp4attn_quantize_v_e4m3(dv)
         fn = lambda: Bd.fp4attn_fwd(qd0, kd0, v8, out=O_alt, status=status)
@@ -495,6 +504,14 @@ def run_cuda(args, w):
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     probe_tflops = sms * iters * 2.0 * 128 * 128 * 64 / (p0.elapsed_time(p1) * 1e-3) / 1e12
     probe_flop_per_clk_sm = iters * 2.0 * 128 * 128 * 64 / max(1, int(cyc.item()))
+
+    # ---- measured ceiling of the softmax arithmetic alone (second roofline of the attention kernel)
+    cyc2 = torch.zeros(2, dtype=torch.int64, device=dev)
+    arith_iters = 8192
+    Bd.fp4attn_softmax_arith_probe(pmap, pairs, arith_iters, cyc2)
+    Bd.fp4attn_softmax_arith_probe(pmap, pairs, arith_iters, cyc2)
+    torch.cuda.synchronize()
+    arith_clk_per_block = int(cyc2[0].item()) / (4.0 * arith_iters)      # per scheduler, four warps each
 
     # ---- parity sample inputs of the headline workload, taken before its tensors are released
     sample = None
@@ -565,6 +582,22 @@ def run_cuda(args, w):
     roof = roofline_record(w, attn_launch_ms, fp4_peak, peaks, "attn_fwd_2q_kernel" if args.schedule == "two-query" else "attn_fwd_kernel")
     roof.update({"fp4_issue_probe_tflops": probe_tflops, "fp4_issue_probe_flop_per_clk_per_sm": probe_flop_per_clk_sm,
                  "launch_ms_mean": attn_launch_ms, "launch_ms_median": statistics.median(attn_ms)})
+    # Softmax-arithmetic roofline: an SM converts four 32x32 blocks (one per scheduler) in `arith_clk_per_block`
+    # clocks when it does nothing else; a block carries 4*32*32*d flop of the two products.  Clock: the median SM
+    # clock sampled during the timed steps (the nominal maximum where NVML gives no samples).
+    sm_hz = clk.summary().get("sm_mhz") or clk.max_mhz or 0
+    arith_peak = sms * 4 * (4.0 * 32 * 32 * w.d) / arith_clk_per_block * sm_hz * 1e6 / 1e12 if sm_hz else None
+    roof_softmax = {"kernel": roof["kernel"], "bound": "alu", "achieved": attn_tflops, "peak": arith_peak, "unit": UNIT,
+                    "frac": attn_tflops / arith_peak if arith_peak else None, "traffic": None,
+                    "clk_per_32x32_block_per_scheduler": arith_clk_per_block,
+                    "peak_source": "measured on this device: the kernel's score -> code arithmetic for map '%s' run alone, four "
+                                   "warps per scheduler (fp4attn_softmax_arith_probe), at the median SM clock of the timed steps; "
+                                   "for exact codes the SFU's 16 ex2/clk/SM (12 of 16 pairs -> 192 clk per block) is the unit "
+                                   "that binds" % args.p_map}
+    for rec in other_maps.values():                                  # the same arithmetic ceiling for the other code maps
+        if "softmax_arith_clk_per_block" in rec and sm_hz:
+            pk = sms * 4 * (4.0 * 32 * 32 * w.d) / rec["softmax_arith_clk_per_block"] * sm_hz * 1e6 / 1e12
+            rec["softmax_arith_frac"] = rec["attn_tflops"] / pk
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": n_warm, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -577,6 +610,7 @@ def run_cuda(args, w):
                       "note": "attention kernel alone (the paper's timing boundary excludes quantization)",
                       "other_code_maps": other_maps},
         "roofline": roof,
+        "roofline_softmax_arith": roof_softmax,
         "window": window,
         "roofline_quantize": {"kernel": q_kernel, "bound": "hbm", "achieved": q_bytes / (quant["rows"] * 1e-3) / 1e9,
                               "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -339,6 +339,19 @@ int fp4attn_release(void);
 int fp4attn_mma_peak_probe(int iters, unsigned long long* cycles_out, fp4attn_stream_t stream);
 
 /*
+ * Arithmetic ceiling of the softmax warps on the current device, measured: on every SM, sixteen warps (four per
+ * scheduler, as in the attention kernel) each run the score -> code arithmetic of Algorithm "direct-p-pack" -
+ * block maximum, block exponent (ceiling rule), the code map (`p_map` and `exact_pairs` as in
+ * fp4attn_operands; other values: FP4ATTN_ERR_INVALID_ARG), E2M1 conversion and packing - on `iters` blocks of 32 rows x 32 scores held in shared memory, with no tensor product, tensor-memory
+ * access or hand-off around it.  Enqueues one kernel; cycles_out (device, TWO 64-bit words, the second is scratch)
+ * receives in its first word the slowest warp's clock count, so that cycles / (4 * iters) is the clocks one
+ * scheduler needs per block.  Used by the benchmark for the roofline of the softmax arithmetic; not part of the
+ * attention path.
+ */
+int fp4attn_softmax_arith_probe(int p_map, int exact_pairs, int iters, unsigned long long* cycles_out,
+                                fp4attn_stream_t stream);
+
+/*
  * Self-test of the bounded in-kernel waits (the failure-detection path; the paper has no
  * counterpart).  Launches one warp that waits on a barrier nothing completes, with a limit of
  * `limit_cycles` SM clocks (1 .. 2^31), and writes to *device_status what the attention kernel

@@ -28,7 +28,7 @@ LIB_PATH = os.path.join(_HERE, "libfp4attn.so")
 EXPORTS = [
     "fp4attn_status_string", "fp4attn_version", "fp4attn_packed_bytes", "fp4attn_scale_bytes",
     "fp4attn_quantize_workspace_bytes", "fp4attn_quantize", "fp4attn_fwd",
-    "fp4attn_attention_host_workspace_bytes", "fp4attn_attention_host", "fp4attn_mma_peak_probe",
+    "fp4attn_attention_host_workspace_bytes", "fp4attn_attention_host", "fp4attn_mma_peak_probe", "fp4attn_softmax_arith_probe",
     "fp4attn_quantize_nvfp4_noalloc", "fp4attn_selftest_bounded_wait", "fp4attn_quantize_mxfp4_rule",
     "fp4attn_quantize_nvfp4_per_head_workspace_bytes", "fp4attn_quantize_nvfp4_per_head", "fp4attn_release",
     "fp4attn_quantize_v_e4m3_workspace_bytes", "fp4attn_quantize_v_e4m3",
@@ -91,6 +91,8 @@ def _load() -> ctypes.CDLL:
     lib.fp4attn_selftest_bounded_wait.argtypes = [ctypes.c_longlong, vp, vp]
     lib.fp4attn_mma_peak_probe.restype = i
     lib.fp4attn_mma_peak_probe.argtypes = [i, vp, vp]
+    lib.fp4attn_softmax_arith_probe.restype = i
+    lib.fp4attn_softmax_arith_probe.argtypes = [i, i, i, vp, vp]
     return lib
 
 
@@ -271,6 +273,13 @@ def fp4attn_release() -> None:
 
 def fp4attn_mma_peak_probe(iters: int, cycles_out: torch.Tensor) -> None:
     _check(lib().fp4attn_mma_peak_probe(iters, cycles_out.data_ptr(), _stream()), "fp4attn_mma_peak_probe")
+
+
+def fp4attn_softmax_arith_probe(p_map: int, exact_pairs: int, iters: int, cycles_out: torch.Tensor) -> None:
+    """cycles_out: two int64 words on the device; word 0 receives the slowest warp's clocks."""
+    assert cycles_out.is_cuda and cycles_out.dtype == torch.int64 and cycles_out.numel() >= 2
+    _check(lib().fp4attn_softmax_arith_probe(p_map, exact_pairs, iters, cycles_out.data_ptr(), _stream()),
+           "fp4attn_softmax_arith_probe")
 
 
 def fp4attn_selftest_bounded_wait(limit_cycles: int, status: torch.Tensor) -> None:

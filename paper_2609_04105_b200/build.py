@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfp4attn.so")
-SOURCES = ["api.cu", "quantize.cu", "attn_fwd.cu", "attn_fwd_2q.cu", "attn_fwd_fp8pv.cu"]
+SOURCES = ["api.cu", "quantize.cu", "attn_fwd.cu", "attn_fwd_2q.cu", "attn_fwd_fp8pv.cu", "probes.cu"]
 FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
          "-Xcompiler", "-fPIC", "--shared", "-Xptxas", "-v", "--threads", "4"]
 

@@ -264,6 +264,28 @@ def test_bounded_wait_times_out_and_reports_status():
         Bd.fp4attn_selftest_bounded_wait(0, status)
 
 
+def test_softmax_arithmetic_probe_respects_the_special_function_unit():
+    """The probe runs the kernel's score -> code arithmetic alone.  With exact codes 24 of a block's 32 elements per
+    row take ex2.approx, at 16 per clock and SM = 8 clocks per warp instruction and scheduler: no less than 192
+    clocks per block.  The affine map has no exponential and must come out faster; the hybrid maps lie between."""
+    from paper_2609_04105_b200 import binding as Bd
+    cyc = torch.zeros(2, dtype=torch.int64, device="cuda")
+    iters = 2048
+
+    def clk(p_map, pairs=0):
+        Bd.fp4attn_softmax_arith_probe(p_map, pairs, iters, cyc)
+        torch.cuda.synchronize()
+        return int(cyc[0].item()) / (4.0 * iters)
+
+    ideal, affine, hybrid8 = clk(Bd.PMAP_IDEAL), clk(Bd.PMAP_AFFINE), clk(Bd.PMAP_HYBRID, 0x5555)
+    assert 192.0 <= ideal < 300.0, ideal
+    assert 40.0 < affine < ideal and affine <= hybrid8 <= ideal, (affine, hybrid8, ideal)
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_softmax_arith_probe(Bd.PMAP_HYBRID, 0x0101, iters, cyc)
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_softmax_arith_probe(Bd.PMAP_IDEAL, 0, 0, cyc)
+
+
 # ------------------------------------------------------------------ affine classifier (p_map = AFFINE)
 def run_gpu_affine(w, q, k, v, a=0.0, b=0.0):
     from paper_2609_04105_b200 import binding as Bd
