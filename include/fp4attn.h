@@ -342,7 +342,8 @@ int fp4attn_mma_peak_probe(int iters, unsigned long long* cycles_out, fp4attn_st
  * Arithmetic ceiling of the softmax warps on the current device, measured: on every SM, sixteen warps (four per
  * scheduler, as in the attention kernel) each run the score -> code arithmetic of Algorithm "direct-p-pack" -
  * block maximum, block exponent (ceiling rule), the code map (`p_map` and `exact_pairs` as in
- * fp4attn_operands; other values: FP4ATTN_ERR_INVALID_ARG), E2M1 conversion and packing - on `iters` blocks of 32 rows x 32 scores held in shared memory, with no tensor product, tensor-memory
+ * fp4attn_operands; other values: FP4ATTN_ERR_INVALID_ARG), E2M1 conversion and packing - on `iters`
+ * (1 .. 2^20) blocks of 32 rows x 32 scores held in shared memory, with no tensor product, tensor-memory
  * access or hand-off around it.  Enqueues one kernel; cycles_out (device, TWO 64-bit words, the second is scratch)
  * receives in its first word the slowest warp's clock count, so that cycles / (4 * iters) is the clocks one
  * scheduler needs per block.  Used by the benchmark for the roofline of the softmax arithmetic; not part of the

@@ -55,7 +55,7 @@ using namespace fp4attn;
 
 extern "C" int fp4attn_softmax_arith_probe(int p_map, int exact_pairs, int iters, unsigned long long* cycles_out,
                                            fp4attn_stream_t stream) {
-  if (iters <= 0 || !cycles_out) return FP4ATTN_ERR_INVALID_ARG;
+  if (iters <= 0 || iters > (1 << 20) || !cycles_out) return FP4ATTN_ERR_INVALID_ARG;   // 2^20 blocks per warp: about half a second
   int variant;                                                  // the kernels' template argument, as in fp4attn_fwd
   if (p_map == FP4ATTN_PMAP_IDEAL) variant = 0;
   else if (p_map == FP4ATTN_PMAP_AFFINE) variant = 1;
