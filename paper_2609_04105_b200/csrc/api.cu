@@ -106,6 +106,9 @@ HostPipe* host_pipe() {
   }
   return &hp;
 }
+// First unit of group c when BH units are cut into `groups` groups whose sizes differ by at most one: the larger groups
+// come first, so that what runs after the last copy in (the last group's kernels and copy out) is as short as possible.
+inline int group_begin(int BH, int groups, int c) { return BH - (int)((long long)BH * (groups - c) / groups); }
 int enqueue_groups(HostPipe* hp, int groups, const void* q_host, const void* k_host, const void* v_host, float softmax_scale,
                    int BH, int N, int d, void* O_host, float* LSE_host, char* ws, const HostPlan& p, size_t workspace_bytes,
                    int* dev_status, cudaStream_t st) {
@@ -115,14 +118,14 @@ int enqueue_groups(HostPipe* hp, int groups, const void* q_host, const void* k_h
   const char* src[3] = {(const char*)q_host, (const char*)k_host, (const char*)v_host};
 #define FP4ATTN_CUDA_OK(call) do { if ((call) != cudaSuccess) return FP4ATTN_ERR_CUDA; } while (0)
   for (int c = 0; c < groups; ++c) {
-    const int h0 = (int)((long long)BH * c / groups), nh = (int)((long long)BH * (c + 1) / groups) - h0;
+    const int h0 = group_begin(BH, groups, c), nh = group_begin(BH, groups, c + 1) - h0;
     for (int i = 0; i < 3; ++i)
       FP4ATTN_CUDA_OK(cudaMemcpyAsync(ws + p.x[i] + h0 * head_elems * 2, src[i] + h0 * head_elems * 2, nh * head_elems * 2,
                                       cudaMemcpyHostToDevice, hp->h2d));
     FP4ATTN_CUDA_OK(cudaEventRecord(hp->in[c], hp->h2d));
   }
   for (int c = 0; c < groups; ++c) {
-    const int h0 = (int)((long long)BH * c / groups), nh = (int)((long long)BH * (c + 1) / groups) - h0;
+    const int h0 = group_begin(BH, groups, c), nh = group_begin(BH, groups, c + 1) - h0;
     FP4ATTN_CUDA_OK(cudaStreamWaitEvent(st, hp->in[c], 0));
     const size_t sf_head[3] = {sfq_head, sfq_head, sfv_head};
     for (int i = 0; i < 3; ++i) {
@@ -157,7 +160,8 @@ int attention_host_pipelined(const void* q_host, const void* k_host, const void*
   const int BH = B * H;
   // Groups of heads: at least 4 (8 from 32 heads on), and about one per 32 MB of input, so that the first copy in and
   // the last kernels and copy out - the parts nothing overlaps - stay small against the whole (measured at
-  // B=1, H=16, N=32768: 4 / 8 / 16 groups 9.31 / 8.74 / 8.61 ms; at B=4, H=16, N=4096: 4.34 / 4.39 / 4.64 ms)
+  // B=1, H=16, N=32768: 4 / 8 / 12 / 16 groups 9.31 / 8.74 / 8.28 / 8.62 ms, the copies alone 7.56 ms; at B=4, H=16,
+  // N=4096: 4.34 / 4.39 / 4.64 ms for 4 / 8 / 16)
   int groups = BH < 8 ? 1 : (BH < 2 * kMaxGroups ? 4 : 8);
   if (groups > 1) {
     const long long by_bytes = (long long)(3ull * BH * N * d * 2 / (32ull << 20));
