@@ -6,7 +6,7 @@ this script is the same comparison (tests/parity.py: strict figures, and the pro
 correct value) over ALL units, for the record.  One launch of the configuration as bench.py launches it, then the
 oracle on a pool of host processes, one unit per task.
 
-  python tests/run_full_parity.py cfg4 [--p-map affine] [--route fp8] [--workers 12] [--units 0:32]
+  python tests/run_full_parity.py cfg4 [--p-map affine] [--p-scale mse] [--route fp8] [--workers 12] [--units 0:32]
 
 Prints one JSON line per unit and a summary line.  Needs a B200; imports the oracle (test infrastructure).
 """
@@ -87,6 +87,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("workload", choices=sorted(I.WORKLOADS))
     ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine"])
+    ap.add_argument("--p-scale", default="ceil", choices=["ceil", "thr16", "mse"], help="block-exponent rule of P (mse: ideal map only)")
     ap.add_argument("--route", default="fp4", choices=["fp4", "fp8"], help="probability / value format: Direct-P FP4 or FP8 P/V")
     ap.add_argument("--workers", type=int, default=max(1, len(os.sched_getaffinity(0)) - 2))
     ap.add_argument("--units", default=None, help="begin:end slice of the (batch, head) units, default all")
@@ -101,11 +102,14 @@ def main():
     kg = Bd.fp4attn_quantize(dev(k), w.qk_fmt, Bd.ROLE_K)
     vg = Bd.fp4attn_quantize_v_e4m3(dev(v)) if args.route == "fp8" else Bd.fp4attn_quantize(dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    O, L = Bd.fp4attn_fwd(qg, kg, vg, status=status, p_map=Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_IDEAL)
+    rule = {"ceil": Bd.PSCALE_CEIL, "thr16": Bd.PSCALE_THR16, "mse": Bd.PSCALE_MSE}[args.p_scale]
+    assert args.route == "fp4" or args.p_scale == "ceil", "the FP8 P/V route has one rule"
+    O, L = Bd.fp4attn_fwd(qg, kg, vg, status=status, p_map=Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_IDEAL,
+                          p_scale_rule=rule)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     _G.update(route=args.route, w=w, q=q, k=k, v=v, O=O.float().cpu().numpy(), L=L.cpu().numpy(), Gq=None, Gk=None,
-              okw=dict(p_map=args.p_map))
+              okw=dict(p_map=args.p_map, p_scale=args.p_scale))
     if w.qk_fmt == I.FMT_NVFP4:
         _G["Gq"] = Qz.nv_tensor_scale(Qz.bf16_bits_to_f64(q))
         _G["Gk"] = Qz.nv_tensor_scale(Qz.bf16_bits_to_f64(k))
@@ -122,7 +126,7 @@ def main():
             print(json.dumps(st), flush=True)
             res.append(st)
     good = [r for r in res if r["ok"]]
-    summary = {"workload": w.name, "route": args.route, "p_map": args.p_map, "units": len(res), "units_ok": len(good),
+    summary = {"workload": w.name, "route": args.route, "p_map": args.p_map, "p_scale": args.p_scale, "units": len(res), "units_ok": len(good),
                "rows": int(sum(r["rows"] for r in good)), "wall_s": round(time.perf_counter() - t0, 1)}
     if good:
         summary.update(rel_fro_strict_max=max(r["rel_fro_strict"] for r in good), max_abs_strict=max(r["max_abs_strict"] for r in good),
