@@ -65,6 +65,11 @@ def test_host_detectable_errors_return_codes_without_a_gpu(lib):
     assert lib.fp4attn_quantize(*args(0x1004, 0, 0, 128, 128)) == 4       # misaligned
     assert lib.fp4attn_quantize(*args(0x1000, 1, 2, 128, 128, vp(0x3000))) == 1   # NVFP4 V
     assert lib.fp4attn_quantize(*args(0x1000, 1, 0, 128, 128, vp(0x3000))) == 5   # NVFP4 without workspace
+    lib.fp4attn_softmax_arith_probe.restype = ctypes.c_int
+    assert lib.fp4attn_softmax_arith_probe(0, 0, 0, vp(0x1000), None) == 1          # no iterations
+    assert lib.fp4attn_softmax_arith_probe(0, 0, 1 << 21, vp(0x1000), None) == 1    # more than the cap
+    assert lib.fp4attn_softmax_arith_probe(2, 0x0101, 16, vp(0x1000), None) == 1    # a pattern no kernel has
+    assert lib.fp4attn_softmax_arith_probe(0, 0, 16, None, None) == 1               # nowhere to write
 
 
 def test_header_is_plain_c_and_the_struct_layout_matches_the_binding(lib, tmp_path):
