@@ -143,7 +143,7 @@ def _boundary_neighbours(v: np.ndarray):
 
 def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int = 128, tile_order=None,
                   p_map: str = "ideal", affine=(1.5, 1.2), p_scale: str = "ceil", row_index=None,
-                  exact_pairs: int = 0xFFFF, report=None, flips=None, ambiguity=None):
+                  exact_pairs: int = 0xFFFF, report=None, flips=None, ambiguity=None, kv_len=None):
     """Direct-P online softmax + PV for a set of query rows of one (batch, head).
 
     s32  [R, N] float32 tensor-core-facing scores;  Vhat [N, d] float64 reconstructed V.
@@ -153,6 +153,9 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
     report : optional dict, filled with the near-decisions of every row (thresholds `ambiguity`, default
              AMBIGUITY): "code" bool [R, N] - the element's code could be its neighbour's; "eb" bool
              [R, N/32] - the block exponent could be the other integer; "row" bool [R] - any of the two.
+    kv_len : optional number of keys that exist (sequences shorter than the padded N): keys kv_len..N-1 are masked
+             like the keys a causal row does not see (score -inf: they enter no block maximum, get code 0 and no
+             weight), so the result is that of the operator on the first kv_len keys.
     flips  : optional dict with the same two keys: decisions to take the OTHER way.  A flipped code moves to
              the code across its nearest boundary; a flipped block exponent to the integer on the other side
              of the block maximum, and the block's codes follow from the new exponent.
@@ -161,6 +164,9 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
     assert N % P_BLOCK == 0 and tile % P_BLOCK == 0 and N % tile == 0
     if row_index is not None:                                    # causal: query row i sees keys 0..i
         s32 = np.where(np.arange(N)[None, :] > np.asarray(row_index)[:, None], np.float32(-np.inf), s32).astype(np.float32)
+    if kv_len is not None:                                       # padded sequence: keys kv_len.. do not exist
+        assert 1 <= int(kv_len) <= N
+        s32 = np.where(np.arange(N)[None, :] >= int(kv_len), np.float32(-np.inf), s32).astype(np.float32)
     y32 = (s32 * np.float32(c32)).astype(np.float32)             # decision variable, fp32
     yx = s32.astype(np.float64) * np.float64(c32)                # converter input, fp64
     mu = np.full(R, -np.inf)
@@ -288,8 +294,13 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
 
 def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int = 128,
                      rows=None, heads=None, tile_order=None, p_map: str = "ideal", affine=(1.5, 1.2),
-                     p_scale: str = "ceil", causal: bool = False, kv_group: int = 1, exact_pairs: int = 0xFFFF):
+                     p_scale: str = "ceil", causal: bool = False, kv_group: int = 1, exact_pairs: int = 0xFFFF,
+                     seq_len=None):
     """Whole-operator oracle.  qd/kd/vd come from oracle.quantize.quantize_qk / quantize_v.
+
+    seq_len : optional [B] integers, 1 <= seq_len[b] <= N: batch entry b is a sequence of seq_len[b] tokens padded
+              to N.  Its keys beyond the length are masked; its query rows beyond the length carry no meaning and
+              are returned as NaN (a caller compares rows below the length only).
 
     rows : optional 1-D index array of query rows evaluated for every (b, h) (rows are
            independent); heads : optional list of (b, h) pairs.  Returns O [n_heads, R, d]
@@ -306,7 +317,11 @@ def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int
         s32 = scores_fp32(qd, kd, b, h, rows, hk)
         Vhat = dequantize({**vd, "nib": vd["nib"][b, hk][None, None], "sf": vd["sf"][b, hk][None, None]})[0, 0].T
         O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order, p_map, affine, p_scale,
-                                        ridx if causal else None, exact_pairs)
+                                        ridx if causal else None, exact_pairs,
+                                        kv_len=None if seq_len is None else int(seq_len[b]))
+        if seq_len is not None:
+            O[ridx >= int(seq_len[b])] = np.nan
+            lse[ridx >= int(seq_len[b])] = np.nan
         Os.append(O)
         Ls.append(lse)
     return np.stack(Os), np.stack(Ls)

@@ -617,3 +617,50 @@ def test_mse_rule_reproduces_table_p_range_mxfp4_row_and_reports_near_ties():
     fl[0, b] = True
     _, _, _, E3, _ = A.direct_p_rows(y[i:i + 1], np.float32(1.0), V, tile=128, p_scale="mse", flips={"eb": fl})
     assert abs(int(E3[0, b]) - int(EB[i, b])) == 1 and np.array_equal(np.delete(E3[0], b), np.delete(EB[i], b))
+
+
+# ------------------------------------------------------------------ padded sequences (seq_len)
+def test_sequence_length_equal_to_n_changes_nothing_and_rows_beyond_a_length_are_not_returned():
+    w, _, qd, kd, vd = _cfg1(N=256, B=2, H=2)
+    O, L = A.direct_p_forward(qd, kd, vd)
+    O2, L2 = A.direct_p_forward(qd, kd, vd, seq_len=[256, 256])
+    assert np.array_equal(O, O2) and np.array_equal(L, L2)
+    O3, L3 = A.direct_p_forward(qd, kd, vd, seq_len=[256, 100])
+    assert np.array_equal(O3[:2], O[:2]) and np.array_equal(L3[:2], L[:2])          # batch entry 0 is complete
+    assert np.isnan(O3[2:, 100:]).all() and np.isnan(L3[2:, 100:]).all() and np.isfinite(O3[2:, :100]).all()
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_sequence_length_on_a_block_boundary_equals_the_operator_on_the_truncated_operands(causal):
+    """A length that is a multiple of 32 cuts between blocks of Q/K rows, of V's key blocks and of P: the padded
+    operator must return what the plain operator returns on the first `len` tokens of the quantized operands."""
+    w, _, qd, kd, vd = _cfg1(N=384, H=2)
+    for n in (32, 160, 256, 352):
+        O, L = A.direct_p_forward(qd, kd, vd, seq_len=[n], causal=causal)
+        cut = lambda t: {**t, "nib": t["nib"][:, :, :n], "sf": t["sf"][:, :, :n]}
+        vcut = {**vd, "nib": vd["nib"][..., :n], "sf": vd["sf"][..., : n // 32]}
+        Ot, Lt = A.direct_p_forward(cut(qd), cut(kd), vcut, tile=32, causal=causal)
+        assert np.abs(O[:, :n] - Ot).max() < 1e-13 and np.abs(L[:, :n] - Lt).max() < 1e-12
+
+
+def test_sequence_length_inside_a_block_against_the_plain_definition():
+    """A length that cuts a 32-key block: the block maximum, hence the block exponent, is taken over the keys that
+    exist; the others carry no code.  Checked against Eq. "represented-output" written out over the existing keys."""
+    w, _, qd, kd, vd = _cfg1(N=128, H=1)
+    n = 77
+    c32 = A.score_constant(qd, kd, w.d)
+    s32 = A.scores_fp32(qd, kd, 0, 0)
+    Vhat = np.ascontiguousarray(np.swapaxes(Qz.dequantize(vd), -1, -2)[0, 0])
+    O, L, codes, EB, _ = A.direct_p_rows(s32[:8], c32, Vhat, kv_len=n)
+    assert not codes[:, n:].any()
+    y32 = (s32[:8] * np.float32(c32)).astype(np.float32)
+    for i in range(8):
+        E_B = [math.ceil(float(y32[i, b:min(b + 32, n)].max())) for b in range(0, n, 32)]
+        assert E_B == [int(e) for e in EB[i, : len(E_B)]]
+        cd = []
+        for j in range(n):                                       # codes of the ideal map, from its definition
+            v = 6.0 * 2.0 ** (float(s32[i, j]) * float(c32) - E_B[j // 32])
+            cd.append(int(F.e2m1_encode_mag(np.array([v]))[0]))
+        assert cd == [int(c) for c in codes[i, :n]]
+        Oi, Li = _plain_definition(y32[i, :n], E_B, cd, Vhat[:n])
+        assert np.abs(O[i] - Oi).max() < 1e-13 and abs(L[i] - Li) < 1e-12
