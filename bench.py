@@ -555,6 +555,11 @@ def run_cuda(args, w):
                 variants += [("two_query_", dict(schedule=Bd.SCHEDULE_TWO_QUERY), 1.0),
                              ("two_query_affine_", dict(schedule=Bd.SCHEDULE_TWO_QUERY, p_map=Bd.PMAP_AFFINE), 1.0)]
             variants.append(("fp8_pv_", None, 1.0))
+            if ww.B >= 4:                                            # padded sequences: a fixed mix of token counts
+                mix = [ww.N, ww.N * 5 // 8 - 120, ww.N // 2 + 1, 300] + [ww.N] * (ww.B - 4)
+                sl = torch.tensor(mix, dtype=torch.int32, device=dev)
+                variants.append(("length_mix_", dict(seq_len=sl), sum(float(n) * n for n in mix) / (ww.B * float(ww.N) ** 2)))
+                rec["length_mix_tokens"] = mix
             for key, kw, share in variants:
                 fn = (lambda: Bd.fp4attn_fwd(sq, sk, sv8, out=so, status=status)) if kw is None else \
                      (lambda: Bd.fp4attn_fwd(sq, sk, sv, out=so, status=status, **kw))
@@ -562,7 +567,8 @@ def run_cuda(args, w):
                     fn()
                 torch.cuda.synchronize()
                 ms = statistics.median(timed_launches(fn, n_it, flush, E, torch.cuda.synchronize))
-                # causal: flops counted as half of the full product (the usual convention)
+                # causal: flops counted as half of the full product (the usual convention); length mix: the scores of
+                # the tokens that exist
                 rec[key + "attn_ms"] = ms
                 rec[key + "attn_tflops"] = share * ww.flops / (ms * 1e-3) / 1e12
                 if not key:

@@ -226,6 +226,9 @@ typedef struct {
                                        [B, kv_heads, d, N] from fp4attn_quantize_v_e4m3, v_sf is ignored, v_G is required;
                                        with the ideal map, the ceiling rule and the one-query schedule only          */
   const float* v_G;                 /* FP4ATTN_PV_E4M3: device fp32 encode factors of V, one per (batch, K/V head)    */
+  const int* seq_len;               /* NULL, or B device integers: batch entry b is a sequence of seq_len[b] tokens
+                                       padded to N (see fp4attn_fwd); values are clamped into 1..N.  With the ideal and
+                                       the affine map, the one-query schedule and FP4ATTN_PV_MXFP4 only              */
 } fp4attn_operands;
 
 /*
@@ -250,6 +253,14 @@ typedef struct {
  * keys j > i are removed from row i before anything else: they never raise a block maximum, always
  * code to 0, and a block without a visible key contributes nothing.  B, H, N, d describe Q and O;
  * K and V have kv_heads heads.
+ *
+ * Padded sequences.  With seq_len != NULL, batch entry b holds a sequence of L = seq_len[b] tokens (1 <= L <= N) in
+ * buffers laid out for N: keys L..N-1 are removed from every row of that entry exactly as a causal row's invisible
+ * keys are (a block's maximum, hence its exponent, is taken over the keys that exist), key tiles that lie entirely
+ * beyond L are neither loaded nor multiplied, query tiles that lie entirely beyond L walk one key tile only, and rows
+ * L..N-1 of O and LSE receive unspecified finite values.  What the padding positions of Q, K and V hold is irrelevant as long as the quantizers were given
+ * finite numbers there (a 32-key block of V that straddles L takes its scale from all 32 keys).  Combines with
+ * causal = 1 and with grouped K/V heads.
  *
  * What FP4ATTN_PMAP_IDEAL guarantees.  x is one fused multiply-add in float32, x = fma(S, c, fl32(log2 6 - E_B)).
  * Of the 16 element pairs (keys 2k, 2k+1) of a block, pairs 0, 5, 10 and 15 evaluate 2^x by a degree-6

@@ -47,7 +47,7 @@ class _Operands(ctypes.Structure):
                 ("p_map", ctypes.c_int), ("affine_a", ctypes.c_float), ("affine_b", ctypes.c_float),
                 ("p_scale_rule", ctypes.c_int), ("causal", ctypes.c_int), ("kv_heads", ctypes.c_int),
                 ("exact_pairs", ctypes.c_int), ("g_per_head", ctypes.c_int), ("schedule", ctypes.c_int),
-                ("pv_fmt", ctypes.c_int), ("v_G", ctypes.c_void_p)]
+                ("pv_fmt", ctypes.c_int), ("v_G", ctypes.c_void_p), ("seq_len", ctypes.c_void_p)]
 
 
 def _load() -> ctypes.CDLL:
@@ -227,14 +227,17 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
                 out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
                 status: Optional[torch.Tensor] = None, p_map: int = PMAP_IDEAL, affine_a: float = 0.0,
                 affine_b: float = 0.0, p_scale_rule: int = PSCALE_CEIL, causal: bool = False,
-                exact_pairs: int = 0, schedule: int = SCHEDULE_ONE_QUERY) -> Tuple[torch.Tensor, torch.Tensor]:
+                exact_pairs: int = 0, schedule: int = SCHEDULE_ONE_QUERY,
+                seq_len: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
     """Direct-P attention forward on quantized operands -> (O bf16 [B,H,N,d], LSE fp32 [B,H,N]).
-    p_map selects the exact code map or the affine classifier (affine_a = 0: A = 1.5, B = 1.2)."""
+    p_map selects the exact code map or the affine classifier (affine_a = 0: A = 1.5, B = 1.2).
+    seq_len: optional CUDA int32 tensor [B], the token count of every batch entry (padded to N)."""
     B, H, N, d = q.shape
     Hkv = k.shape[1]                                   # grouped-query attention when Hkv < H
     assert k.shape == v.shape and k.shape == (B, Hkv, N, d) and H % Hkv == 0 and q.fmt == k.fmt and v.fmt in (FMT_MXFP4, FMT_E4M3)
     fp8 = v.fmt == FMT_E4M3
     assert q.per_head == k.per_head, "Q and K must both carry per-head factors, or neither"
+    assert seq_len is None or (seq_len.is_cuda and seq_len.dtype == torch.int32 and seq_len.numel() == B and seq_len.is_contiguous())
     dev = q.packed.device
     if out is None:
         out = torch.empty((B, H, N, d), dtype=torch.bfloat16, device=dev)
@@ -243,7 +246,8 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
     ops = _Operands(q.packed.data_ptr(), k.packed.data_ptr(), v.packed.data_ptr(),
                     q.scales.data_ptr(), k.scales.data_ptr(), None if fp8 else v.scales.data_ptr(),
                     _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b), int(p_scale_rule), int(bool(causal)), int(Hkv),
-                    int(exact_pairs), int(q.per_head), int(schedule), PV_E4M3 if fp8 else PV_MXFP4, _ptr(v.G) if fp8 else None)
+                    int(exact_pairs), int(q.per_head), int(schedule), PV_E4M3 if fp8 else PV_MXFP4, _ptr(v.G) if fp8 else None,
+                    _ptr(seq_len))
     _check(lib().fp4attn_fwd(ctypes.byref(ops), B, H, N, d, out.data_ptr(), lse.data_ptr(), _ptr(status), _stream()),
            "fp4attn_fwd")
     return out, lse

@@ -34,7 +34,7 @@ extern "C" const char* fp4attn_status_string(int status) {
   }
 }
 
-extern "C" int fp4attn_version(void) { return 200; }
+extern "C" int fp4attn_version(void) { return 300; }
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 

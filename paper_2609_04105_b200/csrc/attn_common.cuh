@@ -76,6 +76,8 @@ struct AttnParams {
   int H, Hkv;              // query heads, K/V heads (H % Hkv == 0: grouped-query attention)
   int BH;                  // B * H
   unsigned long long recip_qtiles, recip_bh;   // ceil(2^64 / (N / 128)), ceil(2^64 / BH); 0 for a divisor of 1
+  const int* seq_len;      // NULL, or B token counts: batch entry b is seq_len[b] tokens padded to N (masked kernels only)
+  unsigned long long recip_h;                  // ceil(2^64 / H); 0 for H = 1
 };
 
 // One work item = one 128-row query tile of one (batch, query head).
@@ -85,15 +87,19 @@ struct WorkItem {
   int qtile_lin;           // (b*H + h) * qtiles + qt: index of the tile's Q scale atom(s)
   int kvh;                 // b*Hkv + h / (H/Hkv): the K/V head this query head reads
   int bh;                  // b*H + h
-  int T2;                  // 128-key stages to walk (causal: up to and including the diagonal)
+  int T2;                  // 128-key stages to walk (causal: up to and including the diagonal; padded: those with a key)
+  int len;                 // keys that exist for this unit (N unless the batch entry is a padded sequence)
 };
 // floor(n / d) for n < 2^31 through the precomputed reciprocal ceil(2^64 / d) (0 stands for d = 1): the
 // roles decode a work item on their critical path, and a 32-bit division costs some fifty instructions
 __device__ __forceinline__ int fast_div(int n, unsigned long long recip) {
   return recip ? (int)__umul64hi((unsigned long long)n, recip) : n;
 }
-template <bool CAUSAL>
+// MASKED: the kernels that mask the last stage of an item - the causal mask (p.causal), padded sequences
+// (p.seq_len), or both.  The unmasked kernels ignore both fields.
+template <bool MASKED>
 __device__ __forceinline__ WorkItem decode_item(int item, const AttnParams& p, int qtiles) {
+  constexpr bool CAUSAL = MASKED;
   WorkItem w;
   int bh;
   if (CAUSAL) {             // longest items first, so the persistent CTAs finish together
@@ -112,7 +118,16 @@ __device__ __forceinline__ WorkItem decode_item(int item, const AttnParams& p, i
     const int b = bh / p.H, h = bh - b * p.H;
     w.kvh = b * p.Hkv + h / (p.H / p.Hkv);
   }
-  w.T2 = CAUSAL ? w.qt + 1 : p.stages;
+  w.len = p.N;
+  w.T2 = p.stages;
+  if (MASKED) {
+    if (p.seq_len) {
+      const int len = __ldg(p.seq_len + fast_div(bh, p.recip_h));
+      w.len = len < 1 ? 1 : (len > p.N ? p.N : len);
+      w.T2 = w.qt * BM < w.len ? (w.len + BS - 1) / BS : 1;   // a query tile beyond the length: one stage, results unused
+    }
+    if (p.causal && w.qt + 1 < w.T2) w.T2 = w.qt + 1;
+  }
   return w;
 }
 

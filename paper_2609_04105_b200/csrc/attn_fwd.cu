@@ -408,11 +408,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     bool ok = true;
     int T2 = 0;
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, g0 += T2) {
-      uint32_t gdiag;                                           // global index of the causal diagonal stage (none: ~0)
+      uint32_t gdiag;                                           // global index of the item's masked stage, its last (none: ~0)
+      int vis;                                                  // keys of that stage this row sees
       {
         const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
         T2 = wi.T2;
-        gdiag = CAUSAL ? g0 + (uint32_t)wi.qt : 0xFFFFFFFFu;
+        gdiag = CAUSAL ? g0 + (uint32_t)(T2 - 1) : 0xFFFFFFFFu;
+        // causal: keys 0..i of row i = qt * 128 + row; padded sequence: keys 0..len-1; both: the fewer
+        const int seen = (CAUSAL && p.causal) ? min(wi.len, wi.qt * BM + row + 1) : wi.len;
+        vis = seen - (T2 - 1) * BS;
         if (NV == 2)                                            // this unit's own pair of encode factors
           c32 = __fdiv_rn(p.c_base, __fmul_rn(__ldg(p.q_G + wi.bh), __ldg(p.k_G + wi.kvh)));
       }
@@ -434,8 +438,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (lane == 0) mbar_arrive(sempty);                   // pair may take the stage after next
           direct_p_block<PMAP, false, THR16>(sraw, c32, p.aff_a, p.aff_b, 32, E1, w1);
         } else {
-          // causal diagonal stage: this row sees keys 0..row of the stage; the team's tile starts at key 64*(team&1)
-          const int v0 = row - 64 * (team & 1) + 1;
+          // masked stage: this row sees the first `vis` keys of the stage; the team's tile starts at key 64*(team&1)
+          const int v0 = vis - 64 * (team & 1);
           direct_p_block<PMAP, true, THR16>(sraw, c32, p.aff_a, p.aff_b, v0, E0, w0);
           tmem_ld_32x32b_x32(tS + 32, sraw);
           tmem_wait_ld();
@@ -649,7 +653,7 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   int pmap = ops->p_map;                                          // kernel instance: 0 ideal, 1 affine, 2..4 mixed patterns
   if (ops->p_map == FP4ATTN_PMAP_HYBRID) {
     pmap = ops->exact_pairs == 0x1111 ? 2 : ops->exact_pairs == 0x5555 ? 3 : ops->exact_pairs == 0x7777 ? 4 : -1;
-    if (pmap < 0 || ops->causal) return FP4ATTN_ERR_INVALID_ARG;    // three patterns, noncausal only
+    if (pmap < 0 || ops->causal || ops->seq_len) return FP4ATTN_ERR_INVALID_ARG;    // three patterns, no masks
   }
   if (ops->p_scale_rule != FP4ATTN_PSCALE_CEIL && ops->p_scale_rule != FP4ATTN_PSCALE_THR16 && ops->p_scale_rule != FP4ATTN_PSCALE_MSE)
     return FP4ATTN_ERR_INVALID_ARG;
@@ -676,6 +680,9 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.recip_qtiles = (N / BM) > 1 ? ~0ull / (unsigned long long)(N / BM) + 1 : 0;
   prm.recip_bh = prm.BH > 1 ? ~0ull / (unsigned long long)prm.BH + 1 : 0;
   prm.causal = ops->causal ? 1 : 0;
+  prm.seq_len = ops->seq_len;
+  prm.recip_h = H > 1 ? ~0ull / (unsigned long long)H + 1 : 0;
+  const bool masked = prm.causal || prm.seq_len;                  // kernels that mask an item's last stage
   prm.H = H;
   prm.Hkv = ops->kv_heads > 0 ? ops->kv_heads : H;
   const float scale = ops->softmax_scale > 0.f ? ops->softmax_scale : (float)(1.0 / sqrt((double)d));
@@ -687,10 +694,12 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.thr16 = ops->p_scale_rule == FP4ATTN_PSCALE_THR16;
   if (ops->schedule != FP4ATTN_SCHEDULE_ONE_QUERY && ops->schedule != FP4ATTN_SCHEDULE_TWO_QUERY) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->pv_fmt != FP4ATTN_PV_MXFP4 && ops->pv_fmt != FP4ATTN_PV_E4M3) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->seq_len && (ops->pv_fmt != FP4ATTN_PV_MXFP4 || ops->schedule != FP4ATTN_SCHEDULE_ONE_QUERY)) return FP4ATTN_ERR_INVALID_ARG;
+  if (((uintptr_t)ops->seq_len & 3) != 0) return FP4ATTN_ERR_ALIGNMENT;
   if (ops->pv_fmt == FP4ATTN_PV_E4M3) return launch_attn_fp8pv(ops, B, H, N, d, prm, st);
   if (ops->schedule == FP4ATTN_SCHEDULE_TWO_QUERY) return launch_attn_two_query(ops, B, H, N, d, pmap, prm, st);
   if (ops->p_scale_rule == FP4ATTN_PSCALE_MSE) {
-    const int sel = (d == 128 ? 4 : 0) | (nv ? 2 : 0) | (prm.causal ? 1 : 0);
+    const int sel = (d == 128 ? 4 : 0) | (nv ? 2 : 0) | (masked ? 1 : 0);
     switch (sel) {
       case 0: return launch_attn<64, 0, 0, false, 2>(ops, B, H, N, prm, st);
       case 1: return launch_attn<64, 0, 0, true, 2>(ops, B, H, N, prm, st);
@@ -717,7 +726,7 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
     default: return launch_attn<128, 1, PM_, CAU_, THR_>(ops, B, H, N, prm, st);         \
   }
 #define FP4ATTN_MASKS(PM_)                                         \
-  if (prm.causal) {                                                \
+  if (masked) {                                                    \
     if (prm.thr16) { FP4ATTN_SHAPES(PM_, true, true) }             \
     else           { FP4ATTN_SHAPES(PM_, true, false) }            \
   } else {                                                         \

@@ -411,6 +411,136 @@ def test_causal_and_gqa_match_oracle_elementwise(name, kw, group, p_map):
     check_heads(Og, Lg, Oo, Lo, heads)
 
 
+# ------------------------------------------------------------------ padded sequences (seq_len)
+SEQLEN_CASES = [
+    # name, shrink, lengths per batch entry, causal, K/V group, map, block-exponent rule
+    ("cfg1", dict(B=3, H=2, N=512), [512, 300, 77], False, 1, "ideal", "ceil"),      # full, inside a tile, inside a block
+    ("cfg1", dict(B=4, H=2, N=384), [1, 32, 128, 383], False, 1, "ideal", "ceil"),   # one key; block and tile boundaries
+    ("cfg1", dict(B=2, H=4, N=640), [129, 600], True, 2, "ideal", "ceil"),           # causal, grouped K/V heads
+    ("cfg1", dict(B=2, H=2, N=512), [200, 470], True, 1, "affine", "thr16"),
+    ("cfg3", dict(B=2, H=2, N=512), [5, 257], False, 1, "affine", "ceil"),           # NVFP4 Q/K, d = 64
+    ("cfg3", dict(B=2, H=2, N=768), [700, 330], True, 1, "ideal", "ceil"),
+    ("cfg2", dict(B=2, H=2, N=1024), [1000, 640], False, 1, "ideal", "mse"),         # d = 128, MSE-selected exponents
+    ("cfg4", dict(B=1, H=2, N=1024), [900], False, 1, "ideal", "ceil"),              # outlier channels
+]
+
+
+@pytest.mark.parametrize("name,kw,lens,causal,group,p_map,p_scale", SEQLEN_CASES)
+def test_padded_sequences_match_oracle_on_the_rows_that_exist(name, kw, lens, causal, group, p_map, p_scale):
+    """Per-batch token counts: keys beyond a count are masked, key tiles beyond it skipped; the rows below the count
+    are compared with the oracle (whole-head protocol), the rows beyond it must at least be finite."""
+    import parity
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    k, v = np.ascontiguousarray(k[:, : w.H // group]), np.ascontiguousarray(v[:, : w.H // group])
+    sl = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    rule = {"ceil": Bd.PSCALE_CEIL, "thr16": Bd.PSCALE_THR16, "mse": Bd.PSCALE_MSE}[p_scale]
+    Og, Lg = run_gpu_general(w, q, k, v, causal=causal, seq_len=sl, p_scale_rule=rule,
+                             p_map=Bd.PMAP_AFFINE if p_map == "affine" else Bd.PMAP_IDEAL)
+    fmt = "mx" if w.qk_fmt == I.FMT_MXFP4 else "nv"
+    qd, kd, vd = Qz.quantize_qk(q, fmt), Qz.quantize_qk(k, fmt), Qz.quantize_v(v)
+    for b in range(w.B):
+        n = lens[b]
+        for h in range(w.H):
+            st = parity.compare_head(Og[b, h], Lg[b, h], qd, kd, vd, b, h, rows=np.arange(n), kv_group=group, causal=causal,
+                                     p_map=p_map, p_scale=p_scale, kv_len=n)
+            assert st["lse_err"] <= parity.LSE_ABS, st
+            # rows of the last tile that holds a token are computed (over the keys that exist); none may be NaN or Inf
+            last = min(w.N, (n + 127) // 128 * 128)
+            assert np.isfinite(Og[b, h][:last]).all() and np.isfinite(Lg[b, h][:last]).all()
+
+
+def test_padded_sequences_full_size_length_mix_sampled_rows_and_timing():
+    """B4 H16 N8192 d128 with a mix of lengths (full, inside a tile, one key past a tile boundary, short): sampled rows
+    of two heads per batch entry against the oracle, noncausal and causal; and the launch takes less time than the full
+    one (key tiles beyond a length are skipped, query tiles beyond it walk a single stage)."""
+    import parity
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.WORKLOADS["cfg5_N8192"]
+    lens = [8192, 5000, 4097, 300]
+    q, k, v = I.make_qkv(w)
+    qg, kg = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+    vg = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    sl = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    qd, kd, vd = oracle_operands(w, q, k, v)
+    rng = np.random.default_rng(11)
+    for causal in (False, True):
+        O, L = Bd.fp4attn_fwd(qg, kg, vg, status=status, seq_len=sl, causal=causal)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        Og, Lg = O.float().cpu().numpy().astype(np.float64), L.cpu().numpy().astype(np.float64)
+        for b, n in enumerate(lens):
+            rows = np.unique(np.concatenate([[0, n - 1], rng.choice(n, size=min(n, 96), replace=False)]))
+            for h in rng.choice(w.H, size=2, replace=False):
+                st = parity.compare_head(Og[b, h], Lg[b, h], qd, kd, vd, b, int(h), rows=rows, causal=causal, kv_len=n)
+                assert st["lse_err"] <= parity.LSE_ABS, st
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    for _ in range(2):
+        Bd.fp4attn_fwd(qg, kg, vg, status=status)
+    ev[0].record()
+    Bd.fp4attn_fwd(qg, kg, vg, status=status)
+    ev[1].record()
+    Bd.fp4attn_fwd(qg, kg, vg, status=status, seq_len=sl)
+    ev[2].record()
+    torch.cuda.synchronize()
+    full, part = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
+    work = sum(float(n) * n for n in lens) / (len(lens) * float(w.N) ** 2)          # 0.41 of the full launch's scores
+    print(f"full {full:.3f} ms, length mix {part:.3f} ms, share of the scores {work:.2f}")
+    assert part < 0.75 * full
+
+
+def test_padded_sequences_full_length_is_bit_identical_and_padding_content_is_irrelevant():
+    """seq_len = N must give the bits of the call without seq_len (another kernel instance: the masked one).  And what
+    sits in the padding of Q and K, and in V beyond the 32-key block that holds the last token, cannot change the
+    rows that exist."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg2"], B=2, H=2, N=768)
+    q, k, v = I.make_qkv(w)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def run(q, k, v, lens):
+        qg, kg = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+        vg = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+        sl = None if lens is None else torch.tensor(lens, dtype=torch.int32, device="cuda")
+        O, L = Bd.fp4attn_fwd(qg, kg, vg, status=status, seq_len=sl)
+        torch.cuda.synchronize()
+        return O, L
+
+    O0, L0 = run(q, k, v, None)
+    O1, L1 = run(q, k, v, [768, 768])
+    assert torch.equal(O0, O1) and torch.equal(L0, L1)
+    lens = [500, 290]
+    O2, L2 = run(q, k, v, lens)
+    q2, k2, v2 = q.copy(), k.copy(), v.copy()
+    rng = np.random.default_rng(5)
+    for b, n in enumerate(lens):
+        pad = (n + 31) // 32 * 32                                # V: the straddling block keeps its scale
+        for t, lo in ((q2, n), (k2, n), (v2, pad)):
+            shape = t[b, :, lo:].shape                           # finite bf16 of either sign, magnitudes 2^-7 .. 2^9
+            t[b, :, lo:] = (rng.integers(0x3C00, 0x4400, size=shape) | (rng.integers(0, 2, size=shape) << 15)).astype(t.dtype)
+    O3, L3 = run(q2, k2, v2, lens)
+    for b, n in enumerate(lens):
+        assert torch.equal(O2[b, :, :n], O3[b, :, :n]) and torch.equal(L2[b, :, :n], L3[b, :, :n])
+    assert int(status.item()) == 0
+
+
+def test_padded_sequences_reject_what_they_do_not_cover():
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg3"], B=2, H=2, N=512)
+    q, k, v = I.make_qkv(w)
+    qg, kg = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+    vg = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    sl = torch.tensor([100, 200], dtype=torch.int32, device="cuda")
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_fwd(qg, kg, vg, seq_len=sl, schedule=Bd.SCHEDULE_TWO_QUERY)
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_fwd(qg, kg, vg, seq_len=sl, p_map=Bd.PMAP_HYBRID, exact_pairs=0x5555)
+    with pytest.raises(Bd.Fp4AttnError):
+        Bd.fp4attn_fwd(qg, kg, Bd.fp4attn_quantize_v_e4m3(_dev(v)), seq_len=sl)
+
+
 def test_gqa_noncausal_matches_oracle():
     w = I.shrink(I.WORKLOADS["cfg1"], N=384, H=6)
     q, k, v = I.make_qkv(w)
