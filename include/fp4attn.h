@@ -258,8 +258,10 @@ typedef struct {
  * buffers laid out for N: keys L..N-1 are removed from every row of that entry exactly as a causal row's invisible
  * keys are (a block's maximum, hence its exponent, is taken over the keys that exist), key tiles that lie entirely
  * beyond L are neither loaded nor multiplied, query tiles that lie entirely beyond L walk one key tile only, and rows
- * L..N-1 of O and LSE receive unspecified finite values.  What the padding positions of Q, K and V hold is irrelevant as long as the quantizers were given
- * finite numbers there (a 32-key block of V that straddles L takes its scale from all 32 keys).  Combines with
+ * L..N-1 of O and LSE receive unspecified finite values.  The quantizers see the padded buffers: MXFP4 rows of Q and K
+ * are quantized one by one, so their padding rows only have to be finite; a 32-key block of V that straddles L takes its
+ * scale from all 32 keys, and an NVFP4 encode factor from the maximum over the whole tensor (or unit), so V's padding
+ * keys and, with NVFP4, all padding should hold zeros unless they are meant to take part in those maxima.  Combines with
  * causal = 1 and with grouped K/V heads.
  *
  * What FP4ATTN_PMAP_IDEAL guarantees.  x is one fused multiply-add in float32, x = fma(S, c, fl32(log2 6 - E_B)).

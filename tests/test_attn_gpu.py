@@ -704,6 +704,41 @@ def test_random_configurations_match_oracle(seed):
         check_heads(O.float().cpu().numpy().astype(np.float64), L.cpu().numpy().astype(np.float64), Oo, Lo, heads, rows)
 
 
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_padded_configurations_match_oracle(seed):
+    """Thirty seeded draws per seed of (d, Q/K format, N, B, heads, K/V head sharing, mask, code map, block-exponent
+    rule, token counts per batch entry): sampled existing rows of two heads each against the oracle."""
+    from paper_2609_04105_b200 import binding as Bd
+    rng = np.random.default_rng(seed)
+    for _ in range(30):
+        d = int(rng.choice([64, 128])); nv = bool(rng.integers(0, 2))
+        N = 128 * int(rng.integers(1, 9)); B = int(rng.integers(1, 5))
+        group = int(rng.choice([1, 1, 2, 4])); Hkv = int(rng.integers(1, 4)); H = Hkv * group
+        causal = bool(rng.integers(0, 2)); pm = int(rng.integers(0, 2))
+        rule = int(rng.choice([Bd.PSCALE_CEIL, Bd.PSCALE_THR16, Bd.PSCALE_MSE])) if pm == 0 else int(rng.integers(0, 2))
+        lens = [int(rng.choice([1, N, int(rng.integers(1, N + 1)), 32 * int(rng.integers(1, N // 32 + 1))])) for _ in range(B)]
+        x = [rng.standard_normal((B, h, N, d)).astype(np.float32) for h in (H, Hkv, Hkv)]
+        bits = [I.f32_to_bf16_bits(a) for a in x]
+        fmt = Bd.FMT_NVFP4 if nv else Bd.FMT_MXFP4
+        ops = [Bd.fp4attn_quantize(_dev(bits[0]), fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(bits[1]), fmt, Bd.ROLE_K),
+               Bd.fp4attn_quantize(_dev(bits[2]), Bd.FMT_MXFP4, Bd.ROLE_V)]
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        O, L = Bd.fp4attn_fwd(*ops, status=status, p_map=pm, p_scale_rule=rule, causal=causal,
+                              seq_len=torch.tensor(lens, dtype=torch.int32, device="cuda"))
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        name = "nv" if nv else "mx"
+        qd, kd, vd = Qz.quantize_qk(bits[0], name), Qz.quantize_qk(bits[1], name), Qz.quantize_v(bits[2])
+        Og, Lg = O.float().cpu().numpy().astype(np.float64), L.cpu().numpy().astype(np.float64)
+        okw = dict(p_map=["ideal", "affine"][pm], p_scale=["ceil", "thr16", "mse"][rule], causal=causal, kv_group=group, seq_len=lens)
+        for _ in range(2):
+            b, h = int(rng.integers(0, B)), int(rng.integers(0, H))
+            n = lens[b]
+            rows = np.unique(np.concatenate([[0, n - 1], rng.choice(n, size=min(n, 40), replace=False)]))
+            Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=[(b, h)], rows=rows, **okw)
+            check_heads(Og, Lg, Oo, Lo, [(b, h)], rows)
+
+
 @pytest.mark.parametrize("kw,group,causal", [(dict(B=2, H=4, N=512), 1, False), (dict(B=1, H=4, N=384, d=128), 2, True),
                                              (dict(B=2, H=6, N=256), 3, False)])
 def test_nvfp4_per_head_factors_attention_matches_oracle(kw, group, causal):
