@@ -228,7 +228,7 @@ typedef struct {
   const float* v_G;                 /* FP4ATTN_PV_E4M3: device fp32 encode factors of V, one per (batch, K/V head)    */
   const int* seq_len;               /* NULL, or B device integers: batch entry b is a sequence of seq_len[b] tokens
                                        padded to N (see fp4attn_fwd); values are clamped into 1..N.  With the ideal and
-                                       the affine map, the one-query schedule and FP4ATTN_PV_MXFP4 only              */
+                                       the affine map (and with FP4ATTN_PV_E4M3), one-query schedule only            */
 } fp4attn_operands;
 
 /*

@@ -331,7 +331,7 @@ def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int
 P8_SHIFT = 8      # probabilities are carried as 2**8 * p, so the largest (p = 1) is 256 <= 448, the E4M3 maximum
 
 
-def fp8_pv_rows(s32: np.ndarray, c32: np.float32, V8hat: np.ndarray, row_index=None):
+def fp8_pv_rows(s32: np.ndarray, c32: np.float32, V8hat: np.ndarray, row_index=None, kv_len=None):
     """FP8 probabilities and values for a set of query rows of one (batch, head) (the route the paper retains for
     training, Section "Training stability selects FP8 P/V"; it prints no algorithm, reading taken here).
 
@@ -342,11 +342,15 @@ def fp8_pv_rows(s32: np.ndarray, c32: np.float32, V8hat: np.ndarray, row_index=N
               of 2**-9; below 2**-10 the value is 0): one 8-bit float per probability, NO block scales;
       O_i   = sum_j p8_ij V^_j / sum_j p8_ij (the same rounded values in numerator and denominator, Eq.
               "represented-output" carried over), LSE_i = ln2 (mu_i - 8 + log2 sum_j p8_ij).
-    Returns O [R, d], LSE [R], the E4M3 bytes [R, N] and mu [R]."""
+    kv_len: optional number of keys that exist (padded sequence); the others are masked like a causal row's
+    invisible keys.  Returns O [R, d], LSE [R], the E4M3 bytes [R, N] and mu [R]."""
     from .formats import e4m3_decode, e4m3_encode_unsigned
     R, N = s32.shape
     if row_index is not None:
         s32 = np.where(np.arange(N)[None, :] > np.asarray(row_index)[:, None], np.float32(-np.inf), s32).astype(np.float32)
+    if kv_len is not None:
+        assert 1 <= int(kv_len) <= N
+        s32 = np.where(np.arange(N)[None, :] >= int(kv_len), np.float32(-np.inf), s32).astype(np.float32)
     y32 = (s32 * np.float32(c32)).astype(np.float32)
     mu = np.ceil(y32.max(axis=1).astype(np.float64))
     b32 = np.float32(np.float32(P8_SHIFT) - mu.astype(np.float32))
@@ -360,8 +364,9 @@ def fp8_pv_rows(s32: np.ndarray, c32: np.float32, V8hat: np.ndarray, row_index=N
 
 
 def fp8_pv_forward(qd: dict, kd: dict, v8: dict, softmax_scale=None, rows=None, heads=None, causal: bool = False,
-                   kv_group: int = 1):
-    """Whole-operator oracle of the FP8-P/V route: FP4 Q, K as in direct_p_forward, v8 from quantize_v_e4m3."""
+                   kv_group: int = 1, seq_len=None):
+    """Whole-operator oracle of the FP8-P/V route: FP4 Q, K as in direct_p_forward, v8 from quantize_v_e4m3;
+    seq_len as in direct_p_forward (rows beyond a length come back as NaN)."""
     from .quantize import dequantize_v_e4m3
     B, H, N, d = qd["nib"].shape
     heads = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
@@ -371,7 +376,11 @@ def fp8_pv_forward(qd: dict, kd: dict, v8: dict, softmax_scale=None, rows=None, 
         hk = h // kv_group
         c32 = score_constant(qd, kd, d, softmax_scale, (b, h, hk))
         s32 = scores_fp32(qd, kd, b, h, rows, hk)
-        O, lse, _, _ = fp8_pv_rows(s32, c32, np.ascontiguousarray(dequantize_v_e4m3(v8, b, hk).T), ridx if causal else None)
+        O, lse, _, _ = fp8_pv_rows(s32, c32, np.ascontiguousarray(dequantize_v_e4m3(v8, b, hk).T), ridx if causal else None,
+                                   kv_len=None if seq_len is None else int(seq_len[b]))
+        if seq_len is not None:
+            O[ridx >= int(seq_len[b])] = np.nan
+            lse[ridx >= int(seq_len[b])] = np.nan
         Os.append(O)
         Ls.append(lse)
     return np.stack(Os), np.stack(Ls)

@@ -694,7 +694,7 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   prm.thr16 = ops->p_scale_rule == FP4ATTN_PSCALE_THR16;
   if (ops->schedule != FP4ATTN_SCHEDULE_ONE_QUERY && ops->schedule != FP4ATTN_SCHEDULE_TWO_QUERY) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->pv_fmt != FP4ATTN_PV_MXFP4 && ops->pv_fmt != FP4ATTN_PV_E4M3) return FP4ATTN_ERR_INVALID_ARG;
-  if (ops->seq_len && (ops->pv_fmt != FP4ATTN_PV_MXFP4 || ops->schedule != FP4ATTN_SCHEDULE_ONE_QUERY)) return FP4ATTN_ERR_INVALID_ARG;
+  if (ops->seq_len && ops->schedule != FP4ATTN_SCHEDULE_ONE_QUERY) return FP4ATTN_ERR_INVALID_ARG;
   if (((uintptr_t)ops->seq_len & 3) != 0) return FP4ATTN_ERR_ALIGNMENT;
   if (ops->pv_fmt == FP4ATTN_PV_E4M3) return launch_attn_fp8pv(ops, B, H, N, d, prm, st);
   if (ops->schedule == FP4ATTN_SCHEDULE_TWO_QUERY) return launch_attn_two_query(ops, B, H, N, d, pmap, prm, st);

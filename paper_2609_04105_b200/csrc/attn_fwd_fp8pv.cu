@@ -394,13 +394,19 @@ attn_fwd_fp8pv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     bool ok = true;
     uint32_t g = 0;                                             // steps so far (both kinds, all pairs)
     uint32_t nbt = 0;                                           // B-visits of this team so far
-    const int v0 = row - 64 * h + 1;                            // visible keys of the team's tile on a causal diagonal stage
+    // keys of the team's tile that this row sees in an item's last stage, the masked one (causal: keys 0..i of row
+    // i = qt * 128 + row; padded sequence: keys 0..len-1; both: the fewer)
+    auto tile_keys = [&](const WorkItem& w) {
+      const int seen = p.causal ? min(w.len, w.qt * BM + row + 1) : w.len;
+      return seen - (w.T2 - 1) * BS - 64 * h;
+    };
     float b = 0.f;                                              // 8 - mu of the item in its second sweep
     for (int phs = 0; ok && phs <= n_my; ++phs) {
       WorkItem wa = {}, wb = {};
       int TA = 0, TB = 0;
       if (phs < n_my) { wa = decode_item<CAUSAL>(item_of(phs), p, qtiles); TA = wa.T2; }
       if (phs >= 1) { wb = decode_item<CAUSAL>(item_of(phs - 1), p, qtiles); TB = wb.T2; }
+      const int va = CAUSAL ? tile_keys(wa) : 64, vb = CAUSAL ? tile_keys(wb) : 64;
       float smax = -INFINITY;                                   // this team's share of the maxima of item phs
       const int TM = TA > TB ? TA : TB;
       for (int s2 = 0; ok && s2 < TM; ++s2) {
@@ -415,12 +421,12 @@ attn_fwd_fp8pv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           uint32_t sraw[32];
           if (kind == 0) {
             // ---- first sweep of item phs: maxima only
-            const bool diag = CAUSAL && s2 == wa.qt;
+            const bool diag = CAUSAL && s2 == TA - 1;
             tmem_ld_32x32b_x32(tS, sraw);
             tmem_wait_ld();
             if (diag) {
 #pragma unroll
-              for (int e = 0; e < 32; ++e) sraw[e] = (e < v0) ? sraw[e] : 0xFF800000u;
+              for (int e = 0; e < 32; ++e) sraw[e] = (e < va) ? sraw[e] : 0xFF800000u;
             }
             smax = fmaxf(smax, max32(sraw));
             tmem_ld_32x32b_x32(tS + 32, sraw);
@@ -430,23 +436,23 @@ attn_fwd_fp8pv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             if (lane == 0) mbar_arrive(sempty);
             if (diag) {
 #pragma unroll
-              for (int e = 0; e < 32; ++e) sraw[e] = (e < v0 - 32) ? sraw[e] : 0xFF800000u;
+              for (int e = 0; e < 32; ++e) sraw[e] = (e < va - 32) ? sraw[e] : 0xFF800000u;
             }
             smax = fmaxf(smax, max32(sraw));
           } else {
             // ---- second sweep of item phs - 1: bytes against its final reference
             uint32_t w[16];
-            const bool diag = CAUSAL && s2 == wb.qt;
+            const bool diag = CAUSAL && s2 == TB - 1;
             tmem_ld_32x32b_x32(tS, sraw);
             tmem_wait_ld();
-            if (diag) fp8_p_block<true>(sraw, c32, b, v0, w);
+            if (diag) fp8_p_block<true>(sraw, c32, b, vb, w);
             else      fp8_p_block<false>(sraw, c32, b, 32, w);
             tmem_ld_32x32b_x32(tS + 32, sraw);
             tmem_wait_ld();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(sempty);
-            if (diag) fp8_p_block<true>(sraw, c32, b, v0 - 32, w + 8);
+            if (diag) fp8_p_block<true>(sraw, c32, b, vb - 32, w + 8);
             else      fp8_p_block<false>(sraw, c32, b, 32, w + 8);
             // the pair's probability slot was last read by the PV product of this team's previous B-visit
             if (nbt > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (nbt - 1) & 1, abortf));
@@ -520,7 +526,7 @@ int launch_attn_fp8pv(const fp4attn_operands* ops, int B, int H, int N, int d, A
     return FP4ATTN_ERR_INVALID_ARG;                               // the code maps and block rules belong to the FP4 probability path
   Fp8Params pp{prm, ops->v_G};
   const bool nv = ops->qk_fmt == FP4ATTN_FMT_NVFP4;
-  const int sel = (d == 128 ? 4 : 0) | (nv ? 2 : 0) | (prm.causal ? 1 : 0);
+  const int sel = (d == 128 ? 4 : 0) | (nv ? 2 : 0) | ((prm.causal || prm.seq_len) ? 1 : 0);   // masked instances
   switch (sel) {
     case 0: return launch_fp8<64, 0, false>(ops, B, H, N, pp, st);
     case 1: return launch_fp8<64, 0, true>(ops, B, H, N, pp, st);

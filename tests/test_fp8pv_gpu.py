@@ -114,6 +114,44 @@ def test_fp8_pv_config2_full_size_sampled_rows_and_many_small_heads():
     _check(w, q, k, v, Og, Lg, heads)
 
 
+FP8_SEQLEN_CASES = [
+    ("cfg1", dict(B=3, H=2, N=512), [512, 300, 77], False, 1),
+    ("cfg1", dict(B=4, H=2, N=384), [1, 32, 128, 383], False, 1),
+    ("cfg1", dict(B=2, H=4, N=640), [129, 600], True, 2),
+    ("cfg3", dict(B=2, H=2, N=768), [700, 330], True, 1),
+    ("cfg2", dict(B=2, H=2, N=1024), [1000, 640], False, 1),
+]
+
+
+@pytest.mark.parametrize("name,kw,lens,causal,group", FP8_SEQLEN_CASES)
+def test_fp8_pv_padded_sequences_match_oracle_on_the_rows_that_exist(name, kw, lens, causal, group):
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    k, v = np.ascontiguousarray(k[:, : w.H // group]), np.ascontiguousarray(v[:, : w.H // group])
+    qg, kg = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+    vg = Bd.fp4attn_quantize_v_e4m3(_dev(v))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    O, L = Bd.fp4attn_fwd(qg, kg, vg, status=status, causal=causal, seq_len=torch.tensor(lens, dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    Og, Lg = O.float().cpu().numpy().astype(np.float64), L.cpu().numpy().astype(np.float64)
+    fmt = "mx" if w.qk_fmt == I.FMT_MXFP4 else "nv"
+    qd, kd, v8 = Qz.quantize_qk(q, fmt), Qz.quantize_qk(k, fmt), Qz.quantize_v_e4m3(v)
+    for b, n in enumerate(lens):
+        heads = [(b, h) for h in range(w.H)]
+        Oo, Lo = A.fp8_pv_forward(qd, kd, v8, heads=heads, rows=np.arange(n), causal=causal, kv_group=group, seq_len=lens)
+        for i, (_, h) in enumerate(heads):
+            g, l = Og[b, h][:n], Lg[b, h][:n]
+            assert np.linalg.norm(g - Oo[i]) / np.linalg.norm(Oo[i]) <= REL_FRO and np.abs(g - Oo[i]).max() <= MAX_ABS
+            assert (np.abs(l - Lo[i]) - 1e-5 * np.abs(Lo[i])).max() <= 1e-3
+            last = min(w.N, (n + 127) // 128 * 128)
+            assert np.isfinite(Og[b, h][:last]).all() and np.isfinite(Lg[b, h][:last]).all()
+    O1, L1 = Bd.fp4attn_fwd(qg, kg, vg, status=status, causal=causal)
+    O2, L2 = Bd.fp4attn_fwd(qg, kg, vg, status=status, causal=causal, seq_len=torch.full((w.B,), w.N, dtype=torch.int32, device="cuda"))
+    assert torch.equal(O1, O2) and torch.equal(L1, L2)           # full lengths: the bits of the call without seq_len
+
+
 def test_fp8_pv_rejects_the_fp4_only_options():
     from paper_2609_04105_b200 import binding as Bd
     w = I.shrink(I.WORKLOADS["cfg1"], N=128)

@@ -132,3 +132,23 @@ def test_fp8_pv_accuracy_sits_where_the_paper_reports_it():
     O2, _ = A.fp8_pv_forward(qd, {**kd, "nib": kd["nib"][:, 1:], "sf": kd["sf"][:, 1:]},
                              {**Qz.quantize_v_e4m3(v[:, 1:])}, heads=[(0, 1)], kv_group=2)
     assert np.abs(O2[0] - O8[0]).max() < 1e-13
+
+
+def test_fp8_rows_of_a_padded_sequence_equal_the_rows_on_the_truncated_keys():
+    """No block structure in this route: keys beyond the length are simply absent, for any length."""
+    rng = np.random.default_rng(9)
+    R, N, d = 5, 256, 8
+    y = (rng.standard_normal((R, N)) * 2).astype(np.float32)
+    V = rng.standard_normal((N, d))
+    for n in (1, 31, 32, 100, 129, 256):
+        O, lse, byte, mu = A.fp8_pv_rows(y, np.float32(1.0), V, kv_len=n)
+        Ot, lt, bt, mt = A.fp8_pv_rows(y[:, :n], np.float32(1.0), V[:n])
+        assert np.abs(O - Ot).max() < 1e-13 and np.abs(lse - lt).max() < 1e-13 and np.array_equal(mu, mt)
+        assert np.array_equal(byte[:, :n], bt) and not byte[:, n:].any()
+    w = I.shrink(I.WORKLOADS["cfg1"], B=2, H=1, N=256)
+    q, k, v = I.make_qkv(w)
+    qd, kd, v8 = Qz.quantize_qk(q, "mx"), Qz.quantize_qk(k, "mx"), Qz.quantize_v_e4m3(v)
+    O, L = A.fp8_pv_forward(qd, kd, v8, seq_len=[256, 90], causal=True)
+    O0, L0 = A.fp8_pv_forward(qd, kd, v8, causal=True)
+    assert np.array_equal(O[0], O0[0]) and np.isnan(O[1, 90:]).all()
+    assert np.array_equal(O[1, :90], O0[1, :90])                # causal rows below the length never saw the masked keys
