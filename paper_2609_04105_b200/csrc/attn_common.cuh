@@ -219,7 +219,7 @@ __device__ __forceinline__ void direct_p_block(uint32_t* sraw, float c32, float 
   constexpr bool THR16 = RULE == 1;
   constexpr uint32_t kExact = exact_pairs_of(PMAP);
   const float LOG2_6 = 2.5849625007211560f;
-  if (MASKED) {                                                 // causal diagonal: keys beyond the query get -inf
+  if (MASKED) {                                                 // keys the row does not see (causal mask, padding) get -inf
 #pragma unroll
     for (int i = 0; i < 32; ++i) sraw[i] = (i < visible) ? sraw[i] : 0xFF800000u;
   }

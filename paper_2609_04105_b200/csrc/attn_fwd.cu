@@ -1,4 +1,5 @@
-// Full-FP4 attention forward with Direct-P for sm_100a (noncausal or causal, optional grouped K/V heads).
+// Full-FP4 attention forward with Direct-P for sm_100a (noncausal or causal, optional grouped K/V heads, optional
+// per-batch token counts for padded sequences).
 //
 // Persistent kernel, one CTA per SM.  A CTA takes work items (one 128-row query tile of one
 // (batch, head)) round-robin and walks the keys of an item in stages of 128 (two 64-key tiles, four
@@ -31,6 +32,8 @@
 namespace fp4attn {
 using namespace ptx;
 
+// CAUSAL: the instances that mask the last stage of an item.  They serve the causal mask (p.causal), padded
+// sequences (p.seq_len) and both together; the other instances never look at either field.
 // NV: 0 - MXFP4 Q, K; 1 - NVFP4 with one encode factor per tensor; 2 - NVFP4 with one factor per (batch, head)
 // unit (an instance of its own: a score constant that changes per work item costs the tensor-wide variant
 // 2-8 % when it is only a run-time branch)
