@@ -6,7 +6,7 @@ this script is the same comparison (tests/parity.py: strict figures, and the pro
 correct value) over ALL units, for the record.  One launch of the configuration as bench.py launches it, then the
 oracle on a pool of host processes, one unit per task.
 
-  python tests/run_full_parity.py cfg4 [--p-map affine] [--p-scale mse] [--route fp8] [--workers 12] [--units 0:32]
+  python tests/run_full_parity.py cfg4 [--p-map affine] [--p-scale mse] [--route fp8] [--length-mix] [--workers 12] [--units 0:32]
 
 Prints one JSON line per unit and a summary line.  Needs a B200; imports the oracle (test infrastructure).
 """
@@ -51,10 +51,13 @@ def _unit(task):
         qd, kd = Qz.quantize_qk(one(q), "mx"), Qz.quantize_qk(one(k), "mx")
     t0 = time.perf_counter()
     try:
+        n = None if _G["lens"] is None else int(_G["lens"][b])     # padded sequence: the rows and keys that exist
         if _G["route"] == "fp8":
-            st = _fp8_head(Og[b, h].astype(np.float64), Lg[b, h].astype(np.float64), qd, kd, Qz.quantize_v_e4m3(one(v)))
+            st = _fp8_head(Og[b, h].astype(np.float64), Lg[b, h].astype(np.float64), qd, kd, Qz.quantize_v_e4m3(one(v)), n=n)
         else:
-            st = parity.compare_head(Og[b, h].astype(np.float64), Lg[b, h].astype(np.float64), qd, kd, Qz.quantize_v(one(v)), 0, 0, **okw)
+            extra = {} if n is None else dict(rows=np.arange(n), kv_len=n)
+            st = parity.compare_head(Og[b, h].astype(np.float64), Lg[b, h].astype(np.float64), qd, kd, Qz.quantize_v(one(v)), 0, 0,
+                                     **extra, **okw)
         st["ok"] = True
     except AssertionError as e:
         st = {"ok": False, "error": str(e)[:400]}
@@ -63,16 +66,17 @@ def _unit(task):
     return st
 
 
-def _fp8_head(Og, Lg, qd, kd, v8, chunk=1024):
-    """FP8 P/V route: strict comparison of one unit, all rows (no alternative evaluations are defined for it)."""
+def _fp8_head(Og, Lg, qd, kd, v8, chunk=1024, n=None):
+    """FP8 P/V route: strict comparison of one unit, all rows (no alternative evaluations are defined for it); with
+    n, the first n rows of a sequence of n tokens."""
     import parity
     from oracle import attention as A
-    N = Og.shape[0]
+    N = Og.shape[0] if n is None else n
     num = den = 0.0
     worst = lse_err = 0.0
     for r0 in range(0, N, chunk):
         rows = np.arange(r0, min(N, r0 + chunk))
-        Oo, Lo = A.fp8_pv_forward(qd, kd, v8, rows=rows, heads=[(0, 0)])
+        Oo, Lo = A.fp8_pv_forward(qd, kd, v8, rows=rows, heads=[(0, 0)], seq_len=None if n is None else [n])
         num += ((Og[rows] - Oo[0]) ** 2).sum()
         den += (Oo[0] ** 2).sum()
         worst = max(worst, float(np.abs(Og[rows] - Oo[0]).max()))
@@ -88,6 +92,8 @@ def main():
     ap.add_argument("workload", choices=sorted(I.WORKLOADS))
     ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine"])
     ap.add_argument("--p-scale", default="ceil", choices=["ceil", "thr16", "mse"], help="block-exponent rule of P (mse: ideal map only)")
+    ap.add_argument("--length-mix", action="store_true",
+                    help="padded sequences: N, 5N/8 - 120, N/2 + 1 and 300 tokens in the first four batch entries (B >= 4)")
     ap.add_argument("--route", default="fp4", choices=["fp4", "fp8"], help="probability / value format: Direct-P FP4 or FP8 P/V")
     ap.add_argument("--workers", type=int, default=max(1, len(os.sched_getaffinity(0)) - 2))
     ap.add_argument("--units", default=None, help="begin:end slice of the (batch, head) units, default all")
@@ -102,13 +108,17 @@ def main():
     kg = Bd.fp4attn_quantize(dev(k), w.qk_fmt, Bd.ROLE_K)
     vg = Bd.fp4attn_quantize_v_e4m3(dev(v)) if args.route == "fp8" else Bd.fp4attn_quantize(dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lens = None
+    if args.length_mix:
+        assert w.B >= 4, "the length mix needs four batch entries"
+        lens = [w.N, w.N * 5 // 8 - 120, w.N // 2 + 1, 300] + [w.N] * (w.B - 4)
     rule = {"ceil": Bd.PSCALE_CEIL, "thr16": Bd.PSCALE_THR16, "mse": Bd.PSCALE_MSE}[args.p_scale]
     assert args.route == "fp4" or args.p_scale == "ceil", "the FP8 P/V route has one rule"
     O, L = Bd.fp4attn_fwd(qg, kg, vg, status=status, p_map=Bd.PMAP_AFFINE if args.p_map == "affine" else Bd.PMAP_IDEAL,
-                          p_scale_rule=rule)
+                          p_scale_rule=rule, seq_len=None if lens is None else torch.tensor(lens, dtype=torch.int32, device="cuda"))
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    _G.update(route=args.route, w=w, q=q, k=k, v=v, O=O.float().cpu().numpy(), L=L.cpu().numpy(), Gq=None, Gk=None,
+    _G.update(lens=lens, route=args.route, w=w, q=q, k=k, v=v, O=O.float().cpu().numpy(), L=L.cpu().numpy(), Gq=None, Gk=None,
               okw=dict(p_map=args.p_map, p_scale=args.p_scale))
     if w.qk_fmt == I.FMT_NVFP4:
         _G["Gq"] = Qz.nv_tensor_scale(Qz.bf16_bits_to_f64(q))
@@ -126,7 +136,7 @@ def main():
             print(json.dumps(st), flush=True)
             res.append(st)
     good = [r for r in res if r["ok"]]
-    summary = {"workload": w.name, "route": args.route, "p_map": args.p_map, "p_scale": args.p_scale, "units": len(res), "units_ok": len(good),
+    summary = {"workload": w.name, "route": args.route, "p_map": args.p_map, "p_scale": args.p_scale, "length_mix": lens, "units": len(res), "units_ok": len(good),
                "rows": int(sum(r["rows"] for r in good)), "wall_s": round(time.perf_counter() - t0, 1)}
     if good:
         summary.update(rel_fro_strict_max=max(r["rel_fro_strict"] for r in good), max_abs_strict=max(r["max_abs_strict"] for r in good),
