@@ -505,6 +505,28 @@ def run_cuda(args, w):
     probe_tflops = sms * iters * 2.0 * 128 * 128 * 64 / (p0.elapsed_time(p1) * 1e-3) / 1e12
     probe_flop_per_clk_sm = iters * 2.0 * 128 * 128 * 64 / max(1, int(cyc.item()))
 
+    # ---- the library's dense block-scaled FP4 GEMM (cuBLASLt through torch._scaled_mm, NVFP4 operands, 8192^3) as a
+    # cross-check of the roofline denominator; context only, None where this torch build does not offer it
+    lib_fp4_tflops = None
+    try:
+        Mg = 8192
+        ga = torch.randint(0, 256, (Mg, Mg // 2), dtype=torch.uint8, device=dev).view(torch.float4_e2m1fn_x2)
+        gb = torch.randint(0, 256, (Mg, Mg // 2), dtype=torch.uint8, device=dev).view(torch.float4_e2m1fn_x2)
+        gs = torch.full((Mg * (Mg // 16),), 1.0, device=dev).to(torch.float8_e4m3fn)      # one scale per 16 elements
+        gemm = lambda: torch._scaled_mm(ga, gb.t(), scale_a=gs, scale_b=gs, out_dtype=torch.bfloat16)
+        for _ in range(3):
+            gemm()
+        g0, g1 = E(), E()
+        g0.record()
+        for _ in range(10):
+            gemm()
+        g1.record()
+        torch.cuda.synchronize()
+        lib_fp4_tflops = 10 * 2.0 * Mg ** 3 / (g0.elapsed_time(g1) * 1e-3) / 1e12
+        del ga, gb, gs
+    except Exception:
+        lib_fp4_tflops = None
+
     # ---- measured ceiling of the softmax arithmetic alone (second roofline of the attention kernel)
     cyc2 = torch.zeros(2, dtype=torch.int64, device=dev)
     arith_iters = 8192
@@ -586,7 +608,7 @@ def run_cuda(args, w):
         return
 
     roof = roofline_record(w, attn_launch_ms, fp4_peak, peaks, "attn_fwd_2q_kernel" if args.schedule == "two-query" else "attn_fwd_kernel")
-    roof.update({"fp4_issue_probe_tflops": probe_tflops, "fp4_issue_probe_flop_per_clk_per_sm": probe_flop_per_clk_sm,
+    roof.update({"fp4_gemm_library_tflops": lib_fp4_tflops, "fp4_issue_probe_tflops": probe_tflops, "fp4_issue_probe_flop_per_clk_per_sm": probe_flop_per_clk_sm,
                  "launch_ms_mean": attn_launch_ms, "launch_ms_median": statistics.median(attn_ms)})
     # Softmax-arithmetic roofline: an SM converts four 32x32 blocks (one per scheduler) in `arith_clk_per_block`
     # clocks when it does nothing else; a block carries 4*32*32*d flop of the two products.  Clock: the median SM
