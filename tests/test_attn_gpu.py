@@ -651,6 +651,37 @@ def test_many_small_heads_more_items_than_one_wave():
     check_heads(Og, Lg, Oo, Lo, heads)
 
 
+# ------------------------------------------------------------------ metamorphic checks (no oracle involved)
+@pytest.mark.parametrize("name,kw", [("cfg2", dict(B=2, H=3, N=1024)), ("cfg3", dict(B=2, H=2, N=768))])
+def test_exact_rescaling_of_q_and_head_permutation_leave_the_bits_unchanged(name, kw):
+    """Q times 2^k with the softmax scale times 2^-k is the same operator: MXFP4 moves the power into the scale bytes,
+    NVFP4 into the encode factor, the float32 scores and the score constant scale exactly, so O and LSE must come out
+    bit for bit.  And the (batch, head) units are independent: permuting the heads permutes the output."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    scale = 1.0 / np.sqrt(w.d)
+
+    def run(q, k, v, s):
+        qg, kg = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+        vg = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        O, L = Bd.fp4attn_fwd(qg, kg, vg, softmax_scale=s, status=st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        return O, L
+
+    O0, L0 = run(q, k, v, scale)
+    for kpow in (-3, 5):
+        q2 = I.f32_to_bf16_bits(I.bf16_bits_to_f32(q) * np.float32(2.0 ** kpow))       # exact in bf16
+        O1, L1 = run(q2, k, v, scale * 2.0 ** -kpow)
+        assert torch.equal(O0, O1) and torch.equal(L0, L1)
+    perm = np.random.default_rng(3).permutation(w.H)
+    O2, L2 = run(np.ascontiguousarray(q[:, perm]), np.ascontiguousarray(k[:, perm]), np.ascontiguousarray(v[:, perm]), scale)
+    idx = torch.from_numpy(perm).cuda()
+    assert torch.equal(O0[:, idx], O2) and torch.equal(L0[:, idx], L2)      # (a tensor-wide NVFP4 factor does not move)
+
+
 # ------------------------------------------------------------------ seeded random configurations
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_random_configurations_match_oracle(seed):
