@@ -505,6 +505,22 @@ def run_cuda(args, w):
     probe_tflops = sms * iters * 2.0 * 128 * 128 * 64 / (p0.elapsed_time(p1) * 1e-3) / 1e12
     probe_flop_per_clk_sm = iters * 2.0 * 128 * 128 * 64 / max(1, int(cyc.item()))
 
+    # ---- the vendor library's BF16 attention forward on the same unquantized tensors (torch SDPA, cuDNN backend):
+    # context for the paper's "x times BF16 attention" figures, not a target and not part of any path of this library
+    bf16_lib = None
+    if world == 1:
+        try:
+            import torch.nn.functional as Fnn
+            from torch.nn.attention import SDPBackend, sdpa_kernel
+            with sdpa_kernel(SDPBackend.CUDNN_ATTENTION):
+                sd = lambda: Fnn.scaled_dot_product_attention(dq, dk, dv)
+                for _ in range(3):
+                    sd()
+                ms_sd = statistics.median(timed_launches(sd, 10, flush, E, torch.cuda.synchronize))
+            bf16_lib = {"attn_ms": ms_sd, "attn_tflops": w.flops / (ms_sd * 1e-3) / 1e12, "what": "torch SDPA, cuDNN backend, bf16, noncausal"}
+        except Exception:
+            bf16_lib = None
+
     # ---- the library's dense block-scaled FP4 GEMM (cuBLASLt through torch._scaled_mm, NVFP4 operands, 8192^3) as a
     # cross-check of the roofline denominator; context only, None where this torch build does not offer it
     lib_fp4_tflops = None
@@ -636,7 +652,7 @@ def run_cuda(args, w):
                    "flops": "4*B*H*N^2*d", "parallelism": f"replica x{world}, (batch, head) units, no collective"},
         "attn_only": {"value": attn_tflops, "unit": UNIT, "ms": attn_launch_ms,
                       "note": "attention kernel alone (the paper's timing boundary excludes quantization)",
-                      "other_code_maps": other_maps},
+                      "other_code_maps": other_maps, "bf16_attention_library": bf16_lib},
         "roofline": roof,
         "roofline_softmax_arith": roof_softmax,
         "window": window,
