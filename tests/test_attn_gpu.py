@@ -651,6 +651,34 @@ def test_many_small_heads_more_items_than_one_wave():
     check_heads(Og, Lg, Oo, Lo, heads)
 
 
+# ------------------------------------------------------------------ degenerate inputs
+@pytest.mark.parametrize("causal", [False, True])
+def test_degenerate_inputs_zero_queries_zero_values_identical_keys(causal):
+    """Q = 0: every score is 0, every visible key gets the same code, O is the mean of the reconstructed V over the
+    visible keys and LSE the log of their number.  V = 0: O is exactly 0.  Identical keys: the same.  Each against the
+    closed form and against the oracle."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg1"], B=1, H=2, N=384)
+    q, k, v = I.make_qkv(w)
+    zero = np.zeros_like(q)
+    vd = Qz.quantize_v(v)
+    Vhat = np.swapaxes(Qz.dequantize(vd), -1, -2)                                  # [B, H, N, d]
+    n_vis = (np.arange(w.N) + 1.0) if causal else np.full(w.N, float(w.N))
+    mean_v = (np.cumsum(Vhat, axis=2) / n_vis[None, None, :, None]) if causal else np.broadcast_to(Vhat.mean(axis=2, keepdims=True), Vhat.shape)
+    kk = np.ascontiguousarray(np.broadcast_to(k[:, :, :1], k.shape))               # every key equals key 0
+    for qq, kx in ((zero, k), (q, kk)):
+        Og, Lg = run_gpu_general(w, qq, kx, v, causal=causal)
+        assert np.abs(Og - mean_v).max() <= 2.0 ** -8 * max(1.0, np.abs(mean_v).max()) + 1e-6        # bf16 rounding of O
+        if qq is zero:
+            assert np.abs(Lg - np.log(n_vis)[None, None]).max() <= 1e-3
+        qd, kd = Qz.quantize_qk(qq, "mx"), Qz.quantize_qk(kx, "mx")
+        heads = [(0, 0), (0, 1)]
+        Oo, Lo = A.direct_p_forward(qd, kd, vd, heads=heads, causal=causal)
+        check_heads(Og, Lg, Oo, Lo, heads)
+    Og, Lg = run_gpu_general(w, q, k, zero, causal=causal)
+    assert not Og.any() and np.isfinite(Lg).all()
+
+
 # ------------------------------------------------------------------ metamorphic checks (no oracle involved)
 @pytest.mark.parametrize("name,kw", [("cfg2", dict(B=2, H=3, N=1024)), ("cfg3", dict(B=2, H=2, N=768))])
 def test_exact_rescaling_of_q_and_head_permutation_leave_the_bits_unchanged(name, kw):
