@@ -249,6 +249,10 @@ typedef struct {
  * block-scaled FP4 product; the output is normalised by the sum of the same rounded values:
  *   O = sum_j p~_j V^_j / sum_j p~_j,   p~_j = 2^(E_B) q_j / 6,   LSE = ln sum_j p~_j.
  *
+ * Range of the logits: |y| < 2^21 is assumed (the block exponent is formed by a float32 rounding trick that is exact
+ * there, and block maxima are clamped to that range); inputs whose scaled scores exceed two million octaves lie
+ * outside any softmax's useful range and give finite but unspecified results.
+ *
  * With causal = 1 (the forward the paper's training section starts from, Section "Causal backward")
  * keys j > i are removed from row i before anything else: they never raise a block maximum, always
  * code to 0, and a block without a visible key contributes nothing.  B, H, N, d describe Q and O;
