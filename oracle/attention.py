@@ -143,7 +143,8 @@ def _boundary_neighbours(v: np.ndarray):
 
 def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int = 128, tile_order=None,
                   p_map: str = "ideal", affine=(1.5, 1.2), p_scale: str = "ceil", row_index=None,
-                  exact_pairs: int = 0xFFFF, report=None, flips=None, ambiguity=None, kv_len=None):
+                  exact_pairs: int = 0xFFFF, report=None, flips=None, ambiguity=None, kv_len=None,
+                  fixed_reference=None):
     """Direct-P online softmax + PV for a set of query rows of one (batch, head).
 
     s32  [R, N] float32 tensor-core-facing scores;  Vhat [N, d] float64 reconstructed V.
@@ -156,6 +157,12 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
     kv_len : optional number of keys that exist (sequences shorter than the padded N): keys kv_len..N-1 are masked
              like the keys a causal row does not see (score -inf: they enter no block maximum, get code 0 and no
              weight), so the result is that of the operator on the first kv_len keys.
+    fixed_reference : optional integer: the row reference is this constant for every row and never moves (the
+             shiftless path of Section "Fix 3: guard only extreme model logits"; the `fast` policy of Table
+             "policy-definition" has no anchor, i.e. reference 0).  A block's E8M0 byte is then E_B - reference +
+             127: a block whose byte would fall below 1 is a zero block, a byte above 254 or a row left without any
+             live block is outside the policy's range and raises ValueError.  Inside the range the result is that of
+             the running reference (codes do not depend on the reference, rescales are exact powers of two).
     flips  : optional dict with the same two keys: decisions to take the OTHER way.  A flipped code moves to
              the code across its nearest boundary; a flipped block exponent to the integer on the other side
              of the block maximum, and the block's codes follow from the new exponent.
@@ -169,7 +176,7 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
         s32 = np.where(np.arange(N)[None, :] >= int(kv_len), np.float32(-np.inf), s32).astype(np.float32)
     y32 = (s32 * np.float32(c32)).astype(np.float32)             # decision variable, fp32
     yx = s32.astype(np.float64) * np.float64(c32)                # converter input, fp64
-    mu = np.full(R, -np.inf)
+    mu = np.full(R, -np.inf) if fixed_reference is None else np.full(R, float(int(fixed_reference)))
     L = np.zeros(R)
     O = np.zeros((R, Vhat.shape[1]))
     codes_all = np.zeros((R, N), dtype=np.uint8)
@@ -230,7 +237,7 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
         j0 = t * tile
         exps = [exponent_of(bj) for bj in range(j0, j0 + tile, P_BLOCK)]
         m_tile = np.max(np.stack([e for e, _ in exps]), axis=0)
-        mu_new = np.maximum(mu, m_tile)
+        mu_new = np.maximum(mu, m_tile) if fixed_reference is None else mu
         f = np.where(np.isinf(mu), 0.0, np.exp2(mu - mu_new))     # exact power of two
         L *= f
         O *= f[:, None]
@@ -240,6 +247,8 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
             E_B = np.where(seen, E_B, 0.0)
             e_B = np.where(seen, E_B - mu, -np.inf)
             live = (e_B + 127) >= 1
+            if fixed_reference is not None and np.any(seen & (e_B + 127 > 254)):
+                raise ValueError("a block exponent lies more than 127 octaves above the fixed reference")
             b_B32 = np.float32(LOG2_6_32 - E_B.astype(np.float32))
             sl = slice(bj, bj + P_BLOCK)
             if p_map in ("ideal", "hybrid"):
@@ -276,6 +285,8 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
             O += (alpha / 6.0)[:, None] * (q @ Vhat[sl])
             codes_all[:, sl] = code
             EB_all[:, bj // P_BLOCK] = np.where(seen, E_B, -(1 << 40)).astype(np.int64)
+    if fixed_reference is not None and np.any(L <= 0):
+        raise ValueError("a row has no block within 126 octaves below the fixed reference")
     Oout = O / L[:, None]
     lse = math.log(2.0) * (mu + np.log2(L))
     if report is not None:
@@ -295,8 +306,9 @@ def direct_p_rows(s32: np.ndarray, c32: np.float32, Vhat: np.ndarray, tile: int 
 def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int = 128,
                      rows=None, heads=None, tile_order=None, p_map: str = "ideal", affine=(1.5, 1.2),
                      p_scale: str = "ceil", causal: bool = False, kv_group: int = 1, exact_pairs: int = 0xFFFF,
-                     seq_len=None):
+                     seq_len=None, fixed_reference=None):
     """Whole-operator oracle.  qd/kd/vd come from oracle.quantize.quantize_qk / quantize_v.
+    fixed_reference: see direct_p_rows (the shiftless path: a constant row reference).
 
     seq_len : optional [B] integers, 1 <= seq_len[b] <= N: batch entry b is a sequence of seq_len[b] tokens padded
               to N.  Its keys beyond the length are masked; its query rows beyond the length carry no meaning and
@@ -318,7 +330,7 @@ def direct_p_forward(qd: dict, kd: dict, vd: dict, softmax_scale=None, tile: int
         Vhat = dequantize({**vd, "nib": vd["nib"][b, hk][None, None], "sf": vd["sf"][b, hk][None, None]})[0, 0].T
         O, lse, _, _, _ = direct_p_rows(s32, c32, np.ascontiguousarray(Vhat), tile, tile_order, p_map, affine, p_scale,
                                         ridx if causal else None, exact_pairs,
-                                        kv_len=None if seq_len is None else int(seq_len[b]))
+                                        kv_len=None if seq_len is None else int(seq_len[b]), fixed_reference=fixed_reference)
         if seq_len is not None:
             O[ridx >= int(seq_len[b])] = np.nan
             lse[ridx >= int(seq_len[b])] = np.nan

@@ -664,3 +664,31 @@ def test_sequence_length_inside_a_block_against_the_plain_definition():
         assert cd == [int(c) for c in codes[i, :n]]
         Oi, Li = _plain_definition(y32[i, :n], E_B, cd, Vhat[:n])
         assert np.abs(O[i] - Oi).max() < 1e-13 and abs(L[i] - Li) < 1e-12
+
+
+# ------------------------------------------------------------------ fixed row reference (the shiftless path)
+def test_fixed_reference_equals_the_running_reference_inside_its_range_and_refuses_what_lies_outside():
+    """Codes do not depend on the row reference and every rescale is an exact power of two, so any constant reference
+    that keeps all E8M0 bytes within 1..254 must reproduce the running-reference result; a block more than 126
+    octaves below the reference is dropped like any zero block; a block above the byte range, or a row left with
+    nothing, is outside the policy and must be refused, not answered."""
+    w, _, qd, kd, vd = _cfg1(N=256, H=2)
+    O, L = A.direct_p_forward(qd, kd, vd)
+    for ref in (0, 17, -40):
+        O2, L2 = A.direct_p_forward(qd, kd, vd, fixed_reference=ref)
+        assert np.abs(O2 - O).max() < 1e-13 and np.abs(L2 - L).max() < 1e-12
+    O3, L3 = A.direct_p_forward(qd, kd, vd, fixed_reference=0, causal=True, seq_len=[200])
+    O4, L4 = A.direct_p_forward(qd, kd, vd, causal=True, seq_len=[200])
+    assert np.abs(O3[:, :200] - O4[:, :200]).max() < 1e-13
+    rng = np.random.default_rng(2)
+    V = rng.standard_normal((64, 4))
+    y = np.zeros((1, 64), dtype=np.float32)
+    y[0, 32:] = -140.0                                           # second block: byte 0 - 140 + 127 < 1 -> zero block
+    O5, L5, codes, _, _ = A.direct_p_rows(y, np.float32(1.0), V, tile=32, fixed_reference=0)
+    assert np.abs(O5[0] - V[:32].mean(axis=0)).max() < 1e-14 and abs(L5[0] - math.log(32.0)) < 1e-12
+    assert not codes[0, 32:].any()
+    y[0, :32] = 130.0                                            # byte 130 + 127 > 254
+    with pytest.raises(ValueError):
+        A.direct_p_rows(y, np.float32(1.0), V, tile=32, fixed_reference=0)
+    with pytest.raises(ValueError):                              # every block of the row below the range
+        A.direct_p_rows(np.full((1, 64), -200.0, dtype=np.float32), np.float32(1.0), V, tile=32, fixed_reference=0)
