@@ -466,10 +466,13 @@ def run_cuda(args, w):
         qd0, kd0, vd0 = state["ops"]
         O_alt = torch.empty_like(O)                                 # O keeps the timed map's result for the parity sample
         for name, kw in (("ideal", dict(p_map=Bd.PMAP_IDEAL)), ("hybrid8", dict(p_map=Bd.PMAP_HYBRID, exact_pairs=0x5555)),
-                         ("affine", dict(p_map=Bd.PMAP_AFFINE))):
-            if name == args.p_map:
+                         ("affine", dict(p_map=Bd.PMAP_AFFINE)),
+                         ("affine_shiftless", dict(p_map=Bd.PMAP_AFFINE, fixed_reference=0))):
+            if name == args.p_map or ("fixed_reference" in kw and w.outliers):     # (outlier logits span more than a fixed reference holds)
                 continue
             rule = pscale if (pscale != Bd.PSCALE_MSE or name == "ideal") else Bd.PSCALE_CEIL     # the MSE rule exists for the ideal map
+            if "fixed_reference" in kw:
+                rule = Bd.PSCALE_CEIL                                # the fixed reference comes with the ceiling rule
             fn = lambda: Bd.fp4attn_fwd(qd0, kd0, vd0, out=O_alt, status=status, p_scale_rule=rule, **kw)
             for _ in range(3):
                 fn()
@@ -589,6 +592,8 @@ def run_cuda(args, w):
             so = torch.empty((ww.B, ww.H, ww.N, ww.d), dtype=torch.bfloat16, device=dev)
             rec = {"workload": _workload_text(ww), "launches": n_it, "inputs": "seeded recipe of the configuration"}
             variants = [("", {}, 1.0), ("affine_", dict(p_map=Bd.PMAP_AFFINE), 1.0), ("causal_", dict(causal=True), 0.5)]
+            if not ww.outliers:                                      # config 4's logits span more than a fixed reference holds
+                variants.append(("affine_shiftless_", dict(p_map=Bd.PMAP_AFFINE, fixed_reference=0), 1.0))
             if ww.d == 64 and ww.N % 256 == 0:                       # the two-query schedule beside the one-query one
                 variants += [("two_query_", dict(schedule=Bd.SCHEDULE_TWO_QUERY), 1.0),
                              ("two_query_affine_", dict(schedule=Bd.SCHEDULE_TWO_QUERY, p_map=Bd.PMAP_AFFINE), 1.0)]

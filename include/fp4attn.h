@@ -46,11 +46,16 @@ enum {
   FP4ATTN_ERR_ALIGNMENT = 4,          /* a pointer violates the stated alignment               */
   FP4ATTN_ERR_WORKSPACE = 5,          /* workspace missing or too small                        */
   FP4ATTN_ERR_CUDA = 6,               /* a CUDA runtime / driver call failed                   */
-  FP4ATTN_ERR_TIMEOUT = 7             /* written to *device_status by a kernel whose bounded
+  FP4ATTN_ERR_TIMEOUT = 7,            /* written to *device_status by a kernel whose bounded
                                          wait ran out; never returned synchronously            */
+  FP4ATTN_ERR_RANGE = 8               /* written to *device_status by a kernel running with a
+                                         fixed row reference when a block exponent or a whole row
+                                         fell outside the E8M0 range around it; never returned
+                                         synchronously                                          */
 };
 
 enum { FP4ATTN_FMT_MXFP4 = 0, FP4ATTN_FMT_NVFP4 = 1 };
+enum { FP4ATTN_REFERENCE_RUNNING = 0, FP4ATTN_REFERENCE_FIXED = 1 };
 enum { FP4ATTN_ROLE_Q = 0, FP4ATTN_ROLE_K = 1, FP4ATTN_ROLE_V = 2 };
 /* how a normalised score x = y - E_B + log2 6 becomes an E2M1 probability code */
 enum { FP4ATTN_PMAP_IDEAL = 0,    /* q = Q_E2M1(2^x)              (Eq. "ideal-code-path"); how 2^x is evaluated
@@ -226,6 +231,11 @@ typedef struct {
                                        [B, kv_heads, d, N] from fp4attn_quantize_v_e4m3, v_sf is ignored, v_G is required;
                                        with the ideal map, the ceiling rule and the one-query schedule only          */
   const float* v_G;                 /* FP4ATTN_PV_E4M3: device fp32 encode factors of V, one per (batch, K/V head)    */
+  int row_reference;                /* FP4ATTN_REFERENCE_RUNNING (0, default) or FP4ATTN_REFERENCE_FIXED: the row
+                                       reference is the constant fixed_reference for every row (see fp4attn_fwd); with
+                                       the ideal and the affine map, the ceiling rule, one factor per tensor, the
+                                       one-query schedule and FP4ATTN_PV_MXFP4 only                                   */
+  int fixed_reference;              /* FP4ATTN_REFERENCE_FIXED: the reference in octaves (log2 units), -1000 .. 1000    */
   const int* seq_len;               /* NULL, or B device integers: batch entry b is a sequence of seq_len[b] tokens
                                        padded to N (see fp4attn_fwd); values are clamped into 1..N.  With the ideal and
                                        the affine map (and with FP4ATTN_PV_E4M3), one-query schedule only            */
@@ -248,6 +258,17 @@ typedef struct {
  * construction (blocks whose byte would drop below 1 are zero blocks).  P V runs as a second
  * block-scaled FP4 product; the output is normalised by the sum of the same rounded values:
  *   O = sum_j p~_j V^_j / sum_j p~_j,   p~_j = 2^(E_B) q_j / 6,   LSE = ln sum_j p~_j.
+ *
+ * Row reference.  By default (FP4ATTN_REFERENCE_RUNNING) mu follows the running maximum as described, which places no
+ * limit on the spread of the logits.  FP4ATTN_REFERENCE_FIXED is the shiftless path of the paper's `fast` policy
+ * (Section "Fix 3: guard only extreme model logits"; Table "policy-definition": no anchor): mu is the constant
+ * fixed_reference for every row, the softmax warps publish the byte E_B - mu + 127 themselves and nothing is ever
+ * rescaled, which takes the row-reference pass out of the chain between the score and the second product.  Codes do
+ * not depend on mu, so inside the range the result is that of the running reference (O to the last bit, LSE to float32
+ * rounding).  The range: a block whose byte would fall below 1 is a zero block (correct when it lies more than 126
+ * octaves below its row's maximum, wrong otherwise); a byte above 254, or a row whose represented sum comes out as 0,
+ * cannot be represented - the kernel then writes FP4ATTN_ERR_RANGE to *device_status and the affected rows are
+ * unspecified.  With fixed_reference = 0 every row whose largest logit y lies between about -120 and +127 is inside.
  *
  * Range of the logits: |y| < 2^21 is assumed (the block exponent is formed by a float32 rounding trick that is exact
  * there, and block maxima are clamped to that range); inputs whose scaled scores exceed two million octaves lie
@@ -277,8 +298,8 @@ typedef struct {
  * out.  FP4ATTN_PMAP_AFFINE has no such band: its arithmetic is exact float32 as written above.
  *
  * O_bf16 [B,H,N,d]; LSE [B,H,N] (may be NULL); device_status (may be NULL) receives
- * FP4ATTN_ERR_TIMEOUT if a bounded in-kernel wait ran out, and is otherwise left untouched, so
- * the caller clears it beforehand.
+ * FP4ATTN_ERR_TIMEOUT if a bounded in-kernel wait ran out (or FP4ATTN_ERR_RANGE, see above), and is otherwise left
+ * untouched, so the caller clears it beforehand.
  */
 int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int d,
                 void* O_bf16, float* LSE, int* device_status, fp4attn_stream_t stream);

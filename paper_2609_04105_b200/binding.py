@@ -20,7 +20,7 @@ SCHEDULE_ONE_QUERY, SCHEDULE_TWO_QUERY = 0, 1
 PV_MXFP4, PV_E4M3 = 0, 1
 QSCALE_CEIL, QSCALE_THR16, QSCALE_FLOOR, QSCALE_MSE = 0, 1, 2, 3
 (OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_ARCH, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA,
- ERR_TIMEOUT) = range(8)
+ ERR_TIMEOUT, ERR_RANGE) = range(9)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libfp4attn.so")
@@ -47,7 +47,8 @@ class _Operands(ctypes.Structure):
                 ("p_map", ctypes.c_int), ("affine_a", ctypes.c_float), ("affine_b", ctypes.c_float),
                 ("p_scale_rule", ctypes.c_int), ("causal", ctypes.c_int), ("kv_heads", ctypes.c_int),
                 ("exact_pairs", ctypes.c_int), ("g_per_head", ctypes.c_int), ("schedule", ctypes.c_int),
-                ("pv_fmt", ctypes.c_int), ("v_G", ctypes.c_void_p), ("seq_len", ctypes.c_void_p)]
+                ("pv_fmt", ctypes.c_int), ("v_G", ctypes.c_void_p), ("row_reference", ctypes.c_int),
+                ("fixed_reference", ctypes.c_int), ("seq_len", ctypes.c_void_p)]
 
 
 def _load() -> ctypes.CDLL:
@@ -228,10 +229,11 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
                 status: Optional[torch.Tensor] = None, p_map: int = PMAP_IDEAL, affine_a: float = 0.0,
                 affine_b: float = 0.0, p_scale_rule: int = PSCALE_CEIL, causal: bool = False,
                 exact_pairs: int = 0, schedule: int = SCHEDULE_ONE_QUERY,
-                seq_len: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+                seq_len: Optional[torch.Tensor] = None, fixed_reference: Optional[int] = None) -> Tuple[torch.Tensor, torch.Tensor]:
     """Direct-P attention forward on quantized operands -> (O bf16 [B,H,N,d], LSE fp32 [B,H,N]).
     p_map selects the exact code map or the affine classifier (affine_a = 0: A = 1.5, B = 1.2).
-    seq_len: optional CUDA int32 tensor [B], the token count of every batch entry (padded to N)."""
+    seq_len: optional CUDA int32 tensor [B], the token count of every batch entry (padded to N).
+    fixed_reference: None - running row reference; an integer - that constant row reference (the shiftless path)."""
     B, H, N, d = q.shape
     Hkv = k.shape[1]                                   # grouped-query attention when Hkv < H
     assert k.shape == v.shape and k.shape == (B, Hkv, N, d) and H % Hkv == 0 and q.fmt == k.fmt and v.fmt in (FMT_MXFP4, FMT_E4M3)
@@ -247,7 +249,7 @@ def fp4attn_fwd(q: QuantizedOperand, k: QuantizedOperand, v: QuantizedOperand, s
                     q.scales.data_ptr(), k.scales.data_ptr(), None if fp8 else v.scales.data_ptr(),
                     _ptr(q.G), _ptr(k.G), q.fmt, float(softmax_scale), int(p_map), float(affine_a), float(affine_b), int(p_scale_rule), int(bool(causal)), int(Hkv),
                     int(exact_pairs), int(q.per_head), int(schedule), PV_E4M3 if fp8 else PV_MXFP4, _ptr(v.G) if fp8 else None,
-                    _ptr(seq_len))
+                    0 if fixed_reference is None else 1, 0 if fixed_reference is None else int(fixed_reference), _ptr(seq_len))
     _check(lib().fp4attn_fwd(ctypes.byref(ops), B, H, N, d, out.data_ptr(), lse.data_ptr(), _ptr(status), _stream()),
            "fp4attn_fwd")
     return out, lse

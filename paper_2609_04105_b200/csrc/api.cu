@@ -30,6 +30,7 @@ extern "C" const char* fp4attn_status_string(int status) {
     case FP4ATTN_ERR_WORKSPACE: return "workspace missing or too small";
     case FP4ATTN_ERR_CUDA: return "CUDA call failed";
     case FP4ATTN_ERR_TIMEOUT: return "bounded in-kernel wait ran out";
+    case FP4ATTN_ERR_RANGE: return "logits outside the range of the fixed row reference";
     default: return "unknown status";
   }
 }

@@ -76,6 +76,7 @@ struct AttnParams {
   int H, Hkv;              // query heads, K/V heads (H % Hkv == 0: grouped-query attention)
   int BH;                  // B * H
   unsigned long long recip_qtiles, recip_bh;   // ceil(2^64 / (N / 128)), ceil(2^64 / BH); 0 for a divisor of 1
+  int ref_fixed;           // the constant row reference of the FIXREF instances (octaves)
   const int* seq_len;      // NULL, or B token counts: batch entry b is seq_len[b] tokens padded to N (masked kernels only)
   unsigned long long recip_h;                  // ceil(2^64 / H); 0 for H = 1
 };

@@ -37,7 +37,10 @@ using namespace ptx;
 // NV: 0 - MXFP4 Q, K; 1 - NVFP4 with one encode factor per tensor; 2 - NVFP4 with one factor per (batch, head)
 // unit (an instance of its own: a score constant that changes per work item costs the tensor-wide variant
 // 2-8 % when it is only a run-time branch)
-template <int D, int NV, int PMAP, bool CAUSAL, int THR16>
+// FIXREF: the row reference is the constant p.ref_fixed (the shiftless path): the teams publish the E8M0 bytes of
+// their blocks themselves, the PV issuer waits for the teams, nothing is ever rescaled, and the correction warps are
+// left with the epilogue.
+template <int D, int NV, int PMAP, bool CAUSAL, int THR16, bool FIXREF = false>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -211,7 +214,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       for (int s2 = 0; ok && s2 < T2; ++s2, ++g) {
         const int pr = g & 1;
         const uint32_t m = g >> 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_PFULL0 + pr), m & 1, abortf));   // codes and scale bytes of both tiles are in smem
+        // codes of both tiles are in tensor memory, their scale bytes in shared memory (written by the correction
+        // warps, or with a fixed reference by the teams themselves)
+        ok = __all_sync(0xffffffffu, mbar_wait(bar((FIXREF ? BAR_SMDONE0 : BAR_PFULL0) + pr), m & 1, abortf));
         if (!ok) break;
         tc_fence_after();
         const uint32_t tSFP = tmem + kColSFP + 4 * pr, tSFV = tmem + kColSFV + 8 * pr;
@@ -259,11 +264,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const WorkItem wi = decode_item<CAUSAL>(item, p, qtiles);
       T2 = wi.T2;
       const bool has_next = item + (int)gridDim.x < p.n_items;
-      int mu = first_served ? mu_next : -(1 << 28);
+      int mu = FIXREF ? p.ref_fixed : (first_served ? mu_next : -(1 << 28));
       int runmax = first_served ? mu_next - kRefHeadroom : -(1 << 28);   // largest block exponent of the row so far
       // One pass per 128-key stage (both of its tiles).  The item's first stage may already have been served
       // from inside the previous item's epilogue.
-      for (uint32_t g = g0 + (first_served ? 1u : 0u); g < g0 + (uint32_t)T2; ++g) {
+      for (uint32_t g = FIXREF ? g0 + (uint32_t)T2 : g0 + (first_served ? 1u : 0u); g < g0 + (uint32_t)T2; ++g) {
         const bool first_of_item = g == g0;
         const int pr = g & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SMDONE0 + pr), (g >> 1) & 1, abortf));
@@ -327,6 +332,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         Lhw = __uint_as_float(r16[0]);
       }
       const float inv = __frcp_rn(6.0f * Lhw);
+      if (FIXREF && !(Lhw > 0.f && Lhw < INFINITY) && p.status) *p.status = FP4ATTN_ERR_RANGE;   // nothing of the row is inside the byte range
       const size_t grow = (size_t)wi.qrow0 + row;
       // stage the bf16 tile in shared memory (128-byte rows, 128B-swizzled like the tensor map) and
       // let TMA write it out, so O is released after four TMEM reads instead of after 16 global stores
@@ -362,7 +368,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
       }
-      if (PMAP != 1 && has_next) {
+      if (!FIXREF && PMAP != 1 && has_next) {
         // O is released; before the stores go out, serve the next item's first stage (the teams run ahead and
         // have it encoded, or will shortly - nothing they need depends on this epilogue), so that its PV waits
         // for neither the rest of this epilogue nor a pass after it.  A first stage starts a fresh reference,
@@ -453,11 +459,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         if (m > 0) ok = __all_sync(0xffffffffu, mbar_wait(pfree, (m - 1) & 1, abortf));   // PV of the pair's previous stage is done
         if (!ok) break;
+        // fixed reference: E8M0 bytes of the two blocks against the constant; below the range a zero block (no codes,
+        // so that a row without any live block shows as a zero row sum), above it an error
+        const int b0 = FIXREF ? E0 - p.ref_fixed + 127 : 0, b1 = FIXREF ? E1 - p.ref_fixed + 127 : 0;
+        if (FIXREF && __any_sync(0xffffffffu, min(b0, b1) < 1)) {    // rare: some row of the warp has a block below the range
+          if (b0 < 1) w0[0] = w0[1] = w0[2] = w0[3] = 0u;
+          if (b1 < 1) w1[0] = w1[1] = w1[2] = w1[3] = 0u;
+        }
         {
           const uint32_t pw[8] = {w0[0], w0[1], w0[2], w0[3], w1[0], w1[1], w1[2], w1[3]};
           tmem_st_32x32b_x8(tP, pw);
         }
-        *meta = make_int2(E0, E1);
+        if (FIXREF) {
+          if (max(b0, b1) > 254 && p.status) *p.status = FP4ATTN_ERR_RANGE;      // (the byte written below is then meaningless)
+          const uint32_t u0 = (uint32_t)max(b0, 0) & 0xFFu, u1 = (uint32_t)max(b1, 0) & 0xFFu;
+          *reinterpret_cast<uint16_t*>(sgen + C::OFF_PSF + 512 * pr + lane * 16 + quarter * 4 + 2 * (team & 1)) = (uint16_t)(u0 | (u1 << 8));
+          fence_proxy_async_smem();
+        } else {
+          *meta = make_int2(E0, E1);
+        }
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -612,7 +632,7 @@ const CUtensorMap* attention_tensor_maps_fp8v(int D, const fp4attn_operands* ops
   return D == 128 ? tensor_maps<128>(ops, O, B, H, Hkv, N, true) : tensor_maps<64>(ops, O, B, H, Hkv, N, true);
 }
 
-template <int D, int NV, int PMAP, bool CAUSAL, int THR16>
+template <int D, int NV, int PMAP, bool CAUSAL, int THR16, bool FIXREF = false>
 static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnParams prm, cudaStream_t st) {
   const int Hkv = prm.Hkv;
   using C = Cfg<D, (NV != 0)>;
@@ -623,14 +643,14 @@ static int launch_attn(const fp4attn_operands* ops, int B, int H, int N, AttnPar
   static std::atomic<bool> attr_set[kMaxDevices];
   if (dev < 0 || dev >= kMaxDevices) return FP4ATTN_ERR_CUDA;
   if (!attr_set[dev].load(std::memory_order_acquire)) {
-    if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16, FIXREF>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
       return FP4ATTN_ERR_CUDA;
     attr_set[dev].store(true, std::memory_order_release);
   }
   const CUtensorMap* tm = tensor_maps<D>(ops, prm.O, B, H, Hkv, N);
   if (!tm) return FP4ATTN_ERR_CUDA;
   const unsigned grid = (unsigned)(prm.n_items < sms ? prm.n_items : sms);     // persistent: one CTA per SM
-  attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tm[0], tm[1], tm[2], tm[3], prm);
+  attn_fwd_kernel<D, NV, PMAP, CAUSAL, THR16, FIXREF><<<grid, kAttnThreads, C::SMEM_BYTES, st>>>(tm[0], tm[1], tm[2], tm[3], prm);
   return cudaGetLastError() == cudaSuccess ? FP4ATTN_OK : FP4ATTN_ERR_CUDA;
 }
 
@@ -699,6 +719,33 @@ extern "C" int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int
   if (ops->pv_fmt != FP4ATTN_PV_MXFP4 && ops->pv_fmt != FP4ATTN_PV_E4M3) return FP4ATTN_ERR_INVALID_ARG;
   if (ops->seq_len && ops->schedule != FP4ATTN_SCHEDULE_ONE_QUERY) return FP4ATTN_ERR_INVALID_ARG;
   if (((uintptr_t)ops->seq_len & 3) != 0) return FP4ATTN_ERR_ALIGNMENT;
+  if (ops->row_reference != FP4ATTN_REFERENCE_RUNNING && ops->row_reference != FP4ATTN_REFERENCE_FIXED) return FP4ATTN_ERR_INVALID_ARG;
+  prm.ref_fixed = ops->fixed_reference;
+  if (ops->row_reference == FP4ATTN_REFERENCE_FIXED) {
+    // the shiftless path: ideal or affine map, ceiling rule, one factor per tensor, one query tile, FP4 P and V
+    if (pmap > 1 || ops->p_scale_rule != FP4ATTN_PSCALE_CEIL || ops->g_per_head || ops->schedule != FP4ATTN_SCHEDULE_ONE_QUERY ||
+        ops->pv_fmt != FP4ATTN_PV_MXFP4 || ops->fixed_reference < -1000 || ops->fixed_reference > 1000)
+      return FP4ATTN_ERR_INVALID_ARG;
+    const int sel = (d == 128 ? 8 : 0) | (nv ? 4 : 0) | (pmap ? 2 : 0) | (masked ? 1 : 0);
+    switch (sel) {
+      case 0: return launch_attn<64, 0, 0, false, 0, true>(ops, B, H, N, prm, st);
+      case 1: return launch_attn<64, 0, 0, true, 0, true>(ops, B, H, N, prm, st);
+      case 2: return launch_attn<64, 0, 1, false, 0, true>(ops, B, H, N, prm, st);
+      case 3: return launch_attn<64, 0, 1, true, 0, true>(ops, B, H, N, prm, st);
+      case 4: return launch_attn<64, 1, 0, false, 0, true>(ops, B, H, N, prm, st);
+      case 5: return launch_attn<64, 1, 0, true, 0, true>(ops, B, H, N, prm, st);
+      case 6: return launch_attn<64, 1, 1, false, 0, true>(ops, B, H, N, prm, st);
+      case 7: return launch_attn<64, 1, 1, true, 0, true>(ops, B, H, N, prm, st);
+      case 8: return launch_attn<128, 0, 0, false, 0, true>(ops, B, H, N, prm, st);
+      case 9: return launch_attn<128, 0, 0, true, 0, true>(ops, B, H, N, prm, st);
+      case 10: return launch_attn<128, 0, 1, false, 0, true>(ops, B, H, N, prm, st);
+      case 11: return launch_attn<128, 0, 1, true, 0, true>(ops, B, H, N, prm, st);
+      case 12: return launch_attn<128, 1, 0, false, 0, true>(ops, B, H, N, prm, st);
+      case 13: return launch_attn<128, 1, 0, true, 0, true>(ops, B, H, N, prm, st);
+      case 14: return launch_attn<128, 1, 1, false, 0, true>(ops, B, H, N, prm, st);
+      default: return launch_attn<128, 1, 1, true, 0, true>(ops, B, H, N, prm, st);
+    }
+  }
   if (ops->pv_fmt == FP4ATTN_PV_E4M3) return launch_attn_fp8pv(ops, B, H, N, d, prm, st);
   if (ops->schedule == FP4ATTN_SCHEDULE_TWO_QUERY) return launch_attn_two_query(ops, B, H, N, d, pmap, prm, st);
   if (ops->p_scale_rule == FP4ATTN_PSCALE_MSE) {

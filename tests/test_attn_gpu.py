@@ -651,6 +651,76 @@ def test_many_small_heads_more_items_than_one_wave():
     check_heads(Og, Lg, Oo, Lo, heads)
 
 
+# ------------------------------------------------------------------ fixed row reference (the shiftless path)
+FIXREF_CASES = [
+    # name, shrink, map, causal, token counts, K/V group, reference
+    ("cfg1", dict(), "ideal", False, None, 1, 0),
+    ("cfg1", dict(N=640, H=3), "affine", False, None, 1, 0),
+    ("cfg1", dict(N=512, H=4), "ideal", True, None, 2, 0),
+    ("cfg1", dict(B=3, H=2, N=512), "affine", False, [512, 300, 77], 1, 5),
+    ("cfg3", dict(B=2, H=2, N=768), "ideal", True, [700, 330], 1, -20),       # NVFP4 Q/K, d = 64
+    ("cfg3", dict(B=2, H=2, N=512), "affine", False, None, 1, 0),
+    ("cfg2", dict(B=2, H=3, N=2304), "ideal", False, None, 1, 0),             # d = 128, many stages
+    ("cfg2", dict(B=2, H=3, N=2304), "affine", True, None, 1, 30),
+]
+
+
+@pytest.mark.parametrize("name,kw,p_map,causal,lens,group,ref", FIXREF_CASES)
+def test_fixed_row_reference_matches_oracle_and_the_running_reference(name, kw, p_map, causal, lens, group, ref):
+    """The shiftless path: a constant row reference, bytes published by the softmax warps, no rescale.  Against the
+    oracle run with the same reference, and against this library's running reference: O bit for bit (codes do not
+    depend on the reference; numerator and row sum differ by the same power of two), LSE to float32 rounding."""
+    import parity
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS[name], **kw)
+    q, k, v = I.make_qkv(w)
+    k, v = np.ascontiguousarray(k[:, : w.H // group]), np.ascontiguousarray(v[:, : w.H // group])
+    sl = None if lens is None else torch.tensor(lens, dtype=torch.int32, device="cuda")
+    pm = Bd.PMAP_AFFINE if p_map == "affine" else Bd.PMAP_IDEAL
+    Og, Lg = run_gpu_general(w, q, k, v, causal=causal, seq_len=sl, p_map=pm, fixed_reference=ref)
+    Or, Lr = run_gpu_general(w, q, k, v, causal=causal, seq_len=sl, p_map=pm)
+    fmt = "mx" if w.qk_fmt == I.FMT_MXFP4 else "nv"
+    qd, kd, vd = Qz.quantize_qk(q, fmt), Qz.quantize_qk(k, fmt), Qz.quantize_v(v)
+    for b in range(w.B):
+        n = w.N if lens is None else lens[b]
+        assert np.array_equal(Og[b, :, :n], Or[b, :, :n])
+        assert np.abs(Lg[b, :, :n] - Lr[b, :, :n]).max() <= 1e-5 * max(1.0, np.abs(Lr[b, :, :n]).max())
+        for h in range(w.H):
+            okw = {} if lens is None else dict(kv_len=n)
+            st = parity.compare_head(Og[b, h], Lg[b, h], qd, kd, vd, b, h, rows=np.arange(n), kv_group=group, causal=causal,
+                                     p_map=p_map, fixed_reference=ref, **okw)
+            assert st["lse_err"] <= parity.LSE_ABS, st
+
+
+def test_fixed_row_reference_reports_logits_outside_its_range_and_rejects_other_options():
+    """Config 4's rows reach |y| ~ 300 and differ by hundreds of octaves: no constant reference holds them, and the
+    kernel must say so through the status word instead of returning numbers.  A reference far above Gaussian logits
+    loses whole rows the same way."""
+    from paper_2609_04105_b200 import binding as Bd
+    w = I.shrink(I.WORKLOADS["cfg4"], H=2, N=1024)
+    q, k, v = I.make_qkv(w)
+    qg, kg = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+    vg = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Bd.fp4attn_fwd(qg, kg, vg, status=status, fixed_reference=0)
+    torch.cuda.synchronize()
+    assert int(status.item()) == Bd.ERR_RANGE
+    status.zero_()
+    Bd.fp4attn_fwd(qg, kg, vg, status=status)                     # the running reference takes the same input
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    w = I.shrink(I.WORKLOADS["cfg1"], N=256)
+    q, k, v = I.make_qkv(w)
+    qg, kg = Bd.fp4attn_quantize(_dev(q), w.qk_fmt, Bd.ROLE_Q), Bd.fp4attn_quantize(_dev(k), w.qk_fmt, Bd.ROLE_K)
+    vg = Bd.fp4attn_quantize(_dev(v), Bd.FMT_MXFP4, Bd.ROLE_V)
+    Bd.fp4attn_fwd(qg, kg, vg, status=status, fixed_reference=400)                  # every block below the byte range
+    torch.cuda.synchronize()
+    assert int(status.item()) == Bd.ERR_RANGE
+    for kw in (dict(p_scale_rule=Bd.PSCALE_THR16), dict(p_map=Bd.PMAP_HYBRID, exact_pairs=0x5555), dict(fixed_reference=5000)):
+        with pytest.raises(Bd.Fp4AttnError):
+            Bd.fp4attn_fwd(qg, kg, vg, **{**dict(fixed_reference=0), **kw})
+
+
 # ------------------------------------------------------------------ degenerate inputs
 @pytest.mark.parametrize("causal", [False, True])
 def test_degenerate_inputs_zero_queries_zero_values_identical_keys(causal):
