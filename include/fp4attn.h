@@ -306,7 +306,7 @@ int fp4attn_fwd(const fp4attn_operands* ops, int B, int H, int N, int d,
 
 /*
  * E4M3 quantizer of V for the FP8 P/V route (Section "Training stability selects FP8 P/V": the retained training
- * route keeps "E4M3 V views"; the paper states no scale rule).  Every (batch, head) unit gets one encode factor
+ * route keeps V in E4M3; the paper states no scale rule).  Every (batch, head) unit gets one encode factor
  * G[b*H + h] = fl32(448 / max|V[b, h]|) (1 for an all-zero unit), written to unit_scale_out (B*H floats), and
  * every value the byte Q_E4M3(fl32(v * G)), round to nearest even; a value is reconstructed as decode(byte) / G.
  * bytes_out receives V^T, [B, H, d, N] bytes (key index contiguous: the contraction-major layout of the second

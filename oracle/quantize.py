@@ -192,7 +192,7 @@ def quantize_v(bits: np.ndarray, rule: str = "ceil"):
 def quantize_v_e4m3(bits: np.ndarray):
     """V bf16 [B,H,N,d] -> E4M3 bytes of V^T, dict(byte [B,H,d,N] uint8, G float32 [B,H], fmt "e4m3").
 
-    The FP8 value operand of the FP8-P/V route (Section "Training stability selects FP8 P/V": "E4M3 V views"); the
+    The FP8 value operand of the FP8-P/V route (Section "Training stability selects FP8 P/V": V is kept in E4M3 there); the
     paper gives no scale rule, reading taken here: one encode factor per (batch, head) unit, like the per-head
     NVFP4 factors, G = fl32(448 / max|V[b,h]|) (1 for an all-zero unit), byte = Q_E4M3(fl32(v * G)) round to nearest
     even; a value is reconstructed as decode(byte) / G."""
