@@ -179,14 +179,15 @@ def oracle_operands_of_heads(w, q, k, v, amax_qk=None):
     return qd, kd, Qz.quantize_v(v)
 
 
-def oracle_sample(w, q, k, v, n_heads, rows, p_map="ideal", p_scale="ceil", amax_qk=None):
+def oracle_sample(w, q, k, v, n_heads, rows, p_map="ideal", p_scale="ceil", amax_qk=None, fixed_reference=None):
     """Runs the oracle (as it stands) on a bounded sample: `n_heads` units (held by q, k, v) and the given query
     rows.  Returns seconds, equivalent TFLOP/s, its outputs and the quantized operands."""
     from oracle import attention as A
     t0 = time.perf_counter()
     qd, kd, vd = oracle_operands_of_heads(w, q, k, v, amax_qk)
     okw = dict(p_map="hybrid", exact_pairs=HYBRID_PATTERNS[p_map]) if p_map in HYBRID_PATTERNS else dict(p_map=p_map)
-    O, lse = A.direct_p_forward(qd, kd, vd, rows=rows, heads=[(0, i) for i in range(n_heads)], p_scale=p_scale, **okw)
+    O, lse = A.direct_p_forward(qd, kd, vd, rows=rows, heads=[(0, i) for i in range(n_heads)], p_scale=p_scale,
+                                fixed_reference=fixed_reference, **okw)
     dt = time.perf_counter() - t0
     n_rows = w.N if rows is None else len(rows)
     flops = 4.0 * n_heads * n_rows * w.N * w.d
@@ -347,7 +348,7 @@ def run_cuda(args, w):
         if ev is not None:
             ev[0].record()
         Bd.fp4attn_fwd(qd, kd, vd, out=O, lse=lse, status=status, p_map=pmap, p_scale_rule=pscale, exact_pairs=pairs,
-                       schedule=sched)
+                       schedule=sched, fixed_reference=args.fixed_reference)
         if ev is not None:
             ev[1].record()
         state["ops"] = (qd, kd, vd)
@@ -651,7 +652,7 @@ def run_cuda(args, w):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": n_warm, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate)", "data": "synthetic",
-        "config": {"workload": _workload_text(w), "step": "quantize Q,K,V + attention forward", "p_map": args.p_map, "p_scale": args.p_scale,
+        "config": {"workload": _workload_text(w), "step": "quantize Q,K,V + attention forward", "p_map": args.p_map, "p_scale": args.p_scale, "row_reference": "running" if args.fixed_reference is None else f"fixed at {args.fixed_reference}",
                    "schedule": args.schedule, "l2": "flushed between steps (256 MiB fill, outside the step's events)",
                    "warmup": f"{n_warm} steps (at least --warmup and 300 ms)",
                    "flops": "4*B*H*N^2*d", "parallelism": f"replica x{world}, (batch, head) units, no collective"},
@@ -678,7 +679,7 @@ def run_cuda(args, w):
     if sample is not None:
         rows, heads = sample["rows"], sample["heads"]
         dt, tf, Oo, Lo, ops = oracle_sample(w, sample["q"], sample["k"], sample["v"], len(heads), rows, args.p_map, args.p_scale,
-                                            sample["amax"])
+                                            sample["amax"], fixed_reference=args.fixed_reference)
         Og = sample["Og"]
         rel = max(float(np.linalg.norm(Og[i] - Oo[i]) / np.linalg.norm(Oo[i])) for i in range(len(heads)))
         text = f"{len(heads)} (batch, head) units x {len(rows)} seeded query rows of {w.name}, {dt:.1f} s"
@@ -711,6 +712,8 @@ def main():
                          "the two neighbouring exponents by squared error (ideal map only)")
     ap.add_argument("--schedule", default="one-query", choices=["one-query", "two-query"],
                     help="query tiles per thread block in the timed step (two-query: d = 64 workloads only)")
+    ap.add_argument("--fixed-reference", type=int, default=None,
+                    help="time the step with this constant row reference (the shiftless path; ideal or affine map, ceiling rule)")
     ap.add_argument("--p-map", default="ideal", choices=["ideal", "affine", "hybrid4", "hybrid8", "hybrid12"],
                     help="score->code map of the timed path: exact codes (default), the paper's affine classifier, or "
                          "4 / 8 / 12 of every 16 element pairs exact and the rest affine (EX2-density control)")
